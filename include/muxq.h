@@ -1,0 +1,189 @@
+/*
+ * libmuxq -- MUXQ quantized linear layer (Y = X.W with outlier-channel redistribution) for
+ * NVIDIA B200 (sm_100a).  C ABI: plain pointers and sizes, no C++ or framework types.
+ *
+ * Method (paper notation): X [M,K] fp16 activations, W [K,N] fp16 weights.
+ *   - outlier channel = column k of X holding at least one |x| > threshold (Section III-C);
+ *     O = ascending list of such k, r = |O|.
+ *   - Body = X with the columns in O multiplied by 2^-exp (Eq. 4); Aux = Body[:, O] (Eq. 5);
+ *     X[:, O] = Body[:, O] + (2^exp - 1) Aux (Eq. 6).
+ *   - abs-max quantization (Eq. 1, Eq. 2): s = max|.| / qmax, code = round_half_even(v / s),
+ *     qmax = 2^(bits-1) - 1, codes clamped to [-qmax, qmax] and stored as int8.  An all-zero
+ *     unit gets s = 1.  Granularity: per tensor, or per vector = per token (row of X) and per
+ *     output channel (column of W) (Section II-A, Fig. 2).
+ *   - Y = dequant( Body_q.W_q + (2^exp - 1) Aux_q.W_q[O,:] ) (Eq. 7, Eq. 3), int32 accumulation.
+ *
+ * Conventions for every entry point
+ *   - All tensor pointers are DEVICE pointers unless the name says "host".  Row-major; "ld" is
+ *     the row pitch in ELEMENTS.  fp16 is IEEE binary16 passed as void*.
+ *   - The caller owns every buffer, including the workspace; the library allocates no device
+ *     memory and keeps no state between calls.  `stream` is a cudaStream_t passed as void*
+ *     (NULL = the legacy default stream).
+ *   - Calls only enqueue work; nothing synchronizes except muxq_read_status and
+ *     muxq_linear_host's final copy-back wait when asked.
+ *   - The int return value reports what the host can see at call time (bad arguments,
+ *     unsupported shapes, workspace too small, CUDA launch errors).  Data-dependent conditions
+ *     (more outlier channels than the capacity, an expired bounded device-side wait) are
+ *     written to the device status word; a kernel never traps and never writes out of bounds.
+ *   - Inputs must be finite.  NaN/Inf give unspecified (but memory-safe) results.
+ *   - Alignment: X, W, Y, workspace 16-byte aligned; K % 16 == 0; ldx % 8 == 0; N % 8 == 0.
+ */
+#ifndef MUXQ_H
+#define MUXQ_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    MUXQ_OK = 0,
+    MUXQ_ERR_INVALID_ARG = 1,
+    MUXQ_ERR_UNSUPPORTED = 2,
+    MUXQ_ERR_WORKSPACE = 3,
+    MUXQ_ERR_CUDA = 4,
+    MUXQ_ERR_CAPACITY = 5, /* device status: r > max_outliers */
+    MUXQ_ERR_TIMEOUT = 6   /* device status: a bounded wait inside a kernel expired */
+} muxq_status;
+
+typedef enum { MUXQ_PER_TENSOR = 0, MUXQ_PER_VECTOR = 1 /* per-token X, per-channel W */ } muxq_gran;
+/* Scale of the Aux block: shared with Body (Aux_q == Body_q[:,O], integer combine) or its own
+ * abs-max.  The paper does not say (Eq. 5 only states Aux = Body_outlier); shared is the default. */
+typedef enum { MUXQ_AUX_SHARED = 0, MUXQ_AUX_OWN = 1 } muxq_aux_scale;
+typedef enum { MUXQ_OUT_F16 = 0, MUXQ_OUT_F32 = 1, MUXQ_OUT_ACC_I32 = 2 /* raw combined accumulator */ } muxq_out;
+
+typedef struct muxq_params {
+    float threshold;  /* outlier criterion, 6.0 (Section III-C) */
+    int exp_factor;   /* 1..3; the paper uses 2 (Section III-C) */
+    int act_bits;     /* 2..8 (Eq. 1 uses 8) */
+    int w_bits;       /* 2..8 (Eq. 2 uses 8) */
+    int gran;         /* muxq_gran */
+    int aux_scale;    /* muxq_aux_scale; only MUXQ_AUX_SHARED runs on the GPU path */
+    int max_outliers; /* capacity of O, 1..64 */
+} muxq_params;
+
+/* threshold 6, exp factor 2, 8/8 bits, per tensor, shared Aux scale, capacity 64. */
+void muxq_default_params(muxq_params *p);
+
+/* Width in bytes/columns of the Aux block in GEMM operand layout:
+ * round_up((2^exp - 1) * max_outliers, 128).  0 on invalid params. */
+int muxq_aux_cols(const muxq_params *p);
+
+/* Bytes of workspace muxq_linear needs for a [M,K] x [K,N] call (0 on invalid arguments). */
+size_t muxq_workspace_bytes(int M, int K, int N, const muxq_params *p);
+/* Bytes of workspace muxq_detect_outliers / muxq_quantize need (small; independent of M). */
+size_t muxq_small_workspace_bytes(int cols);
+/* Bytes of workspace muxq_linear_host needs: muxq_workspace_bytes + device staging of X and Y. */
+size_t muxq_host_workspace_bytes(int M, int K, int N, const muxq_params *p, int out_kind);
+
+/*
+ * Outlier-channel detection (Section III-C: a channel with at least one element of magnitude
+ * greater than `threshold`, strict).
+ *   X          [M,K] fp16, pitch ldx
+ *   col_absmax [K] fp32 out: max_m |X[m,k]|
+ *   outlier_idx[cap] int32 out: the first min(r,cap) outlier channels, ascending
+ *   n_outliers [1] int32 out: r, the true count (may exceed cap)
+ *   workspace  >= muxq_small_workspace_bytes(K); contents need not be initialised
+ * r > cap is not an error here; muxq_linear reports it as MUXQ_ERR_CAPACITY.
+ */
+int muxq_detect_outliers(const void *X_f16, int M, int K, int ldx, float threshold,
+                         float *col_absmax, int32_t *outlier_idx, int32_t *n_outliers, int cap,
+                         void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * Real-domain decomposition (Eq. 4, Eq. 5), for inspection and tests.
+ *   Aux  [M, ld_aux >= cap] fp32 out: Aux[m,j] = X[m,O_j] * 2^-exp for j < min(r,cap), else 0
+ *   Body [M, ld_body >= K] fp32 out, or NULL: X with the columns in O multiplied by 2^-exp
+ * fp32 outputs keep Eq. 6 exact: Body[:,O] + (2^exp - 1) Aux == X[:,O] bit for bit.
+ */
+int muxq_build_aux(const void *X_f16, int M, int K, int ldx, const int32_t *outlier_idx,
+                   const int32_t *n_outliers, int cap, int exp_factor, float *Aux, int ld_aux,
+                   float *Body_or_null, int ld_body, void *stream);
+
+/*
+ * Abs-max quantization (Eq. 1 for activations, Eq. 2 for weights).
+ *
+ * is_weight = 1: A is W [rows=K, cols=N] fp16.  Writes W_q TRANSPOSED, [N, ld_q >= K] int8
+ *   (K contiguous: the tensor-core B operand layout), scales [1] (per tensor) or [N] (per
+ *   vector).  col_absmax / outlier_idx / n_outliers / Aux_q are ignored (pass NULL).
+ *
+ * is_weight = 0: A is X [rows=M, cols=K] fp16; fused redistribute-and-quantize (Eq. 4-5 then
+ *   Eq. 1).  col_absmax [K] must hold muxq_detect_outliers' output for this X.
+ *   outlier_idx/n_outliers from the same call, or both NULL for naive quantization (O empty).
+ *   Writes Body_q [M, ld_q >= K] int8 and, when Aux_q != NULL, the Aux block in operand layout:
+ *   Aux_q [M, ld_aux >= muxq_aux_cols(p)] with Aux_q[m, c*j + t] = Body_q[m, O_j] for j < r,
+ *   t < c = 2^exp - 1 (each Aux column repeated c times so that one integer accumulation yields
+ *   Body_q.W_q + c Aux_q.W_q[O,:]); remaining columns zero.  scales: [1] or [M].
+ *   r > p->max_outliers: only the first max_outliers channels are treated (muxq_linear flags it).
+ *
+ * workspace >= muxq_small_workspace_bytes(cols).
+ */
+int muxq_quantize(const void *A_f16, int rows, int cols, int ld, const muxq_params *p, int is_weight,
+                  const float *col_absmax, const int32_t *outlier_idx, const int32_t *n_outliers,
+                  int8_t *A_q, int ld_q, int8_t *Aux_q, int ld_aux, float *scales,
+                  void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * The integer products, weighted sum and dequantization alone (Eq. 7, Eq. 3) on already
+ * quantized operands:
+ *   acc[m,n] = sum_k Body_q[m,k] W_q[n,k] + sum_{i < c*min(r,cap)} Aux_q[m,i] W_aux[n,i]
+ *   Y[m,n]   = (s_x[m or 0] * s_w[n or 0]) * float(acc[m,n])   (F16: then rounded to fp16)
+ *   Body_q [M, ld_a >= K], Aux_q [M, ld_aux], W_q [N, ldw >= K], W_aux [N, ld_waux], all int8,
+ *   pitches multiples of 16.  W_aux[n, c*j+t] = W_q[n, O_j].  Aux_q/W_aux/n_outliers may be NULL
+ *   (no Aux term).  s_x has M entries if gran is per vector else 1; s_w has N or 1.
+ *   Y: [M, ldy] fp16 / fp32 / int32 by out_kind (int32: the raw acc).
+ *   dev_status: device int32, set to MUXQ_ERR_TIMEOUT if a bounded wait expires (else untouched).
+ */
+int muxq_gemm(const int8_t *Body_q, int ld_a, const int8_t *Aux_q, int ld_aux, const int8_t *W_q,
+              int ldw, const int8_t *W_aux, int ld_waux, const int32_t *n_outliers, int M, int K,
+              int N, const muxq_params *p, const float *s_x, const float *s_w, void *Y, int ldy,
+              int out_kind, int32_t *dev_status, void *stream);
+
+/*
+ * The whole layer: detect -> redistribute + quantize -> INT8 products + Aux correction ->
+ * dequantize (Section III-C, Eq. 1-7).  W_q [N, ldw] and s_w come from muxq_quantize(is_weight=1)
+ * with the same params.  M <= 16 takes the memory-bound decode path; larger M the tensor-core
+ * path.  Y: [M, ldy] by out_kind.  workspace >= muxq_workspace_bytes(M,K,N,p), contents need
+ * not be initialised.  dev_status: device int32; the call sets it to 0 first, kernels raise it
+ * to MUXQ_ERR_CAPACITY (r > max_outliers; Y then unspecified but in bounds) or MUXQ_ERR_TIMEOUT.
+ * Intermediate results stay in the workspace afterwards; muxq_workspace_view locates them.
+ */
+int muxq_linear(const void *X_f16, int M, int K, int ldx, const int8_t *W_q, int ldw,
+                const float *s_w, int N, const muxq_params *p, void *Y, int ldy, int out_kind,
+                void *workspace, size_t workspace_bytes, int32_t *dev_status, void *stream);
+
+/* Where muxq_linear leaves its intermediates inside the workspace (byte offsets). */
+typedef struct muxq_ws_view {
+    size_t col_absmax;  /* float [K] */
+    size_t outlier_idx; /* int32 [max_outliers] */
+    size_t n_outliers;  /* int32 [1] */
+    size_t s_x;         /* float [1] or [M] */
+    size_t body_q;      /* int8 [M, ld_body_q] */
+    size_t aux_q;       /* int8 [M, aux_cols] */
+    size_t w_aux;       /* int8 [N, aux_cols] */
+    int ld_body_q;
+    int aux_cols;
+} muxq_ws_view;
+int muxq_workspace_view(int M, int K, int N, const muxq_params *p, muxq_ws_view *view);
+
+/*
+ * muxq_linear with X and Y in HOST memory (pinned for true asynchrony): copies X to the device,
+ * runs the layer, copies Y back, all on `stream`.  W_q, s_w, workspace and dev_status stay
+ * device pointers.  workspace >= muxq_host_workspace_bytes(...).  X_host must be dense
+ * (pitch K), Y_host dense (pitch N).  Does not synchronize.
+ */
+int muxq_linear_host(const void *X_f16_host, int M, int K, const int8_t *W_q, int ldw,
+                     const float *s_w, int N, const muxq_params *p, void *Y_host, int out_kind,
+                     void *workspace, size_t workspace_bytes, int32_t *dev_status, void *stream);
+
+/* Synchronizes `stream` and returns the device status word (or MUXQ_ERR_CUDA). */
+int muxq_read_status(const int32_t *dev_status, void *stream);
+
+const char *muxq_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MUXQ_H */

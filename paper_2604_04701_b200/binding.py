@@ -1,0 +1,250 @@
+"""ctypes binding of libmuxq.so.  Function names and argument order follow include/muxq.h;
+tensors are torch CUDA tensors whose data_ptr() is passed straight through."""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+from typing import Optional, Tuple
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libmuxq.so")
+
+MUXQ_OK, MUXQ_ERR_INVALID_ARG, MUXQ_ERR_UNSUPPORTED, MUXQ_ERR_WORKSPACE = 0, 1, 2, 3
+MUXQ_ERR_CUDA, MUXQ_ERR_CAPACITY, MUXQ_ERR_TIMEOUT = 4, 5, 6
+MUXQ_PER_TENSOR, MUXQ_PER_VECTOR = 0, 1
+MUXQ_AUX_SHARED, MUXQ_AUX_OWN = 0, 1
+MUXQ_OUT_F16, MUXQ_OUT_F32, MUXQ_OUT_ACC_I32 = 0, 1, 2
+
+EXPORTS = (
+    "muxq_default_params", "muxq_aux_cols", "muxq_workspace_bytes", "muxq_small_workspace_bytes",
+    "muxq_host_workspace_bytes", "muxq_workspace_view", "muxq_detect_outliers", "muxq_build_aux",
+    "muxq_quantize", "muxq_gemm", "muxq_linear", "muxq_linear_host", "muxq_read_status",
+    "muxq_status_string",
+)
+
+
+class MuxqError(RuntimeError):
+    def __init__(self, fn: str, status: int):
+        super().__init__(f"{fn}: {muxq_status_string(status)} (status {status})")
+        self.status = status
+
+
+class _CParams(ctypes.Structure):
+    _fields_ = [("threshold", ctypes.c_float), ("exp_factor", ctypes.c_int), ("act_bits", ctypes.c_int),
+                ("w_bits", ctypes.c_int), ("gran", ctypes.c_int), ("aux_scale", ctypes.c_int),
+                ("max_outliers", ctypes.c_int)]
+
+
+class _CWsView(ctypes.Structure):
+    _fields_ = [("col_absmax", ctypes.c_size_t), ("outlier_idx", ctypes.c_size_t),
+                ("n_outliers", ctypes.c_size_t), ("s_x", ctypes.c_size_t), ("body_q", ctypes.c_size_t),
+                ("aux_q", ctypes.c_size_t), ("w_aux", ctypes.c_size_t), ("ld_body_q", ctypes.c_int),
+                ("aux_cols", ctypes.c_int)]
+
+
+@dataclass
+class MuxqParams:
+    threshold: float = 6.0
+    exp_factor: int = 2
+    act_bits: int = 8
+    w_bits: int = 8
+    gran: int = MUXQ_PER_TENSOR
+    aux_scale: int = MUXQ_AUX_SHARED
+    max_outliers: int = 64
+
+    def c(self) -> _CParams:
+        return _CParams(self.threshold, self.exp_factor, self.act_bits, self.w_bits, self.gran,
+                        self.aux_scale, self.max_outliers)
+
+
+_lib = None
+
+
+def library_path() -> str:
+    return _LIB_PATH
+
+
+def lib() -> ctypes.CDLL:
+    """Loads libmuxq.so; raises if it has not been built (there is no fallback path)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_LIB_PATH):
+            raise RuntimeError(
+                f"{_LIB_PATH} is missing: build it with `python -m paper_2604_04701_b200.build` "
+                "(nvcc, sm_100a).  There is no CPU fallback.")
+        L = ctypes.CDLL(_LIB_PATH)
+        vp, i, sz, f = ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t, ctypes.c_float
+        pp = ctypes.POINTER(_CParams)
+        L.muxq_default_params.argtypes = [pp]; L.muxq_default_params.restype = None
+        L.muxq_aux_cols.argtypes = [pp]; L.muxq_aux_cols.restype = i
+        L.muxq_workspace_bytes.argtypes = [i, i, i, pp]; L.muxq_workspace_bytes.restype = sz
+        L.muxq_small_workspace_bytes.argtypes = [i]; L.muxq_small_workspace_bytes.restype = sz
+        L.muxq_host_workspace_bytes.argtypes = [i, i, i, pp, i]; L.muxq_host_workspace_bytes.restype = sz
+        L.muxq_workspace_view.argtypes = [i, i, i, pp, ctypes.POINTER(_CWsView)]; L.muxq_workspace_view.restype = i
+        L.muxq_detect_outliers.argtypes = [vp, i, i, i, f, vp, vp, vp, i, vp, sz, vp]; L.muxq_detect_outliers.restype = i
+        L.muxq_build_aux.argtypes = [vp, i, i, i, vp, vp, i, i, vp, i, vp, i, vp]; L.muxq_build_aux.restype = i
+        L.muxq_quantize.argtypes = [vp, i, i, i, pp, i, vp, vp, vp, vp, i, vp, i, vp, vp, sz, vp]; L.muxq_quantize.restype = i
+        L.muxq_gemm.argtypes = [vp, i, vp, i, vp, i, vp, i, vp, i, i, i, pp, vp, vp, vp, i, i, vp, vp]; L.muxq_gemm.restype = i
+        L.muxq_linear.argtypes = [vp, i, i, i, vp, i, vp, i, pp, vp, i, i, vp, sz, vp, vp]; L.muxq_linear.restype = i
+        L.muxq_linear_host.argtypes = [vp, i, i, vp, i, vp, i, pp, vp, i, vp, sz, vp, vp]; L.muxq_linear_host.restype = i
+        L.muxq_read_status.argtypes = [vp, vp]; L.muxq_read_status.restype = i
+        L.muxq_status_string.argtypes = [i]; L.muxq_status_string.restype = ctypes.c_char_p
+        _lib = L
+    return _lib
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream() -> ctypes.c_void_p:
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _check(fn: str, rc: int):
+    if rc != MUXQ_OK:
+        raise MuxqError(fn, rc)
+
+
+def muxq_status_string(status: int) -> str:
+    return lib().muxq_status_string(int(status)).decode()
+
+
+def muxq_aux_cols(p: MuxqParams) -> int:
+    return int(lib().muxq_aux_cols(ctypes.byref(p.c())))
+
+
+def muxq_workspace_bytes(M: int, K: int, N: int, p: MuxqParams) -> int:
+    return int(lib().muxq_workspace_bytes(M, K, N, ctypes.byref(p.c())))
+
+
+def muxq_small_workspace_bytes(cols: int) -> int:
+    return int(lib().muxq_small_workspace_bytes(cols))
+
+
+def muxq_host_workspace_bytes(M: int, K: int, N: int, p: MuxqParams, out_kind: int) -> int:
+    return int(lib().muxq_host_workspace_bytes(M, K, N, ctypes.byref(p.c()), out_kind))
+
+
+def muxq_workspace_view(M: int, K: int, N: int, p: MuxqParams) -> _CWsView:
+    v = _CWsView()
+    _check("muxq_workspace_view", lib().muxq_workspace_view(M, K, N, ctypes.byref(p.c()), ctypes.byref(v)))
+    return v
+
+
+class Workspace:
+    """Caller-owned device scratch (a torch uint8 tensor) plus the device status word."""
+
+    def __init__(self, nbytes: int, device="cuda"):
+        self.buf = torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=device)
+        self.status = torch.zeros(1, dtype=torch.int32, device=device)
+
+    @property
+    def nbytes(self) -> int:
+        return self.buf.numel()
+
+
+def muxq_detect_outliers(X: torch.Tensor, threshold: float, cap: int, ws: Workspace
+                         ) -> Tuple[torch.Tensor, torch.Tensor, torch.Tensor]:
+    """Returns (col_absmax [K] f32, outlier_idx [cap] i32, n_outliers [1] i32), all on device."""
+    assert X.is_cuda and X.dtype == torch.float16 and X.dim() == 2 and X.stride(1) == 1
+    M, K = X.shape
+    col_absmax = torch.empty(K, dtype=torch.float32, device=X.device)
+    idx = torch.full((cap,), -1, dtype=torch.int32, device=X.device)
+    n = torch.empty(1, dtype=torch.int32, device=X.device)
+    _check("muxq_detect_outliers",
+           lib().muxq_detect_outliers(_ptr(X), M, K, X.stride(0), float(threshold), _ptr(col_absmax), _ptr(idx),
+                                      _ptr(n), cap, _ptr(ws.buf), ws.nbytes, _stream()))
+    return col_absmax, idx, n
+
+
+def muxq_build_aux(X: torch.Tensor, outlier_idx: torch.Tensor, n_outliers: torch.Tensor, exp_factor: int,
+                   want_body: bool = True):
+    """Real-domain Eq. 4-5: returns (Aux [M,cap] f32, Body [M,K] f32 or None)."""
+    M, K = X.shape
+    cap = outlier_idx.numel()
+    aux = torch.empty(M, cap, dtype=torch.float32, device=X.device)
+    body = torch.empty(M, K, dtype=torch.float32, device=X.device) if want_body else None
+    _check("muxq_build_aux",
+           lib().muxq_build_aux(_ptr(X), M, K, X.stride(0), _ptr(outlier_idx), _ptr(n_outliers), cap, exp_factor,
+                                _ptr(aux), cap, _ptr(body), K, _stream()))
+    return aux, body
+
+
+def muxq_quantize(A: torch.Tensor, p: MuxqParams, is_weight: bool, ws: Workspace,
+                  col_absmax: Optional[torch.Tensor] = None, outlier_idx: Optional[torch.Tensor] = None,
+                  n_outliers: Optional[torch.Tensor] = None, want_aux: bool = True):
+    """Weights: returns (W_q [N,K] i8, s_w).  Activations: returns (Body_q [M,K] i8, Aux_q [M,aux_cols] i8
+    or None, s_x)."""
+    assert A.is_cuda and A.dtype == torch.float16 and A.dim() == 2 and A.stride(1) == 1
+    rows, cols = A.shape
+    per_vec = p.gran == MUXQ_PER_VECTOR
+    if is_weight:
+        A_q = torch.empty(cols, rows, dtype=torch.int8, device=A.device)
+        scales = torch.empty(cols if per_vec else 1, dtype=torch.float32, device=A.device)
+        _check("muxq_quantize",
+               lib().muxq_quantize(_ptr(A), rows, cols, A.stride(0), ctypes.byref(p.c()), 1, None, None, None,
+                                   _ptr(A_q), rows, None, 0, _ptr(scales), _ptr(ws.buf), ws.nbytes, _stream()))
+        return A_q, scales
+    A_q = torch.empty(rows, cols, dtype=torch.int8, device=A.device)
+    aux_cols = muxq_aux_cols(p)
+    aux_q = torch.empty(rows, aux_cols, dtype=torch.int8, device=A.device) if want_aux else None
+    scales = torch.empty(rows if per_vec else 1, dtype=torch.float32, device=A.device)
+    _check("muxq_quantize",
+           lib().muxq_quantize(_ptr(A), rows, cols, A.stride(0), ctypes.byref(p.c()), 0, _ptr(col_absmax),
+                               _ptr(outlier_idx), _ptr(n_outliers), _ptr(A_q), cols, _ptr(aux_q), aux_cols,
+                               _ptr(scales), _ptr(ws.buf), ws.nbytes, _stream()))
+    return A_q, aux_q, scales
+
+
+def _alloc_out(M: int, N: int, out_kind: int, device) -> torch.Tensor:
+    dt = {MUXQ_OUT_F16: torch.float16, MUXQ_OUT_F32: torch.float32, MUXQ_OUT_ACC_I32: torch.int32}[out_kind]
+    return torch.empty(M, N, dtype=dt, device=device)
+
+
+def muxq_gemm(body_q: torch.Tensor, aux_q: Optional[torch.Tensor], w_q: torch.Tensor,
+              w_aux: Optional[torch.Tensor], n_outliers: Optional[torch.Tensor], p: MuxqParams,
+              s_x: Optional[torch.Tensor], s_w: Optional[torch.Tensor], out_kind: int, ws: Workspace,
+              out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    M, K = body_q.shape
+    N = w_q.shape[0]
+    Y = out if out is not None else _alloc_out(M, N, out_kind, body_q.device)
+    _check("muxq_gemm",
+           lib().muxq_gemm(_ptr(body_q), body_q.stride(0), _ptr(aux_q), aux_q.stride(0) if aux_q is not None else 0,
+                           _ptr(w_q), w_q.stride(0), _ptr(w_aux), w_aux.stride(0) if w_aux is not None else 0,
+                           _ptr(n_outliers), M, K, N, ctypes.byref(p.c()), _ptr(s_x), _ptr(s_w), _ptr(Y),
+                           Y.stride(0), out_kind, _ptr(ws.status), _stream()))
+    return Y
+
+
+def muxq_linear(X: torch.Tensor, w_q: torch.Tensor, s_w: torch.Tensor, p: MuxqParams, ws: Workspace,
+                out_kind: int = MUXQ_OUT_F16, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """Y = MUXQ-quantized X.W; w_q [N,K] int8 and s_w from muxq_quantize(is_weight=True)."""
+    assert X.is_cuda and X.dtype == torch.float16 and X.dim() == 2 and X.stride(1) == 1
+    M, K = X.shape
+    N = w_q.shape[0]
+    Y = out if out is not None else _alloc_out(M, N, out_kind, X.device)
+    _check("muxq_linear",
+           lib().muxq_linear(_ptr(X), M, K, X.stride(0), _ptr(w_q), w_q.stride(0), _ptr(s_w), N,
+                             ctypes.byref(p.c()), _ptr(Y), Y.stride(0), out_kind, _ptr(ws.buf), ws.nbytes,
+                             _ptr(ws.status), _stream()))
+    return Y
+
+
+def muxq_linear_host(X_host: torch.Tensor, w_q: torch.Tensor, s_w: torch.Tensor, p: MuxqParams, ws: Workspace,
+                     Y_host: torch.Tensor, out_kind: int = MUXQ_OUT_F16) -> torch.Tensor:
+    """X_host / Y_host are CPU tensors (pinned for asynchronous copies); everything else on device."""
+    assert not X_host.is_cuda and not Y_host.is_cuda and X_host.is_contiguous() and Y_host.is_contiguous()
+    M, K = X_host.shape
+    N = w_q.shape[0]
+    _check("muxq_linear_host",
+           lib().muxq_linear_host(_ptr(X_host), M, K, _ptr(w_q), w_q.stride(0), _ptr(s_w), N, ctypes.byref(p.c()),
+                                  _ptr(Y_host), out_kind, _ptr(ws.buf), ws.nbytes, _ptr(ws.status), _stream()))
+    return Y_host
+
+
+def muxq_read_status(ws: Workspace) -> int:
+    return int(lib().muxq_read_status(_ptr(ws.status), _stream()))

@@ -1,0 +1,104 @@
+// Internal launch interface between the C-ABI host layer (api.cu) and the kernels.
+#pragma once
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace muxq {
+
+// Device control block at the start of every workspace (zeroed by one memset per call together
+// with the column abs-max accumulators that follow it).
+struct Ctrl {
+    uint32_t blocks_done;  // K1: CTAs that have merged their partial maxima
+    int32_t n_outliers;    // r, true count of outlier channels
+    float s_x;             // per-tensor Body scale (Eq. 1)
+    uint32_t reserved[61];
+};
+static_assert(sizeof(Ctrl) == 256, "Ctrl is one 256-byte block");
+
+struct DetectArgs {
+    const __half *X;
+    int M, K, ldx;
+    float tau;
+    int exp_factor;   // e
+    int qmax;         // 2^(bits-1)-1
+    int cap;
+    uint32_t *colmax_bits;  // [K] zero-initialised; bit patterns of non-negative floats
+    Ctrl *ctrl;             // zero-initialised
+    int32_t *outlier_idx;   // [cap] out
+    int32_t *n_outliers;    // [1] out (may alias &ctrl->n_outliers)
+    float *colmul;          // [K] out or NULL: 2^-e on outlier channels (first cap of them), else 1
+    uint8_t *grpflag;       // [K/8] out or NULL: 1 if the 8-column group holds an outlier channel
+    float *s_x;             // [1] out or NULL: per-tensor Body scale
+    int32_t *dev_status;    // out or NULL: raised to MUXQ_ERR_CAPACITY when r > cap
+};
+cudaError_t launch_detect(const DetectArgs &a, cudaStream_t s);
+
+// Finalize-only: colmax already complete (used by muxq_quantize on a caller-provided col_absmax).
+cudaError_t launch_detect_finalize(const DetectArgs &a, cudaStream_t s);
+
+struct QuantActArgs {
+    const __half *X;
+    int M, K, ldx;
+    int exp_factor, qmax, cap, per_token;
+    const int32_t *outlier_idx;  // may be NULL (no outliers)
+    const int32_t *n_outliers;   // may be NULL
+    const float *colmul;         // [K] or NULL when outlier_idx is NULL
+    const uint8_t *grpflag;      // [K/8] or NULL
+    const float *s_x_tensor;     // [1] per-tensor scale (device), used when !per_token
+    float *s_x_rows;             // [M] out when per_token
+    int8_t *body_q;  int ld_q;
+    int8_t *aux_q;   int ld_aux; int aux_cols;   // aux_q may be NULL
+    // W_aux gather fused into the same launch (all NULL/0 to skip)
+    const int8_t *w_q; int ldw; int N;
+    int8_t *w_aux; int ld_waux;
+};
+cudaError_t launch_quant_act(const QuantActArgs &a, cudaStream_t s);
+
+struct QuantWeightArgs {
+    const __half *W;  // [K,N]
+    int K, N, ldw;
+    int qmax, per_channel;
+    const uint32_t *colmax_bits;  // [N] abs-max per output channel (complete)
+    const float *s_tensor;        // [1] per-tensor scale (complete)
+    float *s_w;                   // [1] or [N] out
+    int8_t *w_q; int ld_q;        // [N, ld_q] out
+};
+cudaError_t launch_quant_weight(const QuantWeightArgs &a, cudaStream_t s);
+
+struct BuildAuxArgs {
+    const __half *X; int M, K, ldx;
+    const int32_t *outlier_idx; const int32_t *n_outliers; int cap, exp_factor;
+    float *aux; int ld_aux; float *body; int ld_body;
+};
+cudaError_t launch_build_aux(const BuildAuxArgs &a, cudaStream_t s);
+
+struct GemmArgs {
+    const int8_t *body_q; int ld_a;
+    const int8_t *aux_q;  int ld_aux;
+    const int8_t *w_q;    int ldw;
+    const int8_t *w_aux;  int ld_waux;
+    const int32_t *n_outliers;  // may be NULL
+    int M, K, N;
+    int c, cap, aux_cols;
+    const float *s_x; int s_x_per_row;
+    const float *s_w; int s_w_per_col;
+    void *Y; int ldy; int out_kind;
+    int32_t *dev_status;
+};
+cudaError_t launch_gemm(const GemmArgs &a, cudaStream_t s);
+
+struct DecodeArgs {
+    const int8_t *body_q; int ld_a;   // [M, K]
+    const int8_t *w_q; int ldw;       // [N, K]
+    const int32_t *outlier_idx; const int32_t *n_outliers;
+    int M, K, N, c, cap;
+    const float *s_x; int s_x_per_row;
+    const float *s_w; int s_w_per_col;
+    void *Y; int ldy; int out_kind;
+};
+cudaError_t launch_decode(const DecodeArgs &a, cudaStream_t s);
+
+int num_sms();
+
+}  // namespace muxq

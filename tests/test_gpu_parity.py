@@ -1,0 +1,337 @@
+"""GPU parity: every stage of the CUDA path (through the C-ABI binding) against the CPU oracle on
+the same seeded inputs.  Integer results (codes, accumulators, outlier sets) and fp32 scales must
+match bit for bit; fp32 outputs within 1e-5 relative; fp16 outputs within 1 ulp."""
+import numpy as np
+import pytest
+
+import muxq_synth as synth
+import oracle
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def mx():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    import paper_2604_04701_b200 as m
+    m.lib()
+    return m
+
+
+def dev(a):
+    return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+def f16_ulp_diff(a, b):
+    """Distance in units of fp16 spacing between two float16 arrays (as ordered integers)."""
+    def key(x):
+        u = x.view(np.uint16).astype(np.int32)
+        return np.where(u & 0x8000, -(u & 0x7FFF), u)
+    return np.abs(key(a) - key(b))
+
+
+def rel_err32(y, ref):
+    den = np.maximum(np.abs(ref), 1e-6 * np.abs(ref).max())
+    return (np.abs(y.astype(np.float64) - ref.astype(np.float64)) / den).max()
+
+
+def make_case(seed, M, K, N, n_out=4, mult=50.0, bulk="normal", bulk_scale=1.0):
+    x, ch = synth.make_x(seed, 3, M, K, n_out, mult, mult, bulk, bulk_scale)
+    w = synth.make_w(seed, 3, K, N)
+    return x, w, ch
+
+
+def run_linear(mx, x, w, p, out_kind, rows=None):
+    """GPU: quantize W, run the layer; returns (Y, workspace tensors) and oracle result."""
+    M, K = x.shape
+    N = w.shape[1]
+    wsw = mx.Workspace(mx.muxq_small_workspace_bytes(N))
+    w_q, s_w = mx.muxq_quantize(dev(w), p, True, wsw)
+    ws = mx.Workspace(mx.muxq_workspace_bytes(M, K, N, p))
+    ws.buf.fill_(0xA5)  # the workspace need not be initialised
+    y = mx.muxq_linear(dev(x), w_q, s_w, p, ws, out_kind)
+    st = mx.muxq_read_status(ws)
+    return y, ws, st, w_q, s_w
+
+
+def oracle_linear(x, w, p, rows=None):
+    per_vec = p.gran == 1
+    wq, sw = oracle.quantize_weight(w, bits=p.w_bits, per_channel=per_vec)
+    res = oracle.linear(x, wq, sw, tau=p.threshold, e=p.exp_factor, act_bits=p.act_bits, per_vector=per_vec,
+                        cap=p.max_outliers, rows=rows)
+    return wq, sw, res
+
+
+def ws_views(mx, ws, M, K, N, p):
+    v = mx.muxq_workspace_view(M, K, N, p)
+    b = ws.buf.cpu().numpy()
+    cap = p.max_outliers
+    out = {
+        "col_absmax": b[v.col_absmax: v.col_absmax + 4 * K].view(np.float32),
+        "outlier_idx": b[v.outlier_idx: v.outlier_idx + 4 * cap].view(np.int32),
+        "n_outliers": int(b[v.n_outliers: v.n_outliers + 4].view(np.int32)[0]),
+        "s_x": b[v.s_x: v.s_x + 4 * (M if p.gran == 1 else 1)].view(np.float32),
+        "body_q": b[v.body_q: v.body_q + M * v.ld_body_q].view(np.int8).reshape(M, v.ld_body_q)[:, :K],
+        "aux_q": b[v.aux_q: v.aux_q + M * v.aux_cols].view(np.int8).reshape(M, v.aux_cols),
+        "w_aux": b[v.w_aux: v.w_aux + N * v.aux_cols].view(np.int8).reshape(N, v.aux_cols),
+    }
+    return out
+
+
+# ------------------------------------------------------------------ K1
+@pytest.mark.parametrize("M,K", [(128, 768), (1, 1280), (333, 1040), (4096, 3072), (37, 16)])
+def test_detect_matches_oracle(mx, M, K):
+    x, _, ch = make_case(10 + M, M, K, 8, n_out=min(5, K // 4))
+    x[0, 0] = 6.0  # exactly the threshold somewhere: must not flag by itself
+    cap = 64
+    ws = mx.Workspace(mx.muxq_small_workspace_bytes(K))
+    ws.buf.fill_(0x5A)
+    cm, idx, n = mx.muxq_detect_outliers(dev(x), 6.0, cap, ws)
+    cm_o = oracle.colmax(x)
+    O, r, _ = oracle.detect(cm_o, 6.0, cap)
+    assert np.array_equal(cm.cpu().numpy().view(np.uint32), cm_o.view(np.uint32))
+    assert int(n.item()) == r
+    assert np.array_equal(idx.cpu().numpy()[:min(r, cap)], O)
+
+
+def test_detect_pitched_input_and_capacity_overflow(mx):
+    M, K, ld = 64, 256, 320
+    x, _, _ = make_case(5, M, K, 8, n_out=12)
+    xp = torch.zeros(M, ld, dtype=torch.float16, device="cuda")
+    xp[:, :K] = dev(x)
+    xp[:, K:] = 1000.0  # padding beyond K must be ignored
+    ws = mx.Workspace(mx.muxq_small_workspace_bytes(K))
+    cm, idx, n = mx.muxq_detect_outliers(xp[:, :K], 6.0, 4, ws)
+    cm_o = oracle.colmax(x)
+    O, r, rc = oracle.detect(cm_o, 6.0, 4)
+    assert rc == oracle.ERR_CAPACITY and r >= 12
+    assert int(n.item()) == r and np.array_equal(idx.cpu().numpy(), O)
+    assert np.array_equal(cm.cpu().numpy(), cm_o)
+
+
+# ------------------------------------------------------------------ Eq. 4-5 in the real domain
+def test_build_aux_reconstructs_x(mx):
+    x, _, _ = make_case(6, 200, 512, 8, n_out=6, mult=70.0)
+    ws = mx.Workspace(mx.muxq_small_workspace_bytes(512))
+    xd = dev(x)
+    cm, idx, n = mx.muxq_detect_outliers(xd, 6.0, 16, ws)
+    for e in (1, 2, 3):
+        aux, body = mx.muxq_build_aux(xd, idx, n, e)
+        O, r, _ = oracle.detect(oracle.colmax(x), 6.0, 16)
+        body_o, aux_o = oracle.decompose(x, O, e)
+        assert np.array_equal(body.cpu().numpy(), body_o)
+        a = aux.cpu().numpy()
+        assert np.array_equal(a[:, :r], aux_o) and not a[:, r:].any()
+        recon = body_o.copy()
+        recon[:, O] = body.cpu().numpy()[:, O] + np.float32(2 ** e - 1) * a[:, :r]   # Eq. 6
+        assert np.array_equal(recon, x.astype(np.float32))
+
+
+# ------------------------------------------------------------------ K5 / K2
+@pytest.mark.parametrize("gran", [0, 1])
+@pytest.mark.parametrize("K,N,bits", [(768, 768, 8), (1040, 200, 8), (512, 264, 5)])
+def test_weight_quantization_matches_oracle(mx, gran, K, N, bits):
+    w = synth.make_w(7, K * 3 + N, K, N)
+    p = mx.MuxqParams(gran=gran, w_bits=bits)
+    ws = mx.Workspace(mx.muxq_small_workspace_bytes(N))
+    ws.buf.fill_(0x33)
+    w_q, s_w = mx.muxq_quantize(dev(w), p, True, ws)
+    wq_o, sw_o = oracle.quantize_weight(w, bits=bits, per_channel=bool(gran))
+    assert np.array_equal(s_w.cpu().numpy().view(np.uint32), sw_o.view(np.uint32))
+    assert np.array_equal(w_q.cpu().numpy(), wq_o.T)
+
+
+@pytest.mark.parametrize("gran", [0, 1])
+@pytest.mark.parametrize("M,K,e,bits", [(128, 768, 2, 8), (77, 1040, 2, 8), (300, 512, 3, 6), (64, 256, 1, 8)])
+def test_activation_quantization_matches_oracle(mx, gran, M, K, e, bits):
+    x, _, _ = make_case(20 + M, M, K, 8, n_out=5, mult=60.0)
+    x[3] = 0  # an all-zero token row (per-token scale must become 1)
+    p = mx.MuxqParams(gran=gran, exp_factor=e, act_bits=bits, max_outliers=16)
+    ws = mx.Workspace(mx.muxq_small_workspace_bytes(K))
+    xd = dev(x)
+    cm, idx, n = mx.muxq_detect_outliers(xd, p.threshold, p.max_outliers, ws)
+    body_q, aux_q, s_x = mx.muxq_quantize(xd, p, False, ws, cm, idx, n)
+    O, r, _ = oracle.detect(oracle.colmax(x), 6.0, 16)
+    body, aux = oracle.decompose(x, O, e)
+    sx_o, sa_o, bq_o, aq_o = oracle.quantize_act(body, aux, bits, bool(gran), False)
+    assert np.array_equal(s_x.cpu().numpy().view(np.uint32), sx_o.view(np.uint32))
+    assert np.array_equal(body_q.cpu().numpy(), bq_o)
+    c = 2 ** e - 1
+    a = aux_q.cpu().numpy()
+    assert a.shape[1] == mx.muxq_aux_cols(p)
+    for j in range(r):
+        for t in range(c):
+            assert np.array_equal(a[:, c * j + t], aq_o[:, j])
+    assert not a[:, c * r:].any()
+    # naive quantization (no outlier handling): Eq. 1 alone
+    nq, _, ns = mx.muxq_quantize(xd, p, False, ws, cm, None, None, want_aux=False)
+    sx_n, _, bq_n, _ = oracle.quantize_act(x.astype(np.float32), np.zeros((M, 0), np.float32), bits, bool(gran), False)
+    assert np.array_equal(ns.cpu().numpy(), sx_n) and np.array_equal(nq.cpu().numpy(), bq_n)
+
+
+# ------------------------------------------------------------------ K3 alone
+@pytest.mark.parametrize("M,K,N", [(128, 128, 128), (128, 256, 256), (256, 768, 768), (300, 1040, 520),
+                                   (1000, 512, 1288), (128, 32, 64), (129, 4096, 264)])
+def test_gemm_accumulators_bit_exact(mx, M, K, N):
+    rng = np.random.default_rng(M * 7 + K + N)
+    a = rng.integers(-127, 128, (M, K), dtype=np.int8)
+    b = rng.integers(-127, 128, (N, K), dtype=np.int8)
+    p = mx.MuxqParams()
+    ws = mx.Workspace(256)
+    acc = mx.muxq_gemm(dev(a), None, dev(b), None, None, p, None, None, mx.MUXQ_OUT_ACC_I32, ws)
+    assert mx.muxq_read_status(ws) == 0
+    ref = a.astype(np.int32) @ b.astype(np.int32).T
+    assert np.array_equal(acc.cpu().numpy(), ref)
+
+
+def test_gemm_worst_case_magnitudes(mx):
+    M, K, N = 128, 5120, 256
+    a = np.full((M, K), 127, np.int8)
+    b = np.full((N, K), -127, np.int8)
+    b[::2] = 127
+    acc = mx.muxq_gemm(dev(a), None, dev(b), None, None, mx.MuxqParams(), None, None, 2, mx.Workspace(256))
+    ref = a.astype(np.int32) @ b.astype(np.int32).T
+    assert np.array_equal(acc.cpu().numpy(), ref)
+
+
+# ------------------------------------------------------------------ whole layer
+@pytest.mark.parametrize("gran", [0, 1])
+@pytest.mark.parametrize("M,K,N,n_out", [(128, 768, 768, 4), (300, 1040, 520, 7), (512, 256, 1288, 0),
+                                         (1024, 1280, 1280, 21)])
+def test_linear_matches_oracle(mx, gran, M, K, N, n_out):
+    x, w, ch = make_case(40 + M, M, K, N, n_out=n_out, mult=50.0)
+    p = mx.MuxqParams(gran=gran, max_outliers=32)
+    wq_o, sw_o, res = oracle_linear(x, w, p)
+    assert res.r >= n_out
+    # raw accumulators
+    acc, ws, st, w_q, s_w = run_linear(mx, x, w, p, mx.MUXQ_OUT_ACC_I32)
+    assert st == 0
+    v = ws_views(mx, ws, M, K, N, p)
+    assert v["n_outliers"] == res.r and np.array_equal(v["outlier_idx"][:res.r], res.O)
+    assert np.array_equal(v["col_absmax"].view(np.uint32), res.colmax.view(np.uint32))
+    assert np.array_equal(v["s_x"].view(np.uint32), res.s_x.view(np.uint32))
+    assert np.array_equal(v["body_q"], res.body_q)
+    assert np.array_equal(w_q.cpu().numpy(), wq_o.T)
+    c = 3
+    for j in range(res.r):
+        assert np.array_equal(v["w_aux"][:, c * j], wq_o[res.O[j]])
+        assert np.array_equal(v["aux_q"][:, c * j + 2], res.aux_q[:, j])
+    assert np.array_equal(acc.cpu().numpy(), res.acc)
+    # fp32 and fp16 outputs
+    y32, _, st, _, _ = run_linear(mx, x, w, p, mx.MUXQ_OUT_F32)
+    assert st == 0 and rel_err32(y32.cpu().numpy(), res.y32) <= 1e-5
+    assert np.array_equal(y32.cpu().numpy(), res.y32)  # same operands, same two roundings
+    y16, _, st, _, _ = run_linear(mx, x, w, p, mx.MUXQ_OUT_F16)
+    assert st == 0 and f16_ulp_diff(y16.cpu().numpy(), res.y16).max() <= 1
+
+
+def test_handworked_example_on_gpu(mx):
+    from conftest import load_golden
+    g = load_golden("handworked_exp2.txt")
+    K, N = 16, 8  # the 2x4 / 4x2 example embedded in zero padding
+    x = np.zeros((2, K), np.float16); x[:, :4] = g["X"]
+    w = np.zeros((K, N), np.float16); w[:4, :2] = g["W"]
+    p = mx.MuxqParams(max_outliers=4)
+    # decode path (M = 2)
+    y, ws, st, w_q, s_w = run_linear(mx, x, w, p, mx.MUXQ_OUT_F32)
+    assert st == 0 and np.array_equal(y.cpu().numpy()[:, :2].astype(np.float64), g["Y"])
+    # tensor-core path: repeat the two rows to M = 32
+    xx = np.tile(x, (16, 1))
+    acc, ws, st, _, _ = run_linear(mx, xx, w, p, mx.MUXQ_OUT_ACC_I32)
+    assert st == 0 and np.array_equal(acc.cpu().numpy()[:2, :2], g["acc"].astype(np.int32))
+    y16, _, _, _, _ = run_linear(mx, xx, w, p, mx.MUXQ_OUT_F16)
+    assert np.array_equal(y16.cpu().numpy()[:2, :2].astype(np.float64), g["Y16"])
+
+
+@pytest.mark.parametrize("M", [1, 2, 4, 7, 16])
+@pytest.mark.parametrize("K,N", [(1280, 1280), (1280, 3840), (5120, 1280), (256, 72)])
+def test_decode_matches_oracle(mx, M, K, N):
+    x, w, _ = make_case(60 + M + K, M, K, N, n_out=8, mult=60.0)
+    for gran in (0, 1):
+        p = mx.MuxqParams(gran=gran, max_outliers=32)
+        _, _, res = oracle_linear(x, w, p)
+        acc, ws, st, _, _ = run_linear(mx, x, w, p, mx.MUXQ_OUT_ACC_I32)
+        assert st == 0 and np.array_equal(acc.cpu().numpy(), res.acc)
+        y32, _, _, _, _ = run_linear(mx, x, w, p, mx.MUXQ_OUT_F32)
+        assert np.array_equal(y32.cpu().numpy(), res.y32)
+        y16, _, _, _, _ = run_linear(mx, x, w, p, mx.MUXQ_OUT_F16)
+        assert f16_ulp_diff(y16.cpu().numpy(), res.y16).max() <= 1
+
+
+# ------------------------------------------------------------------ edge cases
+def test_zero_outliers_equals_naive_int8(mx):
+    x, w, _ = make_case(70, 256, 512, 256, n_out=0)
+    p = mx.MuxqParams(threshold=1e4)
+    _, _, res = oracle_linear(x, w, p)
+    assert res.r == 0
+    acc, ws, st, _, _ = run_linear(mx, x, w, p, mx.MUXQ_OUT_ACC_I32)
+    assert st == 0 and np.array_equal(acc.cpu().numpy(), res.acc)
+
+
+def test_capacity_overflow_sets_status_and_stays_in_bounds(mx):
+    M, K, N = 256, 512, 256
+    x, w, _ = make_case(71, M, K, N, n_out=12)
+    p = mx.MuxqParams(max_outliers=4)
+    wsw = mx.Workspace(mx.muxq_small_workspace_bytes(N))
+    w_q, s_w = mx.muxq_quantize(dev(w), p, True, wsw)
+    nbytes = mx.muxq_workspace_bytes(M, K, N, p)
+    ws = mx.Workspace(nbytes + 4096)
+    ws.buf.fill_(0x77)  # canary behind the workspace proper
+    ybuf = torch.full((M + 2, N), 1234.0, dtype=torch.float16, device="cuda")
+    ws_use = mx.Workspace(0)
+    ws_use.buf = ws.buf[:nbytes]
+    y = mx.muxq_linear(dev(x), w_q, s_w, p, ws_use, mx.MUXQ_OUT_F16, out=ybuf[1:M + 1])
+    assert mx.muxq_read_status(ws_use) == mx.MUXQ_ERR_CAPACITY
+    assert (ws.buf[nbytes:] == 0x77).all()
+    assert (ybuf[0] == 1234.0).all() and (ybuf[M + 1] == 1234.0).all()
+    v = ws_views(mx, ws_use, M, K, N, p)
+    O, r, _ = oracle.detect(oracle.colmax(x), 6.0, 4)
+    assert v["n_outliers"] == r and np.array_equal(v["outlier_idx"][:4], O)
+
+
+def test_all_zero_activations(mx):
+    x = np.zeros((128, 256), np.float16)
+    w = synth.make_w(1, 1, 256, 128)
+    for gran in (0, 1):
+        y, ws, st, _, _ = run_linear(mx, x, w, mx.MuxqParams(gran=gran), mx.MUXQ_OUT_F32)
+        assert st == 0 and not y.cpu().numpy().any()
+
+
+def test_argument_errors(mx):
+    p = mx.MuxqParams()
+    ws = mx.Workspace(1 << 20)
+    x = torch.zeros(32, 24, dtype=torch.float16, device="cuda")   # K % 16 != 0
+    w_q = torch.zeros(64, 24, dtype=torch.int8, device="cuda")
+    s_w = torch.ones(1, device="cuda")
+    with pytest.raises(mx.MuxqError) as ei:
+        mx.muxq_linear(x, w_q, s_w, p, ws)
+    assert ei.value.status == mx.MUXQ_ERR_UNSUPPORTED
+    x = torch.zeros(32, 32, dtype=torch.float16, device="cuda")
+    w_q = torch.zeros(64, 32, dtype=torch.int8, device="cuda")
+    small = mx.Workspace(256)
+    with pytest.raises(mx.MuxqError) as ei:
+        mx.muxq_linear(x, w_q, s_w, p, small)
+    assert ei.value.status == mx.MUXQ_ERR_WORKSPACE
+    with pytest.raises(mx.MuxqError) as ei:
+        mx.muxq_linear(x, w_q, s_w, mx.MuxqParams(exp_factor=5), ws)
+    assert ei.value.status == mx.MUXQ_ERR_INVALID_ARG
+    with pytest.raises(mx.MuxqError) as ei:
+        mx.muxq_linear(x, w_q, s_w, mx.MuxqParams(aux_scale=1), ws)
+    assert ei.value.status == mx.MUXQ_ERR_UNSUPPORTED
+
+
+def test_host_buffer_entry_point(mx):
+    M, K, N = 256, 512, 264
+    x, w, _ = make_case(80, M, K, N, n_out=3)
+    p = mx.MuxqParams()
+    wsw = mx.Workspace(mx.muxq_small_workspace_bytes(N))
+    w_q, s_w = mx.muxq_quantize(dev(w), p, True, wsw)
+    ws = mx.Workspace(mx.muxq_host_workspace_bytes(M, K, N, p, mx.MUXQ_OUT_F16))
+    xh = torch.from_numpy(x).pin_memory()
+    yh = torch.empty(M, N, dtype=torch.float16).pin_memory()
+    mx.muxq_linear_host(xh, w_q, s_w, p, ws, yh, mx.MUXQ_OUT_F16)
+    assert mx.muxq_read_status(ws) == 0
+    _, _, res = oracle_linear(x, w, p)
+    assert f16_ulp_diff(yh.numpy(), res.y16).max() <= 1
