@@ -1,0 +1,322 @@
+#!/usr/bin/env python
+"""Benchmark of the MUXQ linear hot path on B200.
+
+A "step" is one pass of the whole hot path -- outlier detection, redistribute + quantize, INT8
+tensor-core GEMM with the Aux correction and dequantization -- over the four GPT-2-small-shaped
+linears (768->2304, 768->768, 768->3072, 3072->768) at M = 8192 tokens, per-tensor INT8, on seeded
+synthetic activations with 6 outlier channels.  Weights are quantized once before timing.
+
+    python bench.py --gpus 1 --steps K --warmup W          # the CUDA library (one JSON line)
+    python bench.py --impl reference ...                    # the CPU oracle on a bounded sample
+
+Metric: effective INT8 TOPS = sum over layers of 2*M*N*K / time (Aux ops are not credited).
+Multi-GPU: the path does not shard (one GPU per problem); N ranks run N independent replicas.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import muxq_synth as synth  # noqa: E402
+
+METRIC = "muxq_linear_effective_int8_tops_prefill"
+UNIT = "TOPS"
+CONFIG_ID = 1
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return {"hbm_gbs": d["hbm_gbs"], "bf16_burst": d["bf16_tflops"],
+                "bf16_sustained": d.get("bf16_tflops_sustained", d["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_burst": 1590.0, "bf16_sustained": 1400.0, "source": "fallback"}
+
+
+def workload(M=None):
+    specs = synth.config_layers(CONFIG_ID, M=M)
+    ops = sum(2.0 * s.M * s.N * s.K for s in specs)
+    return specs, ops
+
+
+def config_dict(specs, extra=None):
+    d = {"workload": "configs[1]: GPT-2-small linear set (768->2304, 768->768, 768->3072, 3072->768), "
+                     f"M={specs[0].M} tokens, 6 outlier channels x40-80, per-tensor INT8, fp16 in/out",
+         "layers_per_step": len(specs), "granularity": "per-tensor",
+         "l2": "no explicit flush: one step streams ~250 MB (X 88 MB, codes 50 MB, Y 113 MB) > 126 MB L2"}
+    if extra:
+        d.update(extra)
+    return d
+
+
+# --------------------------------------------------------------------------- clocks
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, uuid):
+        self.uuid = uuid
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", self.uuid], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, mx, pw = [], [], []
+        reasons = set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in out.strip().splitlines():
+            parts = [p.strip() for p in ln.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0])); mx.append(float(parts[1])); pw.append(float(parts[2]))
+            except ValueError:
+                continue
+            for nm, v in zip(names, parts[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(nm)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "power_w_max": max(pw),
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# --------------------------------------------------------------------------- CPU oracle leg
+def oracle_sample(specs, rows_per_layer):
+    """Times the oracle (as it stands) on the first `rows_per_layer` token rows of every layer."""
+    import oracle
+    oracle.build()
+    prepared = []
+    for s in specs:
+        x, _ = synth.make_x(s.seed, s.tensor_id, rows_per_layer, s.K, s.n_outliers, s.mult_lo, s.mult_hi,
+                            s.bulk, s.bulk_scale)
+        wq, sw = oracle.quantize_weight(s.w())
+        prepared.append((x, wq, sw, s))
+    t0 = time.perf_counter()
+    for x, wq, sw, s in prepared:
+        oracle.linear(x, wq, sw, want_codes=False)
+    dt = time.perf_counter() - t0
+    ops = sum(2.0 * rows_per_layer * s.N * s.K for s in specs)
+    return ops / dt / 1e12, dt, oracle.num_threads()
+
+
+def run_reference(args, rank):
+    if rank != 0:
+        return
+    specs, _ = workload()
+    rows = 2048
+    vals = []
+    oracle_sample(specs, rows)  # one untimed pass
+    t_all = 0.0
+    steps = max(1, min(args.steps, 5))
+    for _ in range(steps):
+        v, dt, cores = oracle_sample(specs, rows)
+        vals.append(v); t_all += dt
+    value = statistics.mean(vals)
+    sample = f"first {rows} of {specs[0].M} token rows of each of the 4 layers per step, {steps} steps"
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": steps, "warmup": 1, "ms_per_step": 1e3 * t_all / steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "int8", "data": "synthetic",
+            "config": config_dict(specs),
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+# --------------------------------------------------------------------------- CUDA arm
+def run_muxq(args, rank, world):
+    import torch
+    import torch.distributed as dist
+
+    import paper_2604_04701_b200 as mx
+
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    mx.lib()  # fails loudly if the CUDA library is missing
+
+    specs, ops_per_step = workload()
+    p = mx.MuxqParams(max_outliers=32)
+    layers = []
+    for s in specs:
+        x, _ = s.x()
+        w = s.w()
+        xd = torch.from_numpy(x).to(dev)
+        w_q, s_w = mx.muxq_quantize(torch.from_numpy(w).to(dev), p, True,
+                                    mx.Workspace(mx.muxq_small_workspace_bytes(s.N), dev))
+        ws = mx.Workspace(mx.muxq_host_workspace_bytes(s.M, s.K, s.N, p, mx.MUXQ_OUT_F16), dev)
+        y = torch.empty(s.M, s.N, dtype=torch.float16, device=dev)
+        layers.append({"spec": s, "x": xd, "w_q": w_q, "s_w": s_w, "ws": ws, "y": y, "x_host": x})
+    torch.cuda.synchronize()
+
+    def step():
+        for L in layers:
+            mx.muxq_linear(L["x"], L["w_q"], L["s_w"], p, L["ws"], mx.MUXQ_OUT_F16, out=L["y"])
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+    for L in layers:
+        st = mx.muxq_read_status(L["ws"])
+        if st != 0:
+            raise RuntimeError(f"device status {st} ({mx.muxq_status_string(st)}) on {L['spec'].name}")
+
+    uuid = str(torch.cuda.get_device_properties(dev).uuid)
+    sampler = ClockSampler(uuid if uuid.startswith("GPU-") else "GPU-" + uuid)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier(); torch.cuda.synchronize()
+    sampler.start()
+    e0.record()
+    for _ in range(args.steps):
+        step()
+    e1.record()
+    torch.cuda.synchronize(); barrier()
+    clocks = sampler.stop()
+    ms = e0.elapsed_time(e1)
+    if world > 1:
+        t = torch.tensor([ms], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    ms_per_step = ms / args.steps
+    value = world * ops_per_step / (ms_per_step * 1e-3) / 1e12
+
+    # ---- per-kernel durations (CUDA events at the kernel boundaries, same stream, same buffers)
+    ksteps = min(args.steps, 100)
+    evs = [[[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in layers] for _ in range(ksteps)]
+    for per_step in evs:
+        for per_layer in per_step:
+            for e in per_layer:
+                e.record()  # creates the CUDA handle
+    torch.cuda.synchronize()
+    for i in range(ksteps):
+        for li, L in enumerate(layers):
+            mx.muxq_linear_events(L["x"], L["w_q"], L["s_w"], p, L["ws"], evs[i][li], mx.MUXQ_OUT_F16, out=L["y"])
+    torch.cuda.synchronize()
+    kern_us = {"detect": [], "quantize": [], "gemm": []}
+    per_layer_gemm_us = []
+    for li, L in enumerate(layers):
+        d = [[evs[i][li][j].elapsed_time(evs[i][li][j + 1]) * 1e3 for i in range(ksteps)] for j in range(3)]
+        kern_us["detect"].append(statistics.mean(d[0]))
+        kern_us["quantize"].append(statistics.mean(d[1]))
+        kern_us["gemm"].append(statistics.mean(d[2]))
+        per_layer_gemm_us.append(statistics.mean(d[2]))
+    gemm_us_per_step = sum(kern_us["gemm"])
+    peaks = load_peaks()
+    int8_peak = 2.0 * peaks["bf16_sustained"]  # INT8 dense rate = 2 x bf16 (nominal 4.5 vs 2.25 POPS)
+    achieved = ops_per_step / (gemm_us_per_step * 1e-6) / 1e12
+    roofline = {"kernel": "k_gemm_i8 (tcgen05 kind::i8, fused Aux + dequant epilogue)", "bound": "tensor",
+                "achieved": achieved, "peak": int8_peak, "unit": "TOPS", "frac": achieved / int8_peak,
+                "peak_source": f"2 x bf16_tflops_sustained of {peaks['source']}",
+                "traffic": None,
+                "per_layer": [{"layer": L["spec"].name, "M": L["spec"].M, "K": L["spec"].K, "N": L["spec"].N,
+                               "gemm_us": per_layer_gemm_us[i], "detect_us": kern_us["detect"][i],
+                               "quantize_us": kern_us["quantize"][i],
+                               "gemm_tops": 2.0 * L["spec"].M * L["spec"].N * L["spec"].K /
+                               (per_layer_gemm_us[i] * 1e-6) / 1e12} for i, L in enumerate(layers)],
+                "share_of_step": {k: sum(v) / (sum(kern_us["detect"]) + sum(kern_us["quantize"]) + gemm_us_per_step)
+                                  for k, v in kern_us.items()}}
+
+    # ---- end to end: host buffers, copies inside the timed region
+    esteps = max(3, min(args.steps, 20))
+    hosts = []
+    for L in layers:
+        xh = torch.from_numpy(L["x_host"]).pin_memory()
+        yh = torch.empty(L["spec"].M, L["spec"].N, dtype=torch.float16).pin_memory()
+        hosts.append((xh, yh))
+
+    def step_host():
+        for L, (xh, yh) in zip(layers, hosts):
+            mx.muxq_linear_host(xh, L["w_q"], L["s_w"], p, L["ws"], yh, mx.MUXQ_OUT_F16)
+
+    for _ in range(2):
+        step_host()
+    torch.cuda.synchronize(); barrier()
+    h0, h1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    h0.record()
+    for _ in range(esteps):
+        step_host()
+    h1.record()
+    torch.cuda.synchronize(); barrier()
+    ems = h0.elapsed_time(h1)
+    if world > 1:
+        t = torch.tensor([ems], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ems = float(t.item())
+    e2e = {"value": world * ops_per_step / (ems / esteps * 1e-3) / 1e12, "unit": UNIT,
+           "h2d_bytes_per_step": int(sum(xh.numel() * 2 for xh, _ in hosts)),
+           "d2h_bytes_per_step": int(sum(yh.numel() * 2 for _, yh in hosts)), "steps": esteps,
+           "ms_per_step": ems / esteps}
+
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        rows = specs[0].M
+        v, dt, cores = oracle_sample(specs, rows)
+        cpu_baseline = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "seconds": dt,
+                        "sample": f"all {rows} token rows of each of the 4 layers, one pass (one step)"}
+
+    if rank == 0:
+        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
+                "scaling": "weak", "vs_baseline": None, "dtype": "int8", "data": "synthetic",
+                "config": config_dict(specs, {"parallelism": "replicas only" if world > 1 else "single GPU"}),
+                "us_per_layer": ms_per_step * 1e3 / len(layers),
+                "pct_of_nominal_int8_peak_4500": 100.0 * value / world / 4500.0,
+                "clocks": clocks, "e2e": e2e, "gpu_launches": args.steps * len(layers) * 3,
+                "roofline": roofline, "cpu_baseline": cpu_baseline}
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5000)
+    ap.add_argument("--warmup", type=int, default=50)
+    ap.add_argument("--impl", default="muxq", choices=["muxq", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if args.impl == "reference":
+        run_reference(args, rank)
+    else:
+        run_muxq(args, rank, world)
+
+
+if __name__ == "__main__":
+    main()

@@ -154,6 +154,17 @@ int muxq_linear(const void *X_f16, int M, int K, int ldx, const int8_t *W_q, int
                 const float *s_w, int N, const muxq_params *p, void *Y, int ldy, int out_kind,
                 void *workspace, size_t workspace_bytes, int32_t *dev_status, void *stream);
 
+/*
+ * muxq_linear that also records four caller-created CUDA events (cudaEvent_t passed as void*;
+ * NULL entries are skipped) on `stream` at its kernel boundaries, for per-kernel timing:
+ * events[0] before detection, [1] after detection, [2] after redistribute-and-quantize,
+ * [3] after the GEMM (or decode) kernel.  Same results as muxq_linear.
+ */
+int muxq_linear_events(const void *X_f16, int M, int K, int ldx, const int8_t *W_q, int ldw,
+                       const float *s_w, int N, const muxq_params *p, void *Y, int ldy, int out_kind,
+                       void *workspace, size_t workspace_bytes, int32_t *dev_status, void *stream,
+                       void *const *events);
+
 /* Where muxq_linear leaves its intermediates inside the workspace (byte offsets). */
 typedef struct muxq_ws_view {
     size_t col_absmax;  /* float [K] */
@@ -177,6 +188,17 @@ int muxq_workspace_view(int M, int K, int N, const muxq_params *p, muxq_ws_view 
 int muxq_linear_host(const void *X_f16_host, int M, int K, const int8_t *W_q, int ldw,
                      const float *s_w, int N, const muxq_params *p, void *Y_host, int out_kind,
                      void *workspace, size_t workspace_bytes, int32_t *dev_status, void *stream);
+
+/*
+ * Measurement aid: runs `ctas` CTAs (one per SM when ctas = SM count) that each issue `iters`
+ * back-to-back tcgen05.mma kind::i8 instructions of shape M128 x N(mma_n = 128 or 256) x K32 on
+ * operands resident in shared memory -- the issue-bound INT8 tensor rate of the GPU as it is clocked
+ * right now.  cycles_per_cta [ctas] (device, uint64) receives each CTA's SM-clock cycle count from
+ * first issue to completion; time the launch with CUDA events for ops/s =
+ * ctas * iters * 2 * 128 * mma_n * 32 / seconds.
+ */
+int muxq_int8_mma_peak(int mma_n, int iters, int ctas, unsigned long long *cycles_per_cta,
+                       int32_t *dev_status, void *stream);
 
 /* Synchronizes `stream` and returns the device status word (or MUXQ_ERR_CUDA). */
 int muxq_read_status(const int32_t *dev_status, void *stream);

@@ -21,7 +21,7 @@ MUXQ_OUT_F16, MUXQ_OUT_F32, MUXQ_OUT_ACC_I32 = 0, 1, 2
 EXPORTS = (
     "muxq_default_params", "muxq_aux_cols", "muxq_workspace_bytes", "muxq_small_workspace_bytes",
     "muxq_host_workspace_bytes", "muxq_workspace_view", "muxq_detect_outliers", "muxq_build_aux",
-    "muxq_quantize", "muxq_gemm", "muxq_linear", "muxq_linear_host", "muxq_read_status",
+    "muxq_quantize", "muxq_gemm", "muxq_linear", "muxq_linear_events", "muxq_linear_host", "muxq_int8_mma_peak", "muxq_read_status",
     "muxq_status_string",
 )
 
@@ -89,7 +89,9 @@ def lib() -> ctypes.CDLL:
         L.muxq_quantize.argtypes = [vp, i, i, i, pp, i, vp, vp, vp, vp, i, vp, i, vp, vp, sz, vp]; L.muxq_quantize.restype = i
         L.muxq_gemm.argtypes = [vp, i, vp, i, vp, i, vp, i, vp, i, i, i, pp, vp, vp, vp, i, i, vp, vp]; L.muxq_gemm.restype = i
         L.muxq_linear.argtypes = [vp, i, i, i, vp, i, vp, i, pp, vp, i, i, vp, sz, vp, vp]; L.muxq_linear.restype = i
+        L.muxq_linear_events.argtypes = [vp, i, i, i, vp, i, vp, i, pp, vp, i, i, vp, sz, vp, vp, vp]; L.muxq_linear_events.restype = i
         L.muxq_linear_host.argtypes = [vp, i, i, vp, i, vp, i, pp, vp, i, vp, sz, vp, vp]; L.muxq_linear_host.restype = i
+        L.muxq_int8_mma_peak.argtypes = [i, i, i, vp, vp, vp]; L.muxq_int8_mma_peak.restype = i
         L.muxq_read_status.argtypes = [vp, vp]; L.muxq_read_status.restype = i
         L.muxq_status_string.argtypes = [i]; L.muxq_status_string.restype = ctypes.c_char_p
         _lib = L
@@ -234,6 +236,21 @@ def muxq_linear(X: torch.Tensor, w_q: torch.Tensor, s_w: torch.Tensor, p: MuxqPa
     return Y
 
 
+def muxq_linear_events(X: torch.Tensor, w_q: torch.Tensor, s_w: torch.Tensor, p: MuxqParams, ws: Workspace,
+                       events, out_kind: int = MUXQ_OUT_F16, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """muxq_linear recording four torch.cuda.Event objects (created with enable_timing=True and already
+    recorded once, so that their CUDA handles exist) at the kernel boundaries."""
+    M, K = X.shape
+    N = w_q.shape[0]
+    Y = out if out is not None else _alloc_out(M, N, out_kind, X.device)
+    arr = (ctypes.c_void_p * 4)(*[ctypes.c_void_p(e.cuda_event) for e in events])
+    _check("muxq_linear_events",
+           lib().muxq_linear_events(_ptr(X), M, K, X.stride(0), _ptr(w_q), w_q.stride(0), _ptr(s_w), N,
+                                    ctypes.byref(p.c()), _ptr(Y), Y.stride(0), out_kind, _ptr(ws.buf), ws.nbytes,
+                                    _ptr(ws.status), _stream(), arr))
+    return Y
+
+
 def muxq_linear_host(X_host: torch.Tensor, w_q: torch.Tensor, s_w: torch.Tensor, p: MuxqParams, ws: Workspace,
                      Y_host: torch.Tensor, out_kind: int = MUXQ_OUT_F16) -> torch.Tensor:
     """X_host / Y_host are CPU tensors (pinned for asynchronous copies); everything else on device."""
@@ -244,6 +261,13 @@ def muxq_linear_host(X_host: torch.Tensor, w_q: torch.Tensor, s_w: torch.Tensor,
            lib().muxq_linear_host(_ptr(X_host), M, K, _ptr(w_q), w_q.stride(0), _ptr(s_w), N, ctypes.byref(p.c()),
                                   _ptr(Y_host), out_kind, _ptr(ws.buf), ws.nbytes, _ptr(ws.status), _stream()))
     return Y_host
+
+
+def muxq_int8_mma_peak(mma_n: int, iters: int, ctas: int, ws: Workspace) -> torch.Tensor:
+    """Enqueues the issue-bound INT8 MMA loop; returns the per-CTA cycle counts (device uint64 as int64)."""
+    cycles = torch.zeros(ctas, dtype=torch.int64, device=ws.buf.device)
+    _check("muxq_int8_mma_peak", lib().muxq_int8_mma_peak(mma_n, iters, ctas, _ptr(cycles), _ptr(ws.status), _stream()))
+    return cycles
 
 
 def muxq_read_status(ws: Workspace) -> int:

@@ -61,7 +61,11 @@ int cuda_rc(cudaError_t e) { return e == cudaSuccess ? MUXQ_OK : MUXQ_ERR_CUDA; 
 
 }  // namespace
 
+namespace muxq { extern int g_peak_mode; void set_gemm_dbg(int v); void set_gemm_tl(long long *p); }
 extern "C" {
+void muxq_debug_set(int v) { muxq::set_gemm_dbg(v); }
+void muxq_debug_tl(long long *p) { muxq::set_gemm_tl(p); }
+void muxq_debug_peak_mode(int m) { muxq::g_peak_mode = m; }
 
 void muxq_default_params(muxq_params *p) {
     if (!p) return;
@@ -211,6 +215,7 @@ int muxq_quantize(const void *A, int rows, int cols, int ld, const muxq_params *
     q.n_outliers = &d.ctrl->n_outliers;
     q.colmul = d.colmul; q.grpflag = d.grpflag;
     q.s_x_tensor = &d.ctrl->s_x;
+    q.inv_s_x_tensor = &d.ctrl->inv_s_x;
     q.s_x_rows = scales;
     q.body_q = A_q; q.ld_q = ld_q;
     q.aux_q = Aux_q; q.ld_aux = ld_aux; q.aux_cols = aux_cols;
@@ -251,9 +256,9 @@ int muxq_gemm(const int8_t *Body_q, int ld_a, const int8_t *Aux_q, int ld_aux, c
     return cuda_rc(launch_gemm(g, static_cast<cudaStream_t>(stream)));
 }
 
-int muxq_linear(const void *X, int M, int K, int ldx, const int8_t *W_q, int ldw, const float *s_w, int N,
-                const muxq_params *p, void *Y, int ldy, int out_kind, void *workspace, size_t workspace_bytes,
-                int32_t *dev_status, void *stream) {
+static int linear_impl(const void *X, int M, int K, int ldx, const int8_t *W_q, int ldw, const float *s_w, int N,
+                       const muxq_params *p, void *Y, int ldy, int out_kind, void *workspace, size_t workspace_bytes,
+                       int32_t *dev_status, void *stream, void *const *events) {
     if (!X || !W_q || !s_w || !Y || !workspace || !dev_status || M <= 0 || K <= 0 || N <= 0 || ldx < K ||
         ldw < K || ldy < N || !params_ok(p) || out_kind < 0 || out_kind > 2)
         return MUXQ_ERR_INVALID_ARG;
@@ -274,6 +279,10 @@ int muxq_linear(const void *X, int M, int K, int ldx, const int8_t *W_q, int ldw
     const bool per_vec = p->gran == MUXQ_PER_VECTOR;
     const bool decode = M <= 16;
     Ctrl *ctrl = reinterpret_cast<Ctrl *>(ws);
+    auto mark = [&](int i) {
+        if (events && events[i]) cudaEventRecord(static_cast<cudaEvent_t>(events[i]), s);
+    };
+    mark(0);
 
     DetectArgs d{};
     d.X = static_cast<const __half *>(X);
@@ -287,6 +296,7 @@ int muxq_linear(const void *X, int M, int K, int ldx, const int8_t *W_q, int ldw
     d.dev_status = dev_status;
     e = launch_detect(d, s);
     if (e != cudaSuccess) return MUXQ_ERR_CUDA;
+    mark(1);
 
     QuantActArgs q{};
     q.X = d.X; q.M = M; q.K = K; q.ldx = ldx;
@@ -295,6 +305,7 @@ int muxq_linear(const void *X, int M, int K, int ldx, const int8_t *W_q, int ldw
     q.n_outliers = &ctrl->n_outliers;
     q.colmul = d.colmul; q.grpflag = d.grpflag;
     q.s_x_tensor = &ctrl->s_x;
+    q.inv_s_x_tensor = &ctrl->inv_s_x;
     q.s_x_rows = reinterpret_cast<float *>(ws + w.sx_rows);
     q.body_q = reinterpret_cast<int8_t *>(ws + w.body_q); q.ld_q = w.ld_q;
     if (!decode) {
@@ -304,6 +315,7 @@ int muxq_linear(const void *X, int M, int K, int ldx, const int8_t *W_q, int ldw
     }
     e = launch_quant_act(q, s);
     if (e != cudaSuccess) return MUXQ_ERR_CUDA;
+    mark(2);
 
     const float *s_x = per_vec ? q.s_x_rows : &ctrl->s_x;
     const int c = (1 << p->exp_factor) - 1;
@@ -316,7 +328,9 @@ int muxq_linear(const void *X, int M, int K, int ldx, const int8_t *W_q, int ldw
         k.s_x = s_x; k.s_x_per_row = per_vec;
         k.s_w = s_w; k.s_w_per_col = per_vec;
         k.Y = Y; k.ldy = ldy; k.out_kind = out_kind;
-        return cuda_rc(launch_decode(k, s));
+        e = launch_decode(k, s);
+        mark(3);
+        return cuda_rc(e);
     }
     GemmArgs g{};
     g.body_q = q.body_q; g.ld_a = w.ld_q;
@@ -329,7 +343,24 @@ int muxq_linear(const void *X, int M, int K, int ldx, const int8_t *W_q, int ldw
     g.s_w = s_w; g.s_w_per_col = per_vec;
     g.Y = Y; g.ldy = ldy; g.out_kind = out_kind;
     g.dev_status = dev_status;
-    return cuda_rc(launch_gemm(g, s));
+    e = launch_gemm(g, s);
+    mark(3);
+    return cuda_rc(e);
+}
+
+int muxq_linear(const void *X, int M, int K, int ldx, const int8_t *W_q, int ldw, const float *s_w, int N,
+                const muxq_params *p, void *Y, int ldy, int out_kind, void *workspace, size_t workspace_bytes,
+                int32_t *dev_status, void *stream) {
+    return linear_impl(X, M, K, ldx, W_q, ldw, s_w, N, p, Y, ldy, out_kind, workspace, workspace_bytes, dev_status,
+                       stream, nullptr);
+}
+
+int muxq_linear_events(const void *X, int M, int K, int ldx, const int8_t *W_q, int ldw, const float *s_w, int N,
+                       const muxq_params *p, void *Y, int ldy, int out_kind, void *workspace,
+                       size_t workspace_bytes, int32_t *dev_status, void *stream, void *const *events) {
+    if (!events) return MUXQ_ERR_INVALID_ARG;
+    return linear_impl(X, M, K, ldx, W_q, ldw, s_w, N, p, Y, ldy, out_kind, workspace, workspace_bytes, dev_status,
+                       stream, events);
 }
 
 int muxq_linear_host(const void *X_host, int M, int K, const int8_t *W_q, int ldw, const float *s_w, int N,
@@ -349,6 +380,13 @@ int muxq_linear_host(const void *X_host, int M, int K, const int8_t *W_q, int ld
     const int rc = muxq_linear(x_dev, M, K, K, W_q, ldw, s_w, N, p, y_dev, N, out_kind, ws, base, dev_status, stream);
     if (rc != MUXQ_OK) return rc;
     return cuda_rc(cudaMemcpyAsync(Y_host, y_dev, (size_t)M * N * out_elem_bytes(out_kind), cudaMemcpyDeviceToHost, s));
+}
+
+int muxq_int8_mma_peak(int mma_n, int iters, int ctas, unsigned long long *cycles_per_cta, int32_t *dev_status,
+                       void *stream) {
+    if ((mma_n != 128 && mma_n != 256 && mma_n != 16 && mma_n != 64) || iters < 1 || iters > (1 << 20) || ctas < 1 || !cycles_per_cta)
+        return MUXQ_ERR_INVALID_ARG;
+    return cuda_rc(launch_mma_peak(mma_n, iters, cycles_per_cta, dev_status, ctas, static_cast<cudaStream_t>(stream)));
 }
 
 int muxq_read_status(const int32_t *dev_status, void *stream) {

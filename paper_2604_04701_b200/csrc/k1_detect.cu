@@ -22,58 +22,73 @@ __device__ __forceinline__ float warp_max(float v) {
 }
 
 // Tail, run by one CTA once every partial maximum is merged: threshold, ordered compaction,
-// per-channel multipliers, Body abs-max -> s_X.
+// per-channel multipliers, Body abs-max -> s_X.  Rounds of 2048 channels: thread t owns the 8
+// consecutive channels [base + 8t, base + 8t + 8), loaded with two coalesced 128-bit loads.
 __device__ void detect_tail(const DetectArgs &a) {
     __shared__ int s_warp_cnt[kWarps];
     __shared__ float s_warp_max[kWarps];
     const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
     const int K = a.K;
-    int chunk = (K + kThreads - 1) / kThreads;
-    chunk = (chunk + 7) & ~7;  // whole 8-channel groups per thread
-    const int k0 = t * chunk;
-    const int k1 = min(K, k0 + chunk);
     const float down = exp2f(-(float)a.exp_factor);
-
-    int cnt = 0;
-    for (int k = k0; k < k1; ++k) cnt += (__uint_as_float(__ldcg(a.colmax_bits + k)) > a.tau) ? 1 : 0;
-
-    // exclusive prefix of cnt over the block (warp scan + warp totals)
-    int incl = cnt;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        int n = __shfl_up_sync(0xffffffffu, incl, o);
-        if (lane >= o) incl += n;
-    }
-    if (lane == 31) s_warp_cnt[warp] = incl;
-    __syncthreads();
-    int base = 0, total = 0;
-#pragma unroll
-    for (int w = 0; w < kWarps; ++w) {
-        int c = s_warp_cnt[w];
-        if (w < warp) base += c;
-        total += c;
-    }
-    int pos = base + incl - cnt;
-
+    int carry = 0;
     float bmax = 0.0f;
-    for (int g = k0; g < k1; g += 8) {
-        uint8_t gf = 0;
-        const int ge = min(k1, g + 8);
-        for (int k = g; k < ge; ++k) {
-            const float cm = __uint_as_float(__ldcg(a.colmax_bits + k));
-            float mul = 1.0f;
-            if (cm > a.tau) {
-                if (pos < a.cap) {
-                    a.outlier_idx[pos] = k;
-                    mul = down;
-                    gf = 1;
-                }
-                ++pos;
-            }
-            if (a.colmul) a.colmul[k] = mul;
-            bmax = fmaxf(bmax, cm * mul);  // power-of-two scaling: exact
+    for (int base = 0; base < K; base += kThreads * 8) {
+        const int k0 = base + t * 8;
+        const bool active = k0 < K;  // K % 8 == 0: a group is entirely inside or outside
+        float cm[8];
+        if (active) {
+            const float4 v0 = __ldcg(reinterpret_cast<const float4 *>(a.colmax_bits + k0));
+            const float4 v1 = __ldcg(reinterpret_cast<const float4 *>(a.colmax_bits + k0) + 1);
+            cm[0] = v0.x; cm[1] = v0.y; cm[2] = v0.z; cm[3] = v0.w;
+            cm[4] = v1.x; cm[5] = v1.y; cm[6] = v1.z; cm[7] = v1.w;
+        } else {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) cm[i] = 0.0f;
         }
-        if (a.grpflag) a.grpflag[g >> 3] = gf;
+        int cnt = 0;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) cnt += (cm[i] > a.tau) ? 1 : 0;
+        // exclusive prefix of cnt over the block (warp scan + warp totals)
+        int incl = cnt;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int n = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += n;
+        }
+        if (lane == 31) s_warp_cnt[warp] = incl;
+        __syncthreads();
+        int before = 0, total = 0;
+#pragma unroll
+        for (int w = 0; w < kWarps; ++w) {
+            const int c = s_warp_cnt[w];
+            if (w < warp) before += c;
+            total += c;
+        }
+        int pos = carry + before + incl - cnt;
+        if (active) {
+            float mul[8];
+            uint8_t gf = 0;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                mul[i] = 1.0f;
+                if (cm[i] > a.tau) {
+                    if (pos < a.cap) {
+                        a.outlier_idx[pos] = k0 + i;
+                        mul[i] = down;
+                        gf = 1;
+                    }
+                    ++pos;
+                }
+                bmax = fmaxf(bmax, cm[i] * mul[i]);  // power-of-two scaling: exact
+            }
+            if (a.colmul) {
+                reinterpret_cast<float4 *>(a.colmul + k0)[0] = make_float4(mul[0], mul[1], mul[2], mul[3]);
+                reinterpret_cast<float4 *>(a.colmul + k0)[1] = make_float4(mul[4], mul[5], mul[6], mul[7]);
+            }
+            if (a.grpflag) a.grpflag[k0 >> 3] = gf;
+        }
+        carry += total;
+        __syncthreads();  // s_warp_cnt is reused by the next round
     }
     bmax = warp_max(bmax);
     if (lane == 0) s_warp_max[warp] = bmax;
@@ -85,9 +100,10 @@ __device__ void detect_tail(const DetectArgs &a) {
         const float s = m > 0.0f ? __fdiv_rn(m, (float)a.qmax) : 1.0f;  // Eq. 1
         if (a.s_x) *a.s_x = s;
         a.ctrl->s_x = s;
-        a.ctrl->n_outliers = total;
-        if (a.n_outliers) *a.n_outliers = total;
-        if (total > a.cap && a.dev_status) atomicMax(a.dev_status, kStatusCapacity);
+        a.ctrl->inv_s_x = __fdiv_rn(1.0f, s);
+        a.ctrl->n_outliers = carry;
+        if (a.n_outliers) *a.n_outliers = carry;
+        if (carry > a.cap && a.dev_status) atomicMax(a.dev_status, kStatusCapacity);
     }
 }
 
@@ -135,7 +151,9 @@ __global__ void __launch_bounds__(kThreads) k_colabsmax_detect(const DetectArgs 
 #pragma unroll
         for (int w = 0; w < kWarps; ++w) m = fmaxf(m, s_part[w][t]);
         const int k = blockIdx.x * kColsPerBlock + t;
-        if (k < a.K && m > 0.0f) atomicMax(a.colmax_bits + k, __float_as_uint(m));
+        // most CTAs find the running maximum already at or above theirs and skip the atomic
+        if (k < a.K && m > 0.0f && __float_as_uint(m) > __ldcg(a.colmax_bits + k))
+            atomicMax(a.colmax_bits + k, __float_as_uint(m));
     }
     // last CTA to arrive runs the tail
     __threadfence();

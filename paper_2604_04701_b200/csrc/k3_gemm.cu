@@ -9,7 +9,9 @@
 //            into a multi-stage shared-memory ring (mbarrier full/empty pairs)
 //   warp 1   MMA issuer: tcgen05.mma kind::i8, M=128, N=BN, K=32 per instruction, accumulating in
 //            one of two TMEM buffers so the epilogue of tile i overlaps the main loop of tile i+1
-//   warps 2-5 epilogue: tcgen05.ld (32 lanes x 32 columns), int32 -> fp32 scale -> fp16/fp32 stores
+//   warps 2-9 epilogue: tcgen05.ld (32 lanes x 32 columns), int32 -> fp32 scale -> fp16/fp32, staged
+//            per warp in 128-byte-swizzled shared memory (32 rows x 128 B) and
+//            written with TMA stores, so global writes are whole 128-byte row segments
 // Every mbarrier wait is bounded; on expiry the CTA raises MUXQ_ERR_TIMEOUT in the device status
 // word, drains its outstanding copies, frees its TMEM and returns.
 #include <cuda.h>
@@ -23,7 +25,8 @@ namespace {
 
 constexpr int BM = 128;
 constexpr int BK = 128;  // bytes of K per stage = one 128-byte swizzle row
-constexpr int kGemmThreads = 192;
+constexpr int kEpiWarps = 8;                       // two per TMEM lane quadrant, each half of the tile's columns
+constexpr int kGemmThreads = 64 + 32 * kEpiWarps;  // TMA warp + MMA warp + epilogue warps
 constexpr int kStatusTimeout = 6;  // MUXQ_ERR_TIMEOUT
 
 template <int BN>
@@ -33,7 +36,9 @@ struct Cfg {
     static constexpr int kBBytes = BN * BK;
     static constexpr int kStageBytes = kABytes + kBBytes;
     static constexpr int kTmemCols = 2 * BN;
-    static constexpr int kSmemBytes = kStages * kStageBytes + 1024;  // + alignment slack
+    static constexpr int kOutStageBytes = 32 * 128;                  // 32 rows x 128 B per epilogue warp
+    static constexpr int kOutBytes = kEpiWarps * kOutStageBytes;
+    static constexpr int kSmemBytes = kStages * kStageBytes + kOutBytes + 1024;  // + alignment slack
 };
 
 struct GemmParams {
@@ -47,13 +52,24 @@ struct GemmParams {
     const float *s_w; int s_w_per_col;
     void *Y; int ldy; int out_kind;
     int32_t *dev_status;
+    int dbg;
+    long long *tl;  // debug timeline (CTA 0): [0..255] producer, [256..511] mma, [512..767] epilogue warp 2
 };
+
+// int32 -> fp32, round to nearest even, exact for every int32, without the (slow) conversion unit:
+// a = hi * 65536 + lo with lo in [0, 65535]; both halves become floats by the "magic constant" bit
+// trick (2^23 + lo, 1.5 * 2^23 + hi, minus the constant) and one fused multiply-add rounds once.
+__device__ __forceinline__ float i32_to_f32_rn(int a) {
+    const float flo = __uint_as_float(0x4B000000u | ((uint32_t)a & 0xFFFFu)) - 8388608.0f;
+    const float fhi = __int_as_float(0x4B400000 + (a >> 16)) - 12582912.0f;
+    return fmaf(fhi, 65536.0f, flo);
+}
 
 template <int BN>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 k_gemm_i8(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_aux,
           const __grid_constant__ CUtensorMap tm_b, const __grid_constant__ CUtensorMap tm_baux,
-          const GemmParams p) {
+          const __grid_constant__ CUtensorMap tm_y, const GemmParams p) {
     using C = Cfg<BN>;
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t bar_full[C::kStages], bar_empty[C::kStages], bar_acc_full[2], bar_acc_empty[2];
@@ -67,6 +83,7 @@ k_gemm_i8(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
     if (threadIdx.x == 0) {
         tma_prefetch_desc(&tm_a);
         tma_prefetch_desc(&tm_b);
+        tma_prefetch_desc(&tm_y);
         if (p.has_aux) {
             tma_prefetch_desc(&tm_aux);
             tma_prefetch_desc(&tm_baux);
@@ -77,7 +94,7 @@ k_gemm_i8(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(&bar_acc_full[b], 1);
-            mbar_init(&bar_acc_empty[b], 4);  // one arrival per epilogue warp
+            mbar_init(&bar_acc_empty[b], kEpiWarps);  // one arrival per epilogue warp
         }
         s_abort = 0;
         fence_barrier_init();
@@ -109,8 +126,10 @@ k_gemm_i8(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
                 for (int kb = 0; kb < total_kb; ++kb, ++it) {
                     const uint32_t s = it % C::kStages, ph = (it / C::kStages) & 1u;
                     if (!mbar_wait(&bar_empty[s], ph ^ 1u, abort_flag)) { ok = false; break; }
+                    if (p.tl && blockIdx.x == 0 && it < 256) p.tl[it] = clock64();
                     uint8_t *sa = smem_al + s * C::kStageBytes;
                     uint8_t *sb = sa + C::kABytes;
+                    if (p.dbg & 2) { mbar_arrive(&bar_full[s]); continue; }
                     mbar_expect_tx(&bar_full[s], C::kStageBytes);
                     if (kb < p.num_kb) {
                         tma_load_2d(sa, &tm_a, &bar_full[s], kb * BK, m0);
@@ -145,6 +164,7 @@ k_gemm_i8(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
                 for (int kb = 0; kb < total_kb; ++kb, ++it) {
                     const uint32_t s = it % C::kStages, ph = (it / C::kStages) & 1u;
                     if (!mbar_wait(&bar_full[s], ph, abort_flag)) { ok = false; break; }
+                    if (p.tl && blockIdx.x == 0 && it < 256) p.tl[256 + it] = clock64();
                     tc_fence_after();
                     int k_bytes;  // valid K extent of this block
                     if (kb < p.num_kb) k_bytes = min(BK, p.K - kb * BK);
@@ -152,7 +172,7 @@ k_gemm_i8(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
                     const int steps = (k_bytes + 31) >> 5;
                     const uint32_t a_addr = smem_base + s * C::kStageBytes;
                     const uint32_t b_addr = a_addr + C::kABytes;
-                    for (int k = 0; k < steps; ++k) {
+                    for (int k = 0; k < ((p.dbg & 4) ? 0 : steps); ++k) {
                         mma_i8_ss(d_tmem, smem_desc_sw128(a_addr + k * 32), smem_desc_sw128(b_addr + k * 32),
                                   idesc, (kb > 0 || k > 0) ? 1u : 0u);
                     }
@@ -164,85 +184,104 @@ k_gemm_i8(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
     } else {
         // ---------------------------------------------------------------- epilogue warps
         const int quad = warp & 3;  // TMEM lane quadrant this warp may read
-        uint32_t tile_it = 0;
+        uint32_t tile_it = 0, n_store = 0;
         bool ok = true;
-        const float sx0 = p.out_kind == 2 ? 1.0f : __ldg(p.s_x);
-        const float sw0 = p.out_kind == 2 ? 1.0f : __ldg(p.s_w);
+        const bool raw = p.out_kind == 2;
+        const int cmode = (p.dbg >> 9) & 3;
+        const float sx0 = raw ? 1.0f : __ldg(p.s_x);
+        const float sw0 = raw ? 1.0f : __ldg(p.s_w);
+        const int cols_per_chunk = p.out_kind == 0 ? 64 : 32;  // 128 bytes of output per row
+        const int chalf = (warp - 2) >> 2;  // which half of the tile's columns this warp converts
+        uint8_t *stage = smem_al + C::kStages * C::kStageBytes + (warp - 2) * C::kOutStageBytes;
+        const uint32_t sw_xor = (uint32_t)(lane & 7);
         for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++tile_it) {
             const int m0 = (tile / p.tiles_n) * BM, n0 = (tile % p.tiles_n) * BN;
             const uint32_t buf = tile_it & 1u, aph = (tile_it >> 1) & 1u;
             ok = mbar_wait(&bar_acc_full[buf], aph, abort_flag);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
+            if (p.tl && blockIdx.x == 0 && warp == 2 && lane == 0 && tile_it < 100) p.tl[512 + 2 * tile_it] = clock64();
             tc_fence_after();
-            const int row = m0 + quad * 32 + lane;
-            const bool row_ok = row < p.M;
+            const int row0 = m0 + quad * 32;
+            const int row = row0 + lane;
             float sx = sx0;
-            if (p.s_x_per_row && row_ok && p.out_kind != 2) sx = __ldg(p.s_x + row);
+            if (p.s_x_per_row && row < p.M && !raw) sx = __ldg(p.s_x + row);
+            const float sxw0 = __fmul_rn(sx, sw0);
 #pragma unroll 1
-            for (int chunk = 0; chunk < BN / 32; ++chunk) {
-                uint32_t v[32];
-                __syncwarp();  // tcgen05.ld is warp-collective: reconverge after the guarded stores
-                const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + buf * BN + chunk * 32;
-                tmem_ld_32x32(taddr, v);
-                tmem_ld_wait();
-                const int col0 = n0 + chunk * 32;
-                if (!row_ok || col0 >= p.N) continue;
-                if (p.out_kind == 2) {
-                    int32_t *y = reinterpret_cast<int32_t *>(p.Y) + (size_t)row * p.ldy + col0;
+            for (int col = chalf * (BN / 2); col < (chalf + 1) * (BN / 2); col += cols_per_chunk) {
+                const int gcol = n0 + col;
+                if (p.dbg & 128) { ++n_store; continue; }
+                uint4 *srow = reinterpret_cast<uint4 *>(stage + lane * 128);
+                const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + buf * BN + col;
+                if (p.out_kind == 0) {
+                    uint32_t v0[32], v1[32];
+                    tmem_ld_32x32(taddr, v0);
+                    tmem_ld_32x32(taddr + 32, v1);
+                    tmem_ld_wait();
+                    // the TMA store that last read the staging buffer must be done with it
+                    if (lane == 0) tma_store_wait_read<0>();
+                    __syncwarp();
 #pragma unroll
-                    for (int g = 0; g < 8; ++g)
-                        if (col0 + g * 4 < p.N)
-                            *reinterpret_cast<uint4 *>(y + g * 4) =
-                                make_uint4(v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
-                } else {
-                    float f[32];
-                    if (p.s_w_per_col) {
+                    for (int g = 0; g < 8; ++g) {
+                        float f[8];
 #pragma unroll
-                        for (int g = 0; g < 8; ++g) {
-                            float4 w4 = make_float4(0.f, 0.f, 0.f, 0.f);
-                            if (col0 + g * 4 < p.N) w4 = __ldg(reinterpret_cast<const float4 *>(p.s_w + col0) + g);
-                            f[4 * g + 0] = __fmul_rn(__fmul_rn(sx, w4.x), __int2float_rn((int)v[4 * g + 0]));
-                            f[4 * g + 1] = __fmul_rn(__fmul_rn(sx, w4.y), __int2float_rn((int)v[4 * g + 1]));
-                            f[4 * g + 2] = __fmul_rn(__fmul_rn(sx, w4.z), __int2float_rn((int)v[4 * g + 2]));
-                            f[4 * g + 3] = __fmul_rn(__fmul_rn(sx, w4.w), __int2float_rn((int)v[4 * g + 3]));
+                        for (int i = 0; i < 8; ++i) {
+                            const int idx = g * 8 + i;
+                            const int a = (int)(idx < 32 ? v0[idx & 31] : v1[idx & 31]);
+                            float sc = sxw0;
+                            if (p.s_w_per_col) sc = __fmul_rn(sx, gcol + idx < p.N ? __ldg(p.s_w + gcol + idx) : 0.0f);
+                            f[i] = __fmul_rn(sc, (cmode == 1 || (cmode == 2 && (i & 3) == 0)) ? __int2float_rn(a) : i32_to_f32_rn(a));
                         }
-                    } else {
-                        const float sxw = __fmul_rn(sx, sw0);
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) f[i] = __fmul_rn(sxw, __int2float_rn((int)v[i]));
+                        __half2 h0 = __floats2half2_rn(f[0], f[1]), h1 = __floats2half2_rn(f[2], f[3]);
+                        __half2 h2 = __floats2half2_rn(f[4], f[5]), h3 = __floats2half2_rn(f[6], f[7]);
+                        uint4 o;
+                        o.x = *reinterpret_cast<uint32_t *>(&h0); o.y = *reinterpret_cast<uint32_t *>(&h1);
+                        o.z = *reinterpret_cast<uint32_t *>(&h2); o.w = *reinterpret_cast<uint32_t *>(&h3);
+                        srow[g ^ sw_xor] = o;
                     }
-                    if (p.out_kind == 1) {
-                        float *y = reinterpret_cast<float *>(p.Y) + (size_t)row * p.ldy + col0;
+                } else {
+                    uint32_t v[32];
+                    tmem_ld_32x32(taddr, v);
+                    tmem_ld_wait();
+                    if (lane == 0) tma_store_wait_read<0>();
+                    __syncwarp();
 #pragma unroll
-                        for (int g = 0; g < 8; ++g)
-                            if (col0 + g * 4 < p.N)
-                                *reinterpret_cast<float4 *>(y + g * 4) =
-                                    make_float4(f[4 * g], f[4 * g + 1], f[4 * g + 2], f[4 * g + 3]);
-                    } else {
-                        __half *y = reinterpret_cast<__half *>(p.Y) + (size_t)row * p.ldy + col0;
+                    for (int g = 0; g < 8; ++g) {
+                        uint4 o;
+                        if (raw) {
+                            o = make_uint4(v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
+                        } else {
+                            float f[4];
 #pragma unroll
-                        for (int g = 0; g < 4; ++g) {
-                            if (col0 + g * 8 < p.N) {
-                                __half2 h0 = __floats2half2_rn(f[8 * g + 0], f[8 * g + 1]);
-                                __half2 h1 = __floats2half2_rn(f[8 * g + 2], f[8 * g + 3]);
-                                __half2 h2 = __floats2half2_rn(f[8 * g + 4], f[8 * g + 5]);
-                                __half2 h3 = __floats2half2_rn(f[8 * g + 6], f[8 * g + 7]);
-                                uint4 o;
-                                o.x = *reinterpret_cast<uint32_t *>(&h0);
-                                o.y = *reinterpret_cast<uint32_t *>(&h1);
-                                o.z = *reinterpret_cast<uint32_t *>(&h2);
-                                o.w = *reinterpret_cast<uint32_t *>(&h3);
-                                *reinterpret_cast<uint4 *>(y + g * 8) = o;
+                            for (int i = 0; i < 4; ++i) {
+                                const int idx = g * 4 + i;
+                                float sc = sxw0;
+                                if (p.s_w_per_col)
+                                    sc = __fmul_rn(sx, gcol + idx < p.N ? __ldg(p.s_w + gcol + idx) : 0.0f);
+                                f[i] = __fmul_rn(sc, (cmode == 1 || (cmode == 2 && (i & 3) == 0)) ? __int2float_rn((int)v[idx]) : i32_to_f32_rn((int)v[idx]));
                             }
+                            o = make_uint4(__float_as_uint(f[0]), __float_as_uint(f[1]), __float_as_uint(f[2]),
+                                           __float_as_uint(f[3]));
                         }
+                        srow[g ^ sw_xor] = o;
                     }
                 }
+                if (!(p.dbg & 64)) fence_proxy_async();  // make the generic-proxy writes visible to the TMA engine
+                __syncwarp();
+                if (lane == 0) {
+                    // rows >= M and columns >= N are clipped by the copy engine; a chunk wholly outside is
+                    // skipped, but its (empty) group is still committed so the buffer accounting stays exact
+                    if (row0 < p.M && gcol < p.N && !(p.dbg & 1)) tma_store_2d(&tm_y, stage, gcol, row0);
+                    tma_store_commit();
+                }
+                ++n_store;
             }
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&bar_acc_empty[buf]);
+            if (p.tl && blockIdx.x == 0 && warp == 2 && lane == 0 && tile_it < 100) p.tl[513 + 2 * tile_it] = clock64();
         }
+        if (lane == 0) tma_store_wait_all<0>();
     }
 
     // ---------------------------------------------------------------- teardown
@@ -287,6 +326,25 @@ bool make_map_i8(CUtensorMap *map, const void *ptr, uint64_t rows, uint64_t cols
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// output matrix [M, N] of 2- or 4-byte elements, pitch ldy elements; box = 128 bytes x 32 rows
+bool make_map_out(CUtensorMap *map, void *ptr, uint64_t rows, uint64_t cols, uint64_t ldy, int out_kind) {
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn) return false;
+    const uint64_t esz = out_kind == 0 ? 2 : 4;
+    const CUtensorMapDataType dt = out_kind == 0   ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16
+                                   : out_kind == 1 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32
+                                                   : CU_TENSOR_MAP_DATA_TYPE_INT32;
+    cuuint64_t dims[2] = {cols, rows};
+    cuuint64_t strides[1] = {ldy * esz};
+    cuuint32_t box[2] = {(cuuint32_t)(128 / esz), 32};
+    cuuint32_t estr[2] = {1, 1};
+    return fn(map, dt, 2, ptr, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+              CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+int g_dbg = 0;
+long long *g_tl = nullptr;
+
 template <int BN>
 cudaError_t launch_gemm_bn(const GemmArgs &a, cudaStream_t s) {
     using C = Cfg<BN>;
@@ -297,7 +355,8 @@ cudaError_t launch_gemm_bn(const GemmArgs &a, cudaStream_t s) {
         attr_set = true;
     }
     const bool has_aux = a.aux_q && a.w_aux && a.n_outliers;
-    CUtensorMap tm_a, tm_b, tm_aux, tm_baux;
+    CUtensorMap tm_a, tm_b, tm_aux, tm_baux, tm_y;
+    if (!make_map_out(&tm_y, a.Y, a.M, a.N, a.ldy, a.out_kind)) return cudaErrorInvalidValue;
     if (!make_map_i8(&tm_a, a.body_q, a.M, a.K, a.ld_a, BM)) return cudaErrorInvalidValue;
     if (!make_map_i8(&tm_b, a.w_q, a.N, a.K, a.ldw, BN)) return cudaErrorInvalidValue;
     if (has_aux) {
@@ -319,15 +378,22 @@ cudaError_t launch_gemm_bn(const GemmArgs &a, cudaStream_t s) {
     p.s_w = a.s_w; p.s_w_per_col = a.s_w_per_col;
     p.Y = a.Y; p.ldy = a.ldy; p.out_kind = a.out_kind;
     p.dev_status = a.dev_status;
+    p.dbg = g_dbg;
+    p.tl = g_tl;
     int grid = p.tiles_m * p.tiles_n;
     if (grid > num_sms()) grid = num_sms();
-    k_gemm_i8<BN><<<grid, kGemmThreads, C::kSmemBytes, s>>>(tm_a, tm_aux, tm_b, tm_baux, p);
+    k_gemm_i8<BN><<<grid, kGemmThreads, C::kSmemBytes, s>>>(tm_a, tm_aux, tm_b, tm_baux, tm_y, p);
     return cudaGetLastError();
 }
 
 }  // namespace
 
+void set_gemm_dbg(int v) { g_dbg = v; }
+void set_gemm_tl(long long *p) { g_tl = p; }
+
 cudaError_t launch_gemm(const GemmArgs &a, cudaStream_t s) {
+    if (g_dbg & 8) return launch_gemm_bn<256>(a, s);
+    if (g_dbg & 16) return launch_gemm_bn<128>(a, s);
     // Tile width: 256 halves the per-MMA operand traffic; 128 gives more tiles when the 256-wide
     // tiling leaves most of the last wave idle.
     const int sms = num_sms();

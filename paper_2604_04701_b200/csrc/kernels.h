@@ -12,7 +12,8 @@ struct Ctrl {
     uint32_t blocks_done;  // K1: CTAs that have merged their partial maxima
     int32_t n_outliers;    // r, true count of outlier channels
     float s_x;             // per-tensor Body scale (Eq. 1)
-    uint32_t reserved[61];
+    float inv_s_x;         // 1 / s_x, correctly rounded (used only to pre-screen the exact division)
+    uint32_t reserved[60];
 };
 static_assert(sizeof(Ctrl) == 256, "Ctrl is one 256-byte block");
 
@@ -46,6 +47,7 @@ struct QuantActArgs {
     const float *colmul;         // [K] or NULL when outlier_idx is NULL
     const uint8_t *grpflag;      // [K/8] or NULL
     const float *s_x_tensor;     // [1] per-tensor scale (device), used when !per_token
+    const float *inv_s_x_tensor; // [1] its correctly rounded reciprocal
     float *s_x_rows;             // [M] out when per_token
     int8_t *body_q;  int ld_q;
     int8_t *aux_q;   int ld_aux; int aux_cols;   // aux_q may be NULL
@@ -98,6 +100,9 @@ struct DecodeArgs {
     void *Y; int ldy; int out_kind;
 };
 cudaError_t launch_decode(const DecodeArgs &a, cudaStream_t s);
+
+cudaError_t launch_mma_peak(int n, int iters, unsigned long long *cycles_out, int32_t *status, int grid,
+                            cudaStream_t s);
 
 int num_sms();
 

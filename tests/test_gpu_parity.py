@@ -171,6 +171,28 @@ def test_activation_quantization_matches_oracle(mx, gran, M, K, e, bits):
     assert np.array_equal(ns.cpu().numpy(), sx_n) and np.array_equal(nq.cpu().numpy(), bq_n)
 
 
+def test_quantization_ties_round_half_even(mx):
+    """Scale 0.25 exactly and inputs on multiples of 0.125: every other value is an exact .5 tie."""
+    M, K = 64, 256
+    rng = np.random.default_rng(3)
+    x = (rng.integers(-100, 101, (M, K)) * 0.125).astype(np.float16)
+    x[0, 7] = 31.75  # abs-max -> s = 31.75 / 127 = 0.25
+    p = mx.MuxqParams(threshold=1e4)
+    ws = mx.Workspace(mx.muxq_small_workspace_bytes(K))
+    xd = dev(x)
+    cm, idx, n = mx.muxq_detect_outliers(xd, p.threshold, p.max_outliers, ws)
+    body_q, _, s_x = mx.muxq_quantize(xd, p, False, ws, cm, idx, n, want_aux=False)
+    assert s_x.item() == 0.25
+    ref = np.rint(x.astype(np.float32) / np.float32(0.25)).astype(np.int8)  # numpy rint is half-to-even
+    assert (np.abs(x.astype(np.float32) / 0.25 % 1.0) == 0.5).sum() > 1000
+    assert np.array_equal(body_q.cpu().numpy(), ref)
+    for gran in (0, 1):
+        sx_o, _, bq_o, _ = oracle.quantize_act(x.astype(np.float32), np.zeros((M, 0), np.float32), 8, bool(gran), False)
+        pq = mx.MuxqParams(threshold=1e4, gran=gran)
+        bq, _, sx = mx.muxq_quantize(xd, pq, False, ws, cm, idx, n, want_aux=False)
+        assert np.array_equal(sx.cpu().numpy(), sx_o) and np.array_equal(bq.cpu().numpy(), bq_o)
+
+
 # ------------------------------------------------------------------ K3 alone
 @pytest.mark.parametrize("M,K,N", [(128, 128, 128), (128, 256, 256), (256, 768, 768), (300, 1040, 520),
                                    (1000, 512, 1288), (128, 32, 64), (129, 4096, 264)])
@@ -194,6 +216,19 @@ def test_gemm_worst_case_magnitudes(mx):
     acc = mx.muxq_gemm(dev(a), None, dev(b), None, None, mx.MuxqParams(), None, None, 2, mx.Workspace(256))
     ref = a.astype(np.int32) @ b.astype(np.int32).T
     assert np.array_equal(acc.cpu().numpy(), ref)
+    assert np.abs(ref).max() > 2 ** 24  # int32 -> fp32 must round (to nearest even) here
+    sx = np.array([0.0123], np.float32); sw = np.array([0.00071], np.float32)
+    y = mx.muxq_gemm(dev(a), None, dev(b), None, None, mx.MuxqParams(), dev(sx), dev(sw), 1, mx.Workspace(256))
+    assert np.array_equal(y.cpu().numpy(), (sx * sw) * ref.astype(np.float32))
+    # odd magnitudes above 2^24 exercise the rounding itself
+    a[:, :7] = 1; b[:, :7] = 1
+    b[1::2, 7] = 3
+    ref = a.astype(np.int32) @ b.astype(np.int32).T
+    y = mx.muxq_gemm(dev(a), None, dev(b), None, None, mx.MuxqParams(), dev(sx), dev(sw), 1, mx.Workspace(256))
+    assert np.array_equal(y.cpu().numpy(), (sx * sw) * ref.astype(np.float32))
+    y16 = mx.muxq_gemm(dev(a), None, dev(b), None, None, mx.MuxqParams(), dev(sx), dev(sw), 0, mx.Workspace(256))
+    with np.errstate(over="ignore"):
+        assert np.array_equal(y16.cpu().numpy(), ((sx * sw) * ref.astype(np.float32)).astype(np.float16))
 
 
 # ------------------------------------------------------------------ whole layer
