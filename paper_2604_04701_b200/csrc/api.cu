@@ -61,11 +61,7 @@ int cuda_rc(cudaError_t e) { return e == cudaSuccess ? MUXQ_OK : MUXQ_ERR_CUDA; 
 
 }  // namespace
 
-namespace muxq { extern int g_peak_mode; void set_gemm_dbg(int v); void set_gemm_tl(long long *p); }
 extern "C" {
-void muxq_debug_set(int v) { muxq::set_gemm_dbg(v); }
-void muxq_debug_tl(long long *p) { muxq::set_gemm_tl(p); }
-void muxq_debug_peak_mode(int m) { muxq::g_peak_mode = m; }
 
 void muxq_default_params(muxq_params *p) {
     if (!p) return;

@@ -9,9 +9,13 @@
 //            into a multi-stage shared-memory ring (mbarrier full/empty pairs)
 //   warp 1   MMA issuer: tcgen05.mma kind::i8, M=128, N=BN, K=32 per instruction, accumulating in
 //            one of two TMEM buffers so the epilogue of tile i overlaps the main loop of tile i+1
-//   warps 2-9 epilogue: tcgen05.ld (32 lanes x 32 columns), int32 -> fp32 scale -> fp16/fp32, staged
-//            per warp in 128-byte-swizzled shared memory (32 rows x 128 B) and
-//            written with TMA stores, so global writes are whole 128-byte row segments
+//   warps 2-9 epilogue: tcgen05.ld (32 lanes x 32 columns, the next chunk in flight while the current
+//            one is converted), int32 -> fp32 -> scale -> fp16/fp32, staged per warp in
+//            128-byte-swizzled shared memory (32 rows x 128 B) and written with TMA stores, so
+//            global writes are whole 128-byte row segments
+// Role dispatch uses a warp index broadcast with a shuffle, which keeps each role's control flow
+// and its descriptors / addresses warp-uniform; the producer and the MMA issuer run as whole warps
+// with one elected lane issuing (a divergent single-thread loop issues MMAs several times slower).
 // Every mbarrier wait is bounded; on expiry the CTA raises MUXQ_ERR_TIMEOUT in the device status
 // word, drains its outstanding copies, frees its TMEM and returns.
 #include <cuda.h>
@@ -28,17 +32,20 @@ constexpr int BK = 128;  // bytes of K per stage = one 128-byte swizzle row
 constexpr int kEpiWarps = 8;                       // two per TMEM lane quadrant, each half of the tile's columns
 constexpr int kGemmThreads = 64 + 32 * kEpiWarps;  // TMA warp + MMA warp + epilogue warps
 constexpr int kStatusTimeout = 6;  // MUXQ_ERR_TIMEOUT
+constexpr int kOutF16 = 0, kOutF32 = 1, kOutI32 = 2;
 
 template <int BN>
 struct Cfg {
-    static constexpr int kStages = BN == 256 ? 4 : 6;
     static constexpr int kABytes = BM * BK;
     static constexpr int kBBytes = BN * BK;
     static constexpr int kStageBytes = kABytes + kBBytes;
     static constexpr int kTmemCols = 2 * BN;
-    static constexpr int kOutStageBytes = 32 * 128;                  // 32 rows x 128 B per epilogue warp
-    static constexpr int kOutBytes = kEpiWarps * kOutStageBytes;
+    static constexpr int kOutBufBytes = 32 * 128;  // one TMA store box: 32 rows x 128 B
+    static constexpr int kOutBufs = BN == 256 ? 1 : 2;  // staging buffers per epilogue warp
+    static constexpr int kOutBytes = kEpiWarps * kOutBufs * kOutBufBytes;
+    static constexpr int kStages = (227 * 1024 - 1024 - kOutBytes - 1024) / kStageBytes;
     static constexpr int kSmemBytes = kStages * kStageBytes + kOutBytes + 1024;  // + alignment slack
+    static_assert(kStages >= 3, "operand ring too shallow");
 };
 
 struct GemmParams {
@@ -48,24 +55,59 @@ struct GemmParams {
     int has_aux;   // Aux operands present
     int c, cap;
     const int32_t *n_outliers;
-    const float *s_x; int s_x_per_row;
-    const float *s_w; int s_w_per_col;
-    void *Y; int ldy; int out_kind;
+    const float *s_x;
+    const float *s_w;
     int32_t *dev_status;
-    int dbg;
-    long long *tl;  // debug timeline (CTA 0): [0..255] producer, [256..511] mma, [512..767] epilogue warp 2
 };
 
-// int32 -> fp32, round to nearest even, exact for every int32, without the (slow) conversion unit:
-// a = hi * 65536 + lo with lo in [0, 65535]; both halves become floats by the "magic constant" bit
-// trick (2^23 + lo, 1.5 * 2^23 + hi, minus the constant) and one fused multiply-add rounds once.
-__device__ __forceinline__ float i32_to_f32_rn(int a) {
-    const float flo = __uint_as_float(0x4B000000u | ((uint32_t)a & 0xFFFFu)) - 8388608.0f;
-    const float fhi = __int_as_float(0x4B400000 + (a >> 16)) - 12582912.0f;
-    return fmaf(fhi, 65536.0f, flo);
+// One 32-column chunk of one accumulator row: int32 -> fp32 (round to nearest even, exact below
+// 2^24) -> times the scale -> output type, written as 16-byte pieces into the warp's staging row
+// with the 128-byte swizzle the TMA store expects (16-byte piece g of row `lane` sits at g ^ (lane & 7)).
+template <int kOut, bool kPerVec>
+__device__ __forceinline__ void convert_chunk(const uint32_t (&v)[32], uint4 *srow, int piece0, uint32_t sw_xor,
+                                              float sx, float sxw, const float *s_w_col, int cols_left) {
+    if (kOut == kOutI32) {
+#pragma unroll
+        for (int g = 0; g < 8; ++g)
+            srow[(piece0 + g) ^ sw_xor] = make_uint4(v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
+        return;
+    }
+    float f[32];
+#pragma unroll
+    for (int g = 0; g < 8; ++g) {
+        float4 sc = make_float4(sxw, sxw, sxw, sxw);
+        if (kPerVec) {
+            // same address in every lane: one broadcast transaction; columns past N read as 0
+            const float4 w = 4 * g < cols_left ? __ldg(reinterpret_cast<const float4 *>(s_w_col) + g)
+                                               : make_float4(0.f, 0.f, 0.f, 0.f);
+            sc = make_float4(__fmul_rn(sx, w.x), __fmul_rn(sx, w.y), __fmul_rn(sx, w.z), __fmul_rn(sx, w.w));
+        }
+        f[4 * g + 0] = __fmul_rn(sc.x, __int2float_rn((int)v[4 * g + 0]));
+        f[4 * g + 1] = __fmul_rn(sc.y, __int2float_rn((int)v[4 * g + 1]));
+        f[4 * g + 2] = __fmul_rn(sc.z, __int2float_rn((int)v[4 * g + 2]));
+        f[4 * g + 3] = __fmul_rn(sc.w, __int2float_rn((int)v[4 * g + 3]));
+    }
+    if (kOut == kOutF32) {
+#pragma unroll
+        for (int g = 0; g < 8; ++g)
+            srow[(piece0 + g) ^ sw_xor] = make_uint4(__float_as_uint(f[4 * g]), __float_as_uint(f[4 * g + 1]),
+                                                     __float_as_uint(f[4 * g + 2]), __float_as_uint(f[4 * g + 3]));
+    } else {
+#pragma unroll
+        for (int g = 0; g < 4; ++g) {
+            const __half2 h0 = __floats2half2_rn(f[8 * g + 0], f[8 * g + 1]);
+            const __half2 h1 = __floats2half2_rn(f[8 * g + 2], f[8 * g + 3]);
+            const __half2 h2 = __floats2half2_rn(f[8 * g + 4], f[8 * g + 5]);
+            const __half2 h3 = __floats2half2_rn(f[8 * g + 6], f[8 * g + 7]);
+            uint4 o;
+            o.x = *reinterpret_cast<const uint32_t *>(&h0); o.y = *reinterpret_cast<const uint32_t *>(&h1);
+            o.z = *reinterpret_cast<const uint32_t *>(&h2); o.w = *reinterpret_cast<const uint32_t *>(&h3);
+            srow[(piece0 + g) ^ sw_xor] = o;
+        }
+    }
 }
 
-template <int BN>
+template <int BN, int kOut, bool kPerVec>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 k_gemm_i8(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_aux,
           const __grid_constant__ CUtensorMap tm_b, const __grid_constant__ CUtensorMap tm_baux,
@@ -76,7 +118,8 @@ k_gemm_i8(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
     __shared__ uint32_t s_tmem_base;
     __shared__ uint32_t s_abort;
 
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0);  // warp-uniform by construction
+    const int lane = threadIdx.x & 31;
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *smem_al = smem_raw + (smem_base - smem_u32(smem_raw));
 
@@ -106,180 +149,143 @@ k_gemm_i8(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    const uint32_t tmem_base = s_tmem_base;
+    const uint32_t tmem_base = __shfl_sync(0xffffffffu, s_tmem_base, 0);
     volatile uint32_t *abort_flag = &s_abort;
 
-    // Aux extent: c*r replicated columns -> K blocks and MMA steps of 32
+    // Aux extent: c*r replicated columns -> at most one extra K block, ceil(c*r/32) MMA steps
     int aux_cols_used = 0;
-    if (p.has_aux && p.n_outliers) aux_cols_used = p.c * min(__ldg(p.n_outliers), p.cap);
+    if (p.has_aux) aux_cols_used = p.c * min(__ldg(p.n_outliers), p.cap);
+    aux_cols_used = __shfl_sync(0xffffffffu, aux_cols_used, 0);
     const int aux_kb = (aux_cols_used + BK - 1) / BK;
     const int total_kb = p.num_kb + aux_kb;
     const int num_tiles = p.tiles_m * p.tiles_n;
 
     if (warp == 0) {
-        if (lane == 0) {
-            // ------------------------------------------------------------ TMA producer
-            uint32_t it = 0;
-            bool ok = true;
-            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
-                const int m0 = (tile / p.tiles_n) * BM, n0 = (tile % p.tiles_n) * BN;
-                for (int kb = 0; kb < total_kb; ++kb, ++it) {
-                    const uint32_t s = it % C::kStages, ph = (it / C::kStages) & 1u;
-                    if (!mbar_wait(&bar_empty[s], ph ^ 1u, abort_flag)) { ok = false; break; }
-                    if (p.tl && blockIdx.x == 0 && it < 256) p.tl[it] = clock64();
-                    uint8_t *sa = smem_al + s * C::kStageBytes;
-                    uint8_t *sb = sa + C::kABytes;
-                    if (p.dbg & 2) { mbar_arrive(&bar_full[s]); continue; }
-                    mbar_expect_tx(&bar_full[s], C::kStageBytes);
-                    if (kb < p.num_kb) {
-                        tma_load_2d(sa, &tm_a, &bar_full[s], kb * BK, m0);
-                        tma_load_2d(sb, &tm_b, &bar_full[s], kb * BK, n0);
-                    } else {
-                        tma_load_2d(sa, &tm_aux, &bar_full[s], (kb - p.num_kb) * BK, m0);
-                        tma_load_2d(sb, &tm_baux, &bar_full[s], (kb - p.num_kb) * BK, n0);
-                    }
+        // ------------------------------------------------------------ TMA producer (whole warp, one lane issues)
+        uint32_t it = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+            const int m0 = (tile / p.tiles_n) * BM, n0 = (tile % p.tiles_n) * BN;
+            for (int kb = 0; kb < total_kb; ++kb, ++it) {
+                const uint32_t s = it % C::kStages, ph = (it / C::kStages) & 1u;
+                if (!mbar_wait_warp(&bar_empty[s], ph ^ 1u, abort_flag)) { ok = false; break; }
+                uint8_t *sa = smem_al + s * C::kStageBytes;
+                uint8_t *sb = sa + C::kABytes;
+                mbar_expect_tx_elect(&bar_full[s], C::kStageBytes);
+                if (kb < p.num_kb) {
+                    tma_load_2d_elect(sa, &tm_a, &bar_full[s], kb * BK, m0);
+                    tma_load_2d_elect(sb, &tm_b, &bar_full[s], kb * BK, n0);
+                } else {
+                    tma_load_2d_elect(sa, &tm_aux, &bar_full[s], (kb - p.num_kb) * BK, m0);
+                    tma_load_2d_elect(sb, &tm_baux, &bar_full[s], (kb - p.num_kb) * BK, n0);
                 }
             }
-            if (!ok) {
-                // drain: wait (bounded) until every copy this thread issued has landed
-                const uint32_t first = it > (uint32_t)C::kStages ? it - C::kStages : 0u;
-                for (uint32_t j = first; j < it; ++j) {
-                    const uint32_t s = j % C::kStages, ph = (j / C::kStages) & 1u;
-                    for (uint32_t i = 0; i < kSpinLimit; ++i)
-                        if (mbar_try_wait(&bar_full[s], ph)) break;
-                }
+        }
+        if (!ok) {
+            // drain: wait (bounded) until every copy this warp issued has landed
+            const uint32_t first = it > (uint32_t)C::kStages ? it - C::kStages : 0u;
+            for (uint32_t j = first; j < it; ++j) {
+                const uint32_t s = j % C::kStages, ph = (j / C::kStages) & 1u;
+                for (uint32_t i = 0; i < kSpinLimit; ++i)
+                    if (__any_sync(0xffffffffu, mbar_try_wait(&bar_full[s], ph))) break;
             }
         }
     } else if (warp == 1) {
-        if (lane == 0) {
-            // ------------------------------------------------------------ MMA issuer
-            constexpr uint32_t idesc = idesc_i8(BM, BN);
-            uint32_t it = 0, tile_it = 0;
-            bool ok = true;
-            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++tile_it) {
-                const uint32_t buf = tile_it & 1u, aph = (tile_it >> 1) & 1u;
-                if (!mbar_wait(&bar_acc_empty[buf], aph ^ 1u, abort_flag)) { ok = false; break; }
+        // ------------------------------------------------------------ MMA issuer (whole warp, one lane issues)
+        constexpr uint32_t idesc = idesc_i8(BM, BN);
+        const uint64_t a_desc0 = smem_desc_sw128(smem_base);
+        const uint64_t b_desc0 = smem_desc_sw128(smem_base + C::kABytes);
+        const int body_tail_steps = ((p.K - (p.num_kb - 1) * BK) + 31) >> 5;  // valid 32-byte steps of the last body block
+        uint32_t it = 0, tile_it = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++tile_it) {
+            const uint32_t buf = tile_it & 1u, aph = (tile_it >> 1) & 1u;
+            if (!mbar_wait_warp(&bar_acc_empty[buf], aph ^ 1u, abort_flag)) { ok = false; break; }
+            tc_fence_after();
+            const uint32_t d_tmem = tmem_base + buf * BN;
+            for (int kb = 0; kb < total_kb; ++kb, ++it) {
+                const uint32_t s = it % C::kStages, ph = (it / C::kStages) & 1u;
+                if (!mbar_wait_warp(&bar_full[s], ph, abort_flag)) { ok = false; break; }
                 tc_fence_after();
-                const uint32_t d_tmem = tmem_base + buf * BN;
-                for (int kb = 0; kb < total_kb; ++kb, ++it) {
-                    const uint32_t s = it % C::kStages, ph = (it / C::kStages) & 1u;
-                    if (!mbar_wait(&bar_full[s], ph, abort_flag)) { ok = false; break; }
-                    if (p.tl && blockIdx.x == 0 && it < 256) p.tl[256 + it] = clock64();
-                    tc_fence_after();
-                    int k_bytes;  // valid K extent of this block
-                    if (kb < p.num_kb) k_bytes = min(BK, p.K - kb * BK);
-                    else k_bytes = min(BK, aux_cols_used - (kb - p.num_kb) * BK);
-                    const int steps = (k_bytes + 31) >> 5;
-                    const uint32_t a_addr = smem_base + s * C::kStageBytes;
-                    const uint32_t b_addr = a_addr + C::kABytes;
-                    for (int k = 0; k < ((p.dbg & 4) ? 0 : steps); ++k) {
-                        mma_i8_ss(d_tmem, smem_desc_sw128(a_addr + k * 32), smem_desc_sw128(b_addr + k * 32),
-                                  idesc, (kb > 0 || k > 0) ? 1u : 0u);
-                    }
-                    mma_commit(&bar_empty[s]);  // stage reusable once these MMAs have read it
+                // descriptor start addresses are in 16-byte units: a stage is kStageBytes/16 apart, a 32-byte K step 2
+                const uint64_t a_desc = a_desc0 + (uint64_t)(s * (C::kStageBytes >> 4));
+                const uint64_t b_desc = b_desc0 + (uint64_t)(s * (C::kStageBytes >> 4));
+                int steps = 4;
+                if (kb == p.num_kb - 1) steps = body_tail_steps;
+                else if (kb >= p.num_kb) steps = (min(BK, aux_cols_used - (kb - p.num_kb) * BK) + 31) >> 5;
+                if (steps == 4) {
+                    mma_i8_ss_elect(d_tmem, a_desc, b_desc, idesc, kb > 0 ? 1u : 0u);
+                    mma_i8_ss_elect(d_tmem, a_desc + 2, b_desc + 2, idesc, 1u);
+                    mma_i8_ss_elect(d_tmem, a_desc + 4, b_desc + 4, idesc, 1u);
+                    mma_i8_ss_elect(d_tmem, a_desc + 6, b_desc + 6, idesc, 1u);
+                } else {
+                    for (int k = 0; k < steps; ++k)
+                        mma_i8_ss_elect(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (kb > 0 || k > 0) ? 1u : 0u);
                 }
-                if (ok) mma_commit(&bar_acc_full[buf]);
+                mma_commit_elect(&bar_empty[s]);  // stage reusable once these MMAs have read it
             }
+            if (ok) mma_commit_elect(&bar_acc_full[buf]);
         }
     } else {
         // ---------------------------------------------------------------- epilogue warps
-        const int quad = warp & 3;  // TMEM lane quadrant this warp may read
-        uint32_t tile_it = 0, n_store = 0;
-        bool ok = true;
-        const bool raw = p.out_kind == 2;
-        const int cmode = (p.dbg >> 9) & 3;
-        const float sx0 = raw ? 1.0f : __ldg(p.s_x);
-        const float sw0 = raw ? 1.0f : __ldg(p.s_w);
-        const int cols_per_chunk = p.out_kind == 0 ? 64 : 32;  // 128 bytes of output per row
-        const int chalf = (warp - 2) >> 2;  // which half of the tile's columns this warp converts
-        uint8_t *stage = smem_al + C::kStages * C::kStageBytes + (warp - 2) * C::kOutStageBytes;
+        const int quad = warp & 3;           // TMEM lane quadrant this warp may read
+        const int chalf = (warp - 2) >> 2;   // which half of the tile's columns this warp converts
+        constexpr int kChunks = BN / 2 / 32;                          // 32-column chunks per warp and tile
+        constexpr int kChunksPerBox = kOut == kOutF16 ? 2 : 1;        // 128 bytes of output per row and box
+        static_assert(kChunks % kChunksPerBox == 0, "a store box must not straddle two warps' columns");
+        uint8_t *stage0 = smem_al + C::kStages * C::kStageBytes + (warp - 2) * (C::kOutBufs * C::kOutBufBytes);
         const uint32_t sw_xor = (uint32_t)(lane & 7);
+        float sxw = 1.0f, sx = 1.0f;
+        if (kOut != kOutI32 && !kPerVec) sxw = __fmul_rn(__ldg(p.s_x), __ldg(p.s_w));
+        uint32_t tile_it = 0, n_box = 0;
+        bool ok = true;
         for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++tile_it) {
             const int m0 = (tile / p.tiles_n) * BM, n0 = (tile % p.tiles_n) * BN;
             const uint32_t buf = tile_it & 1u, aph = (tile_it >> 1) & 1u;
-            ok = mbar_wait(&bar_acc_full[buf], aph, abort_flag);
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
-            if (p.tl && blockIdx.x == 0 && warp == 2 && lane == 0 && tile_it < 100) p.tl[512 + 2 * tile_it] = clock64();
-            tc_fence_after();
             const int row0 = m0 + quad * 32;
-            const int row = row0 + lane;
-            float sx = sx0;
-            if (p.s_x_per_row && row < p.M && !raw) sx = __ldg(p.s_x + row);
-            const float sxw0 = __fmul_rn(sx, sw0);
-#pragma unroll 1
-            for (int col = chalf * (BN / 2); col < (chalf + 1) * (BN / 2); col += cols_per_chunk) {
-                const int gcol = n0 + col;
-                if (p.dbg & 128) { ++n_store; continue; }
-                uint4 *srow = reinterpret_cast<uint4 *>(stage + lane * 128);
-                const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + buf * BN + col;
-                if (p.out_kind == 0) {
-                    uint32_t v0[32], v1[32];
-                    tmem_ld_32x32(taddr, v0);
-                    tmem_ld_32x32(taddr + 32, v1);
-                    tmem_ld_wait();
-                    // the TMA store that last read the staging buffer must be done with it
-                    if (lane == 0) tma_store_wait_read<0>();
-                    __syncwarp();
+            if (kPerVec && kOut != kOutI32) sx = row0 + lane < p.M ? __ldg(p.s_x + row0 + lane) : 0.0f;
+            ok = mbar_wait_warp(&bar_acc_full[buf], aph, abort_flag);
+            if (!ok) break;
+            tc_fence_after();
+            const int col0 = chalf * (BN / 2);
+            const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + buf * BN + col0;
+            uint32_t v[2][32];
+            tmem_ld_32x32(taddr, v[0]);
 #pragma unroll
-                    for (int g = 0; g < 8; ++g) {
-                        float f[8];
-#pragma unroll
-                        for (int i = 0; i < 8; ++i) {
-                            const int idx = g * 8 + i;
-                            const int a = (int)(idx < 32 ? v0[idx & 31] : v1[idx & 31]);
-                            float sc = sxw0;
-                            if (p.s_w_per_col) sc = __fmul_rn(sx, gcol + idx < p.N ? __ldg(p.s_w + gcol + idx) : 0.0f);
-                            f[i] = __fmul_rn(sc, (cmode == 1 || (cmode == 2 && (i & 3) == 0)) ? __int2float_rn(a) : i32_to_f32_rn(a));
-                        }
-                        __half2 h0 = __floats2half2_rn(f[0], f[1]), h1 = __floats2half2_rn(f[2], f[3]);
-                        __half2 h2 = __floats2half2_rn(f[4], f[5]), h3 = __floats2half2_rn(f[6], f[7]);
-                        uint4 o;
-                        o.x = *reinterpret_cast<uint32_t *>(&h0); o.y = *reinterpret_cast<uint32_t *>(&h1);
-                        o.z = *reinterpret_cast<uint32_t *>(&h2); o.w = *reinterpret_cast<uint32_t *>(&h3);
-                        srow[g ^ sw_xor] = o;
-                    }
+            for (int ch = 0; ch < kChunks; ++ch) {
+                tmem_ld_wait();
+                if (ch + 1 < kChunks) {
+                    tmem_ld_32x32(taddr + 32 * (ch + 1), v[(ch + 1) & 1]);
                 } else {
-                    uint32_t v[32];
-                    tmem_ld_32x32(taddr, v);
-                    tmem_ld_wait();
-                    if (lane == 0) tma_store_wait_read<0>();
+                    // every TMEM read of this warp for this tile has completed: hand the buffer back
+                    tc_fence_before();
                     __syncwarp();
-#pragma unroll
-                    for (int g = 0; g < 8; ++g) {
-                        uint4 o;
-                        if (raw) {
-                            o = make_uint4(v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
-                        } else {
-                            float f[4];
-#pragma unroll
-                            for (int i = 0; i < 4; ++i) {
-                                const int idx = g * 4 + i;
-                                float sc = sxw0;
-                                if (p.s_w_per_col)
-                                    sc = __fmul_rn(sx, gcol + idx < p.N ? __ldg(p.s_w + gcol + idx) : 0.0f);
-                                f[i] = __fmul_rn(sc, (cmode == 1 || (cmode == 2 && (i & 3) == 0)) ? __int2float_rn((int)v[idx]) : i32_to_f32_rn((int)v[idx]));
-                            }
-                            o = make_uint4(__float_as_uint(f[0]), __float_as_uint(f[1]), __float_as_uint(f[2]),
-                                           __float_as_uint(f[3]));
-                        }
-                        srow[g ^ sw_xor] = o;
+                    if (lane == 0) mbar_arrive(&bar_acc_empty[buf]);
+                }
+                const int piece = ch % kChunksPerBox;  // position of this chunk inside its store box
+                uint8_t *stage = stage0 + (n_box % C::kOutBufs) * C::kOutBufBytes;
+                if (piece == 0) {
+                    // the store that last read this staging buffer must be done reading it
+                    if (lane == 0) tma_store_wait_read<C::kOutBufs - 1>();
+                    __syncwarp();
+                }
+                const int gcol = n0 + col0 + 32 * ch;
+                convert_chunk<kOut, kPerVec>(v[ch & 1], reinterpret_cast<uint4 *>(stage + lane * 128),
+                                             kOut == kOutF16 ? 4 * piece : 0, sw_xor, sx, sxw, p.s_w + gcol,
+                                             p.N - gcol);
+                if (piece == kChunksPerBox - 1) {
+                    fence_proxy_async();  // make the generic-proxy writes visible to the TMA engine
+                    __syncwarp();
+                    if (lane == 0) {
+                        // rows >= M and columns >= N are clipped by the copy engine; a box wholly outside is
+                        // skipped, but its (empty) group is still committed so the buffer accounting stays exact
+                        const int bcol = gcol - 32 * piece;
+                        if (row0 < p.M && bcol < p.N) tma_store_2d(&tm_y, stage, bcol, row0);
+                        tma_store_commit();
                     }
+                    ++n_box;
                 }
-                if (!(p.dbg & 64)) fence_proxy_async();  // make the generic-proxy writes visible to the TMA engine
-                __syncwarp();
-                if (lane == 0) {
-                    // rows >= M and columns >= N are clipped by the copy engine; a chunk wholly outside is
-                    // skipped, but its (empty) group is still committed so the buffer accounting stays exact
-                    if (row0 < p.M && gcol < p.N && !(p.dbg & 1)) tma_store_2d(&tm_y, stage, gcol, row0);
-                    tma_store_commit();
-                }
-                ++n_store;
             }
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&bar_acc_empty[buf]);
-            if (p.tl && blockIdx.x == 0 && warp == 2 && lane == 0 && tile_it < 100) p.tl[513 + 2 * tile_it] = clock64();
         }
         if (lane == 0) tma_store_wait_all<0>();
     }
@@ -314,6 +320,7 @@ EncodeTiledFn get_encode_fn() {
 }
 
 // int8 matrix [rows, cols] with pitch ld bytes, K-major; box = 128 bytes x box_rows, 128-byte swizzle.
+// Out-of-range rows and columns read as zero, which a K tail or a ragged tile edge relies on.
 bool make_map_i8(CUtensorMap *map, const void *ptr, uint64_t rows, uint64_t cols, uint64_t ld, uint32_t box_rows) {
     EncodeTiledFn fn = get_encode_fn();
     if (!fn) return false;
@@ -330,10 +337,10 @@ bool make_map_i8(CUtensorMap *map, const void *ptr, uint64_t rows, uint64_t cols
 bool make_map_out(CUtensorMap *map, void *ptr, uint64_t rows, uint64_t cols, uint64_t ldy, int out_kind) {
     EncodeTiledFn fn = get_encode_fn();
     if (!fn) return false;
-    const uint64_t esz = out_kind == 0 ? 2 : 4;
-    const CUtensorMapDataType dt = out_kind == 0   ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16
-                                   : out_kind == 1 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32
-                                                   : CU_TENSOR_MAP_DATA_TYPE_INT32;
+    const uint64_t esz = out_kind == kOutF16 ? 2 : 4;
+    const CUtensorMapDataType dt = out_kind == kOutF16   ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16
+                                   : out_kind == kOutF32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32
+                                                         : CU_TENSOR_MAP_DATA_TYPE_INT32;
     cuuint64_t dims[2] = {cols, rows};
     cuuint64_t strides[1] = {ldy * esz};
     cuuint32_t box[2] = {(cuuint32_t)(128 / esz), 32};
@@ -342,15 +349,13 @@ bool make_map_out(CUtensorMap *map, void *ptr, uint64_t rows, uint64_t cols, uin
               CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-int g_dbg = 0;
-long long *g_tl = nullptr;
-
-template <int BN>
-cudaError_t launch_gemm_bn(const GemmArgs &a, cudaStream_t s) {
+template <int BN, int kOut, bool kPerVec>
+cudaError_t launch_gemm_inst(const GemmArgs &a, cudaStream_t s) {
     using C = Cfg<BN>;
     static bool attr_set = false;
     if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(k_gemm_i8<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
+        cudaError_t e = cudaFuncSetAttribute(k_gemm_i8<BN, kOut, kPerVec>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             C::kSmemBytes);
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
@@ -374,28 +379,30 @@ cudaError_t launch_gemm_bn(const GemmArgs &a, cudaStream_t s) {
     p.has_aux = has_aux ? 1 : 0;
     p.c = a.c; p.cap = a.cap;
     p.n_outliers = a.n_outliers;
-    p.s_x = a.s_x; p.s_x_per_row = a.s_x_per_row;
-    p.s_w = a.s_w; p.s_w_per_col = a.s_w_per_col;
-    p.Y = a.Y; p.ldy = a.ldy; p.out_kind = a.out_kind;
+    p.s_x = a.s_x;
+    p.s_w = a.s_w;
     p.dev_status = a.dev_status;
-    p.dbg = g_dbg;
-    p.tl = g_tl;
     int grid = p.tiles_m * p.tiles_n;
     if (grid > num_sms()) grid = num_sms();
-    k_gemm_i8<BN><<<grid, kGemmThreads, C::kSmemBytes, s>>>(tm_a, tm_aux, tm_b, tm_baux, tm_y, p);
+    k_gemm_i8<BN, kOut, kPerVec><<<grid, kGemmThreads, C::kSmemBytes, s>>>(tm_a, tm_aux, tm_b, tm_baux, tm_y, p);
     return cudaGetLastError();
+}
+
+template <int BN>
+cudaError_t launch_gemm_bn(const GemmArgs &a, cudaStream_t s) {
+    const bool per_vec = a.s_x_per_row || a.s_w_per_col;  // the two granularities come as a pair
+    switch (a.out_kind) {
+        case kOutF16: return per_vec ? launch_gemm_inst<BN, kOutF16, true>(a, s) : launch_gemm_inst<BN, kOutF16, false>(a, s);
+        case kOutF32: return per_vec ? launch_gemm_inst<BN, kOutF32, true>(a, s) : launch_gemm_inst<BN, kOutF32, false>(a, s);
+        default: return launch_gemm_inst<BN, kOutI32, false>(a, s);
+    }
 }
 
 }  // namespace
 
-void set_gemm_dbg(int v) { g_dbg = v; }
-void set_gemm_tl(long long *p) { g_tl = p; }
-
 cudaError_t launch_gemm(const GemmArgs &a, cudaStream_t s) {
-    if (g_dbg & 8) return launch_gemm_bn<256>(a, s);
-    if (g_dbg & 16) return launch_gemm_bn<128>(a, s);
-    // Tile width: 256 halves the per-MMA operand traffic; 128 gives more tiles when the 256-wide
-    // tiling leaves most of the last wave idle.
+    // Tile width: an M128 MMA runs at the full tensor rate for N >= 128, and 256 halves the operand
+    // traffic per MMA; 128 gives more tiles when the 256-wide tiling leaves most of the last wave idle.
     const int sms = num_sms();
     const int tm = (a.M + BM - 1) / BM;
     const int t256 = tm * ((a.N + 255) / 256), t128 = tm * ((a.N + 127) / 128);

@@ -21,7 +21,7 @@ def L():
 def test_every_declared_symbol_is_exported(L):
     hdr = open(os.path.join(ROOT, "include", "muxq.h")).read()
     hdr = re.sub(r"/\*.*?\*/", "", hdr, flags=re.S)
-    declared = set(re.findall(r"\b(muxq_[a-z_]+)\s*\(", hdr))
+    declared = set(re.findall(r"\b(muxq_[a-z0-9_]+)\s*\(", hdr))
     assert {"muxq_detect_outliers", "muxq_build_aux", "muxq_quantize", "muxq_linear"} <= declared
     lib = ctypes.CDLL(L.library_path())
     for name in sorted(declared):
