@@ -157,8 +157,10 @@ int muxq_linear(const void *X_f16, int M, int K, int ldx, const int8_t *W_q, int
 /*
  * muxq_linear that also records four caller-created CUDA events (cudaEvent_t passed as void*;
  * NULL entries are skipped) on `stream` at its kernel boundaries, for per-kernel timing:
- * events[0] before detection, [1] after detection, [2] after redistribute-and-quantize,
- * [3] after the GEMM (or decode) kernel.  Same results as muxq_linear.
+ * events[0] at entry, [1] after the workspace clear (start of the fused detect + redistribute +
+ * quantize kernel), [2] after that kernel, [3] after the GEMM (or decode) kernel.  When `stream`
+ * is being captured into a CUDA graph the records become event-record nodes, re-recorded by every
+ * replay.  Same results as muxq_linear.
  */
 int muxq_linear_events(const void *X_f16, int M, int K, int ldx, const int8_t *W_q, int ldw,
                        const float *s_w, int N, const muxq_params *p, void *Y, int ldy, int out_kind,

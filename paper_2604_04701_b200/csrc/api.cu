@@ -39,7 +39,7 @@ SmallWs small_ws(int cols) {
 // muxq_linear workspace: the small block, then per-token scales, Body_q, Aux_q, W_aux.
 struct LinearWs {
     SmallWs s;
-    size_t sx_rows, body_q, aux_q, w_aux, total;
+    size_t colmax_rep, sx_rows, body_q, aux_q, w_aux, total;
     int ld_q, aux_cols;
 };
 LinearWs linear_ws(int M, int K, int N, const muxq_params *p) {
@@ -47,6 +47,11 @@ LinearWs linear_ws(int M, int K, int N, const muxq_params *p) {
     w.s = small_ws(K);
     w.aux_cols = muxq_aux_cols(p);
     w.ld_q = K;
+    // The replicated abs-max accumulators of the fused kernel sit right behind ctrl | colmax so that
+    // one memset clears all three; the other small arrays follow.
+    w.colmax_rep = align_up(w.s.colmax + (size_t)K * 4, 256);
+    const size_t shift = align_up(w.colmax_rep + (size_t)kPrepColmaxReplicas * K * 4, 256) - w.s.colmul;
+    w.s.colmul += shift; w.s.grpflag += shift; w.s.oidx += shift; w.s.total += shift;
     w.sx_rows = w.s.total;
     w.body_q = align_up(w.sx_rows + (size_t)M * 4, 1024);
     w.aux_q = align_up(w.body_q + (size_t)M * w.ld_q, 1024);
@@ -268,58 +273,86 @@ static int linear_impl(const void *X, int M, int K, int ldx, const int8_t *W_q, 
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     uint8_t *ws = static_cast<uint8_t *>(workspace);
 
-    cudaError_t e = cudaMemsetAsync(ws, 0, w.s.colmax + (size_t)K * 4, s);
-    if (e == cudaSuccess) e = cudaMemsetAsync(dev_status, 0, 4, s);
-    if (e != cudaSuccess) return MUXQ_ERR_CUDA;
-
     const bool per_vec = p->gran == MUXQ_PER_VECTOR;
     const bool decode = M <= 16;
+    const bool fused = prep_supported(M, K);
     Ctrl *ctrl = reinterpret_cast<Ctrl *>(ws);
+    // inside a stream capture the records become event-record nodes that every replay re-records
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    if (events) cudaStreamIsCapturing(s, &cap);
+    const unsigned ev_flags = cap == cudaStreamCaptureStatusActive ? cudaEventRecordExternal : cudaEventRecordDefault;
     auto mark = [&](int i) {
-        if (events && events[i]) cudaEventRecord(static_cast<cudaEvent_t>(events[i]), s);
+        if (events && events[i]) cudaEventRecordWithFlags(static_cast<cudaEvent_t>(events[i]), s, ev_flags);
     };
     mark(0);
-
-    DetectArgs d{};
-    d.X = static_cast<const __half *>(X);
-    d.M = M; d.K = K; d.ldx = ldx;
-    d.tau = p->threshold; d.exp_factor = p->exp_factor; d.qmax = qmax_of(p->act_bits); d.cap = p->max_outliers;
-    d.colmax_bits = reinterpret_cast<uint32_t *>(ws + w.s.colmax);
-    d.ctrl = ctrl;
-    d.outlier_idx = reinterpret_cast<int32_t *>(ws + w.s.oidx);
-    d.colmul = reinterpret_cast<float *>(ws + w.s.colmul);
-    d.grpflag = ws + w.s.grpflag;
-    d.dev_status = dev_status;
-    e = launch_detect(d, s);
+    cudaError_t e = cudaMemsetAsync(ws, 0, fused ? w.colmax_rep + (size_t)kPrepColmaxReplicas * K * 4
+                                                 : w.s.colmax + (size_t)K * 4, s);
+    if (e == cudaSuccess && !fused) e = cudaMemsetAsync(dev_status, 0, 4, s);  // the fused kernel clears it itself
     if (e != cudaSuccess) return MUXQ_ERR_CUDA;
     mark(1);
 
-    QuantActArgs q{};
-    q.X = d.X; q.M = M; q.K = K; q.ldx = ldx;
-    q.exp_factor = p->exp_factor; q.qmax = d.qmax; q.cap = p->max_outliers; q.per_token = per_vec;
-    q.outlier_idx = d.outlier_idx;
-    q.n_outliers = &ctrl->n_outliers;
-    q.colmul = d.colmul; q.grpflag = d.grpflag;
-    q.s_x_tensor = &ctrl->s_x;
-    q.inv_s_x_tensor = &ctrl->inv_s_x;
-    q.s_x_rows = reinterpret_cast<float *>(ws + w.sx_rows);
-    q.body_q = reinterpret_cast<int8_t *>(ws + w.body_q); q.ld_q = w.ld_q;
-    if (!decode) {
-        q.aux_q = reinterpret_cast<int8_t *>(ws + w.aux_q); q.ld_aux = w.aux_cols; q.aux_cols = w.aux_cols;
-        q.w_q = W_q; q.ldw = ldw; q.N = N;
-        q.w_aux = reinterpret_cast<int8_t *>(ws + w.w_aux); q.ld_waux = w.aux_cols;
+    int32_t *oidx = reinterpret_cast<int32_t *>(ws + w.s.oidx);
+    float *s_x_rows = reinterpret_cast<float *>(ws + w.sx_rows);
+    int8_t *body_q = reinterpret_cast<int8_t *>(ws + w.body_q);
+    int8_t *aux_q = decode ? nullptr : reinterpret_cast<int8_t *>(ws + w.aux_q);
+    int8_t *w_aux = decode ? nullptr : reinterpret_cast<int8_t *>(ws + w.w_aux);
+    if (fused) {
+        PrepArgs f{};
+        f.X = static_cast<const __half *>(X);
+        f.M = M; f.K = K; f.ldx = ldx;
+        f.tau = p->threshold; f.exp_factor = p->exp_factor; f.qmax = qmax_of(p->act_bits);
+        f.cap = p->max_outliers; f.per_token = per_vec;
+        f.colmax_rep = reinterpret_cast<uint32_t *>(ws + w.colmax_rep);
+        f.colmax_bits = reinterpret_cast<uint32_t *>(ws + w.s.colmax);
+        f.ctrl = ctrl;
+        f.outlier_idx = oidx;
+        f.s_x_rows = s_x_rows;
+        f.body_q = body_q; f.ld_q = w.ld_q;
+        f.aux_q = aux_q; f.ld_aux = w.aux_cols; f.aux_cols = w.aux_cols;
+        if (!decode) { f.w_q = W_q; f.ldw = ldw; f.N = N; f.w_aux = w_aux; f.ld_waux = w.aux_cols; }
+        f.dev_status = dev_status;
+        e = launch_prep(f, s);
+        if (e != cudaSuccess) return MUXQ_ERR_CUDA;
+    } else {
+        DetectArgs d{};
+        d.X = static_cast<const __half *>(X);
+        d.M = M; d.K = K; d.ldx = ldx;
+        d.tau = p->threshold; d.exp_factor = p->exp_factor; d.qmax = qmax_of(p->act_bits); d.cap = p->max_outliers;
+        d.colmax_bits = reinterpret_cast<uint32_t *>(ws + w.s.colmax);
+        d.ctrl = ctrl;
+        d.outlier_idx = oidx;
+        d.colmul = reinterpret_cast<float *>(ws + w.s.colmul);
+        d.grpflag = ws + w.s.grpflag;
+        d.dev_status = dev_status;
+        e = launch_detect(d, s);
+        if (e != cudaSuccess) return MUXQ_ERR_CUDA;
+        QuantActArgs q{};
+        q.X = d.X; q.M = M; q.K = K; q.ldx = ldx;
+        q.exp_factor = p->exp_factor; q.qmax = d.qmax; q.cap = p->max_outliers; q.per_token = per_vec;
+        q.outlier_idx = oidx;
+        q.n_outliers = &ctrl->n_outliers;
+        q.colmul = d.colmul; q.grpflag = d.grpflag;
+        q.s_x_tensor = &ctrl->s_x;
+        q.inv_s_x_tensor = &ctrl->inv_s_x;
+        q.s_x_rows = s_x_rows;
+        q.body_q = body_q; q.ld_q = w.ld_q;
+        if (!decode) {
+            q.aux_q = aux_q; q.ld_aux = w.aux_cols; q.aux_cols = w.aux_cols;
+            q.w_q = W_q; q.ldw = ldw; q.N = N;
+            q.w_aux = w_aux; q.ld_waux = w.aux_cols;
+        }
+        e = launch_quant_act(q, s);
+        if (e != cudaSuccess) return MUXQ_ERR_CUDA;
     }
-    e = launch_quant_act(q, s);
-    if (e != cudaSuccess) return MUXQ_ERR_CUDA;
     mark(2);
 
-    const float *s_x = per_vec ? q.s_x_rows : &ctrl->s_x;
+    const float *s_x = per_vec ? s_x_rows : &ctrl->s_x;
     const int c = (1 << p->exp_factor) - 1;
     if (decode) {
         DecodeArgs k{};
-        k.body_q = q.body_q; k.ld_a = w.ld_q;
+        k.body_q = body_q; k.ld_a = w.ld_q;
         k.w_q = W_q; k.ldw = ldw;
-        k.outlier_idx = d.outlier_idx; k.n_outliers = &ctrl->n_outliers;
+        k.outlier_idx = oidx; k.n_outliers = &ctrl->n_outliers;
         k.M = M; k.K = K; k.N = N; k.c = c; k.cap = p->max_outliers;
         k.s_x = s_x; k.s_x_per_row = per_vec;
         k.s_w = s_w; k.s_w_per_col = per_vec;
@@ -329,10 +362,10 @@ static int linear_impl(const void *X, int M, int K, int ldx, const int8_t *W_q, 
         return cuda_rc(e);
     }
     GemmArgs g{};
-    g.body_q = q.body_q; g.ld_a = w.ld_q;
-    g.aux_q = q.aux_q; g.ld_aux = w.aux_cols;
+    g.body_q = body_q; g.ld_a = w.ld_q;
+    g.aux_q = aux_q; g.ld_aux = w.aux_cols;
     g.w_q = W_q; g.ldw = ldw;
-    g.w_aux = q.w_aux; g.ld_waux = w.aux_cols;
+    g.w_aux = w_aux; g.ld_waux = w.aux_cols;
     g.n_outliers = &ctrl->n_outliers;
     g.M = M; g.K = K; g.N = N; g.c = c; g.cap = p->max_outliers; g.aux_cols = w.aux_cols;
     g.s_x = s_x; g.s_x_per_row = per_vec;

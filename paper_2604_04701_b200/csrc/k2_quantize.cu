@@ -7,6 +7,7 @@
 // true fp32 division bit for bit; a reciprocal multiply pre-screens the (common) values that are
 // provably far from a rounding tie, the rest take the division.
 #include "kernels.h"
+#include "quant.cuh"
 
 namespace muxq {
 
@@ -14,61 +15,6 @@ namespace {
 
 constexpr int kThreads = 256;
 constexpr int kWarps = kThreads / 32;
-
-__device__ __forceinline__ float warp_max(float v) {
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
-    return v;
-}
-
-// Eq. 1: code = clamp(round_half_even(v / s), -q, q) with a true fp32 division.
-__device__ __forceinline__ int quant_exact(float v, float s, float qf) {
-    float t = rintf(__fdiv_rn(v, s));
-    t = fminf(fmaxf(t, -qf), qf);
-    return __float2int_rn(t);
-}
-
-// The same code, cheaper: t = v * (1/s) differs from the correctly rounded quotient by less than
-// 2.3e-5 for |v/s| <= 128, so whenever t is farther than 1e-4 from every half-integer both round
-// to the same integer.  Returns false when t is too close to a tie; the caller then takes the
-// exact division.
-__device__ __forceinline__ bool quant_screen(float v, float inv_s, float qf, int &code) {
-    const float t = v * inv_s;
-    float n = rintf(t);
-    const bool safe = (0.5f - fabsf(t - n)) > 1e-4f;
-    n = fminf(fmaxf(n, -qf), qf);
-    code = __float2int_rn(n);
-    return safe;
-}
-
-__device__ __forceinline__ void unpack8(const uint4 &v, float (&f)[8]) {
-    const __half2 *h = reinterpret_cast<const __half2 *>(&v);
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        float2 p = __half22float2(h[i]);
-        f[2 * i] = p.x;
-        f[2 * i + 1] = p.y;
-    }
-}
-
-// 8 values (already multiplied by their channel factors) -> 8 codes packed in a uint2
-__device__ __forceinline__ uint2 quant8(const float (&f)[8], float s, float inv_s, float qf) {
-    int c[8];
-    bool safe = true;
-#pragma unroll
-    for (int i = 0; i < 8; ++i) safe &= quant_screen(f[i], inv_s, qf, c[i]);
-    if (!safe) {
-#pragma unroll
-        for (int i = 0; i < 8; ++i) c[i] = quant_exact(f[i], s, qf);
-    }
-    uint32_t lo = 0, hi = 0;
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        lo |= (uint32_t)(c[i] & 0xff) << (8 * i);
-        hi |= (uint32_t)(c[4 + i] & 0xff) << (8 * i);
-    }
-    return make_uint2(lo, hi);
-}
 
 // Aux block word w of row xr: columns 4w..4w+3, column c*j + t holds the code of Body[m, O_j]
 __device__ __forceinline__ uint32_t aux_word(const __half *xr, const int32_t *oidx, int w, int c, int r, float down,

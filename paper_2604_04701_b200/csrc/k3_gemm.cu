@@ -66,12 +66,11 @@ struct GemmParams {
 template <int kOut, bool kPerVec>
 __device__ __forceinline__ void convert_chunk(const uint32_t (&v)[32], uint4 *srow, int piece0, uint32_t sw_xor,
                                               float sx, float sxw, const float *s_w_col, int cols_left) {
-    if (kOut == kOutI32) {
+    if constexpr (kOut == kOutI32) {
 #pragma unroll
         for (int g = 0; g < 8; ++g)
             srow[(piece0 + g) ^ sw_xor] = make_uint4(v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
-        return;
-    }
+    } else {
     float f[32];
 #pragma unroll
     for (int g = 0; g < 8; ++g) {
@@ -104,6 +103,7 @@ __device__ __forceinline__ void convert_chunk(const uint32_t (&v)[32], uint4 *sr
             o.z = *reinterpret_cast<const uint32_t *>(&h2); o.w = *reinterpret_cast<const uint32_t *>(&h3);
             srow[(piece0 + g) ^ sw_xor] = o;
         }
+    }
     }
 }
 

@@ -13,7 +13,8 @@ struct Ctrl {
     int32_t n_outliers;    // r, true count of outlier channels
     float s_x;             // per-tensor Body scale (Eq. 1)
     float inv_s_x;         // 1 / s_x, correctly rounded (used only to pre-screen the exact division)
-    uint32_t reserved[60];
+    uint32_t arrived;      // fused prep kernel: CTAs that have reached the grid-wide barrier
+    uint32_t reserved[59];
 };
 static_assert(sizeof(Ctrl) == 256, "Ctrl is one 256-byte block");
 
@@ -56,6 +57,28 @@ struct QuantActArgs {
     int8_t *w_aux; int ld_waux;
 };
 cudaError_t launch_quant_act(const QuantActArgs &a, cudaStream_t s);
+
+// Fused detect + redistribute + quantize (one cooperative launch, X read from HBM once).
+constexpr int kPrepColmaxReplicas = 8;
+struct PrepArgs {
+    const __half *X;
+    int M, K, ldx;
+    float tau;
+    int exp_factor, qmax, cap, per_token;
+    uint32_t *colmax_rep;    // [kPrepColmaxReplicas, K] zero-initialised accumulators
+    uint32_t *colmax_bits;   // [K] out: channel abs-max (bit patterns of non-negative floats)
+    Ctrl *ctrl;              // zero-initialised
+    int32_t *outlier_idx;    // [cap] out
+    float *s_x_rows;         // [M] out when per_token
+    int8_t *body_q;  int ld_q;
+    int8_t *aux_q;   int ld_aux; int aux_cols;   // aux_q may be NULL (decode path)
+    const int8_t *w_q; int ldw; int N;           // W_aux gather (all NULL/0 to skip)
+    int8_t *w_aux; int ld_waux;
+    int32_t *dev_status;     // set to 0 at kernel start, raised on r > cap or a barrier time-out
+};
+// False when the shape does not fit the fused kernel (the caller then uses the separate kernels).
+bool prep_supported(int M, int K);
+cudaError_t launch_prep(const PrepArgs &a, cudaStream_t s);
 
 struct QuantWeightArgs {
     const __half *W;  // [K,N]
