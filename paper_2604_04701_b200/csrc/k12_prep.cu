@@ -1,0 +1,354 @@
+// Fused activation preparation for muxq_linear: per-channel abs-max and outlier detection
+// (Section III-C), the redistribution of Eq. 4-5 and the abs-max quantization of Eq. 1, in ONE
+// launch that reads X from HBM once.
+//
+// The per-tensor scale and the outlier set depend on every row of X, so the kernel has two passes
+// separated by a grid-wide barrier.  It is launched cooperatively with one CTA per SM; CTA b owns a
+// contiguous slab of token rows and keeps it in shared memory between the passes (a slab of
+// M/148 rows x K fp16 fits for the GPT-2 shapes; rows that do not fit are re-read, normally from L2):
+//   pass 1  stream the slab (128-bit loads, a thread owns 8 channels and walks down the rows),
+//           stash it in shared memory, merge channel maxima CTA-wide in shared memory and then
+//           device-wide with integer atomicMax on the bit patterns (maxima of non-negative floats
+//           are order independent, so the result is exact).  The device-wide accumulators are
+//           replicated kColmaxReplicas times (CTA b uses copy b mod R): same-address atomics
+//           serialise in L2, and one copy would take 148 of them per channel
+//   barrier bounded spin on an arrival counter; a time-out raises MUXQ_ERR_TIMEOUT and returns
+//   pass 2  every CTA derives O, the channel factors and s_X from the K maxima (cheap, redundant),
+//           then quantizes its slab out of shared memory, one warp per token row, writing Body_q,
+//           the Aux block and (spread over the grid) the gathered W_aux rows.
+#include "kernels.h"
+#include "quant.cuh"
+
+namespace muxq {
+
+namespace {
+
+constexpr int kT = 1024;
+constexpr int kWarps = kT / 32;
+constexpr int kMaxK = 8 * kT;  // one group of 8 channels per thread
+constexpr int kMaxOut = 64;
+constexpr int kColmaxReplicas = kPrepColmaxReplicas;
+constexpr int kStatusCapacity = 5;  // MUXQ_ERR_CAPACITY
+constexpr int kStatusTimeout = 6;   // MUXQ_ERR_TIMEOUT
+constexpr uint32_t kBarrierSpin = 1u << 21;
+constexpr int kMaxDynSmem = 227 * 1024 - 1024;
+
+__host__ __device__ inline int fixed_smem_bytes(int K) {
+    const int G = K >> 3;
+    return 8 * K + ((G + 15) & ~15) + kMaxOut * 4;  // colmul | colmax | group flags | outlier indices
+}
+
+__device__ __forceinline__ uint32_t ld_acquire_u32(const uint32_t *p) {
+    uint32_t v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+
+__device__ __forceinline__ void absmax4(__half2 (&m)[4], const uint4 &v) {
+    m[0] = __hmax2(m[0], __habs2(*reinterpret_cast<const __half2 *>(&v.x)));
+    m[1] = __hmax2(m[1], __habs2(*reinterpret_cast<const __half2 *>(&v.y)));
+    m[2] = __hmax2(m[2], __habs2(*reinterpret_cast<const __half2 *>(&v.z)));
+    m[3] = __hmax2(m[3], __habs2(*reinterpret_cast<const __half2 *>(&v.w)));
+}
+
+// 8 values of one 16-byte chunk, channel factors applied when the group holds an outlier channel
+__device__ __forceinline__ void load_chunk(const uint4 *src, int ch, const uint8_t *flag, const float *colmul,
+                                           float (&f)[8]) {
+    const uint4 v = src[ch];
+    unpack8(v, f);
+    if (flag[ch]) {
+        const float4 m0 = reinterpret_cast<const float4 *>(colmul)[2 * ch];
+        const float4 m1 = reinterpret_cast<const float4 *>(colmul)[2 * ch + 1];
+        f[0] *= m0.x; f[1] *= m0.y; f[2] *= m0.z; f[3] *= m0.w;  // 1 or 2^-e: exact
+        f[4] *= m1.x; f[5] *= m1.y; f[6] *= m1.z; f[7] *= m1.w;
+    }
+}
+
+__global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, int rows_base, int rows_extra, int slab_bytes) {
+    extern __shared__ __align__(16) uint8_t smem[];
+    __shared__ int s_warp_cnt[kWarps];
+    __shared__ float s_warp_max[kWarps];
+    __shared__ float s_scale[2];
+    __shared__ int s_fail;
+
+    const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
+    const int K = a.K, G = K >> 3;
+    float *s_colmul = reinterpret_cast<float *>(smem);
+    uint32_t *s_colmax = reinterpret_cast<uint32_t *>(smem + 4 * K);
+    uint8_t *s_flag = smem + 8 * K;
+    int32_t *s_oidx = reinterpret_cast<int32_t *>(smem + 8 * K + ((G + 15) & ~15));
+    uint8_t *slab = smem + fixed_smem_bytes(K);
+
+    const int b = blockIdx.x;
+    const int r0 = b * rows_base + min(b, rows_extra);
+    const int rows = rows_base + (b < rows_extra ? 1 : 0);
+    const int fit = min(rows, slab_bytes / (2 * K));
+    if (b == 0 && t == 0 && a.dev_status) *a.dev_status = 0;
+
+    // ---------------------------------------------------------------- pass 1: channel maxima
+    for (int k = t; k < K; k += kT) s_colmax[k] = 0u;
+    __syncthreads();
+    {
+        const int rstride = kT / G;  // G <= kT: thread = (row offset, channel group)
+        const int cg = t % G, row_off = t / G;
+        if (row_off < rstride) {
+            __half2 m[4];
+            m[0] = m[1] = m[2] = m[3] = __float2half2_rn(0.f);
+            const __half *px = a.X + (size_t)r0 * a.ldx + cg * 8;
+            uint8_t *ps = slab + cg * 16;
+            // up to 8 independent 16-byte loads in flight per thread
+            for (int row = row_off; row < rows; row += 8 * rstride) {
+                uint4 v[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    const int rr = row + u * rstride;
+                    v[u] = rr < rows ? __ldg(reinterpret_cast<const uint4 *>(px + (size_t)rr * a.ldx))
+                                     : make_uint4(0u, 0u, 0u, 0u);
+                }
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    absmax4(m, v[u]);
+                    const int rr = row + u * rstride;
+                    if (rr < fit) *reinterpret_cast<uint4 *>(ps + (size_t)rr * K * 2) = v[u];
+                }
+            }
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const float lo = __low2float(m[i]), hi = __high2float(m[i]);
+                if (lo > 0.0f) atomicMax(&s_colmax[cg * 8 + 2 * i], __float_as_uint(lo));
+                if (hi > 0.0f) atomicMax(&s_colmax[cg * 8 + 2 * i + 1], __float_as_uint(hi));
+            }
+        }
+    }
+    __syncthreads();
+    {
+        uint32_t *rep = a.colmax_rep + (size_t)(b % kColmaxReplicas) * K;
+        for (int k = t; k < K; k += kT) {
+            const uint32_t v = s_colmax[k];
+            // a CTA that finds the running maximum already at or above its own skips the atomic
+            if (v != 0u && v > __ldcg(rep + k)) atomicMax(rep + k, v);
+        }
+    }
+
+    // ---------------------------------------------------------------- grid-wide barrier (bounded)
+    __threadfence();
+    __syncthreads();
+    if (t == 0) {
+        atomicAdd(&a.ctrl->arrived, 1u);
+        bool ok = false;
+        for (uint32_t i = 0; i < kBarrierSpin; ++i) {
+            if (ld_acquire_u32(&a.ctrl->arrived) >= gridDim.x) { ok = true; break; }
+            __nanosleep(32);
+        }
+        s_fail = ok ? 0 : 1;
+        if (!ok && a.dev_status) atomicMax(a.dev_status, kStatusTimeout);
+    }
+    __syncthreads();
+    if (s_fail) return;
+
+    // ---------------------------------------------------------------- O, channel factors, s_X (every CTA)
+    const float down = exp2f(-(float)a.exp_factor);
+    const float qf = (float)a.qmax;
+    int r_true;
+    {
+        // channel maxima = max over the replicas, fetched with coalesced 16-byte loads
+        for (int k4 = t; k4 < (K >> 2); k4 += kT) {
+            uint4 v[kColmaxReplicas];
+#pragma unroll
+            for (int rp = 0; rp < kColmaxReplicas; ++rp)
+                v[rp] = __ldcg(reinterpret_cast<const uint4 *>(a.colmax_rep + (size_t)rp * K) + k4);
+            uint4 mx = v[0];
+#pragma unroll
+            for (int rp = 1; rp < kColmaxReplicas; ++rp) {
+                mx.x = max(mx.x, v[rp].x); mx.y = max(mx.y, v[rp].y);
+                mx.z = max(mx.z, v[rp].z); mx.w = max(mx.w, v[rp].w);
+            }
+            reinterpret_cast<uint4 *>(s_colmax)[k4] = mx;
+            if (b == 0) reinterpret_cast<uint4 *>(a.colmax_bits)[k4] = mx;
+        }
+        __syncthreads();
+        const bool active = t < G;  // thread t owns channels [8t, 8t+8)
+        float cm[8];
+        if (active) {
+            const float4 v0 = reinterpret_cast<const float4 *>(s_colmax)[2 * t];
+            const float4 v1 = reinterpret_cast<const float4 *>(s_colmax)[2 * t + 1];
+            cm[0] = v0.x; cm[1] = v0.y; cm[2] = v0.z; cm[3] = v0.w;
+            cm[4] = v1.x; cm[5] = v1.y; cm[6] = v1.z; cm[7] = v1.w;
+        } else {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) cm[i] = 0.0f;
+        }
+        int cnt = 0;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) cnt += (cm[i] > a.tau) ? 1 : 0;
+        int incl = cnt;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int n = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += n;
+        }
+        if (lane == 31) s_warp_cnt[warp] = incl;
+        __syncthreads();
+        int before = 0, total = 0;
+#pragma unroll
+        for (int w = 0; w < kWarps; ++w) {
+            const int c = s_warp_cnt[w];
+            if (w < warp) before += c;
+            total += c;
+        }
+        r_true = total;
+        int pos = before + incl - cnt;
+        float bmax = 0.0f;
+        if (active) {
+            float mul[8];
+            uint8_t gf = 0;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                mul[i] = 1.0f;
+                if (cm[i] > a.tau) {  // strict: |x| == threshold does not flag the channel
+                    if (pos < a.cap) {
+                        s_oidx[pos] = 8 * t + i;
+                        if (b == 0) a.outlier_idx[pos] = 8 * t + i;
+                        mul[i] = down;
+                        gf = 1;
+                    }
+                    ++pos;
+                }
+                bmax = fmaxf(bmax, cm[i] * mul[i]);  // power-of-two scaling: exact
+            }
+            reinterpret_cast<float4 *>(s_colmul)[2 * t] = make_float4(mul[0], mul[1], mul[2], mul[3]);
+            reinterpret_cast<float4 *>(s_colmul)[2 * t + 1] = make_float4(mul[4], mul[5], mul[6], mul[7]);
+            s_flag[t] = gf;
+        }
+        bmax = warp_max(bmax);
+        if (lane == 0) s_warp_max[warp] = bmax;
+        __syncthreads();
+        if (t == 0) {
+            float mx = 0.0f;
+#pragma unroll
+            for (int w = 0; w < kWarps; ++w) mx = fmaxf(mx, s_warp_max[w]);
+            const float s = mx > 0.0f ? __fdiv_rn(mx, qf) : 1.0f;  // Eq. 1
+            s_scale[0] = s;
+            s_scale[1] = __fdiv_rn(1.0f, s);
+            if (b == 0) {
+                a.ctrl->s_x = s;
+                a.ctrl->inv_s_x = s_scale[1];
+                a.ctrl->n_outliers = total;
+                if (total > a.cap && a.dev_status) atomicMax(a.dev_status, kStatusCapacity);
+            }
+        }
+        __syncthreads();
+    }
+    const int r = min(r_true, a.cap);
+    const int c = (1 << a.exp_factor) - 1;
+    const int used_words = (c * r + 3) >> 2;
+    // W_aux[n, c*j + t] = W_q[n, O_j], one 4-byte word per thread and round, spread over the grid.
+    // The first round's scattered byte loads are issued here and consumed after pass 2, which hides
+    // their latency behind the quantization work.
+    const int wa_words_per_row = a.aux_cols >> 2;
+    const int wa_total = a.w_aux ? a.N * wa_words_per_row : 0;
+    const int wa_first = b * kT + t;
+    uint8_t wa_byte[4] = {0, 0, 0, 0};
+    if (wa_first < wa_total) {
+        const int n = wa_first / wa_words_per_row, w = wa_first - n * wa_words_per_row;
+        if (w < used_words) {
+#pragma unroll
+            for (int bb = 0; bb < 4; ++bb) {
+                const int j = (w * 4 + bb) / c;
+                if (j < r) wa_byte[bb] = (uint8_t)a.w_q[(size_t)n * a.ldw + s_oidx[j]];
+            }
+        }
+    }
+
+    // ---------------------------------------------------------------- pass 2: Body_q and the Aux block
+    for (int row = warp; row < rows; row += kWarps) {
+        const size_t m = (size_t)r0 + row;
+        const uint4 *src = row < fit ? reinterpret_cast<const uint4 *>(slab + (size_t)row * K * 2)
+                                     : reinterpret_cast<const uint4 *>(a.X + m * a.ldx);
+        float s = s_scale[0], inv_s = s_scale[1];
+        if (a.per_token) {
+            // per-token scale from Body's row (after the 2^-e redistribution)
+            float mx = 0.0f;
+            for (int ch = lane; ch < G; ch += 32) {
+                float f[8];
+                load_chunk(src, ch, s_flag, s_colmul, f);
+#pragma unroll
+                for (int i = 0; i < 8; ++i) mx = fmaxf(mx, fabsf(f[i]));
+            }
+            mx = warp_max(mx);
+            s = mx > 0.0f ? __fdiv_rn(mx, qf) : 1.0f;
+            inv_s = __fdiv_rn(1.0f, s);
+            if (lane == 0) a.s_x_rows[m] = s;
+        }
+        int8_t *q = a.body_q + m * a.ld_q;
+        for (int ch = lane; ch < G; ch += 32) {
+            float f[8];
+            load_chunk(src, ch, s_flag, s_colmul, f);
+            *reinterpret_cast<uint2 *>(q + ch * 8) = quant8(f, s, inv_s, qf);
+        }
+        if (a.aux_q) {
+            const __half *xr = reinterpret_cast<const __half *>(src);
+            for (int w = lane; w < (a.aux_cols >> 2); w += 32) {
+                uint32_t packed = 0;
+                if (w < used_words) {
+#pragma unroll
+                    for (int bb = 0; bb < 4; ++bb) {
+                        const int j = (w * 4 + bb) / c;  // column c*j + t holds the code of Body[m, O_j] (Eq. 5)
+                        if (j < r) {
+                            const float v = __half2float(xr[s_oidx[j]]) * down;
+                            packed |= (uint32_t)(quant_exact(v, s, qf) & 0xff) << (8 * bb);
+                        }
+                    }
+                }
+                *reinterpret_cast<uint32_t *>(a.aux_q + m * a.ld_aux + w * 4) = packed;
+            }
+        }
+    }
+
+    // ---------------------------------------------------------------- W_aux: first round, then the rest
+    if (wa_first < wa_total) {
+        const int n = wa_first / wa_words_per_row, w = wa_first - n * wa_words_per_row;
+        const uint32_t packed = (uint32_t)wa_byte[0] | ((uint32_t)wa_byte[1] << 8) | ((uint32_t)wa_byte[2] << 16) |
+                                ((uint32_t)wa_byte[3] << 24);
+        *reinterpret_cast<uint32_t *>(a.w_aux + (size_t)n * a.ld_waux + w * 4) = packed;
+    }
+    for (int i = wa_first + gridDim.x * kT; i < wa_total; i += gridDim.x * kT) {
+        const int n = i / wa_words_per_row, w = i - n * wa_words_per_row;
+        uint32_t packed = 0;
+        if (w < used_words) {
+#pragma unroll
+            for (int bb = 0; bb < 4; ++bb) {
+                const int j = (w * 4 + bb) / c;
+                if (j < r) packed |= (uint32_t)(uint8_t)a.w_q[(size_t)n * a.ldw + s_oidx[j]] << (8 * bb);
+            }
+        }
+        *reinterpret_cast<uint32_t *>(a.w_aux + (size_t)n * a.ld_waux + w * 4) = packed;
+    }
+}
+
+}  // namespace
+
+bool prep_supported(int M, int K) { return M >= 1 && K >= 8 && K % 8 == 0 && K <= kMaxK; }
+
+cudaError_t launch_prep(const PrepArgs &a, cudaStream_t s) {
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(k_prep, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem);
+        if (e != cudaSuccess) return e;
+        attr_set = true;
+    }
+    int grid = num_sms();
+    if (grid > a.M) grid = a.M;
+    int rows_base = a.M / grid, rows_extra = a.M % grid;
+    const int rows_max = rows_base + (rows_extra ? 1 : 0);
+    const int fixed = fixed_smem_bytes(a.K);
+    const long long want = (long long)rows_max * a.K * 2;
+    int slab_bytes = (int)(want < (long long)(kMaxDynSmem - fixed) ? want : (long long)(kMaxDynSmem - fixed));
+    slab_bytes &= ~15;
+    PrepArgs args = a;
+    void *params[] = {&args, &rows_base, &rows_extra, &slab_bytes};
+    return cudaLaunchCooperativeKernel(reinterpret_cast<const void *>(k_prep), dim3(grid), dim3(kT), params,
+                                       (size_t)(fixed + slab_bytes), s);
+}
+
+}  // namespace muxq

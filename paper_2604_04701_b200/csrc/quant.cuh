@@ -1,0 +1,62 @@
+// Device helpers shared by the activation-quantization kernels: Eq. 1 codes equal to
+// round_half_even(v / s) with a true fp32 division (bit for bit), and fp16 unpacking.
+#pragma once
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace muxq {
+
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+}
+
+// Eq. 1: code = clamp(round_half_even(v / s), -q, q) with a true fp32 division.
+__device__ __forceinline__ int quant_exact(float v, float s, float qf) {
+    float t = rintf(__fdiv_rn(v, s));
+    t = fminf(fmaxf(t, -qf), qf);
+    return __float2int_rn(t);
+}
+
+__device__ __forceinline__ void unpack8(const uint4 &v, float (&f)[8]) {
+    const __half2 *h = reinterpret_cast<const __half2 *>(&v);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        float2 p = __half22float2(h[i]);
+        f[2 * i] = p.x;
+        f[2 * i + 1] = p.y;
+    }
+}
+
+// 8 values (already multiplied by their channel factors) -> 8 codes packed in a uint2.
+//
+// Fast path: t = v * (1/s) differs from the correctly rounded quotient v / s by less than 2.3e-5
+// for |v/s| <= 128, so whenever t is farther than 1e-4 from every half-integer both round to the
+// same integer.  Adding 1.5 * 2^23 rounds t to that integer (round half to even) and leaves its
+// two's-complement low byte in the low byte of the float's bit pattern, which a byte permute packs
+// directly.  If any of the 8 values is too close to a tie, or exceeds the code range (possible
+// only when the scale was not derived from these values), all 8 take the exact division.
+__device__ __forceinline__ uint2 quant8(const float (&f)[8], float s, float inv_s, float qf) {
+    const float magic = 12582912.0f;  // 1.5 * 2^23
+    uint32_t b[8];
+    float dmax = 0.0f, amax = 0.0f;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const float t = f[i] * inv_s;
+        const float tm = t + magic;
+        dmax = fmaxf(dmax, fabsf(t - (tm - magic)));
+        amax = fmaxf(amax, fabsf(t));
+        b[i] = __float_as_uint(tm);
+    }
+    if (dmax > 0.4999f || amax > qf + 0.25f) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) b[i] = (uint32_t)quant_exact(f[i], s, qf);
+    }
+    const uint32_t p01 = __byte_perm(b[0], b[1], 0x0040), p23 = __byte_perm(b[2], b[3], 0x0040);
+    const uint32_t p45 = __byte_perm(b[4], b[5], 0x0040), p67 = __byte_perm(b[6], b[7], 0x0040);
+    return make_uint2(__byte_perm(p01, p23, 0x5410), __byte_perm(p45, p67, 0x5410));
+}
+
+}  // namespace muxq
