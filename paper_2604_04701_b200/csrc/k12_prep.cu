@@ -27,6 +27,7 @@ constexpr int kT = 1024;
 constexpr int kWarps = kT / 32;
 constexpr int kMaxK = 8 * kT;  // one group of 8 channels per thread
 constexpr int kMaxOut = 64;
+constexpr int kMaxAuxCols = 512;  // (2^3 - 1) * 64 rounded up to 128
 constexpr int kColmaxReplicas = kPrepColmaxReplicas;
 constexpr int kStatusCapacity = 5;  // MUXQ_ERR_CAPACITY
 constexpr int kStatusTimeout = 6;   // MUXQ_ERR_TIMEOUT
@@ -35,7 +36,8 @@ constexpr int kMaxDynSmem = 227 * 1024 - 1024;
 
 __host__ __device__ inline int fixed_smem_bytes(int K) {
     const int G = K >> 3;
-    return 8 * K + ((G + 15) & ~15) + kMaxOut * 4;  // colmul | colmax | group flags | outlier indices
+    // colmul | colmax | group flags | outlier indices | source channel of every Aux column
+    return 8 * K + ((G + 15) & ~15) + kMaxOut * 4 + kMaxAuxCols * 2;
 }
 
 __device__ __forceinline__ uint32_t ld_acquire_u32(const uint32_t *p) {
@@ -77,6 +79,7 @@ __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, int rows_base,
     uint32_t *s_colmax = reinterpret_cast<uint32_t *>(smem + 4 * K);
     uint8_t *s_flag = smem + 8 * K;
     int32_t *s_oidx = reinterpret_cast<int32_t *>(smem + 8 * K + ((G + 15) & ~15));
+    uint16_t *s_auxsrc = reinterpret_cast<uint16_t *>(s_oidx + kMaxOut);
     uint8_t *slab = smem + fixed_smem_bytes(K);
 
     const int b = blockIdx.x;
@@ -124,22 +127,23 @@ __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, int rows_base,
     {
         uint32_t *rep = a.colmax_rep + (size_t)(b % kColmaxReplicas) * K;
         for (int k = t; k < K; k += kT) {
+            // a warp's 32 consecutive channels travel as one 128-byte reduction request
             const uint32_t v = s_colmax[k];
-            // a CTA that finds the running maximum already at or above its own skips the atomic
-            if (v != 0u && v > __ldcg(rep + k)) atomicMax(rep + k, v);
+            if (v != 0u) atomicMax(rep + k, v);
         }
     }
 
     // ---------------------------------------------------------------- grid-wide barrier (bounded)
-    __threadfence();
     __syncthreads();
     if (t == 0) {
+        __threadfence();  // cumulative: publishes the whole CTA's reductions, ordered before it by the barrier
         atomicAdd(&a.ctrl->arrived, 1u);
         bool ok = false;
         for (uint32_t i = 0; i < kBarrierSpin; ++i) {
             if (ld_acquire_u32(&a.ctrl->arrived) >= gridDim.x) { ok = true; break; }
-            __nanosleep(32);
+            __nanosleep(20);
         }
+        __threadfence();
         s_fail = ok ? 0 : 1;
         if (!ok && a.dev_status) atomicMax(a.dev_status, kStatusTimeout);
     }
@@ -189,9 +193,9 @@ __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, int rows_base,
         }
         if (lane == 31) s_warp_cnt[warp] = incl;
         __syncthreads();
+        const int owner_warps = (G + 31) >> 5;  // warps beyond these own no channel and counted 0
         int before = 0, total = 0;
-#pragma unroll
-        for (int w = 0; w < kWarps; ++w) {
+        for (int w = 0; w < owner_warps; ++w) {
             const int c = s_warp_cnt[w];
             if (w < warp) before += c;
             total += c;
@@ -225,8 +229,7 @@ __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, int rows_base,
         __syncthreads();
         if (t == 0) {
             float mx = 0.0f;
-#pragma unroll
-            for (int w = 0; w < kWarps; ++w) mx = fmaxf(mx, s_warp_max[w]);
+            for (int w = 0; w < owner_warps; ++w) mx = fmaxf(mx, s_warp_max[w]);
             const float s = mx > 0.0f ? __fdiv_rn(mx, qf) : 1.0f;  // Eq. 1
             s_scale[0] = s;
             s_scale[1] = __fdiv_rn(1.0f, s);
@@ -241,7 +244,10 @@ __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, int rows_base,
     }
     const int r = min(r_true, a.cap);
     const int c = (1 << a.exp_factor) - 1;
-    const int used_words = (c * r + 3) >> 2;
+    const int used_cols = c * r, used_words = (used_cols + 3) >> 2;
+    // Aux column c*j + i mirrors channel O_j (Eq. 5), repeated c times for the weighted sum of Eq. 7
+    for (int i = t; i < used_cols; i += kT) s_auxsrc[i] = (uint16_t)s_oidx[i / c];
+    __syncthreads();
     // W_aux[n, c*j + t] = W_q[n, O_j], one 4-byte word per thread and round, spread over the grid.
     // The first round's scattered byte loads are issued here and consumed after pass 2, which hides
     // their latency behind the quantization work.
@@ -253,10 +259,8 @@ __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, int rows_base,
         const int n = wa_first / wa_words_per_row, w = wa_first - n * wa_words_per_row;
         if (w < used_words) {
 #pragma unroll
-            for (int bb = 0; bb < 4; ++bb) {
-                const int j = (w * 4 + bb) / c;
-                if (j < r) wa_byte[bb] = (uint8_t)a.w_q[(size_t)n * a.ldw + s_oidx[j]];
-            }
+            for (int bb = 0; bb < 4; ++bb)
+                if (w * 4 + bb < used_cols) wa_byte[bb] = (uint8_t)a.w_q[(size_t)n * a.ldw + s_auxsrc[w * 4 + bb]];
         }
     }
 
@@ -287,18 +291,14 @@ __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, int rows_base,
             *reinterpret_cast<uint2 *>(q + ch * 8) = quant8(f, s, inv_s, qf);
         }
         if (a.aux_q) {
-            const __half *xr = reinterpret_cast<const __half *>(src);
+            // shared scale: Aux_q[m, c*j + i] is the code Body_q[m, O_j] this warp has just written
+            __syncwarp();
             for (int w = lane; w < (a.aux_cols >> 2); w += 32) {
                 uint32_t packed = 0;
                 if (w < used_words) {
 #pragma unroll
-                    for (int bb = 0; bb < 4; ++bb) {
-                        const int j = (w * 4 + bb) / c;  // column c*j + t holds the code of Body[m, O_j] (Eq. 5)
-                        if (j < r) {
-                            const float v = __half2float(xr[s_oidx[j]]) * down;
-                            packed |= (uint32_t)(quant_exact(v, s, qf) & 0xff) << (8 * bb);
-                        }
-                    }
+                    for (int bb = 0; bb < 4; ++bb)
+                        if (w * 4 + bb < used_cols) packed |= (uint32_t)(uint8_t)q[s_auxsrc[w * 4 + bb]] << (8 * bb);
                 }
                 *reinterpret_cast<uint32_t *>(a.aux_q + m * a.ld_aux + w * 4) = packed;
             }
@@ -317,10 +317,9 @@ __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, int rows_base,
         uint32_t packed = 0;
         if (w < used_words) {
 #pragma unroll
-            for (int bb = 0; bb < 4; ++bb) {
-                const int j = (w * 4 + bb) / c;
-                if (j < r) packed |= (uint32_t)(uint8_t)a.w_q[(size_t)n * a.ldw + s_oidx[j]] << (8 * bb);
-            }
+            for (int bb = 0; bb < 4; ++bb)
+                if (w * 4 + bb < used_cols)
+                    packed |= (uint32_t)(uint8_t)a.w_q[(size_t)n * a.ldw + s_auxsrc[w * 4 + bb]] << (8 * bb);
         }
         *reinterpret_cast<uint32_t *>(a.w_aux + (size_t)n * a.ld_waux + w * 4) = packed;
     }
