@@ -40,9 +40,9 @@ __host__ __device__ inline int fixed_smem_bytes(int K) {
     return 8 * K + ((G + 15) & ~15) + kMaxOut * 4 + kMaxAuxCols * 2;
 }
 
-__device__ __forceinline__ uint32_t ld_acquire_u32(const uint32_t *p) {
+__device__ __forceinline__ uint32_t ld_relaxed_u32(const uint32_t *p) {
     uint32_t v;
-    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
     return v;
 }
 
@@ -140,10 +140,9 @@ __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, int rows_base,
         atomicAdd(&a.ctrl->arrived, 1u);
         bool ok = false;
         for (uint32_t i = 0; i < kBarrierSpin; ++i) {
-            if (ld_acquire_u32(&a.ctrl->arrived) >= gridDim.x) { ok = true; break; }
-            __nanosleep(20);
+            if (ld_relaxed_u32(&a.ctrl->arrived) >= gridDim.x) { ok = true; break; }
         }
-        __threadfence();
+        __threadfence();  // acquire side: the other CTAs' reductions are visible from here on
         s_fail = ok ? 0 : 1;
         if (!ok && a.dev_status) atomicMax(a.dev_status, kStatusTimeout);
     }
@@ -265,12 +264,66 @@ __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, int rows_base,
     }
 
     // ---------------------------------------------------------------- pass 2: Body_q and the Aux block
+    if (!a.per_token) {
+        // Per-tensor scale: the pass-1 mapping again (a thread owns 8 channels and walks down the
+        // rows), so the channel factors stay in registers and consecutive lanes store consecutive codes.
+        const float s = s_scale[0], inv_s = s_scale[1];
+        const int rstride = kT / G;
+        const int cg = t % G, row_off = t / G;
+        if (row_off < rstride) {
+            const float4 m0 = reinterpret_cast<const float4 *>(s_colmul)[2 * cg];
+            const float4 m1 = reinterpret_cast<const float4 *>(s_colmul)[2 * cg + 1];
+            const float mul[8] = {m0.x, m0.y, m0.z, m0.w, m1.x, m1.y, m1.z, m1.w};
+            for (int row = row_off; row < rows; row += 2 * rstride) {
+                uint4 v[2];
+#pragma unroll
+                for (int u = 0; u < 2; ++u) {
+                    const int rr = row + u * rstride;
+                    v[u] = make_uint4(0u, 0u, 0u, 0u);
+                    if (rr < fit) v[u] = *reinterpret_cast<const uint4 *>(slab + (size_t)rr * K * 2 + cg * 16);
+                    else if (rr < rows) v[u] = __ldg(reinterpret_cast<const uint4 *>(a.X + ((size_t)r0 + rr) * a.ldx) + cg);
+                }
+#pragma unroll
+                for (int u = 0; u < 2; ++u) {
+                    const int rr = row + u * rstride;
+                    if (rr < rows) {
+                        float f[8];
+                        unpack8(v[u], f);
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) f[i] *= mul[i];  // 1 or 2^-e: exact
+                        *reinterpret_cast<uint2 *>(a.body_q + ((size_t)r0 + rr) * a.ld_q + cg * 8) = quant8(f, s, inv_s, qf);
+                    }
+                }
+            }
+        }
+        if (a.aux_q) {
+            // Aux block of this CTA's rows: zero everywhere except the first c*r columns, where
+            // Aux_q[m, c*j + i] = code of Body[m, O_j] (Eq. 5, shared scale), recomputed from the slab
+            // with the exact division, one (row, column) pair per thread.
+            const int aux_words = a.aux_cols >> 2;
+            const int zero_from = used_cols >> 2;  // first word that holds a zero byte
+            const int zwords = aux_words - zero_from;
+            for (int i = t; i < rows * zwords; i += kT) {
+                const int row = i / zwords, w = zero_from + (i - row * zwords);
+                *reinterpret_cast<uint32_t *>(a.aux_q + ((size_t)r0 + row) * a.ld_aux + w * 4) = 0u;
+            }
+            __syncthreads();  // the byte stores below may land in a word zeroed above
+            for (int i = t; i < rows * used_cols; i += kT) {
+                const int row = i / used_cols, col = i - row * used_cols;
+                const size_t m = (size_t)r0 + row;
+                const __half *xr = row < fit ? reinterpret_cast<const __half *>(slab + (size_t)row * K * 2)
+                                             : a.X + m * a.ldx;
+                const float x = __half2float(xr[s_auxsrc[col]]) * down;
+                a.aux_q[m * a.ld_aux + col] = (int8_t)quant_exact(x, s, qf);
+            }
+        }
+    } else
     for (int row = warp; row < rows; row += kWarps) {
         const size_t m = (size_t)r0 + row;
         const uint4 *src = row < fit ? reinterpret_cast<const uint4 *>(slab + (size_t)row * K * 2)
                                      : reinterpret_cast<const uint4 *>(a.X + m * a.ldx);
-        float s = s_scale[0], inv_s = s_scale[1];
-        if (a.per_token) {
+        float s, inv_s;
+        {
             // per-token scale from Body's row (after the 2^-e redistribution)
             float mx = 0.0f;
             for (int ch = lane; ch < G; ch += 32) {

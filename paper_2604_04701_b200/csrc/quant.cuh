@@ -32,25 +32,26 @@ __device__ __forceinline__ void unpack8(const uint4 &v, float (&f)[8]) {
 
 // 8 values (already multiplied by their channel factors) -> 8 codes packed in a uint2.
 //
-// Fast path: t = v * (1/s) differs from the correctly rounded quotient v / s by less than 2.3e-5
-// for |v/s| <= 128, so whenever t is farther than 1e-4 from every half-integer both round to the
-// same integer.  Adding 1.5 * 2^23 rounds t to that integer (round half to even) and leaves its
-// two's-complement low byte in the low byte of the float's bit pattern, which a byte permute packs
-// directly.  If any of the 8 values is too close to a tie, or exceeds the code range (possible
-// only when the scale was not derived from these values), all 8 take the exact division.
+// Fast path: p = v * (1/s), taken exactly inside a fused multiply-add, differs from the correctly
+// rounded quotient v / s by less than 1.6e-5 for |v/s| <= 128, so whenever p is farther than 1e-4
+// from every half-integer both round to the same integer.  fma(v, 1/s, 1.5 * 2^23) rounds p to that
+// integer (round half to even) and leaves its two's-complement low byte in the low byte of the
+// float's bit pattern, which a byte permute packs directly; a second fma gives p minus that integer.
+// If any of the 8 values is too close to a tie, or exceeds the code range (possible only when the
+// scale was not derived from these values), all 8 take the exact division.
 __device__ __forceinline__ uint2 quant8(const float (&f)[8], float s, float inv_s, float qf) {
     const float magic = 12582912.0f;  // 1.5 * 2^23
     uint32_t b[8];
     float dmax = 0.0f, amax = 0.0f;
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
-        const float t = f[i] * inv_s;
-        const float tm = t + magic;
-        dmax = fmaxf(dmax, fabsf(t - (tm - magic)));
-        amax = fmaxf(amax, fabsf(t));
+        const float tm = fmaf(f[i], inv_s, magic);
+        const float n = tm - magic;
+        dmax = fmaxf(dmax, fabsf(fmaf(f[i], inv_s, -n)));
+        amax = fmaxf(amax, fabsf(n));
         b[i] = __float_as_uint(tm);
     }
-    if (dmax > 0.4999f || amax > qf + 0.25f) {
+    if (dmax > 0.4999f || amax > qf) {
 #pragma unroll
         for (int i = 0; i < 8; ++i) b[i] = (uint32_t)quant_exact(f[i], s, qf);
     }
