@@ -45,7 +45,8 @@ typedef enum {
     MUXQ_ERR_WORKSPACE = 3,
     MUXQ_ERR_CUDA = 4,
     MUXQ_ERR_CAPACITY = 5, /* device status: r > max_outliers */
-    MUXQ_ERR_TIMEOUT = 6   /* device status: a bounded wait inside a kernel expired */
+    MUXQ_ERR_TIMEOUT = 6,  /* device status: a bounded wait inside a kernel expired */
+    MUXQ_ERR_STATIC_LIMIT = 7 /* muxq_linear_decode_noalloc: M or K beyond its built-in scratch */
 } muxq_status;
 
 typedef enum { MUXQ_PER_TENSOR = 0, MUXQ_PER_VECTOR = 1 /* per-token X, per-channel W */ } muxq_gran;
@@ -190,6 +191,30 @@ int muxq_workspace_view(int M, int K, int N, const muxq_params *p, muxq_ws_view 
 int muxq_linear_host(const void *X_f16_host, int M, int K, const int8_t *W_q, int ldw,
                      const float *s_w, int N, const muxq_params *p, void *Y_host, int out_kind,
                      void *workspace, size_t workspace_bytes, int32_t *dev_status, void *stream);
+
+/*
+ * The decode-shaped layer without a caller-provided workspace.  (The paper has no counterpart:
+ * this entry point exists for the sake of callers, not of the method.)
+ *
+ * Some callers cannot allocate device memory where they call the layer: a decode loop in which a
+ * cudaMalloc would stall every stream of the device, a plug-in inside a host program that has
+ * handed all device memory to its own pool, a process past the point where its memory budget was
+ * frozen.  For them the scratch that muxq_linear takes as `workspace` is a fixed array inside the
+ * library: 426,752 bytes of device memory on every GPU that loads the library, held until the
+ * process exits.  It covers M <= 16 token rows and K <= 8192 input channels, any N; larger M or K
+ * return MUXQ_ERR_STATIC_LIMIT and launch nothing.  The call allocates and frees nothing.
+ *
+ * Arguments, results, alignment rules and the device status word are those of muxq_linear with
+ * M <= 16 (same kernels, same arithmetic).  The first call on each device looks up the array's
+ * device address (the device must be current); make that first call outside any stream capture.
+ * All calls on a device share the one array and it keeps the previous call's contents: the parts
+ * that must start at zero are cleared on `stream` at the head of each call, and two calls whose
+ * GPU work overlaps (different streams, or graphs replayed concurrently) race on it -- keep them
+ * on one stream or order them yourself.  The intermediates are not exposed.
+ */
+int muxq_linear_decode_noalloc(const void *X_f16, int M, int K, int ldx, const int8_t *W_q, int ldw,
+                               const float *s_w, int N, const muxq_params *p, void *Y, int ldy,
+                               int out_kind, int32_t *dev_status, void *stream);
 
 /*
  * Measurement aid: runs `ctas` CTAs (one per SM when ctas = SM count) that each issue `iters`

@@ -13,7 +13,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_HERE, "libmuxq.so")
 
 MUXQ_OK, MUXQ_ERR_INVALID_ARG, MUXQ_ERR_UNSUPPORTED, MUXQ_ERR_WORKSPACE = 0, 1, 2, 3
-MUXQ_ERR_CUDA, MUXQ_ERR_CAPACITY, MUXQ_ERR_TIMEOUT = 4, 5, 6
+MUXQ_ERR_CUDA, MUXQ_ERR_CAPACITY, MUXQ_ERR_TIMEOUT, MUXQ_ERR_STATIC_LIMIT = 4, 5, 6, 7
 MUXQ_PER_TENSOR, MUXQ_PER_VECTOR = 0, 1
 MUXQ_AUX_SHARED, MUXQ_AUX_OWN = 0, 1
 MUXQ_OUT_F16, MUXQ_OUT_F32, MUXQ_OUT_ACC_I32 = 0, 1, 2
@@ -21,7 +21,8 @@ MUXQ_OUT_F16, MUXQ_OUT_F32, MUXQ_OUT_ACC_I32 = 0, 1, 2
 EXPORTS = (
     "muxq_default_params", "muxq_aux_cols", "muxq_workspace_bytes", "muxq_small_workspace_bytes",
     "muxq_host_workspace_bytes", "muxq_workspace_view", "muxq_detect_outliers", "muxq_build_aux",
-    "muxq_quantize", "muxq_gemm", "muxq_linear", "muxq_linear_events", "muxq_linear_host", "muxq_int8_mma_peak", "muxq_read_status",
+    "muxq_quantize", "muxq_gemm", "muxq_linear", "muxq_linear_events", "muxq_linear_host",
+    "muxq_linear_decode_noalloc", "muxq_int8_mma_peak", "muxq_read_status",
     "muxq_status_string",
 )
 
@@ -91,6 +92,7 @@ def lib() -> ctypes.CDLL:
         L.muxq_linear.argtypes = [vp, i, i, i, vp, i, vp, i, pp, vp, i, i, vp, sz, vp, vp]; L.muxq_linear.restype = i
         L.muxq_linear_events.argtypes = [vp, i, i, i, vp, i, vp, i, pp, vp, i, i, vp, sz, vp, vp, vp]; L.muxq_linear_events.restype = i
         L.muxq_linear_host.argtypes = [vp, i, i, vp, i, vp, i, pp, vp, i, vp, sz, vp, vp]; L.muxq_linear_host.restype = i
+        L.muxq_linear_decode_noalloc.argtypes = [vp, i, i, i, vp, i, vp, i, pp, vp, i, i, vp, vp]; L.muxq_linear_decode_noalloc.restype = i
         L.muxq_int8_mma_peak.argtypes = [i, i, i, vp, vp, vp]; L.muxq_int8_mma_peak.restype = i
         L.muxq_read_status.argtypes = [vp, vp]; L.muxq_read_status.restype = i
         L.muxq_status_string.argtypes = [i]; L.muxq_status_string.restype = ctypes.c_char_p
@@ -261,6 +263,24 @@ def muxq_linear_host(X_host: torch.Tensor, w_q: torch.Tensor, s_w: torch.Tensor,
            lib().muxq_linear_host(_ptr(X_host), M, K, _ptr(w_q), w_q.stride(0), _ptr(s_w), N, ctypes.byref(p.c()),
                                   _ptr(Y_host), out_kind, _ptr(ws.buf), ws.nbytes, _ptr(ws.status), _stream()))
     return Y_host
+
+
+def muxq_linear_decode_noalloc(X: torch.Tensor, w_q: torch.Tensor, s_w: torch.Tensor, p: MuxqParams,
+                               status: torch.Tensor, out_kind: int = MUXQ_OUT_F16,
+                               out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """muxq_linear for M <= 16 rows and K <= 8192 channels with no workspace argument: the scratch is
+    a fixed array inside the library, for callers that cannot allocate device memory at the call site.
+    `out` should be given by such callers (otherwise torch allocates it); `status` is a device int32[1].
+    Calls share the scratch, so keep them on one stream."""
+    assert X.is_cuda and X.dtype == torch.float16 and X.dim() == 2 and X.stride(1) == 1
+    M, K = X.shape
+    N = w_q.shape[0]
+    Y = out if out is not None else _alloc_out(M, N, out_kind, X.device)
+    _check("muxq_linear_decode_noalloc",
+           lib().muxq_linear_decode_noalloc(_ptr(X), M, K, X.stride(0), _ptr(w_q), w_q.stride(0), _ptr(s_w), N,
+                                            ctypes.byref(p.c()), _ptr(Y), Y.stride(0), out_kind, _ptr(status),
+                                            _stream()))
+    return Y
 
 
 def muxq_int8_mma_peak(mma_n: int, iters: int, ctas: int, ws: Workspace) -> torch.Tensor:

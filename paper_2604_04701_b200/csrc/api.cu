@@ -436,6 +436,7 @@ const char *muxq_status_string(int st) {
         case MUXQ_ERR_CUDA: return "CUDA runtime error";
         case MUXQ_ERR_CAPACITY: return "more outlier channels than max_outliers";
         case MUXQ_ERR_TIMEOUT: return "bounded device-side wait expired";
+        case MUXQ_ERR_STATIC_LIMIT: return "M or K exceeds the built-in scratch of the no-allocation entry point";
         default: return "unknown status";
     }
 }
