@@ -150,7 +150,7 @@ __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, int rows_base,
     if (s_fail) return;
 
     // ---------------------------------------------------------------- O, channel factors, s_X (every CTA)
-    const float down = exp2f(-(float)a.exp_factor);
+    const float down = __int_as_float((127 - a.exp_factor) << 23);  // 2^-e
     const float qf = (float)a.qmax;
     int r_true;
     {
@@ -170,8 +170,13 @@ __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, int rows_base,
             if (b == 0) reinterpret_cast<uint4 *>(a.colmax_bits)[k4] = mx;
         }
         __syncthreads();
-        const bool active = t < G;  // thread t owns channels [8t, 8t+8)
+        // thread t owns channels [8t, 8t+8); warps beyond owner_warps own none and only follow the barriers
+        const int owner_warps = (G + 31) >> 5;
+        const bool owner = warp < owner_warps;
+        const bool active = t < G;
         float cm[8];
+        int cnt = 0, incl = 0;
+        if (owner) {
         if (active) {
             const float4 v0 = reinterpret_cast<const float4 *>(s_colmax)[2 * t];
             const float4 v1 = reinterpret_cast<const float4 *>(s_colmax)[2 * t + 1];
@@ -181,18 +186,17 @@ __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, int rows_base,
 #pragma unroll
             for (int i = 0; i < 8; ++i) cm[i] = 0.0f;
         }
-        int cnt = 0;
 #pragma unroll
         for (int i = 0; i < 8; ++i) cnt += (cm[i] > a.tau) ? 1 : 0;
-        int incl = cnt;
+        incl = cnt;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
             const int n = __shfl_up_sync(0xffffffffu, incl, o);
             if (lane >= o) incl += n;
         }
         if (lane == 31) s_warp_cnt[warp] = incl;
+        }
         __syncthreads();
-        const int owner_warps = (G + 31) >> 5;  // warps beyond these own no channel and counted 0
         int before = 0, total = 0;
         for (int w = 0; w < owner_warps; ++w) {
             const int c = s_warp_cnt[w];
@@ -200,6 +204,7 @@ __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, int rows_base,
             total += c;
         }
         r_true = total;
+        if (owner) {
         int pos = before + incl - cnt;
         float bmax = 0.0f;
         if (active) {
@@ -225,7 +230,13 @@ __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, int rows_base,
         }
         bmax = warp_max(bmax);
         if (lane == 0) s_warp_max[warp] = bmax;
+        }
+        // Aux column c*j + i mirrors channel O_j (Eq. 5), repeated c times for the weighted sum of Eq. 7
         __syncthreads();
+        {
+            const int cc = (1 << a.exp_factor) - 1, ucols = cc * min(total, a.cap);
+            for (int i = t; i < ucols; i += kT) s_auxsrc[i] = (uint16_t)s_oidx[i / cc];
+        }
         if (t == 0) {
             float mx = 0.0f;
             for (int w = 0; w < owner_warps; ++w) mx = fmaxf(mx, s_warp_max[w]);
@@ -244,9 +255,6 @@ __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, int rows_base,
     const int r = min(r_true, a.cap);
     const int c = (1 << a.exp_factor) - 1;
     const int used_cols = c * r, used_words = (used_cols + 3) >> 2;
-    // Aux column c*j + i mirrors channel O_j (Eq. 5), repeated c times for the weighted sum of Eq. 7
-    for (int i = t; i < used_cols; i += kT) s_auxsrc[i] = (uint16_t)s_oidx[i / c];
-    __syncthreads();
     // W_aux[n, c*j + t] = W_q[n, O_j], one 4-byte word per thread and round, spread over the grid.
     // The first round's scattered byte loads are issued here and consumed after pass 2, which hides
     // their latency behind the quantization work.
@@ -274,6 +282,9 @@ __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, int rows_base,
             const float4 m0 = reinterpret_cast<const float4 *>(s_colmul)[2 * cg];
             const float4 m1 = reinterpret_cast<const float4 *>(s_colmul)[2 * cg + 1];
             const float mul[8] = {m0.x, m0.y, m0.z, m0.w, m1.x, m1.y, m1.z, m1.w};
+            float is[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) is[i] = inv_s * mul[i];  // the channel factor folded into 1/s (power of two: exact)
             for (int row = row_off; row < rows; row += 2 * rstride) {
                 uint4 v[2];
 #pragma unroll
@@ -289,9 +300,8 @@ __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, int rows_base,
                     if (rr < rows) {
                         float f[8];
                         unpack8(v[u], f);
-#pragma unroll
-                        for (int i = 0; i < 8; ++i) f[i] *= mul[i];  // 1 or 2^-e: exact
-                        *reinterpret_cast<uint2 *>(a.body_q + ((size_t)r0 + rr) * a.ld_q + cg * 8) = quant8(f, s, inv_s, qf);
+                        *reinterpret_cast<uint2 *>(a.body_q + ((size_t)r0 + rr) * a.ld_q + cg * 8) =
+                            quant8_scaled(f, mul, is, s, qf);
                     }
                 }
             }

@@ -60,4 +60,27 @@ __device__ __forceinline__ uint2 quant8(const float (&f)[8], float s, float inv_
     return make_uint2(__byte_perm(p01, p23, 0x5410), __byte_perm(p45, p67, 0x5410));
 }
 
+// The same for values whose power-of-two channel factors mul[i] are still to be applied, with
+// is[i] = (1/s) * mul[i] (exact), and for a scale s that was derived from these very values, so that
+// no code can leave [-q, q] and the range check is not needed.
+__device__ __forceinline__ uint2 quant8_scaled(const float (&f)[8], const float (&mul)[8], const float (&is)[8],
+                                               float s, float qf) {
+    const float magic = 12582912.0f;  // 1.5 * 2^23
+    uint32_t b[8];
+    float dmax = 0.0f;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const float tm = fmaf(f[i], is[i], magic);
+        dmax = fmaxf(dmax, fabsf(fmaf(f[i], is[i], magic - tm)));
+        b[i] = __float_as_uint(tm);
+    }
+    if (dmax > 0.4999f) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) b[i] = (uint32_t)quant_exact(f[i] * mul[i], s, qf);
+    }
+    const uint32_t p01 = __byte_perm(b[0], b[1], 0x0040), p23 = __byte_perm(b[2], b[3], 0x0040);
+    const uint32_t p45 = __byte_perm(b[4], b[5], 0x0040), p67 = __byte_perm(b[6], b[7], 0x0040);
+    return make_uint2(__byte_perm(p01, p23, 0x5410), __byte_perm(p45, p67, 0x5410));
+}
+
 }  // namespace muxq
