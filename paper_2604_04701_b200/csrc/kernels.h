@@ -112,6 +112,7 @@ struct GemmArgs {
     int32_t *dev_status;
 };
 cudaError_t launch_gemm(const GemmArgs &a, cudaStream_t s);
+cudaError_t launch_gemm_pair(const GemmArgs &a, int bn, cudaStream_t s);  // two CTAs per 256-row tile
 
 struct DecodeArgs {
     const int8_t *body_q; int ld_a;   // [M, K]
