@@ -254,23 +254,59 @@ def run_muxq(args, rank, world):
             for j in range(3):
                 acc_us[li][j] += evs[li][j].elapsed_time(evs[li][j + 1]) * 1e3 / ksteps
     kern_us = {"clear": [a[0] for a in acc_us], "prepare": [a[1] for a in acc_us], "gemm": [a[2] for a in acc_us]}
-    per_layer_gemm_us = kern_us["gemm"]
-    gemm_us_per_step = sum(kern_us["gemm"])
+    total_us = sum(sum(v) for v in kern_us.values())
+
+    # ---- the dominant kernel on its own: a graph of only the four GEMM launches, fed from the
+    # intermediates the last step left in each layer's workspace (Body_q, Aux_q, W_aux, r, s_X)
+    def ws_tensor(L, off, nbytes, dtype, shape):
+        return L["ws"].buf[off: off + nbytes].view(dtype).view(*shape)
+
+    gemm_calls = []
+    for L in layers:
+        sp = L["spec"]
+        v = mx.muxq_workspace_view(sp.M, sp.K, sp.N, p)
+        gemm_calls.append((
+            ws_tensor(L, v.body_q, sp.M * v.ld_body_q, torch.int8, (sp.M, v.ld_body_q)),
+            ws_tensor(L, v.aux_q, sp.M * v.aux_cols, torch.int8, (sp.M, v.aux_cols)),
+            L["w_q"], ws_tensor(L, v.w_aux, sp.N * v.aux_cols, torch.int8, (sp.N, v.aux_cols)),
+            ws_tensor(L, v.n_outliers, 4, torch.int32, (1,)), ws_tensor(L, v.s_x, 4, torch.float32, (1,)),
+            L["s_w"], L["ws"], L["y"]))
+
+    def gemm_step():
+        for (bq, aq, wq, wa, nout, sx, sw, wsx, y) in gemm_calls:
+            mx.muxq_gemm(bq, aq, wq, wa, nout, p, sx, sw, mx.MUXQ_OUT_F16, wsx, out=y)
+
+    with torch.cuda.stream(side):
+        gemm_step()
+        side.synchronize()
+        g_gemm = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g_gemm, stream=side):
+            gemm_step()
+    torch.cuda.synchronize()
+    for _ in range(3):
+        g_gemm.replay()
+    k0, k1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    k0.record()
+    for _ in range(ksteps):
+        g_gemm.replay()
+    k1.record()
+    torch.cuda.synchronize()
+    check_status()
+    gemm_us_per_step = k0.elapsed_time(k1) * 1e3 / ksteps
     peaks = load_peaks()
     int8_peak = 2.0 * peaks["bf16_sustained"]  # INT8 dense rate = 2 x bf16 (nominal 4.5 vs 2.25 POPS)
     achieved = ops_per_step / (gemm_us_per_step * 1e-6) / 1e12
-    total_us = sum(sum(v) for v in kern_us.values())
-    roofline = {"kernel": "k_gemm_i8 (tcgen05 kind::i8, fused Aux + dequant epilogue)", "bound": "tensor",
-                "achieved": achieved, "peak": int8_peak, "unit": "TOPS", "frac": achieved / int8_peak,
-                "peak_source": f"2 x bf16_tflops_sustained of {peaks['source']}",
-                "traffic": None,
-                "per_layer": [{"layer": L["spec"].name, "M": L["spec"].M, "K": L["spec"].K, "N": L["spec"].N,
-                               "gemm_us": per_layer_gemm_us[i], "clear_us": kern_us["clear"][i],
-                               "prepare_us": kern_us["prepare"][i],
-                               "prepare_gbs": (3.0 * L["spec"].M * L["spec"].K) / (kern_us["prepare"][i] * 1e-6) / 1e9,
-                               "gemm_tops": 2.0 * L["spec"].M * L["spec"].N * L["spec"].K /
-                               (per_layer_gemm_us[i] * 1e-6) / 1e12} for i, L in enumerate(layers)],
-                "share_of_step": {k: sum(v) / total_us for k, v in kern_us.items()}}
+    roofline = {"kernel": "k_gemm_i8_pair (tcgen05 kind::i8 cta_group::2, fused Aux + dequant epilogue)",
+                "bound": "tensor", "achieved": achieved, "peak": int8_peak, "unit": "TOPS",
+                "frac": achieved / int8_peak, "peak_source": f"2 x bf16_tflops_sustained of {peaks['source']}",
+                "traffic": None, "launches_per_step": len(layers), "us_per_step": gemm_us_per_step,
+                "how": "CUDA events around replays of a graph holding only the step's four GEMM launches",
+                "per_layer_in_step": [{"layer": L["spec"].name, "M": L["spec"].M, "K": L["spec"].K, "N": L["spec"].N,
+                                       "clear_us": kern_us["clear"][i], "prepare_us": kern_us["prepare"][i],
+                                       "gemm_us": kern_us["gemm"][i]} for i, L in enumerate(layers)],
+                "share_of_step": {k: sum(v) / total_us for k, v in kern_us.items()},
+                "share_note": "from event-record nodes inside the step graph; each segment carries node overhead"}
 
     # ---- end to end: host buffers, copies inside the timed region
     esteps = max(3, min(args.steps, 20))
