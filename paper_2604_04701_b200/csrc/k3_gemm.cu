@@ -182,19 +182,18 @@ k_gemm_i8(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
             tc_fence_after();
             const int col0 = chalf * (BN / 2);
             const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + buf * BN + col0;
-            uint32_t v[2][32];
-            tmem_ld_32x32(taddr, v[0]);
+            // Pull this warp's whole share of the accumulator (32 rows x BN/2 columns) into registers at once
+            // and hand the TMEM buffer back before converting: the MMA issuer can then start the tile after
+            // next while this tile is still being converted and stored.
+            uint32_t v[kChunks][32];
+#pragma unroll
+            for (int ch = 0; ch < kChunks; ++ch) tmem_ld_32x32(taddr + 32 * ch, v[ch]);
+            tmem_ld_wait();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&bar_acc_empty[buf]);
 #pragma unroll
             for (int ch = 0; ch < kChunks; ++ch) {
-                tmem_ld_wait();
-                if (ch + 1 < kChunks) {
-                    tmem_ld_32x32(taddr + 32 * (ch + 1), v[(ch + 1) & 1]);
-                } else {
-                    // every TMEM read of this warp for this tile has completed: hand the buffer back
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(&bar_acc_empty[buf]);
-                }
                 const int piece = ch % kChunksPerBox;  // position of this chunk inside its store box
                 uint8_t *stage = stage0 + (n_box % C::kOutBufs) * C::kOutBufBytes;
                 if (piece == 0) {
@@ -203,7 +202,7 @@ k_gemm_i8(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
                     __syncwarp();
                 }
                 const int gcol = n0 + col0 + 32 * ch;
-                convert_chunk<kOut, kPerVec>(v[ch & 1], reinterpret_cast<uint4 *>(stage + lane * 128),
+                convert_chunk<kOut, kPerVec>(v[ch], reinterpret_cast<uint4 *>(stage + lane * 128),
                                              kOut == kOutF16 ? 4 * piece : 0, sw_xor, sx, sxw, p.s_w + gcol,
                                              p.N - gcol);
                 if (piece == kChunksPerBox - 1) {
