@@ -13,9 +13,10 @@
 //           replicated kColmaxReplicas times (CTA b uses copy b mod R): same-address atomics
 //           serialise in L2, and one copy would take 148 of them per channel
 //   barrier bounded spin on an arrival counter; a time-out raises MUXQ_ERR_TIMEOUT and returns
-//   pass 2  every CTA derives O, the channel factors and s_X from the K maxima (cheap, redundant),
-//           then quantizes its slab out of shared memory, one warp per token row, writing Body_q,
-//           the Aux block and (spread over the grid) the gathered W_aux rows.
+//   pass 2  every CTA derives the channel factors and s_X from the K maxima (cheap, redundant; warp 0
+//           lists O meanwhile), then quantizes its slab out of shared memory with the pass-1 thread
+//           mapping (per tensor) or one warp per token row (per token), writing Body_q, the Aux block
+//           and (spread over the grid) the gathered W_aux rows.
 #include "kernels.h"
 #include "quant.cuh"
 
@@ -68,9 +69,8 @@ __device__ __forceinline__ void load_chunk(const uint4 *src, int ch, const uint8
 
 __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, int rows_base, int rows_extra, int slab_bytes) {
     extern __shared__ __align__(16) uint8_t smem[];
-    __shared__ int s_warp_cnt[kWarps];
     __shared__ float s_warp_max[kWarps];
-    __shared__ float s_scale[2];
+    __shared__ int s_r_true;
     __shared__ int s_fail;
 
     const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
@@ -149,139 +149,122 @@ __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, int rows_base,
     __syncthreads();
     if (s_fail) return;
 
-    // ---------------------------------------------------------------- O, channel factors, s_X (every CTA)
+    // ---------------------------------------------------------------- channel factors and s_X (every CTA)
     const float down = __int_as_float((127 - a.exp_factor) << 23);  // 2^-e
     const float qf = (float)a.qmax;
-    int r_true;
+    const int c = (1 << a.exp_factor) - 1;
+    // channel maxima = max over the replicas, fetched with coalesced 16-byte loads
+    for (int k4 = t; k4 < (K >> 2); k4 += kT) {
+        uint4 v[kColmaxReplicas];
+#pragma unroll
+        for (int rp = 0; rp < kColmaxReplicas; ++rp)
+            v[rp] = __ldcg(reinterpret_cast<const uint4 *>(a.colmax_rep + (size_t)rp * K) + k4);
+        uint4 mx = v[0];
+#pragma unroll
+        for (int rp = 1; rp < kColmaxReplicas; ++rp) {
+            mx.x = max(mx.x, v[rp].x); mx.y = max(mx.y, v[rp].y);
+            mx.z = max(mx.z, v[rp].z); mx.w = max(mx.w, v[rp].w);
+        }
+        reinterpret_cast<uint4 *>(s_colmax)[k4] = mx;
+        if (b == 0) reinterpret_cast<uint4 *>(a.colmax_bits)[k4] = mx;
+    }
+    __syncthreads();
+    // Every thread derives the factors of the 8 channels it owns in both passes: 2^-e where the channel
+    // holds an element above the threshold (strict), else 1.  (When more channels are flagged than the
+    // capacity allows the call fails with MUXQ_ERR_CAPACITY and Y is unspecified, so no ordering is needed here.)
+    const int rstride = kT / G;
+    const int cg = t % G, row_off = t / G;
+    float mul[8];
     {
-        // channel maxima = max over the replicas, fetched with coalesced 16-byte loads
-        for (int k4 = t; k4 < (K >> 2); k4 += kT) {
-            uint4 v[kColmaxReplicas];
-#pragma unroll
-            for (int rp = 0; rp < kColmaxReplicas; ++rp)
-                v[rp] = __ldcg(reinterpret_cast<const uint4 *>(a.colmax_rep + (size_t)rp * K) + k4);
-            uint4 mx = v[0];
-#pragma unroll
-            for (int rp = 1; rp < kColmaxReplicas; ++rp) {
-                mx.x = max(mx.x, v[rp].x); mx.y = max(mx.y, v[rp].y);
-                mx.z = max(mx.z, v[rp].z); mx.w = max(mx.w, v[rp].w);
-            }
-            reinterpret_cast<uint4 *>(s_colmax)[k4] = mx;
-            if (b == 0) reinterpret_cast<uint4 *>(a.colmax_bits)[k4] = mx;
-        }
-        __syncthreads();
-        // thread t owns channels [8t, 8t+8); warps beyond owner_warps own none and only follow the barriers
-        const int owner_warps = (G + 31) >> 5;
-        const bool owner = warp < owner_warps;
-        const bool active = t < G;
-        float cm[8];
-        int cnt = 0, incl = 0;
-        if (owner) {
-        if (active) {
-            const float4 v0 = reinterpret_cast<const float4 *>(s_colmax)[2 * t];
-            const float4 v1 = reinterpret_cast<const float4 *>(s_colmax)[2 * t + 1];
-            cm[0] = v0.x; cm[1] = v0.y; cm[2] = v0.z; cm[3] = v0.w;
-            cm[4] = v1.x; cm[5] = v1.y; cm[6] = v1.z; cm[7] = v1.w;
-        } else {
-#pragma unroll
-            for (int i = 0; i < 8; ++i) cm[i] = 0.0f;
-        }
-#pragma unroll
-        for (int i = 0; i < 8; ++i) cnt += (cm[i] > a.tau) ? 1 : 0;
-        incl = cnt;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const int n = __shfl_up_sync(0xffffffffu, incl, o);
-            if (lane >= o) incl += n;
-        }
-        if (lane == 31) s_warp_cnt[warp] = incl;
-        }
-        __syncthreads();
-        int before = 0, total = 0;
-        for (int w = 0; w < owner_warps; ++w) {
-            const int c = s_warp_cnt[w];
-            if (w < warp) before += c;
-            total += c;
-        }
-        r_true = total;
-        if (owner) {
-        int pos = before + incl - cnt;
+        const float4 v0 = reinterpret_cast<const float4 *>(s_colmax)[2 * cg];
+        const float4 v1 = reinterpret_cast<const float4 *>(s_colmax)[2 * cg + 1];
+        const float cm[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
         float bmax = 0.0f;
-        if (active) {
-            float mul[8];
-            uint8_t gf = 0;
+        bool any = false;
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                mul[i] = 1.0f;
-                if (cm[i] > a.tau) {  // strict: |x| == threshold does not flag the channel
-                    if (pos < a.cap) {
-                        s_oidx[pos] = 8 * t + i;
-                        if (b == 0) a.outlier_idx[pos] = 8 * t + i;
-                        mul[i] = down;
-                        gf = 1;
-                    }
-                    ++pos;
-                }
-                bmax = fmaxf(bmax, cm[i] * mul[i]);  // power-of-two scaling: exact
-            }
-            reinterpret_cast<float4 *>(s_colmul)[2 * t] = make_float4(mul[0], mul[1], mul[2], mul[3]);
-            reinterpret_cast<float4 *>(s_colmul)[2 * t + 1] = make_float4(mul[4], mul[5], mul[6], mul[7]);
-            s_flag[t] = gf;
+        for (int i = 0; i < 8; ++i) {
+            const bool flagged = cm[i] > a.tau;
+            mul[i] = flagged ? down : 1.0f;
+            any |= flagged;
+            bmax = fmaxf(bmax, cm[i] * mul[i]);  // power-of-two scaling: exact
+        }
+        if (row_off == 0) {  // shared copies for the per-token path
+            reinterpret_cast<float4 *>(s_colmul)[2 * cg] = make_float4(mul[0], mul[1], mul[2], mul[3]);
+            reinterpret_cast<float4 *>(s_colmul)[2 * cg + 1] = make_float4(mul[4], mul[5], mul[6], mul[7]);
+            s_flag[cg] = any ? 1 : 0;
         }
         bmax = warp_max(bmax);
         if (lane == 0) s_warp_max[warp] = bmax;
+    }
+    __syncthreads();
+    float s, inv_s;
+    {
+        const float mx = warp_max(s_warp_max[lane]);
+        s = mx > 0.0f ? __fdiv_rn(mx, qf) : 1.0f;  // Eq. 1
+        inv_s = __fdiv_rn(1.0f, s);
+        if (b == 0 && t == 0) {
+            a.ctrl->s_x = s;
+            a.ctrl->inv_s_x = inv_s;
         }
-        // Aux column c*j + i mirrors channel O_j (Eq. 5), repeated c times for the weighted sum of Eq. 7
-        __syncthreads();
-        {
-            const int cc = (1 << a.exp_factor) - 1, ucols = cc * min(total, a.cap);
-            for (int i = t; i < ucols; i += kT) s_auxsrc[i] = (uint16_t)s_oidx[i / cc];
+    }
+    // Warp 0 lists O in ascending order (the other warps do not need it until the Aux block) and the
+    // source channel of every Aux column: column c*j + i mirrors channel O_j (Eq. 5), repeated c times
+    // for the weighted sum of Eq. 7.
+    if (warp == 0) {
+        int carry = 0;
+        for (int base = 0; base < G; base += 32) {
+            const int g = base + lane;
+            float cm[8];
+            if (g < G) {
+                const float4 v0 = reinterpret_cast<const float4 *>(s_colmax)[2 * g];
+                const float4 v1 = reinterpret_cast<const float4 *>(s_colmax)[2 * g + 1];
+                cm[0] = v0.x; cm[1] = v0.y; cm[2] = v0.z; cm[3] = v0.w;
+                cm[4] = v1.x; cm[5] = v1.y; cm[6] = v1.z; cm[7] = v1.w;
+            } else {
+#pragma unroll
+                for (int i = 0; i < 8; ++i) cm[i] = 0.0f;
+            }
+            int cnt = 0;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) cnt += (cm[i] > a.tau) ? 1 : 0;
+            if (!__any_sync(0xffffffffu, cnt != 0)) continue;
+            int incl = cnt;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int n = __shfl_up_sync(0xffffffffu, incl, o);
+                if (lane >= o) incl += n;
+            }
+            int pos = carry + incl - cnt;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                if (cm[i] > a.tau) {
+                    if (pos < a.cap) {
+                        s_oidx[pos] = 8 * g + i;
+                        if (b == 0) a.outlier_idx[pos] = 8 * g + i;
+                    }
+                    ++pos;
+                }
+            }
+            carry += __shfl_sync(0xffffffffu, incl, 31);
         }
-        if (t == 0) {
-            float mx = 0.0f;
-            for (int w = 0; w < owner_warps; ++w) mx = fmaxf(mx, s_warp_max[w]);
-            const float s = mx > 0.0f ? __fdiv_rn(mx, qf) : 1.0f;  // Eq. 1
-            s_scale[0] = s;
-            s_scale[1] = __fdiv_rn(1.0f, s);
+        __syncwarp();
+        const int ucols = c * min(carry, a.cap);
+        for (int i = lane; i < ucols; i += 32) s_auxsrc[i] = (uint16_t)s_oidx[i / c];
+        if (lane == 0) {
+            s_r_true = carry;
             if (b == 0) {
-                a.ctrl->s_x = s;
-                a.ctrl->inv_s_x = s_scale[1];
-                a.ctrl->n_outliers = total;
-                if (total > a.cap && a.dev_status) atomicMax(a.dev_status, kStatusCapacity);
+                a.ctrl->n_outliers = carry;
+                if (carry > a.cap && a.dev_status) atomicMax(a.dev_status, kStatusCapacity);
             }
         }
-        __syncthreads();
     }
-    const int r = min(r_true, a.cap);
-    const int c = (1 << a.exp_factor) - 1;
-    const int used_cols = c * r, used_words = (used_cols + 3) >> 2;
-    // W_aux[n, c*j + t] = W_q[n, O_j], one 4-byte word per thread and round, spread over the grid.
-    // The first round's scattered byte loads are issued here and consumed after pass 2, which hides
-    // their latency behind the quantization work.
-    const int wa_words_per_row = a.aux_cols >> 2;
-    const int wa_total = a.w_aux ? a.N * wa_words_per_row : 0;
-    const int wa_first = b * kT + t;
-    uint8_t wa_byte[4] = {0, 0, 0, 0};
-    if (wa_first < wa_total) {
-        const int n = wa_first / wa_words_per_row, w = wa_first - n * wa_words_per_row;
-        if (w < used_words) {
-#pragma unroll
-            for (int bb = 0; bb < 4; ++bb)
-                if (w * 4 + bb < used_cols) wa_byte[bb] = (uint8_t)a.w_q[(size_t)n * a.ldw + s_auxsrc[w * 4 + bb]];
-        }
-    }
+    if (a.per_token) __syncthreads();  // the per-token path reads the shared factor copies and the Aux sources
 
     // ---------------------------------------------------------------- pass 2: Body_q and the Aux block
     if (!a.per_token) {
         // Per-tensor scale: the pass-1 mapping again (a thread owns 8 channels and walks down the
         // rows), so the channel factors stay in registers and consecutive lanes store consecutive codes.
-        const float s = s_scale[0], inv_s = s_scale[1];
-        const int rstride = kT / G;
-        const int cg = t % G, row_off = t / G;
         if (row_off < rstride) {
-            const float4 m0 = reinterpret_cast<const float4 *>(s_colmul)[2 * cg];
-            const float4 m1 = reinterpret_cast<const float4 *>(s_colmul)[2 * cg + 1];
-            const float mul[8] = {m0.x, m0.y, m0.z, m0.w, m1.x, m1.y, m1.z, m1.w};
             float is[8];
 #pragma unroll
             for (int i = 0; i < 8; ++i) is[i] = inv_s * mul[i];  // the channel factor folded into 1/s (power of two: exact)
@@ -306,34 +289,13 @@ __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, int rows_base,
                 }
             }
         }
-        if (a.aux_q) {
-            // Aux block of this CTA's rows: zero everywhere except the first c*r columns, where
-            // Aux_q[m, c*j + i] = code of Body[m, O_j] (Eq. 5, shared scale), recomputed from the slab
-            // with the exact division, one (row, column) pair per thread.
-            const int aux_words = a.aux_cols >> 2;
-            const int zero_from = used_cols >> 2;  // first word that holds a zero byte
-            const int zwords = aux_words - zero_from;
-            for (int i = t; i < rows * zwords; i += kT) {
-                const int row = i / zwords, w = zero_from + (i - row * zwords);
-                *reinterpret_cast<uint32_t *>(a.aux_q + ((size_t)r0 + row) * a.ld_aux + w * 4) = 0u;
-            }
-            __syncthreads();  // the byte stores below may land in a word zeroed above
-            for (int i = t; i < rows * used_cols; i += kT) {
-                const int row = i / used_cols, col = i - row * used_cols;
-                const size_t m = (size_t)r0 + row;
-                const __half *xr = row < fit ? reinterpret_cast<const __half *>(slab + (size_t)row * K * 2)
-                                             : a.X + m * a.ldx;
-                const float x = __half2float(xr[s_auxsrc[col]]) * down;
-                a.aux_q[m * a.ld_aux + col] = (int8_t)quant_exact(x, s, qf);
-            }
-        }
-    } else
-    for (int row = warp; row < rows; row += kWarps) {
-        const size_t m = (size_t)r0 + row;
-        const uint4 *src = row < fit ? reinterpret_cast<const uint4 *>(slab + (size_t)row * K * 2)
-                                     : reinterpret_cast<const uint4 *>(a.X + m * a.ldx);
-        float s, inv_s;
-        {
+    } else {
+        const int r = min(s_r_true, a.cap);
+        const int used_cols = c * r, used_words = (used_cols + 3) >> 2;
+        for (int row = warp; row < rows; row += kWarps) {
+            const size_t m = (size_t)r0 + row;
+            const uint4 *src = row < fit ? reinterpret_cast<const uint4 *>(slab + (size_t)row * K * 2)
+                                         : reinterpret_cast<const uint4 *>(a.X + m * a.ldx);
             // per-token scale from Body's row (after the 2^-e redistribution)
             float mx = 0.0f;
             for (int ch = lane; ch < G; ch += 32) {
@@ -343,48 +305,74 @@ __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, int rows_base,
                 for (int i = 0; i < 8; ++i) mx = fmaxf(mx, fabsf(f[i]));
             }
             mx = warp_max(mx);
-            s = mx > 0.0f ? __fdiv_rn(mx, qf) : 1.0f;
-            inv_s = __fdiv_rn(1.0f, s);
-            if (lane == 0) a.s_x_rows[m] = s;
-        }
-        int8_t *q = a.body_q + m * a.ld_q;
-        for (int ch = lane; ch < G; ch += 32) {
-            float f[8];
-            load_chunk(src, ch, s_flag, s_colmul, f);
-            *reinterpret_cast<uint2 *>(q + ch * 8) = quant8(f, s, inv_s, qf);
-        }
-        if (a.aux_q) {
-            // shared scale: Aux_q[m, c*j + i] is the code Body_q[m, O_j] this warp has just written
-            __syncwarp();
-            for (int w = lane; w < (a.aux_cols >> 2); w += 32) {
-                uint32_t packed = 0;
-                if (w < used_words) {
+            const float sr = mx > 0.0f ? __fdiv_rn(mx, qf) : 1.0f;
+            const float inv_sr = __fdiv_rn(1.0f, sr);
+            if (lane == 0) a.s_x_rows[m] = sr;
+            int8_t *q = a.body_q + m * a.ld_q;
+            for (int ch = lane; ch < G; ch += 32) {
+                float f[8];
+                load_chunk(src, ch, s_flag, s_colmul, f);
+                *reinterpret_cast<uint2 *>(q + ch * 8) = quant8(f, sr, inv_sr, qf);
+            }
+            if (a.aux_q) {
+                // shared scale: Aux_q[m, c*j + i] is the code Body_q[m, O_j] this warp has just written
+                __syncwarp();
+                for (int w = lane; w < (a.aux_cols >> 2); w += 32) {
+                    uint32_t packed = 0;
+                    if (w < used_words) {
 #pragma unroll
-                    for (int bb = 0; bb < 4; ++bb)
-                        if (w * 4 + bb < used_cols) packed |= (uint32_t)(uint8_t)q[s_auxsrc[w * 4 + bb]] << (8 * bb);
+                        for (int bb = 0; bb < 4; ++bb)
+                            if (w * 4 + bb < used_cols)
+                                packed |= (uint32_t)(uint8_t)q[s_auxsrc[w * 4 + bb]] << (8 * bb);
+                    }
+                    *reinterpret_cast<uint32_t *>(a.aux_q + m * a.ld_aux + w * 4) = packed;
                 }
-                *reinterpret_cast<uint32_t *>(a.aux_q + m * a.ld_aux + w * 4) = packed;
             }
         }
     }
 
-    // ---------------------------------------------------------------- W_aux: first round, then the rest
-    if (wa_first < wa_total) {
-        const int n = wa_first / wa_words_per_row, w = wa_first - n * wa_words_per_row;
-        const uint32_t packed = (uint32_t)wa_byte[0] | ((uint32_t)wa_byte[1] << 8) | ((uint32_t)wa_byte[2] << 16) |
-                                ((uint32_t)wa_byte[3] << 24);
-        *reinterpret_cast<uint32_t *>(a.w_aux + (size_t)n * a.ld_waux + w * 4) = packed;
-    }
-    for (int i = wa_first + gridDim.x * kT; i < wa_total; i += gridDim.x * kT) {
-        const int n = i / wa_words_per_row, w = i - n * wa_words_per_row;
-        uint32_t packed = 0;
-        if (w < used_words) {
-#pragma unroll
-            for (int bb = 0; bb < 4; ++bb)
-                if (w * 4 + bb < used_cols)
-                    packed |= (uint32_t)(uint8_t)a.w_q[(size_t)n * a.ldw + s_auxsrc[w * 4 + bb]] << (8 * bb);
+    // ---------------------------------------------------------------- Aux block (per tensor) and W_aux
+    __syncthreads();  // warp 0's outlier list and Aux sources are complete
+    const int r = min(s_r_true, a.cap);
+    const int used_cols = c * r, used_words = (used_cols + 3) >> 2;
+    if (a.aux_q && !a.per_token) {
+        // Aux block of this CTA's rows: zero except the first c*r columns, where Aux_q[m, c*j + i] is the
+        // code of Body[m, O_j] (Eq. 5, shared scale), recomputed from the slab with the exact division,
+        // one (row, column) pair per thread.  Whole words beyond the used ones are cleared by other threads.
+        const int aux_words = a.aux_cols >> 2;
+        const int zwords = aux_words - used_words;
+        for (int i = t; i < rows * zwords; i += kT) {
+            const int row = i / zwords, w = used_words + (i - row * zwords);
+            *reinterpret_cast<uint32_t *>(a.aux_q + ((size_t)r0 + row) * a.ld_aux + w * 4) = 0u;
         }
-        *reinterpret_cast<uint32_t *>(a.w_aux + (size_t)n * a.ld_waux + w * 4) = packed;
+        const int bcols = used_words * 4;  // byte columns written here, the tail of the last word as zeros
+        for (int i = t; i < rows * bcols; i += kT) {
+            const int row = i / bcols, col = i - row * bcols;
+            const size_t m = (size_t)r0 + row;
+            int code = 0;
+            if (col < used_cols) {
+                const __half *xr = row < fit ? reinterpret_cast<const __half *>(slab + (size_t)row * K * 2)
+                                             : a.X + m * a.ldx;
+                code = quant_exact(__half2float(xr[s_auxsrc[col]]) * down, s, qf);
+            }
+            a.aux_q[m * a.ld_aux + col] = (int8_t)code;
+        }
+    }
+    // W_aux[n, c*j + i] = W_q[n, O_j], one 4-byte word per thread and round, spread over the grid
+    if (a.w_aux) {
+        const int words_per_row = a.aux_cols >> 2;
+        const int total = a.N * words_per_row;
+        for (int i = b * kT + t; i < total; i += gridDim.x * kT) {
+            const int n = i / words_per_row, w = i - n * words_per_row;
+            uint32_t packed = 0;
+            if (w < used_words) {
+#pragma unroll
+                for (int bb = 0; bb < 4; ++bb)
+                    if (w * 4 + bb < used_cols)
+                        packed |= (uint32_t)(uint8_t)a.w_q[(size_t)n * a.ldw + s_auxsrc[w * 4 + bb]] << (8 * bb);
+            }
+            *reinterpret_cast<uint32_t *>(a.w_aux + (size_t)n * a.ld_waux + w * 4) = packed;
+        }
     }
 }
 
