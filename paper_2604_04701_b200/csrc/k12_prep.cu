@@ -24,7 +24,7 @@ namespace muxq {
 
 namespace {
 
-constexpr int kT = 1024;
+constexpr int kT = 1024;  // the warp-group split of the last phase (512 + 256 + 256 threads) assumes this
 constexpr int kWarps = kT / 32;
 constexpr int kMaxK = 8 * kT;  // one group of 8 channels per thread
 constexpr int kMaxOut = 64;
@@ -180,18 +180,18 @@ __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, int rows_base,
         const float4 v1 = reinterpret_cast<const float4 *>(s_colmax)[2 * cg + 1];
         const float cm[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
         float bmax = 0.0f;
-        bool any = false;
+        uint32_t mask = 0;  // bit i: channel 8*cg + i is an outlier channel
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
             const bool flagged = cm[i] > a.tau;
             mul[i] = flagged ? down : 1.0f;
-            any |= flagged;
+            mask |= flagged ? (1u << i) : 0u;
             bmax = fmaxf(bmax, cm[i] * mul[i]);  // power-of-two scaling: exact
         }
-        if (row_off == 0) {  // shared copies for the per-token path
+        if (row_off == 0) {  // shared copies: the outlier listing below and the per-token path read them
             reinterpret_cast<float4 *>(s_colmul)[2 * cg] = make_float4(mul[0], mul[1], mul[2], mul[3]);
             reinterpret_cast<float4 *>(s_colmul)[2 * cg + 1] = make_float4(mul[4], mul[5], mul[6], mul[7]);
-            s_flag[cg] = any ? 1 : 0;
+            s_flag[cg] = (uint8_t)mask;
         }
         bmax = warp_max(bmax);
         if (lane == 0) s_warp_max[warp] = bmax;
@@ -201,33 +201,22 @@ __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, int rows_base,
     {
         const float mx = warp_max(s_warp_max[lane]);
         s = mx > 0.0f ? __fdiv_rn(mx, qf) : 1.0f;  // Eq. 1
-        inv_s = __fdiv_rn(1.0f, s);
+        inv_s = __frcp_rn(s);  // correctly rounded 1/s
         if (b == 0 && t == 0) {
             a.ctrl->s_x = s;
             a.ctrl->inv_s_x = inv_s;
         }
     }
-    // Warp 0 lists O in ascending order (the other warps do not need it until the Aux block) and the
-    // source channel of every Aux column: column c*j + i mirrors channel O_j (Eq. 5), repeated c times
-    // for the weighted sum of Eq. 7.
-    if (warp == 0) {
+    // The last warp (idle or lightly loaded in the quantization loop) lists O in ascending order from the
+    // per-group flag masks; nothing needs the list before the Aux block.  It also fills the source channel
+    // of every Aux column: column c*j + i mirrors channel O_j (Eq. 5), repeated c times for Eq. 7.
+    if (warp == kWarps - 1) {
         int carry = 0;
         for (int base = 0; base < G; base += 32) {
             const int g = base + lane;
-            float cm[8];
-            if (g < G) {
-                const float4 v0 = reinterpret_cast<const float4 *>(s_colmax)[2 * g];
-                const float4 v1 = reinterpret_cast<const float4 *>(s_colmax)[2 * g + 1];
-                cm[0] = v0.x; cm[1] = v0.y; cm[2] = v0.z; cm[3] = v0.w;
-                cm[4] = v1.x; cm[5] = v1.y; cm[6] = v1.z; cm[7] = v1.w;
-            } else {
-#pragma unroll
-                for (int i = 0; i < 8; ++i) cm[i] = 0.0f;
-            }
-            int cnt = 0;
-#pragma unroll
-            for (int i = 0; i < 8; ++i) cnt += (cm[i] > a.tau) ? 1 : 0;
-            if (!__any_sync(0xffffffffu, cnt != 0)) continue;
+            uint32_t m = g < G ? s_flag[g] : 0u;
+            if (!__any_sync(0xffffffffu, m != 0u)) continue;
+            const int cnt = __popc(m);
             int incl = cnt;
 #pragma unroll
             for (int o = 1; o < 32; o <<= 1) {
@@ -235,15 +224,14 @@ __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, int rows_base,
                 if (lane >= o) incl += n;
             }
             int pos = carry + incl - cnt;
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                if (cm[i] > a.tau) {
-                    if (pos < a.cap) {
-                        s_oidx[pos] = 8 * g + i;
-                        if (b == 0) a.outlier_idx[pos] = 8 * g + i;
-                    }
-                    ++pos;
+            while (m) {
+                const int i = __ffs(m) - 1;
+                m &= m - 1;
+                if (pos < a.cap) {
+                    s_oidx[pos] = 8 * g + i;
+                    if (b == 0) a.outlier_idx[pos] = 8 * g + i;
                 }
+                ++pos;
             }
             carry += __shfl_sync(0xffffffffu, incl, 31);
         }
@@ -335,34 +323,41 @@ __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, int rows_base,
     __syncthreads();  // warp 0's outlier list and Aux sources are complete
     const int r = min(s_r_true, a.cap);
     const int used_cols = c * r, used_words = (used_cols + 3) >> 2;
-    if (a.aux_q && !a.per_token) {
-        // Aux block of this CTA's rows: zero except the first c*r columns, where Aux_q[m, c*j + i] is the
-        // code of Body[m, O_j] (Eq. 5, shared scale), recomputed from the slab with the exact division,
-        // one (row, column) pair per thread.  Whole words beyond the used ones are cleared by other threads.
-        const int aux_words = a.aux_cols >> 2;
-        const int zwords = aux_words - used_words;
-        for (int i = t; i < rows * zwords; i += kT) {
-            const int row = i / zwords, w = used_words + (i - row * zwords);
-            *reinterpret_cast<uint32_t *>(a.aux_q + ((size_t)r0 + row) * a.ld_aux + w * 4) = 0u;
-        }
-        const int bcols = used_words * 4;  // byte columns written here, the tail of the last word as zeros
-        for (int i = t; i < rows * bcols; i += kT) {
-            const int row = i / bcols, col = i - row * bcols;
-            const size_t m = (size_t)r0 + row;
-            int code = 0;
-            if (col < used_cols) {
-                const __half *xr = row < fit ? reinterpret_cast<const __half *>(slab + (size_t)row * K * 2)
-                                             : a.X + m * a.ldx;
-                code = quant_exact(__half2float(xr[s_auxsrc[col]]) * down, s, qf);
+    // Three independent jobs share the CTA's warps so that their latencies overlap instead of adding up:
+    // warps 0-15 the Aux codes, warps 16-23 the Aux zero fill, warps 24-31 the W_aux gather.
+    const bool do_aux = a.aux_q && !a.per_token;
+    if (warp < 16) {
+        if (do_aux) {
+            // Aux_q[m, c*j + i] = code of Body[m, O_j] (Eq. 5, shared scale), recomputed from the slab with the
+            // exact division, one (row, column) pair per thread; the tail of the last used word is zero.
+            const int bcols = used_words * 4;
+            for (int i = t; i < rows * bcols; i += 512) {
+                const int row = i / bcols, col = i - row * bcols;
+                const size_t m = (size_t)r0 + row;
+                int code = 0;
+                if (col < used_cols) {
+                    const __half *xr = row < fit ? reinterpret_cast<const __half *>(slab + (size_t)row * K * 2)
+                                                 : a.X + m * a.ldx;
+                    code = quant_exact(__half2float(xr[s_auxsrc[col]]) * down, s, qf);
+                }
+                a.aux_q[m * a.ld_aux + col] = (int8_t)code;
             }
-            a.aux_q[m * a.ld_aux + col] = (int8_t)code;
         }
-    }
-    // W_aux[n, c*j + i] = W_q[n, O_j], one 4-byte word per thread and round, spread over the grid
-    if (a.w_aux) {
+    } else if (warp < 24) {
+        if (do_aux) {
+            // whole words of the Aux block beyond the used ones
+            const int aux_words = a.aux_cols >> 2;
+            const int zwords = aux_words - used_words;
+            for (int i = t - 512; i < rows * zwords; i += 256) {
+                const int row = i / zwords, w = used_words + (i - row * zwords);
+                *reinterpret_cast<uint32_t *>(a.aux_q + ((size_t)r0 + row) * a.ld_aux + w * 4) = 0u;
+            }
+        }
+    } else if (a.w_aux) {
+        // W_aux[n, c*j + i] = W_q[n, O_j], one 4-byte word per thread and round, spread over the grid
         const int words_per_row = a.aux_cols >> 2;
         const int total = a.N * words_per_row;
-        for (int i = b * kT + t; i < total; i += gridDim.x * kT) {
+        for (int i = b * 256 + (t - 768); i < total; i += gridDim.x * 256) {
             const int n = i / words_per_row, w = i - n * words_per_row;
             uint32_t packed = 0;
             if (w < used_words) {
