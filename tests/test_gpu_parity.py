@@ -370,3 +370,69 @@ def test_host_buffer_entry_point(mx):
     assert mx.muxq_read_status(ws) == 0
     _, _, res = oracle_linear(x, w, p)
     assert f16_ulp_diff(yh.numpy(), res.y16).max() <= 1
+
+
+# ------------------------------------------------------------------ full benchmark sizes, sampled rows
+def _full_size_check(mx, spec, gran, n_rows=48, cap=32):
+    """One layer at its full size through muxq_linear (the launch configuration bench.py times);
+    detection results and scales are compared in full, the products on seeded sample rows (each row of
+    the layer is independent once O and the scales are fixed, so the oracle computes them one by one)."""
+    x, _ = spec.x()
+    w = spec.w()
+    p = mx.MuxqParams(gran=gran, max_outliers=cap)
+    rng = np.random.default_rng(spec.seed * 1000 + spec.tensor_id)
+    rows = np.unique(np.concatenate([[0, spec.M - 1, 127, 128, spec.M // 2],
+                                     rng.integers(0, spec.M, n_rows)])).astype(np.int32)
+    rows = rows[rows < spec.M]
+    wq_o, sw_o, res = oracle_linear(x, w, p, rows=rows)
+    assert res.rc == 0 and res.r >= spec.n_outliers
+    y16, ws, st, w_q, s_w = run_linear(mx, x, w, p, mx.MUXQ_OUT_F16)
+    assert st == 0
+    v = ws_views(mx, ws, spec.M, spec.K, spec.N, p)
+    assert v["n_outliers"] == res.r and np.array_equal(v["outlier_idx"][:res.r], res.O)
+    assert np.array_equal(v["col_absmax"].view(np.uint32), res.colmax.view(np.uint32))
+    assert np.array_equal(v["s_x"].view(np.uint32), res.s_x.view(np.uint32))
+    assert np.array_equal(v["body_q"], res.body_q)          # every code of the full matrix
+    assert np.array_equal(w_q.cpu().numpy(), wq_o.T)
+    assert f16_ulp_diff(y16.cpu().numpy()[rows], res.y16).max() <= 1
+    acc, _, st, _, _ = run_linear(mx, x, w, p, mx.MUXQ_OUT_ACC_I32)
+    assert st == 0 and np.array_equal(acc.cpu().numpy()[rows], res.acc)
+    y32, _, st, _, _ = run_linear(mx, x, w, p, mx.MUXQ_OUT_F32)
+    assert st == 0 and rel_err32(y32.cpu().numpy()[rows], res.y32) <= 1e-5
+
+
+@pytest.mark.parametrize("gran", [0, 1])
+@pytest.mark.parametrize("layer", [0, 1, 2, 3])
+def test_config1_full_size_sampled_rows(mx, layer, gran):
+    _full_size_check(mx, synth.config_layers(1)[layer], gran)
+
+
+@pytest.mark.parametrize("layer", [0, 3])
+def test_config2_heavy_tailed_full_size_sampled_rows(mx, layer):
+    _full_size_check(mx, synth.config_layers(2)[layer], 0, cap=64)
+
+
+@pytest.mark.parametrize("layer", [1, 3])
+def test_config3_prefill_full_size_sampled_rows(mx, layer):
+    _full_size_check(mx, synth.config_layers(3)[layer], 0)
+
+
+@pytest.mark.parametrize("M", [1, 4, 16])
+def test_config3_decode_full_size(mx, M):
+    for spec in synth.config_layers(3, M=M):
+        x, _ = spec.x()
+        w = spec.w()
+        p = mx.MuxqParams(max_outliers=32)
+        _, _, res = oracle_linear(x, w, p)
+        y32, _, st, _, _ = run_linear(mx, x, w, p, mx.MUXQ_OUT_F32)
+        assert st == 0 and np.array_equal(y32.cpu().numpy(), res.y32)
+        y16, ws, st, _, _ = run_linear(mx, x, w, p, mx.MUXQ_OUT_F16)
+        assert st == 0 and f16_ulp_diff(y16.cpu().numpy(), res.y16).max() <= 1
+        v = ws_views(mx, ws, spec.M, spec.K, spec.N, p)
+        assert v["n_outliers"] == res.r and np.array_equal(v["outlier_idx"][:res.r], res.O)
+
+
+@pytest.mark.parametrize("n_out", [0, 2, 8, 32])
+def test_config4_outlier_sweep_full_size_sampled_rows(mx, n_out):
+    spec = synth.config_layers(4, n_outliers=n_out, layers=36)[35 * 4 + 2]   # last layer's c_fc, 8192 x 1280 -> 5120
+    _full_size_check(mx, spec, 0, cap=64)
