@@ -285,6 +285,28 @@ static int linear_impl(const void *X, int M, int K, int ldx, const int8_t *W_q, 
         if (events && events[i]) cudaEventRecordWithFlags(static_cast<cudaEvent_t>(events[i]), s, ev_flags);
     };
     mark(0);
+    if (decode && decode_fused_supported(M, K)) {
+        // M <= 16: one launch does the whole layer and needs no cleared scratch; it leaves colmax, O, r
+        // and the scale(s) in the workspace for inspection
+        DecodeFusedArgs k{};
+        k.X = static_cast<const __half *>(X);
+        k.M = M; k.K = K; k.ldx = ldx;
+        k.w_q = W_q; k.ldw = ldw; k.N = N;
+        k.s_w = s_w; k.per_vec = per_vec;
+        k.tau = p->threshold; k.exp_factor = p->exp_factor; k.qmax = qmax_of(p->act_bits);
+        k.cap = p->max_outliers; k.c = (1 << p->exp_factor) - 1;
+        k.Y = Y; k.ldy = ldy; k.out_kind = out_kind;
+        k.colmax = reinterpret_cast<float *>(ws + w.s.colmax);
+        k.outlier_idx = reinterpret_cast<int32_t *>(ws + w.s.oidx);
+        k.ctrl = ctrl;
+        k.s_x_rows = reinterpret_cast<float *>(ws + w.sx_rows);
+        k.dev_status = dev_status;
+        mark(1);
+        mark(2);
+        const cudaError_t ed = launch_decode_fused(k, s);
+        mark(3);
+        return cuda_rc(ed);
+    }
     cudaError_t e = cudaMemsetAsync(ws, 0, fused ? w.colmax_rep + (size_t)kPrepColmaxReplicas * K * 4
                                                  : w.s.colmax + (size_t)K * 4, s);
     if (e == cudaSuccess && !fused) e = cudaMemsetAsync(dev_status, 0, 4, s);  // the fused kernel clears it itself

@@ -1,0 +1,323 @@
+// K4, fused form: the whole MUXQ layer for M <= 16 token rows in ONE launch -- detection (Section
+// III-C), redistribution (Eq. 4-5), quantization (Eq. 1), the INT8 products with the Aux correction
+// (Eq. 7) and the dequantization (Eq. 3).  At these sizes the layer is a stream over W_q (N*K bytes)
+// and everything else is small, so:
+//   prologue  every CTA reads the few rows of X itself (twice, from L2), derives the channel maxima, the
+//             outlier flags, the scale(s) and the INT8 codes of X into shared memory -- redundant work
+//             per CTA, but no grid-wide barrier, no scratch in global memory and no second launch.
+//   stream    a CTA takes 8 output channels at a time; its 16 warps split K into 64-byte segments.
+//             A lane loads 16 bytes of one W_q row (8 rows x 64 contiguous bytes per warp load), the
+//             matching 16 bytes of X codes come from shared memory, and two mma.sync m16n8k32 (s8 x s8
+//             -> s32) consume them.  The K order inside a segment is permuted the same way for both
+//             operands (lane q of a row holds bytes 16q..16q+15), which a dot product does not notice.
+//             Aux term with the shared scale: Aux_q == Body_q[:, O], so c * sum_{k in O} is a second
+//             accumulation with X masked to the outlier channels, issued only for segments that hold one.
+//   finish    the 16 partial 16x8 tiles are summed through shared memory, combined as acc_b + c*acc_a
+//             (int32, exact), dequantized and stored.
+// Tensor-core use here is the small legacy mma.sync form on purpose: the path is bound by the W_q
+// stream, and mma.sync needs no TMEM or descriptor set-up for 8-column tiles.
+#include "kernels.h"
+#include "quant.cuh"
+
+namespace muxq {
+
+namespace {
+
+constexpr int kT = 512;
+constexpr int kWarps = kT / 32;
+constexpr int kMaxIter = 2;           // channel groups (8 channels) per thread: K <= 8 * kT * kMaxIter
+constexpr int kStatusCapacity = 5;    // MUXQ_ERR_CAPACITY
+
+__device__ __forceinline__ void mma_s8(int (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                       uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k32.row.col.s32.s8.s8.s32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+        "{%0, %1, %2, %3};"
+        : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+struct Smem {
+    int pitch;          // bytes per row of X codes; pitch % 128 == 64 keeps the 8-row x 64-byte reads conflict free
+    int off_mask;       // [K] 0xFF at outlier channels
+    int off_segflag;    // [K/64] segment holds an outlier channel
+    int off_grpmask;    // [K/8] per-group flag bits
+    int off_red;        // [2][kWarps][128] int32 partial tiles
+    int total;
+};
+__host__ __device__ inline Smem smem_layout(int MT, int K) {
+    Smem s;
+    s.pitch = K + ((64 - (K & 127)) & 127);
+    if ((s.pitch & 127) != 64) s.pitch += 64;
+    s.off_mask = MT * s.pitch;
+    s.off_segflag = s.off_mask + K;
+    s.off_grpmask = s.off_segflag + (((K >> 6) + 15) & ~15);
+    s.off_red = (s.off_grpmask + (K >> 3) + 15) & ~15;
+    s.total = s.off_red + 2 * kWarps * 128 * 4;
+    return s;
+}
+
+template <int MT>
+__global__ void __launch_bounds__(kT) k_decode_fused(const DecodeFusedArgs a) {
+    extern __shared__ __align__(16) uint8_t smem[];
+    __shared__ uint32_t s_rowmax[16];  // bit patterns of non-negative floats (per-token row maxima of Body)
+    __shared__ float s_wmax[kWarps];
+    __shared__ float s_rowscale[16];
+    __shared__ int s_r;
+
+    const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
+    const int K = a.K, G = K >> 3, M = a.M;
+    const Smem L = smem_layout(MT, K);
+    int8_t *xq = reinterpret_cast<int8_t *>(smem);
+    uint8_t *s_mask = smem + L.off_mask;
+    uint8_t *s_segflag = smem + L.off_segflag;
+    uint8_t *s_grpmask = smem + L.off_grpmask;
+    int *s_red = reinterpret_cast<int *>(smem + L.off_red);
+    const float down = __int_as_float((127 - a.exp_factor) << 23);  // 2^-e
+    const float qf = (float)a.qmax;
+    const bool first = blockIdx.x == 0;
+
+    if (first && t == 0 && a.dev_status) *a.dev_status = 0;
+    if (t < 16) s_rowmax[t] = 0u;
+    for (int i = t; i < (K >> 6); i += kT) s_segflag[i] = 0;
+    __syncthreads();
+
+    // ---------------------------------------------------------------- pass A: channel maxima, flags, Body maxima
+    uint32_t my_mask[kMaxIter];
+    float bmax = 0.0f;
+#pragma unroll
+    for (int it = 0; it < kMaxIter; ++it) {
+        my_mask[it] = 0;
+        const int cg = t + it * kT;
+        if (cg < G) {
+            __half2 cm[4];
+            cm[0] = cm[1] = cm[2] = cm[3] = __float2half2_rn(0.f);
+            for (int m = 0; m < M; ++m) {
+                const uint4 v = __ldg(reinterpret_cast<const uint4 *>(a.X + (size_t)m * a.ldx) + cg);
+                cm[0] = __hmax2(cm[0], __habs2(*reinterpret_cast<const __half2 *>(&v.x)));
+                cm[1] = __hmax2(cm[1], __habs2(*reinterpret_cast<const __half2 *>(&v.y)));
+                cm[2] = __hmax2(cm[2], __habs2(*reinterpret_cast<const __half2 *>(&v.z)));
+                cm[3] = __hmax2(cm[3], __habs2(*reinterpret_cast<const __half2 *>(&v.w)));
+            }
+            float c8[8];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) { c8[2 * i] = __low2float(cm[i]); c8[2 * i + 1] = __high2float(cm[i]); }
+            uint32_t mask = 0;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const bool flagged = c8[i] > a.tau;  // strict
+                mask |= flagged ? (1u << i) : 0u;
+                bmax = fmaxf(bmax, flagged ? c8[i] * down : c8[i]);
+            }
+            my_mask[it] = mask;
+            s_grpmask[cg] = (uint8_t)mask;
+            if (mask) s_segflag[cg >> 3] = 1;
+            uint2 mb;
+            mb.x = ((mask & 1) ? 0xFFu : 0u) | ((mask & 2) ? 0xFF00u : 0u) | ((mask & 4) ? 0xFF0000u : 0u) |
+                   ((mask & 8) ? 0xFF000000u : 0u);
+            mb.y = ((mask & 16) ? 0xFFu : 0u) | ((mask & 32) ? 0xFF00u : 0u) | ((mask & 64) ? 0xFF0000u : 0u) |
+                   ((mask & 128) ? 0xFF000000u : 0u);
+            *reinterpret_cast<uint2 *>(s_mask + cg * 8) = mb;
+            if (first && a.colmax) {
+                reinterpret_cast<float4 *>(a.colmax)[2 * cg] = make_float4(c8[0], c8[1], c8[2], c8[3]);
+                reinterpret_cast<float4 *>(a.colmax)[2 * cg + 1] = make_float4(c8[4], c8[5], c8[6], c8[7]);
+            }
+        }
+    }
+    if (a.per_vec) {
+        // per-token scales: row maxima of Body (after the 2^-e), a second cheap sweep with the flags known
+#pragma unroll
+        for (int it = 0; it < kMaxIter; ++it) {
+            const int cg = t + it * kT;
+            if (cg < G) {
+                for (int m = 0; m < M; ++m) {
+                    const uint4 v = __ldg(reinterpret_cast<const uint4 *>(a.X + (size_t)m * a.ldx) + cg);
+                    float f[8];
+                    unpack8(v, f);
+                    float rm = 0.0f;
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) rm = fmaxf(rm, fabsf((my_mask[it] >> i) & 1u ? f[i] * down : f[i]));
+                    if (rm > 0.0f) atomicMax(&s_rowmax[m], __float_as_uint(rm));
+                }
+            }
+        }
+    }
+    bmax = warp_max(bmax);
+    if (lane == 0) s_wmax[warp] = bmax;
+    __syncthreads();
+    // ---------------------------------------------------------------- scales (Eq. 1)
+    if (t < 16) {
+        float s;
+        if (a.per_vec) {
+            const float mx = __uint_as_float(s_rowmax[t]);
+            s = mx > 0.0f ? __fdiv_rn(mx, qf) : 1.0f;
+            if (first && t < M && a.s_x_rows) a.s_x_rows[t] = s;
+        } else {
+            float mx = 0.0f;
+#pragma unroll
+            for (int w = 0; w < kWarps; ++w) mx = fmaxf(mx, s_wmax[w]);
+            s = mx > 0.0f ? __fdiv_rn(mx, qf) : 1.0f;
+            if (first && t == 0 && a.ctrl) { a.ctrl->s_x = s; a.ctrl->inv_s_x = __frcp_rn(s); }
+        }
+        s_rowscale[t] = s;
+    }
+    // warp 1 lists O in ascending order for the caller (the products below only need the flags)
+    if (warp == 1 && first) {
+        int carry = 0;
+        for (int base = 0; base < G; base += 32) {
+            const int g = base + lane;
+            uint32_t m = g < G ? s_grpmask[g] : 0u;
+            if (!__any_sync(0xffffffffu, m != 0u)) continue;
+            const int cnt = __popc(m);
+            int incl = cnt;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int n = __shfl_up_sync(0xffffffffu, incl, o);
+                if (lane >= o) incl += n;
+            }
+            int pos = carry + incl - cnt;
+            while (m) {
+                const int i = __ffs(m) - 1;
+                m &= m - 1;
+                if (pos < a.cap && a.outlier_idx) a.outlier_idx[pos] = 8 * g + i;
+                ++pos;
+            }
+            carry += __shfl_sync(0xffffffffu, incl, 31);
+        }
+        if (lane == 0) {
+            if (a.ctrl) a.ctrl->n_outliers = carry;
+            if (carry > a.cap && a.dev_status) atomicMax(a.dev_status, kStatusCapacity);
+        }
+    }
+    if (warp == 2) {  // every CTA needs r only to know whether the capacity was exceeded
+        int cnt = 0;
+        for (int g = lane; g < G; g += 32) cnt += __popc((uint32_t)s_grpmask[g]);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
+        if (lane == 0) s_r = cnt;
+    }
+    __syncthreads();
+
+    // ---------------------------------------------------------------- pass B: codes of X into shared memory
+#pragma unroll
+    for (int it = 0; it < kMaxIter; ++it) {
+        const int cg = t + it * kT;
+        if (cg < G) {
+            float mul[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) mul[i] = (my_mask[it] >> i) & 1u ? down : 1.0f;
+            for (int m = 0; m < MT; ++m) {
+                uint2 code = make_uint2(0u, 0u);
+                if (m < M) {
+                    const uint4 v = __ldg(reinterpret_cast<const uint4 *>(a.X + (size_t)m * a.ldx) + cg);
+                    float f[8];
+                    unpack8(v, f);
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) f[i] *= mul[i];  // exact
+                    const float s = s_rowscale[a.per_vec ? m : 0];
+                    code = quant8(f, s, __frcp_rn(s), qf);
+                }
+                *reinterpret_cast<uint2 *>(xq + m * L.pitch + cg * 8) = code;
+            }
+        }
+    }
+    __syncthreads();
+    if (s_r > a.cap) return;  // MUXQ_ERR_CAPACITY was raised; Y is unspecified
+
+    // ---------------------------------------------------------------- stream W_q, 8 output channels at a time
+    const int r = lane >> 2, q = lane & 3;
+    const int nseg = K >> 6;
+    const int tiles = (a.N + 7) >> 3;
+    for (int tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
+        const int n0 = tile * 8;
+        const int n = n0 + r;
+        const int8_t *wrow = a.w_q + (size_t)min(n, a.N - 1) * a.ldw + q * 16;
+        const int8_t *xlo = xq + r * L.pitch + q * 16;
+        int accb[4] = {0, 0, 0, 0}, acca[4] = {0, 0, 0, 0};
+        for (int seg0 = warp; seg0 < nseg; seg0 += 4 * kWarps) {
+            uint4 wv[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int seg = seg0 + u * kWarps;
+                wv[u] = seg < nseg ? __ldg(reinterpret_cast<const uint4 *>(wrow + seg * 64)) : make_uint4(0u, 0u, 0u, 0u);
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int seg = seg0 + u * kWarps;
+                if (seg < nseg) {
+                    const uint4 alo = *reinterpret_cast<const uint4 *>(xlo + seg * 64);
+                    uint4 ahi = make_uint4(0u, 0u, 0u, 0u);
+                    if (MT == 16) ahi = *reinterpret_cast<const uint4 *>(xlo + 8 * L.pitch + seg * 64);
+                    mma_s8(accb, alo.x, ahi.x, alo.y, ahi.y, wv[u].x, wv[u].y);
+                    mma_s8(accb, alo.z, ahi.z, alo.w, ahi.w, wv[u].z, wv[u].w);
+                    if (s_segflag[seg]) {  // warp-uniform: Aux term on the outlier channels of this segment
+                        const uint4 mk = *reinterpret_cast<const uint4 *>(s_mask + seg * 64 + q * 16);
+                        mma_s8(acca, alo.x & mk.x, ahi.x & mk.x, alo.y & mk.y, ahi.y & mk.y, wv[u].x, wv[u].y);
+                        mma_s8(acca, alo.z & mk.z, ahi.z & mk.z, alo.w & mk.w, ahi.w & mk.w, wv[u].z, wv[u].w);
+                    }
+                }
+            }
+        }
+        // acc = acc_b + c * acc_a (Eq. 7), partial over this warp's K segments; element (row, col) of the
+        // 16 x 8 tile: this lane holds rows r and r+8, columns 2q and 2q+1
+        int *red = s_red + warp * 128;
+        red[r * 8 + 2 * q] = accb[0] + a.c * acca[0];
+        red[r * 8 + 2 * q + 1] = accb[1] + a.c * acca[1];
+        red[(r + 8) * 8 + 2 * q] = accb[2] + a.c * acca[2];
+        red[(r + 8) * 8 + 2 * q + 1] = accb[3] + a.c * acca[3];
+        __syncthreads();
+        if (t < 128) {
+            int acc = 0;
+#pragma unroll
+            for (int w = 0; w < kWarps; ++w) acc += s_red[w * 128 + t];
+            const int m = t >> 3, nn = n0 + (t & 7);
+            if (m < M && nn < a.N) {
+                const size_t o = (size_t)m * a.ldy + nn;
+                if (a.out_kind == 2) {
+                    reinterpret_cast<int32_t *>(a.Y)[o] = acc;
+                } else {
+                    const float sx = s_rowscale[a.per_vec ? m : 0];
+                    const float sw = a.per_vec ? __ldg(a.s_w + nn) : __ldg(a.s_w);
+                    const float y = __fmul_rn(__fmul_rn(sx, sw), __int2float_rn(acc));  // Eq. 3
+                    if (a.out_kind == 1) reinterpret_cast<float *>(a.Y)[o] = y;
+                    else reinterpret_cast<__half *>(a.Y)[o] = __float2half_rn(y);
+                }
+            }
+        }
+        __syncthreads();
+    }
+}
+
+}  // namespace
+
+bool decode_fused_supported(int M, int K) { return M >= 1 && M <= 16 && K % 64 == 0 && K <= 8 * kT * kMaxIter; }
+
+cudaError_t launch_decode_fused(const DecodeFusedArgs &a, cudaStream_t s) {
+    const int MT = a.M <= 8 ? 8 : 16;
+    const Smem L = smem_layout(MT, a.K);
+    static bool attr8 = false, attr16 = false;
+    cudaError_t e;
+    if (MT == 8 && !attr8) {
+        e = cudaFuncSetAttribute(k_decode_fused<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+        if (e != cudaSuccess) return e;
+        attr8 = true;
+    }
+    if (MT == 16 && !attr16) {
+        e = cudaFuncSetAttribute(k_decode_fused<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+        if (e != cudaSuccess) return e;
+        attr16 = true;
+    }
+    if (L.total > 200 * 1024) return cudaErrorInvalidValue;
+    // CTAs per SM by shared memory and by threads (2048 / 512), then a strided loop over the 8-channel tiles
+    int per_sm = (int)((227 * 1024) / (L.total + 2048));
+    if (per_sm > 4) per_sm = 4;
+    if (per_sm < 1) per_sm = 1;
+    const int tiles = (a.N + 7) / 8;
+    int grid = num_sms() * per_sm;
+    if (grid > tiles) grid = tiles;
+    if (MT == 8) k_decode_fused<8><<<grid, kT, L.total, s>>>(a);
+    else k_decode_fused<16><<<grid, kT, L.total, s>>>(a);
+    return cudaGetLastError();
+}
+
+}  // namespace muxq

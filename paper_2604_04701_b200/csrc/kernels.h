@@ -125,6 +125,22 @@ struct DecodeArgs {
 };
 cudaError_t launch_decode(const DecodeArgs &a, cudaStream_t s);
 
+// Whole layer for M <= 16 in one launch (no scratch needed; the optional outputs are for inspection).
+struct DecodeFusedArgs {
+    const __half *X; int M, K, ldx;
+    const int8_t *w_q; int ldw; int N;
+    const float *s_w; int per_vec;      // per-token X scales and per-channel W scales, or one of each
+    float tau; int exp_factor, qmax, cap, c;
+    void *Y; int ldy; int out_kind;
+    float *colmax;                      // [K] out or NULL
+    int32_t *outlier_idx;               // [cap] out or NULL
+    Ctrl *ctrl;                         // out or NULL: n_outliers, s_x
+    float *s_x_rows;                    // [M] out or NULL (per-token scales)
+    int32_t *dev_status;                // set to 0, raised to MUXQ_ERR_CAPACITY when r > cap
+};
+bool decode_fused_supported(int M, int K);
+cudaError_t launch_decode_fused(const DecodeFusedArgs &a, cudaStream_t s);
+
 cudaError_t launch_mma_peak(int n, int iters, unsigned long long *cycles_out, int32_t *status, int grid,
                             cudaStream_t s);
 
