@@ -25,6 +25,7 @@ namespace {
 
 constexpr int kT = 512;
 constexpr int kWarps = kT / 32;
+constexpr int kPre = 8;               // 64-byte W segments per warp fetched ahead of the prologue
 constexpr int kMaxIter = 2;           // channel groups (8 channels) per thread: K <= 8 * kT * kMaxIter
 constexpr int kStatusCapacity = 5;    // MUXQ_ERR_CAPACITY
 
@@ -58,7 +59,7 @@ __host__ __device__ inline Smem smem_layout(int MT, int K) {
 }
 
 template <int MT>
-__global__ void __launch_bounds__(kT) k_decode_fused(const DecodeFusedArgs a) {
+__global__ void __launch_bounds__(kT, 1) k_decode_fused(const DecodeFusedArgs a, int tpg) {
     extern __shared__ __align__(16) uint8_t smem[];
     __shared__ uint32_t s_rowmax[16];  // bit patterns of non-negative floats (per-token row maxima of Body)
     __shared__ float s_wmax[kWarps];
@@ -77,6 +78,28 @@ __global__ void __launch_bounds__(kT) k_decode_fused(const DecodeFusedArgs a) {
     const float qf = (float)a.qmax;
     const bool first = blockIdx.x == 0;
 
+    // The first tile's share of W_q does not depend on X: its loads go out before the prologue, so the
+    // HBM latency of the stream overlaps the detection and quantization work.
+    const int r = lane >> 2, q = lane & 3;
+    const int nseg = K >> 6;
+    const int tiles = (a.N + 7) >> 3;
+    const int ws = kWarps / tpg;             // warps per team
+    const int team = warp / ws, wi = warp - team * ws;
+    uint4 wpre[kPre];
+    {
+        const int n = (blockIdx.x * tpg + team) * 8 + r;
+        const int8_t *wrow = a.w_q + (size_t)min(n, a.N - 1) * a.ldw + q * 16;
+#pragma unroll
+        for (int u = 0; u < kPre; ++u) {
+            const int seg = wi + u * ws;
+            wpre[u] = seg < nseg ? __ldg(reinterpret_cast<const uint4 *>(wrow + seg * 64)) : make_uint4(0u, 0u, 0u, 0u);
+        }
+    }
+    // Everything below reads X or writes results: under programmatic dependent launch it must wait for the
+    // kernel before this one in the stream; the weights above are constants and were fetched ahead of that.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+
     if (first && t == 0 && a.dev_status) *a.dev_status = 0;
     if (t < 16) s_rowmax[t] = 0u;
     for (int i = t; i < (K >> 6); i += kT) s_segflag[i] = 0;
@@ -92,12 +115,19 @@ __global__ void __launch_bounds__(kT) k_decode_fused(const DecodeFusedArgs a) {
         if (cg < G) {
             __half2 cm[4];
             cm[0] = cm[1] = cm[2] = cm[3] = __float2half2_rn(0.f);
-            for (int m = 0; m < M; ++m) {
-                const uint4 v = __ldg(reinterpret_cast<const uint4 *>(a.X + (size_t)m * a.ldx) + cg);
-                cm[0] = __hmax2(cm[0], __habs2(*reinterpret_cast<const __half2 *>(&v.x)));
-                cm[1] = __hmax2(cm[1], __habs2(*reinterpret_cast<const __half2 *>(&v.y)));
-                cm[2] = __hmax2(cm[2], __habs2(*reinterpret_cast<const __half2 *>(&v.z)));
-                cm[3] = __hmax2(cm[3], __habs2(*reinterpret_cast<const __half2 *>(&v.w)));
+            for (int m0 = 0; m0 < M; m0 += 4) {  // four independent row loads in flight
+                uint4 v[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u)
+                    v[u] = m0 + u < M ? __ldg(reinterpret_cast<const uint4 *>(a.X + (size_t)(m0 + u) * a.ldx) + cg)
+                                      : make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    cm[0] = __hmax2(cm[0], __habs2(*reinterpret_cast<const __half2 *>(&v[u].x)));
+                    cm[1] = __hmax2(cm[1], __habs2(*reinterpret_cast<const __half2 *>(&v[u].y)));
+                    cm[2] = __hmax2(cm[2], __habs2(*reinterpret_cast<const __half2 *>(&v[u].z)));
+                    cm[3] = __hmax2(cm[3], __habs2(*reinterpret_cast<const __half2 *>(&v[u].w)));
+                }
             }
             float c8[8];
 #pragma unroll
@@ -206,56 +236,65 @@ __global__ void __launch_bounds__(kT) k_decode_fused(const DecodeFusedArgs a) {
             float mul[8];
 #pragma unroll
             for (int i = 0; i < 8; ++i) mul[i] = (my_mask[it] >> i) & 1u ? down : 1.0f;
-            for (int m = 0; m < MT; ++m) {
-                uint2 code = make_uint2(0u, 0u);
-                if (m < M) {
-                    const uint4 v = __ldg(reinterpret_cast<const uint4 *>(a.X + (size_t)m * a.ldx) + cg);
-                    float f[8];
-                    unpack8(v, f);
+            for (int m0 = 0; m0 < MT; m0 += 4) {  // four independent row loads in flight
+                uint4 v[4];
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) f[i] *= mul[i];  // exact
-                    const float s = s_rowscale[a.per_vec ? m : 0];
-                    code = quant8(f, s, __frcp_rn(s), qf);
+                for (int u = 0; u < 4; ++u)
+                    v[u] = m0 + u < M ? __ldg(reinterpret_cast<const uint4 *>(a.X + (size_t)(m0 + u) * a.ldx) + cg)
+                                      : make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int m = m0 + u;
+                    uint2 code = make_uint2(0u, 0u);
+                    if (m < M) {
+                        float f[8];
+                        unpack8(v[u], f);
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) f[i] *= mul[i];  // exact
+                        const float s = s_rowscale[a.per_vec ? m : 0];
+                        code = quant8(f, s, __frcp_rn(s), qf);
+                    }
+                    *reinterpret_cast<uint2 *>(xq + m * L.pitch + cg * 8) = code;
                 }
-                *reinterpret_cast<uint2 *>(xq + m * L.pitch + cg * 8) = code;
             }
         }
     }
     __syncthreads();
     if (s_r > a.cap) return;  // MUXQ_ERR_CAPACITY was raised; Y is unspecified
 
-    // ---------------------------------------------------------------- stream W_q, 8 output channels at a time
-    const int r = lane >> 2, q = lane & 3;
-    const int nseg = K >> 6;
-    const int tiles = (a.N + 7) >> 3;
-    for (int tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
-        const int n0 = tile * 8;
-        const int n = n0 + r;
-        const int8_t *wrow = a.w_q + (size_t)min(n, a.N - 1) * a.ldw + q * 16;
+    // ---------------------------------------------------------------- stream W_q
+    // A CTA works on a group of tpg 8-channel tiles at a time; team j of its warps takes tile j of the
+    // group and splits K among its members, so that every lane keeps several 16-byte loads in flight
+    // whatever K is.
+    const int groups = (tiles + tpg - 1) / tpg;
+    for (int group = blockIdx.x; group < groups; group += gridDim.x) {
         const int8_t *xlo = xq + r * L.pitch + q * 16;
         int accb[4] = {0, 0, 0, 0}, acca[4] = {0, 0, 0, 0};
-        for (int seg0 = warp; seg0 < nseg; seg0 += 4 * kWarps) {
-            uint4 wv[4];
+        // this warp's segments (at most kPre by the choice of tpg) are already in registers
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const int seg = seg0 + u * kWarps;
-                wv[u] = seg < nseg ? __ldg(reinterpret_cast<const uint4 *>(wrow + seg * 64)) : make_uint4(0u, 0u, 0u, 0u);
-            }
-#pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const int seg = seg0 + u * kWarps;
-                if (seg < nseg) {
-                    const uint4 alo = *reinterpret_cast<const uint4 *>(xlo + seg * 64);
-                    uint4 ahi = make_uint4(0u, 0u, 0u, 0u);
-                    if (MT == 16) ahi = *reinterpret_cast<const uint4 *>(xlo + 8 * L.pitch + seg * 64);
-                    mma_s8(accb, alo.x, ahi.x, alo.y, ahi.y, wv[u].x, wv[u].y);
-                    mma_s8(accb, alo.z, ahi.z, alo.w, ahi.w, wv[u].z, wv[u].w);
-                    if (s_segflag[seg]) {  // warp-uniform: Aux term on the outlier channels of this segment
-                        const uint4 mk = *reinterpret_cast<const uint4 *>(s_mask + seg * 64 + q * 16);
-                        mma_s8(acca, alo.x & mk.x, ahi.x & mk.x, alo.y & mk.y, ahi.y & mk.y, wv[u].x, wv[u].y);
-                        mma_s8(acca, alo.z & mk.z, ahi.z & mk.z, alo.w & mk.w, ahi.w & mk.w, wv[u].z, wv[u].w);
-                    }
+        for (int u = 0; u < kPre; ++u) {
+            const int seg = wi + u * ws;
+            if (seg < nseg) {
+                const uint4 alo = *reinterpret_cast<const uint4 *>(xlo + seg * 64);
+                uint4 ahi = make_uint4(0u, 0u, 0u, 0u);
+                if (MT == 16) ahi = *reinterpret_cast<const uint4 *>(xlo + 8 * L.pitch + seg * 64);
+                mma_s8(accb, alo.x, ahi.x, alo.y, ahi.y, wpre[u].x, wpre[u].y);
+                mma_s8(accb, alo.z, ahi.z, alo.w, ahi.w, wpre[u].z, wpre[u].w);
+                if (s_segflag[seg]) {  // warp-uniform: Aux term on the outlier channels of this segment
+                    const uint4 mk = *reinterpret_cast<const uint4 *>(s_mask + seg * 64 + q * 16);
+                    mma_s8(acca, alo.x & mk.x, ahi.x & mk.x, alo.y & mk.y, ahi.y & mk.y, wpre[u].x, wpre[u].y);
+                    mma_s8(acca, alo.z & mk.z, ahi.z & mk.z, alo.w & mk.w, ahi.w & mk.w, wpre[u].z, wpre[u].w);
                 }
+            }
+        }
+        // fetch the next group's segments now; they arrive while this group is reduced and stored
+        if (group + (int)gridDim.x < groups) {
+            const int nn0 = ((group + gridDim.x) * tpg + team) * 8;
+            const int8_t *wnext = a.w_q + (size_t)min(nn0 + r, a.N - 1) * a.ldw + q * 16;
+#pragma unroll
+            for (int u = 0; u < kPre; ++u) {
+                const int seg = wi + u * ws;
+                if (seg < nseg) wpre[u] = __ldg(reinterpret_cast<const uint4 *>(wnext + seg * 64));
             }
         }
         // acc = acc_b + c * acc_a (Eq. 7), partial over this warp's K segments; element (row, col) of the
@@ -266,11 +305,11 @@ __global__ void __launch_bounds__(kT) k_decode_fused(const DecodeFusedArgs a) {
         red[(r + 8) * 8 + 2 * q] = accb[2] + a.c * acca[2];
         red[(r + 8) * 8 + 2 * q + 1] = accb[3] + a.c * acca[3];
         __syncthreads();
-        if (t < 128) {
+        for (int e = t; e < 128 * tpg; e += kT) {
+            const int j = e >> 7, el = e & 127;  // tile of the group, element of its 16 x 8 tile
             int acc = 0;
-#pragma unroll
-            for (int w = 0; w < kWarps; ++w) acc += s_red[w * 128 + t];
-            const int m = t >> 3, nn = n0 + (t & 7);
+            for (int w = 0; w < ws; ++w) acc += s_red[(j * ws + w) * 128 + el];
+            const int m = el >> 3, nn = (group * tpg + j) * 8 + (el & 7);
             if (m < M && nn < a.N) {
                 const size_t o = (size_t)m * a.ldy + nn;
                 if (a.out_kind == 2) {
@@ -308,16 +347,26 @@ cudaError_t launch_decode_fused(const DecodeFusedArgs &a, cudaStream_t s) {
         attr16 = true;
     }
     if (L.total > 200 * 1024) return cudaErrorInvalidValue;
-    // CTAs per SM by shared memory and by threads (2048 / 512), then a strided loop over the 8-channel tiles
-    int per_sm = (int)((227 * 1024) / (L.total + 2048));
-    if (per_sm > 4) per_sm = 4;
-    if (per_sm < 1) per_sm = 1;
-    const int tiles = (a.N + 7) / 8;
-    int grid = num_sms() * per_sm;
-    if (grid > tiles) grid = tiles;
-    if (MT == 8) k_decode_fused<8><<<grid, kT, L.total, s>>>(a);
-    else k_decode_fused<16><<<grid, kT, L.total, s>>>(a);
-    return cudaGetLastError();
+    // tiles per group: the smallest power of two that gives every warp at least 4 segments of 64 bytes
+    const int nseg = a.K / 64, tiles = (a.N + 7) / 8;
+    int tpg = 1;
+    while (tpg < kWarps && nseg * tpg < 4 * kWarps) tpg *= 2;
+    const int groups = (tiles + tpg - 1) / tpg;
+    // at most one CTA per SM, so that the kernel of the next layer in the stream can become resident beside
+    // this one (programmatic dependent launch) and fetch its weights while this one finishes
+    int grid = num_sms();
+    if (grid > groups) grid = groups;
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(kT);
+    cfg.dynamicSmemBytes = (size_t)L.total;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    if (MT == 8) return cudaLaunchKernelEx(&cfg, k_decode_fused<8>, a, tpg);
+    return cudaLaunchKernelEx(&cfg, k_decode_fused<16>, a, tpg);
 }
 
 }  // namespace muxq
