@@ -339,6 +339,57 @@ def run_muxq(args, rank, world):
            "d2h_bytes_per_step": int(sum(yh.numel() * 2 for _, yh in hosts)), "steps": esteps,
            "ms_per_step": ems / esteps}
 
+    # ---- decode shapes (M <= 16): the 36 x 4 GPT-2-large linears as one stream of layers with distinct
+    # weights (708 MB of W_q, far more than the L2 holds), replayed from a graph; GB/s = W_q bytes / time
+    decode = None
+    if world == 1 and not args.no_decode:
+        d = 1280
+        dshapes = [(d, 3 * d), (d, d), (d, 4 * d), (4 * d, d)]
+        gen = torch.Generator(device=dev)
+        gen.manual_seed(4)
+        dlayers = []
+        for _ in range(36):
+            for (K, N) in dshapes:
+                dlayers.append((K, N, torch.randint(-127, 128, (N, K), dtype=torch.int8, device=dev, generator=gen)))
+        wbytes = sum(K * N for K, N, _ in dlayers)
+        sw1 = torch.full((1,), 0.02 / 127.0, device=dev)
+        decode = {"workload": "configs[3]/[4] decode: 36 x (1280->3840, 1280->1280, 1280->5120, 5120->1280), "
+                              "8 outlier channels x60, per-tensor INT8, one fused launch per layer",
+                  "w_bytes": wbytes, "layers": len(dlayers), "hbm_peak_gbs": peaks["hbm_gbs"]}
+        for Md in (1, 4, 16):
+            dx = {K: torch.from_numpy(synth.make_x(3, 100 + K, Md, K, 8, 60.0, 60.0)[0]).to(dev) for K in (d, 4 * d)}
+            dy = {N: torch.empty(Md, N, dtype=torch.float16, device=dev) for N in (d, 3 * d, 4 * d)}
+            dws = {K: mx.Workspace(mx.muxq_workspace_bytes(Md, K, 4 * d, p), dev) for K in (d, 4 * d)}
+
+            def chain():
+                for (K, N, wq) in dlayers:
+                    mx.muxq_linear(dx[K], wq, sw1, p, dws[K], mx.MUXQ_OUT_F16, out=dy[N])
+
+            with torch.cuda.stream(side):
+                chain()
+                side.synchronize()
+                g_dec = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g_dec, stream=side):
+                    chain()
+            torch.cuda.synchronize()
+            for _ in range(3):
+                g_dec.replay()
+            d0, d1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            d0.record()
+            for _ in range(10):
+                g_dec.replay()
+            d1.record()
+            torch.cuda.synchronize()
+            for K in dws:
+                if mx.muxq_read_status(dws[K]) != 0:
+                    raise RuntimeError("device status raised on the decode chain")
+            us = d0.elapsed_time(d1) * 1e3 / 10
+            gbs = wbytes / us / 1e3
+            decode[f"M{Md}"] = {"us_per_layer": us / len(dlayers), "gb_per_s": gbs, "frac_of_measured_hbm": gbs / peaks["hbm_gbs"]}
+            del g_dec
+        del dlayers
+
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         rows = specs[0].M
@@ -354,7 +405,7 @@ def run_muxq(args, rank, world):
                 "us_per_layer": ms_per_step * 1e3 / len(layers),
                 "pct_of_nominal_int8_peak_4500": 100.0 * value / world / 4500.0,
                 "clocks": clocks, "e2e": e2e, "gpu_launches": args.steps * len(layers) * 2,
-                "roofline": roofline, "cpu_baseline": cpu_baseline}
+                "roofline": roofline, "decode": decode, "cpu_baseline": cpu_baseline}
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
@@ -367,6 +418,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=50)
     ap.add_argument("--impl", default="muxq", choices=["muxq", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-decode", action="store_true")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
