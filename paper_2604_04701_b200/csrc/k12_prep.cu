@@ -248,6 +248,10 @@ __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, int rows_base,
     }
     if (a.per_token) __syncthreads();  // the per-token path reads the shared factor copies and the Aux sources
 
+    // Let a kernel launched as a programmatic dependent (the GEMM) start its set-up on SMs as they free up;
+    // it still waits for this whole grid to finish before it reads anything written here.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+
     // ---------------------------------------------------------------- pass 2: Body_q and the Aux block
     if (!a.per_token) {
         // Per-tensor scale: the pass-1 mapping again (a thread owns 8 channels and walks down the

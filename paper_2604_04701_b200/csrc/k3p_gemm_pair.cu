@@ -88,6 +88,10 @@ k_gemm_i8_pair(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     const uint32_t tmem_base = __shfl_sync(0xffffffffu, s_tmem_base, 0);
     volatile uint32_t *abort_flag = &s_abort;
 
+    // Launched as a programmatic dependent of the kernel before it in the stream (the activation
+    // preparation): the set-up above overlaps that kernel's tail; its results are read only from here on.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+
     int aux_cols_used = 0;
     if (p.has_aux) aux_cols_used = p.c * min(__ldg(p.n_outliers), p.cap);
     aux_cols_used = __shfl_sync(0xffffffffu, aux_cols_used, 0);
@@ -295,10 +299,12 @@ cudaError_t launch_pair_inst(const GemmArgs &a, cudaStream_t s) {
     cfg.blockDim = dim3(kGemmThreads);
     cfg.dynamicSmemBytes = C::kSmemBytes;
     cfg.stream = s;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr; cfg.numAttrs = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 2;
     return cudaLaunchKernelEx(&cfg, kern, tm_a, tm_aux, tm_b, tm_baux, tm_y, p);
 }
 
