@@ -91,6 +91,7 @@ k_gemm_i8_pair(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     // Launched as a programmatic dependent of the kernel before it in the stream (the activation
     // preparation): the set-up above overlaps that kernel's tail; its results are read only from here on.
     asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");  // a dependent still waits for this grid to finish
 
     int aux_cols_used = 0;
     if (p.has_aux) aux_cols_used = p.c * min(__ldg(p.n_outliers), p.cap);
