@@ -339,6 +339,44 @@ def run_muxq(args, rank, world):
            "d2h_bytes_per_step": int(sum(yh.numel() * 2 for _, yh in hosts)), "steps": esteps,
            "ms_per_step": ems / esteps}
 
+    # ---- the per-vector variant of the same workload (per-token X scales, per-channel W scales)
+    per_vector = None
+    if world == 1:
+        pv = mx.MuxqParams(max_outliers=32, gran=mx.MUXQ_PER_VECTOR)
+        pv_layers = []
+        for L in layers:
+            sp = L["spec"]
+            w_q, s_w = mx.muxq_quantize(torch.from_numpy(sp.w()).to(dev), pv, True,
+                                        mx.Workspace(mx.muxq_small_workspace_bytes(sp.N), dev))
+            pv_layers.append((L["x"], w_q, s_w, L["ws"], L["y"]))
+
+        def pv_step():
+            for (xd, w_q, s_w, wsx, y) in pv_layers:
+                mx.muxq_linear(xd, w_q, s_w, pv, wsx, mx.MUXQ_OUT_F16, out=y)
+
+        with torch.cuda.stream(side):
+            pv_step()
+            side.synchronize()
+            check_status()
+            g_pv = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g_pv, stream=side):
+                pv_step()
+        torch.cuda.synchronize()
+        for _ in range(3):
+            g_pv.replay()
+        v0, v1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        v0.record()
+        for _ in range(ksteps):
+            g_pv.replay()
+        v1.record()
+        torch.cuda.synchronize()
+        check_status()
+        pv_ms = v0.elapsed_time(v1) / ksteps
+        per_vector = {"granularity": "per-token X, per-channel W", "ms_per_step": pv_ms,
+                      "value": ops_per_step / (pv_ms * 1e-3) / 1e12, "unit": UNIT}
+        del g_pv, pv_layers
+
     # ---- decode shapes (M <= 16): the 36 x 4 GPT-2-large linears as one stream of layers with distinct
     # weights (708 MB of W_q, far more than the L2 holds), replayed from a graph; GB/s = W_q bytes / time
     decode = None
@@ -405,7 +443,7 @@ def run_muxq(args, rank, world):
                 "us_per_layer": ms_per_step * 1e3 / len(layers),
                 "pct_of_nominal_int8_peak_4500": 100.0 * value / world / 4500.0,
                 "clocks": clocks, "e2e": e2e, "gpu_launches": args.steps * len(layers) * 2,
-                "roofline": roofline, "decode": decode, "cpu_baseline": cpu_baseline}
+                "roofline": roofline, "per_vector": per_vector, "decode": decode, "cpu_baseline": cpu_baseline}
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
