@@ -145,11 +145,13 @@ int muxq_gemm(const int8_t *Body_q, int ld_a, const int8_t *Aux_q, int ld_aux, c
 /*
  * The whole layer: detect -> redistribute + quantize -> INT8 products + Aux correction ->
  * dequantize (Section III-C, Eq. 1-7).  W_q [N, ldw] and s_w come from muxq_quantize(is_weight=1)
- * with the same params.  M <= 16 takes the memory-bound decode path; larger M the tensor-core
- * path.  Y: [M, ldy] by out_kind.  workspace >= muxq_workspace_bytes(M,K,N,p), contents need
- * not be initialised.  dev_status: device int32; the call sets it to 0 first, kernels raise it
- * to MUXQ_ERR_CAPACITY (r > max_outliers; Y then unspecified but in bounds) or MUXQ_ERR_TIMEOUT.
- * Intermediate results stay in the workspace afterwards; muxq_workspace_view locates them.
+ * with the same params.  M > 16: one preparation kernel and one tensor-core GEMM kernel.  M <= 16:
+ * the memory-bound decode path, a single kernel that streams W_q once.  Y: [M, ldy] by out_kind.
+ * workspace >= muxq_workspace_bytes(M,K,N,p), contents need not be initialised.  dev_status: device
+ * int32; the call sets it to 0 first, kernels raise it to MUXQ_ERR_CAPACITY (r > max_outliers; Y
+ * then unspecified but in bounds) or MUXQ_ERR_TIMEOUT.
+ * Intermediates stay in the workspace afterwards; muxq_workspace_view locates them.  For M <= 16
+ * only col_absmax, outlier_idx, n_outliers and s_x are left there (the codes never leave the SMs).
  */
 int muxq_linear(const void *X_f16, int M, int K, int ldx, const int8_t *W_q, int ldw,
                 const float *s_w, int N, const muxq_params *p, void *Y, int ldy, int out_kind,
