@@ -289,7 +289,17 @@ cudaError_t launch_gemm(const GemmArgs &a, cudaStream_t s) {
     // CTA pairs (256-row tiles, a third less operand traffic per SM) unless M is too small to fill them.
     // Measured on B200: with pairs the 256-wide tile is at least as fast as the 128-wide one for every N > 128
     // (the narrower tile needs 1.5x the operand bytes per MMA and becomes load-bound).
-    if (a.M > BM && a.N >= 128) return launch_gemm_pair(a, a.N > 128 ? 256 : 128, s);
+    // A 192-wide tile carries 17 % more operand bytes per MMA, but divides some N (768) into fewer idle
+    // rounds: take it when its estimated makespan, with a 15 % handicap (measured), still beats the 256-wide one.
+    if (a.M > BM && a.N >= 128) {
+        int bn = 128;
+        if (a.N > 128) {
+            const int pairs = num_sms() / 2, tm2 = (a.M + 2 * BM - 1) / (2 * BM);
+            const int r256 = (tm2 * ((a.N + 255) / 256) + pairs - 1) / pairs, r192 = (tm2 * ((a.N + 191) / 192) + pairs - 1) / pairs;
+            bn = r192 * 192 * 1.15 < r256 * 256.0 ? 192 : 256;
+        }
+        return launch_gemm_pair(a, bn, s);
+    }
     // Single-CTA tiles: 256 halves the operand traffic per MMA; 128 gives more tiles when the 256-wide
     // tiling leaves most of the last wave idle.
     const int sms = num_sms();

@@ -31,7 +31,7 @@ struct PairCfg {
     static constexpr int kABytes = BM * BK;          // this CTA's 128 rows of A
     static constexpr int kBBytes = (BN / 2) * BK;    // this CTA's half of B's rows
     static constexpr int kStageBytes = kABytes + kBBytes;
-    static constexpr int kTmemCols = 2 * BN;
+    static constexpr int kTmemCols = BN > 128 ? 512 : 256;  // two accumulator buffers, a power of two
     static constexpr int kOutBufBytes = 32 * 128;
     static constexpr int kOutBufs = 2;
     static constexpr int kOutBytes = kEpiWarps * kOutBufs * kOutBufBytes;
@@ -180,9 +180,14 @@ k_gemm_i8_pair(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
         // ---------------------------------------------------------------- epilogue warps (both CTAs, own 128 rows)
         const int quad = warp & 3;
         const int chalf = (warp - 2) >> 2;
-        constexpr int kChunks = BN / 2 / 32;
+        // The two warps of a TMEM lane quadrant split the tile's columns in units of 64 (one fp16 store box):
+        // the first takes 128 of a 192- or 256-wide tile (64 of a 128-wide one), the second takes the rest.
+        constexpr int kCols0 = BN >= 192 ? 128 : BN / 2;
+        constexpr int kChunks = kCols0 / 32;              // 32-column chunks of the larger share
         constexpr int kChunksPerBox = kOut == kOutF16 ? 2 : 1;
-        static_assert(kChunks % kChunksPerBox == 0, "a store box must not straddle two warps' columns");
+        static_assert(kChunks % kChunksPerBox == 0 && ((BN - kCols0) / 32) % kChunksPerBox == 0,
+                      "a store box must not straddle two warps' columns");
+        const int nch = chalf == 0 ? kChunks : (BN - kCols0) / 32;  // warp-uniform
         uint8_t *stage0 = smem_al + C::kStages * C::kStageBytes + (warp - 2) * (C::kOutBufs * C::kOutBufBytes);
         const uint32_t sw_xor = (uint32_t)(lane & 7);
         float sxw = 1.0f, sx = 1.0f;
@@ -197,20 +202,22 @@ k_gemm_i8_pair(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
             ok = mbar_wait_warp(&bar_acc_full[buf], aph, abort_flag);
             if (!ok) break;
             tc_fence_after();
-            const int col0 = chalf * (BN / 2);
+            const int col0 = chalf * kCols0;
             const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + buf * BN + col0;
             // Pull this warp's whole share of the accumulator (32 rows x BN/2 columns) into registers at once
             // and hand the TMEM buffer back before converting: the MMA issuer can then start the tile after
             // next while this tile is still being converted and stored.
             uint32_t v[kChunks][32];
 #pragma unroll
-            for (int ch = 0; ch < kChunks; ++ch) tmem_ld_32x32(taddr + 32 * ch, v[ch]);
+            for (int ch = 0; ch < kChunks; ++ch)
+                if (ch < nch) tmem_ld_32x32(taddr + 32 * ch, v[ch]);
             tmem_ld_wait();
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(&bar_acc_empty[buf]), 0));
 #pragma unroll
             for (int ch = 0; ch < kChunks; ++ch) {
+                if (ch >= nch) break;
                 const int piece = ch % kChunksPerBox;
                 uint8_t *stage = stage0 + (n_box % C::kOutBufs) * C::kOutBufBytes;
                 if (piece == 0) {
@@ -321,9 +328,9 @@ cudaError_t launch_pair_bn(const GemmArgs &a, cudaStream_t s) {
 
 }  // namespace
 
-// CTA-pair GEMM; bn = 256 or 128 (tile width).
+// CTA-pair GEMM; bn = 256, 192 or 128 (tile width).
 cudaError_t launch_gemm_pair(const GemmArgs &a, int bn, cudaStream_t s) {
-    return bn == 256 ? launch_pair_bn<256>(a, s) : launch_pair_bn<128>(a, s);
+    return bn == 256 ? launch_pair_bn<256>(a, s) : bn == 192 ? launch_pair_bn<192>(a, s) : launch_pair_bn<128>(a, s);
 }
 
 }  // namespace muxq
