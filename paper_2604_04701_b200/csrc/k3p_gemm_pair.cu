@@ -192,6 +192,7 @@ k_gemm_i8_pair(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
         const uint32_t sw_xor = (uint32_t)(lane & 7);
         float sxw = 1.0f, sx = 1.0f;
         if (kOut != kOutI32 && !kPerVec) sxw = __fmul_rn(__ldg(p.s_x), __ldg(p.s_w));
+        const uint64_t y_policy = make_policy_evict_first();
         uint32_t tile_it = 0, n_box = 0;
         bool ok = true;
         for (int tile = pair; tile < num_tiles && ok; tile += num_pairs, ++tile_it) {
@@ -233,7 +234,7 @@ k_gemm_i8_pair(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                     __syncwarp();
                     if (lane == 0) {
                         const int bcol = gcol - 32 * piece;
-                        if (row0 < p.M && bcol < p.N) tma_store_2d(&tm_y, stage, bcol, row0);
+                        if (row0 < p.M && bcol < p.N) tma_store_2d_hint(&tm_y, stage, bcol, row0, y_policy);
                         tma_store_commit();
                     }
                     ++n_box;
