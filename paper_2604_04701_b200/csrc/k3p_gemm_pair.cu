@@ -241,7 +241,8 @@ k_gemm_i8_pair(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                 }
             }
         }
-        if (lane == 0) tma_store_wait_all<0>();
+        // the staging buffers must outlive the copies that read them; the writes themselves complete with the grid
+        if (lane == 0) tma_store_wait_read<0>();
     }
 
     // ---------------------------------------------------------------- teardown
