@@ -436,3 +436,20 @@ def test_config3_decode_full_size(mx, M):
 def test_config4_outlier_sweep_full_size_sampled_rows(mx, n_out):
     spec = synth.config_layers(4, n_outliers=n_out, layers=36)[35 * 4 + 2]   # last layer's c_fc, 8192 x 1280 -> 5120
     _full_size_check(mx, spec, 0, cap=64)
+
+
+@pytest.mark.parametrize("e,act_bits,w_bits,gran", [(1, 8, 8, 0), (3, 6, 5, 0), (3, 7, 4, 1), (2, 5, 8, 1)])
+def test_linear_other_exp_factors_and_bit_widths(mx, e, act_bits, w_bits, gran):
+    """exp factor 1 / 3 and the reduced bit widths of Tables 1-2 through the whole layer (tensor-core path
+    and decode path): the Aux block then repeats each column 2^e - 1 = 1 or 7 times."""
+    for M, K, N in ((384, 768, 520), (5, 1280, 264)):
+        x, w, _ = make_case(300 + e + act_bits, M, K, N, n_out=5, mult=50.0)
+        p = mx.MuxqParams(exp_factor=e, act_bits=act_bits, w_bits=w_bits, gran=gran, max_outliers=16)
+        wq_o, sw_o, res = oracle_linear(x, w, p)
+        acc, ws, st, w_q, s_w = run_linear(mx, x, w, p, mx.MUXQ_OUT_ACC_I32)
+        assert st == 0 and np.array_equal(w_q.cpu().numpy(), wq_o.T)
+        assert np.array_equal(acc.cpu().numpy(), res.acc)
+        y32, _, st, _, _ = run_linear(mx, x, w, p, mx.MUXQ_OUT_F32)
+        assert st == 0 and np.array_equal(y32.cpu().numpy(), res.y32)
+        y16, _, st, _, _ = run_linear(mx, x, w, p, mx.MUXQ_OUT_F16)
+        assert st == 0 and f16_ulp_diff(y16.cpu().numpy(), res.y16).max() <= 1
