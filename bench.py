@@ -316,19 +316,35 @@ def run_muxq(args, rank, world):
         yh = torch.empty(L["spec"].M, L["spec"].N, dtype=torch.float16).pin_memory()
         hosts.append((xh, yh))
 
+    # Consecutive layers alternate between two streams, so one layer's device-to-host copy of Y overlaps the
+    # next layer's host-to-device copy of X (PCIe is full duplex); each layer has its own buffers.
+    h_streams = [torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev)]
+
     def step_host():
-        for L, (xh, yh) in zip(layers, hosts):
-            mx.muxq_linear_host(xh, L["w_q"], L["s_w"], p, L["ws"], yh, mx.MUXQ_OUT_F16)
+        for i, (L, (xh, yh)) in enumerate(zip(layers, hosts)):
+            with torch.cuda.stream(h_streams[i & 1]):
+                mx.muxq_linear_host(xh, L["w_q"], L["s_w"], p, L["ws"], yh, mx.MUXQ_OUT_F16)
+
+    def join_host():
+        for hs in h_streams:
+            torch.cuda.current_stream().wait_stream(hs)
+
+    def fork_host():
+        for hs in h_streams:
+            hs.wait_stream(torch.cuda.current_stream())
 
     for _ in range(2):
         step_host()
     torch.cuda.synchronize(); barrier()
     h0, h1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     h0.record()
+    fork_host()
     for _ in range(esteps):
         step_host()
+    join_host()
     h1.record()
     torch.cuda.synchronize(); barrier()
+    check_status()
     ems = h0.elapsed_time(h1)
     if world > 1:
         t = torch.tensor([ems], device=dev)
