@@ -355,6 +355,17 @@ def run_muxq(args, rank, world):
            "d2h_bytes_per_step": int(sum(yh.numel() * 2 for _, yh in hosts)), "steps": esteps,
            "ms_per_step": ems / esteps}
 
+    # ---- whole-layer roofline: per layer the slower of the INT8 tensor time and the HBM time of its
+    # algorithmic bytes (X fp16 read once, W_q, Y fp16 written once), summed over the step
+    t_roof_us = 0.0
+    for L in layers:
+        sp = L["spec"]
+        t_c = 2.0 * sp.M * sp.N * sp.K / (int8_peak * 1e12) * 1e6
+        t_m = (2.0 * sp.M * sp.K + sp.N * sp.K + 2.0 * sp.M * sp.N) / (peaks["hbm_gbs"] * 1e9) * 1e6
+        t_roof_us += max(t_c, t_m)
+    step_roofline = {"t_roof_us": t_roof_us, "frac": t_roof_us / (ms_per_step * 1e3),
+                     "peaks": {"int8_tops": int8_peak, "hbm_gbs": peaks["hbm_gbs"], "source": peaks["source"]}}
+
     # ---- the per-vector variant of the same workload (per-token X scales, per-channel W scales)
     per_vector = None
     if world == 1:
@@ -459,7 +470,7 @@ def run_muxq(args, rank, world):
                 "us_per_layer": ms_per_step * 1e3 / len(layers),
                 "pct_of_nominal_int8_peak_4500": 100.0 * value / world / 4500.0,
                 "clocks": clocks, "e2e": e2e, "gpu_launches": args.steps * len(layers) * 2,
-                "roofline": roofline, "per_vector": per_vector, "decode": decode, "cpu_baseline": cpu_baseline}
+                "roofline": roofline, "step_roofline": step_roofline, "per_vector": per_vector, "decode": decode, "cpu_baseline": cpu_baseline}
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()

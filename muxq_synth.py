@@ -125,7 +125,7 @@ def _gpt2_linears(d: int) -> List[Tuple[str, int, int]]:
 
 def config_layers(cfg: int, M: int | None = None, n_outliers: int | None = None,
                   layers: int = 1) -> List[LayerSpec]:
-    """The five workloads the benchmark contract lists, as LayerSpecs.
+    """The five benchmark workloads, as LayerSpecs.
 
     0: one 128x768x768 layer, 4 outlier channels x50, seed 0.
     1: GPT-2-small linears at M=8192, 6 outlier channels x U(40,80), seed 1.
