@@ -453,3 +453,21 @@ def test_linear_other_exp_factors_and_bit_widths(mx, e, act_bits, w_bits, gran):
         assert st == 0 and np.array_equal(y32.cpu().numpy(), res.y32)
         y16, _, st, _, _ = run_linear(mx, x, w, p, mx.MUXQ_OUT_F16)
         assert st == 0 and f16_ulp_diff(y16.cpu().numpy(), res.y16).max() <= 1
+
+
+@pytest.mark.parametrize("M", [3, 40])
+@pytest.mark.parametrize("gran", [0, 1])
+def test_wide_k_takes_the_separate_kernels(mx, M, gran):
+    """K beyond what the fused preparation / fused decode kernels hold (8192 channels) falls back to the
+    stand-alone detect and quantize kernels; same results."""
+    K, N = 8320, 136
+    x, w, _ = make_case(500 + M, M, K, N, n_out=9, mult=50.0)
+    p = mx.MuxqParams(gran=gran, max_outliers=32)
+    _, _, res = oracle_linear(x, w, p)
+    acc, ws, st, _, _ = run_linear(mx, x, w, p, mx.MUXQ_OUT_ACC_I32)
+    assert st == 0 and np.array_equal(acc.cpu().numpy(), res.acc)
+    v = ws_views(mx, ws, M, K, N, p)
+    assert v["n_outliers"] == res.r and np.array_equal(v["outlier_idx"][:res.r], res.O)
+    assert np.array_equal(v["body_q"], res.body_q)
+    y32, _, st, _, _ = run_linear(mx, x, w, p, mx.MUXQ_OUT_F32)
+    assert st == 0 and np.array_equal(y32.cpu().numpy(), res.y32)
