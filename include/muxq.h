@@ -17,7 +17,7 @@
  *   - All tensor pointers are DEVICE pointers unless the name says "host".  Row-major; "ld" is
  *     the row pitch in ELEMENTS.  fp16 is IEEE binary16 passed as void*.
  *   - The caller owns every buffer, including the workspace; the library allocates no device
- *     memory and keeps no state between calls.  `stream` is a cudaStream_t passed as void*
+ *     memory and keeps no host state between calls.  `stream` is a cudaStream_t passed as void*
  *     (NULL = the legacy default stream).
  *   - Calls only enqueue work; nothing synchronizes except muxq_read_status and
  *     muxq_linear_host's final copy-back wait when asked.
@@ -78,6 +78,22 @@ size_t muxq_workspace_bytes(int M, int K, int N, const muxq_params *p);
 size_t muxq_small_workspace_bytes(int cols);
 /* Bytes of workspace muxq_linear_host needs: muxq_workspace_bytes + device staging of X and Y. */
 size_t muxq_host_workspace_bytes(int M, int K, int N, const muxq_params *p, int out_kind);
+
+/*
+ * Prepares a workspace for muxq_linear / muxq_linear_events / muxq_linear_host: enqueues on `stream`
+ * a zero fill of the control block and of the abs-max accumulators of the detection step
+ * (Section III-C) at its start (at most 257 KiB; fewer when workspace_bytes is smaller).  The layer
+ * kernels find these words zero and put them back to zero before they finish, so that a layer call
+ * carries no clearing step of its own.  Call it once after allocating the workspace, before its
+ * first layer call, and again
+ *   - after a layer call whose status word read MUXQ_ERR_TIMEOUT,
+ *   - after the same memory was handed to muxq_detect_outliers or muxq_quantize as their workspace,
+ *     or written by anything else.
+ * One workspace may then serve any sequence of layer shapes, one call at a time (calls that share a
+ * workspace must be ordered on one stream or by events).  Returns MUXQ_ERR_INVALID_ARG for a NULL
+ * pointer or fewer than 256 bytes.
+ */
+int muxq_workspace_init(void *workspace, size_t workspace_bytes, void *stream);
 
 /*
  * Outlier-channel detection (Section III-C: a channel with at least one element of magnitude
@@ -147,7 +163,7 @@ int muxq_gemm(const int8_t *Body_q, int ld_a, const int8_t *Aux_q, int ld_aux, c
  * dequantize (Section III-C, Eq. 1-7).  W_q [N, ldw] and s_w come from muxq_quantize(is_weight=1)
  * with the same params.  M > 16: one preparation kernel and one tensor-core GEMM kernel.  M <= 16:
  * the memory-bound decode path, a single kernel that streams W_q once.  Y: [M, ldy] by out_kind.
- * workspace >= muxq_workspace_bytes(M,K,N,p), contents need not be initialised.  dev_status: device
+ * workspace >= muxq_workspace_bytes(M,K,N,p), prepared once by muxq_workspace_init.  dev_status: device
  * int32; the call sets it to 0 first, kernels raise it to MUXQ_ERR_CAPACITY (r > max_outliers; Y
  * then unspecified but in bounds) or MUXQ_ERR_TIMEOUT.
  * Intermediates stay in the workspace afterwards; muxq_workspace_view locates them.  For M <= 16
@@ -160,8 +176,8 @@ int muxq_linear(const void *X_f16, int M, int K, int ldx, const int8_t *W_q, int
 /*
  * muxq_linear that also records four caller-created CUDA events (cudaEvent_t passed as void*;
  * NULL entries are skipped) on `stream` at its kernel boundaries, for per-kernel timing:
- * events[0] at entry, [1] after the workspace clear (start of the fused detect + redistribute +
- * quantize kernel), [2] after that kernel, [3] after the GEMM (or decode) kernel.  When `stream`
+ * events[0] at entry, [1] at the start of the fused detect + redistribute + quantize kernel (after
+ * the clearing step where the shape needs one: K > 8192), [2] after that kernel, [3] after the GEMM (or decode) kernel.  When `stream`
  * is being captured into a CUDA graph the records become event-record nodes, re-recorded by every
  * replay.  Same results as muxq_linear.
  */
@@ -187,7 +203,7 @@ int muxq_workspace_view(int M, int K, int N, const muxq_params *p, muxq_ws_view 
 /*
  * muxq_linear with X and Y in HOST memory (pinned for true asynchrony): copies X to the device,
  * runs the layer, copies Y back, all on `stream`.  W_q, s_w, workspace and dev_status stay
- * device pointers.  workspace >= muxq_host_workspace_bytes(...).  X_host must be dense
+ * device pointers.  workspace >= muxq_host_workspace_bytes(...), prepared by muxq_workspace_init.  X_host must be dense
  * (pitch K), Y_host dense (pitch N).  Does not synchronize.
  */
 int muxq_linear_host(const void *X_f16_host, int M, int K, const int8_t *W_q, int ldw,

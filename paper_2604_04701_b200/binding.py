@@ -20,7 +20,7 @@ MUXQ_OUT_F16, MUXQ_OUT_F32, MUXQ_OUT_ACC_I32 = 0, 1, 2
 
 EXPORTS = (
     "muxq_default_params", "muxq_aux_cols", "muxq_workspace_bytes", "muxq_small_workspace_bytes",
-    "muxq_host_workspace_bytes", "muxq_workspace_view", "muxq_detect_outliers", "muxq_build_aux",
+    "muxq_host_workspace_bytes", "muxq_workspace_init", "muxq_workspace_view", "muxq_detect_outliers", "muxq_build_aux",
     "muxq_quantize", "muxq_gemm", "muxq_linear", "muxq_linear_events", "muxq_linear_host",
     "muxq_linear_decode_noalloc", "muxq_int8_mma_peak", "muxq_read_status",
     "muxq_status_string",
@@ -84,6 +84,7 @@ def lib() -> ctypes.CDLL:
         L.muxq_workspace_bytes.argtypes = [i, i, i, pp]; L.muxq_workspace_bytes.restype = sz
         L.muxq_small_workspace_bytes.argtypes = [i]; L.muxq_small_workspace_bytes.restype = sz
         L.muxq_host_workspace_bytes.argtypes = [i, i, i, pp, i]; L.muxq_host_workspace_bytes.restype = sz
+        L.muxq_workspace_init.argtypes = [vp, sz, vp]; L.muxq_workspace_init.restype = i
         L.muxq_workspace_view.argtypes = [i, i, i, pp, ctypes.POINTER(_CWsView)]; L.muxq_workspace_view.restype = i
         L.muxq_detect_outliers.argtypes = [vp, i, i, i, f, vp, vp, vp, i, vp, sz, vp]; L.muxq_detect_outliers.restype = i
         L.muxq_build_aux.argtypes = [vp, i, i, i, vp, vp, i, i, vp, i, vp, i, vp]; L.muxq_build_aux.restype = i
@@ -145,6 +146,12 @@ class Workspace:
     def __init__(self, nbytes: int, device="cuda"):
         self.buf = torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=device)
         self.status = torch.zeros(1, dtype=torch.int32, device=device)
+        self.init()
+
+    def init(self) -> None:
+        """muxq_workspace_init on the current stream (needed again after a time-out status or foreign writes)."""
+        with torch.cuda.device(self.buf.device):
+            _check("muxq_workspace_init", lib().muxq_workspace_init(_ptr(self.buf), self.nbytes, _stream()))
 
     @property
     def nbytes(self) -> int:

@@ -1,5 +1,5 @@
 // C-ABI host layer of libmuxq: argument checks, workspace carving, kernel launches.
-// No device memory is allocated here and no state survives a call.
+// No device memory is allocated here and no host state survives a call.
 #include <math.h>
 #include <string.h>
 
@@ -47,11 +47,12 @@ LinearWs linear_ws(int M, int K, int N, const muxq_params *p) {
     w.s = small_ws(K);
     w.aux_cols = muxq_aux_cols(p);
     w.ld_q = K;
-    // The replicated abs-max accumulators of the fused kernel sit right behind ctrl | colmax so that
-    // one memset clears all three; the other small arrays follow.
-    w.colmax_rep = align_up(w.s.colmax + (size_t)K * 4, 256);
-    const size_t shift = align_up(w.colmax_rep + (size_t)kPrepColmaxReplicas * K * 4, 256) - w.s.colmul;
-    w.s.colmul += shift; w.s.grpflag += shift; w.s.oidx += shift; w.s.total += shift;
+    // The replicated abs-max accumulators of the fused kernel sit right behind ctrl, in a region of fixed
+    // size: the fused kernel finds it zero and leaves it zero, for every shape that shares the workspace.
+    // Everything a call overwrites with other values follows behind it.
+    w.colmax_rep = sizeof(Ctrl);
+    const size_t shift = align_up(w.colmax_rep + kPrepRepRegionBytes, 256) - w.s.colmax;
+    w.s.colmax += shift; w.s.colmul += shift; w.s.grpflag += shift; w.s.oidx += shift; w.s.total += shift;
     w.sx_rows = w.s.total;
     w.body_q = align_up(w.sx_rows + (size_t)M * 4, 1024);
     w.aux_q = align_up(w.body_q + (size_t)M * w.ld_q, 1024);
@@ -96,6 +97,13 @@ size_t muxq_host_workspace_bytes(int M, int K, int N, const muxq_params *p, int 
     const size_t base = muxq_workspace_bytes(M, K, N, p);
     if (!base || out_kind < 0 || out_kind > 2) return 0;
     return base + align_up((size_t)M * K * 2, 1024) + align_up((size_t)M * N * out_elem_bytes(out_kind), 1024);
+}
+
+int muxq_workspace_init(void *workspace, size_t workspace_bytes, void *stream) {
+    if (!workspace || workspace_bytes < sizeof(Ctrl)) return MUXQ_ERR_INVALID_ARG;
+    const size_t n = sizeof(Ctrl) + kPrepRepRegionBytes;
+    return cuda_rc(cudaMemsetAsync(workspace, 0, workspace_bytes < n ? workspace_bytes : n,
+                                   static_cast<cudaStream_t>(stream)));
 }
 
 int muxq_workspace_view(int M, int K, int N, const muxq_params *p, muxq_ws_view *v) {
@@ -307,9 +315,14 @@ static int linear_impl(const void *X, int M, int K, int ldx, const int8_t *W_q, 
         mark(3);
         return cuda_rc(ed);
     }
-    cudaError_t e = cudaMemsetAsync(ws, 0, fused ? w.colmax_rep + (size_t)kPrepColmaxReplicas * K * 4
-                                                 : w.s.colmax + (size_t)K * 4, s);
-    if (e == cudaSuccess && !fused) e = cudaMemsetAsync(dev_status, 0, 4, s);  // the fused kernel clears it itself
+    // The fused kernel keeps its counters and accumulators zero between calls (muxq_workspace_init zeroed
+    // them once); the separate kernels take a cleared control block and abs-max array per call.
+    cudaError_t e = cudaSuccess;
+    if (!fused) {
+        e = cudaMemsetAsync(ws, 0, sizeof(Ctrl), s);
+        if (e == cudaSuccess) e = cudaMemsetAsync(ws + w.s.colmax, 0, (size_t)K * 4, s);
+        if (e == cudaSuccess) e = cudaMemsetAsync(dev_status, 0, 4, s);  // the fused kernel clears it itself
+    }
     if (e != cudaSuccess) return MUXQ_ERR_CUDA;
     mark(1);
 

@@ -17,6 +17,10 @@
 //           lists O meanwhile), then quantizes its slab out of shared memory with the pass-1 thread
 //           mapping (per tensor) or one warp per token row (per token), writing Body_q, the Aux block
 //           and (spread over the grid) the gathered W_aux rows.
+// The kernel expects the barrier counter, the reader counter and the replicated accumulators to be zero and
+// leaves them zero: once every CTA has fetched the merged maxima (each takes a ticket after doing so; the
+// holder of the last ticket knows), nothing reads them any more, and that CTA clears them during the last phase.
+// A call therefore needs no separate clearing step; a barrier time-out leaves them dirty.
 #include "kernels.h"
 #include "quant.cuh"
 
@@ -27,6 +31,7 @@ namespace {
 constexpr int kT = 1024;  // the warp-group split of the last phase (512 + 256 + 256 threads) assumes this
 constexpr int kWarps = kT / 32;
 constexpr int kMaxK = 8 * kT;  // one group of 8 channels per thread
+static_assert(kMaxK == kPrepMaxK, "the accumulator region of the workspace is sized for kPrepMaxK channels");
 constexpr int kMaxOut = 64;
 constexpr int kMaxAuxCols = 512;  // (2^3 - 1) * 64 rounded up to 128
 constexpr int kColmaxReplicas = kPrepColmaxReplicas;
@@ -72,6 +77,7 @@ __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, int rows_base,
     __shared__ float s_warp_max[kWarps];
     __shared__ int s_r_true;
     __shared__ int s_fail;
+    __shared__ int s_last;
 
     const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
     const int K = a.K, G = K >> 3;
@@ -169,6 +175,14 @@ __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, int rows_base,
         if (b == 0) reinterpret_cast<uint4 *>(a.colmax_bits)[k4] = mx;
     }
     __syncthreads();
+    // This CTA holds its copy of the maxima.  The CTA that takes the last ticket knows that every CTA does
+    // (and has therefore left the barrier), so it may put the accumulators and both counters back to zero for
+    // the next call; the ticket is fetched here and looked at only before the last phase, off the critical path.
+    uint32_t ticket = 0;
+    if (t == 0) {
+        __threadfence();
+        ticket = atomicAdd(&a.ctrl->readers, 1u);
+    }
     // Every thread derives the factors of the 8 channels it owns in both passes: 2^-e where the channel
     // holds an element above the threshold (strict), else 1.  (When more channels are flagged than the
     // capacity allows the call fails with MUXQ_ERR_CAPACITY and Y is unspecified, so no ordering is needed here.)
@@ -324,7 +338,8 @@ __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, int rows_base,
     }
 
     // ---------------------------------------------------------------- Aux block (per tensor) and W_aux
-    __syncthreads();  // warp 0's outlier list and Aux sources are complete
+    if (t == 0) s_last = ticket == gridDim.x - 1 ? 1 : 0;
+    __syncthreads();  // the last warp's outlier list and Aux sources are complete
     const int r = min(s_r_true, a.cap);
     const int used_cols = c * r, used_words = (used_cols + 3) >> 2;
     // Three independent jobs share the CTA's warps so that their latencies overlap instead of adding up:
@@ -348,6 +363,14 @@ __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, int rows_base,
             }
         }
     } else if (warp < 24) {
+        if (s_last) {
+            uint4 *rep4 = reinterpret_cast<uint4 *>(a.colmax_rep);
+            for (int i = t - 512; i < kColmaxReplicas * (K >> 2); i += 256) rep4[i] = make_uint4(0u, 0u, 0u, 0u);
+            if (t == 512) {
+                a.ctrl->arrived = 0u;
+                a.ctrl->readers = 0u;
+            }
+        }
         if (do_aux) {
             // whole words of the Aux block beyond the used ones
             const int aux_words = a.aux_cols >> 2;

@@ -6,15 +6,17 @@
 
 namespace muxq {
 
-// Device control block at the start of every workspace (zeroed by one memset per call together
-// with the column abs-max accumulators that follow it).
+// Device control block at the start of every workspace.  The stand-alone kernels get it zeroed by a
+// memset per call; the fused prep kernel needs `arrived`, `readers` and its replicated abs-max
+// accumulators zero on entry and leaves them zero on exit (see k12_prep.cu).
 struct Ctrl {
     uint32_t blocks_done;  // K1: CTAs that have merged their partial maxima
     int32_t n_outliers;    // r, true count of outlier channels
     float s_x;             // per-tensor Body scale (Eq. 1)
     float inv_s_x;         // 1 / s_x, correctly rounded (used only to pre-screen the exact division)
     uint32_t arrived;      // fused prep kernel: CTAs that have reached the grid-wide barrier
-    uint32_t reserved[59];
+    uint32_t readers;      // fused prep kernel: CTAs that have fetched the merged channel maxima
+    uint32_t reserved[58];
 };
 static_assert(sizeof(Ctrl) == 256, "Ctrl is one 256-byte block");
 
@@ -60,14 +62,18 @@ cudaError_t launch_quant_act(const QuantActArgs &a, cudaStream_t s);
 
 // Fused detect + redistribute + quantize (one cooperative launch, X read from HBM once).
 constexpr int kPrepColmaxReplicas = 8;
+constexpr int kPrepMaxK = 8192;
+// Bytes of replicated accumulators behind Ctrl for the widest supported K.  The region has the same place
+// and size for every shape, so "all zero between calls" holds whatever sequence of shapes uses a workspace.
+constexpr size_t kPrepRepRegionBytes = (size_t)kPrepColmaxReplicas * kPrepMaxK * 4;
 struct PrepArgs {
     const __half *X;
     int M, K, ldx;
     float tau;
     int exp_factor, qmax, cap, per_token;
-    uint32_t *colmax_rep;    // [kPrepColmaxReplicas, K] zero-initialised accumulators
+    uint32_t *colmax_rep;    // [kPrepColmaxReplicas, K] accumulators: zero on entry, zeroed again before exit
     uint32_t *colmax_bits;   // [K] out: channel abs-max (bit patterns of non-negative floats)
-    Ctrl *ctrl;              // zero-initialised
+    Ctrl *ctrl;              // arrived, readers: zero on entry, zero again on exit
     int32_t *outlier_idx;    // [cap] out
     float *s_x_rows;         // [M] out when per_token
     int8_t *body_q;  int ld_q;

@@ -50,7 +50,8 @@ def run_linear(mx, x, w, p, out_kind, rows=None):
     wsw = mx.Workspace(mx.muxq_small_workspace_bytes(N))
     w_q, s_w = mx.muxq_quantize(dev(w), p, True, wsw)
     ws = mx.Workspace(mx.muxq_workspace_bytes(M, K, N, p))
-    ws.buf.fill_(0xA5)  # the workspace need not be initialised
+    ws.buf.fill_(0xA5)  # everything but the words muxq_workspace_init prepares may hold garbage
+    ws.init()
     y = mx.muxq_linear(dev(x), w_q, s_w, p, ws, out_kind)
     st = mx.muxq_read_status(ws)
     return y, ws, st, w_q, s_w
@@ -317,6 +318,7 @@ def test_capacity_overflow_sets_status_and_stays_in_bounds(mx):
     ybuf = torch.full((M + 2, N), 1234.0, dtype=torch.float16, device="cuda")
     ws_use = mx.Workspace(0)
     ws_use.buf = ws.buf[:nbytes]
+    ws_use.init()
     y = mx.muxq_linear(dev(x), w_q, s_w, p, ws_use, mx.MUXQ_OUT_F16, out=ybuf[1:M + 1])
     assert mx.muxq_read_status(ws_use) == mx.MUXQ_ERR_CAPACITY
     assert (ws.buf[nbytes:] == 0x77).all()
@@ -471,3 +473,26 @@ def test_wide_k_takes_the_separate_kernels(mx, M, gran):
     assert np.array_equal(v["body_q"], res.body_q)
     y32, _, st, _, _ = run_linear(mx, x, w, p, mx.MUXQ_OUT_F32)
     assert st == 0 and np.array_equal(y32.cpu().numpy(), res.y32)
+
+
+def test_one_workspace_serves_a_sequence_of_shapes(mx):
+    """The layer kernels leave the prepared words of the workspace as they found them: one
+    muxq_workspace_init, then different shapes, granularities and repeats, each checked against the oracle."""
+    shapes = [(300, 768, 256, 0), (300, 768, 256, 0), (64, 256, 136, 1), (520, 3072, 128, 0), (8, 512, 128, 0),
+              (40, 8320, 136, 0), (300, 768, 256, 1), (1000, 1024, 264, 0)]
+    big = 0
+    for M, K, N, gran in shapes:
+        big = max(big, mx.muxq_workspace_bytes(M, K, N, mx.MuxqParams(gran=gran)))
+    ws = mx.Workspace(big)
+    ws.buf.fill_(0x3C)
+    ws.init()
+    for i, (M, K, N, gran) in enumerate(shapes):
+        p = mx.MuxqParams(gran=gran)
+        x, w, _ = make_case(900 + i, M, K, N, n_out=5)
+        w_q, s_w = mx.muxq_quantize(dev(w), p, True, mx.Workspace(mx.muxq_small_workspace_bytes(N)))
+        y = mx.muxq_linear(dev(x), w_q, s_w, p, ws, mx.MUXQ_OUT_F32)
+        assert mx.muxq_read_status(ws) == 0
+        _, _, res = oracle_linear(x, w, p)
+        v = ws_views(mx, ws, M, K, N, p)
+        assert v["n_outliers"] == res.r and np.array_equal(v["outlier_idx"][:res.r], res.O), (i, M, K, N)
+        assert rel_err32(y.cpu().numpy(), res.y32) <= 1e-5, (i, M, K, N)
