@@ -46,9 +46,9 @@ __host__ __device__ inline int fixed_smem_bytes(int K) {
     return 8 * K + ((G + 15) & ~15) + kMaxOut * 4 + kMaxAuxCols * 2;
 }
 
-__device__ __forceinline__ uint32_t ld_relaxed_u32(const uint32_t *p) {
+__device__ __forceinline__ uint32_t ld_acquire_u32(const uint32_t *p) {
     uint32_t v;
-    asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
     return v;
 }
 
@@ -145,10 +145,11 @@ __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, int rows_base,
         __threadfence();  // cumulative: publishes the whole CTA's reductions, ordered before it by the barrier
         atomicAdd(&a.ctrl->arrived, 1u);
         bool ok = false;
+        // acquire loads: once the full count is seen, the other CTAs' reductions (released before their
+        // arrivals) are visible to this thread, and through the barrier below to the whole CTA
         for (uint32_t i = 0; i < kBarrierSpin; ++i) {
-            if (ld_relaxed_u32(&a.ctrl->arrived) >= gridDim.x) { ok = true; break; }
+            if (ld_acquire_u32(&a.ctrl->arrived) >= gridDim.x) { ok = true; break; }
         }
-        __threadfence();  // acquire side: the other CTAs' reductions are visible from here on
         s_fail = ok ? 0 : 1;
         if (!ok && a.dev_status) atomicMax(a.dev_status, kStatusTimeout);
     }
@@ -178,11 +179,10 @@ __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, int rows_base,
     // This CTA holds its copy of the maxima.  The CTA that takes the last ticket knows that every CTA does
     // (and has therefore left the barrier), so it may put the accumulators and both counters back to zero for
     // the next call; the ticket is fetched here and looked at only before the last phase, off the critical path.
+    // (No fence: the loads above have returned their values, so stores issued after the last ticket was
+    // taken cannot reach them.)
     uint32_t ticket = 0;
-    if (t == 0) {
-        __threadfence();
-        ticket = atomicAdd(&a.ctrl->readers, 1u);
-    }
+    if (t == 0) ticket = atomicAdd(&a.ctrl->readers, 1u);
     // Every thread derives the factors of the 8 channels it owns in both passes: 2^-e where the channel
     // holds an element above the threshold (strict), else 1.  (When more channels are flagged than the
     // capacity allows the call fails with MUXQ_ERR_CAPACITY and Y is unspecified, so no ordering is needed here.)
@@ -274,25 +274,48 @@ __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, int rows_base,
             float is[8];
 #pragma unroll
             for (int i = 0; i < 8; ++i) is[i] = inv_s * mul[i];  // the channel factor folded into 1/s (power of two: exact)
-            for (int row = row_off; row < rows; row += 2 * rstride) {
-                uint4 v[2];
+            // Rows row_off, row_off + rstride, ...: first those held in the slab, two per iteration, then the
+            // rest from global memory (normally L2), four loads in flight.  Addresses advance by constant steps.
+            const uint32_t sstep = (uint32_t)rstride * (uint32_t)K * 2u;
+            const size_t qstep = (size_t)rstride * a.ld_q, xstep = (size_t)rstride * a.ldx;
+            const uint8_t *sp = slab + (size_t)row_off * K * 2 + cg * 16;
+            int8_t *qp = a.body_q + ((size_t)r0 + row_off) * a.ld_q + cg * 8;
+            int row = row_off;
+            for (; row + rstride < fit; row += 2 * rstride) {
+                const uint4 v0 = *reinterpret_cast<const uint4 *>(sp);
+                const uint4 v1 = *reinterpret_cast<const uint4 *>(sp + sstep);
+                float f[8];
+                unpack8(v0, f);
+                *reinterpret_cast<uint2 *>(qp) = quant8_scaled(f, mul, is, s, qf);
+                unpack8(v1, f);
+                *reinterpret_cast<uint2 *>(qp + qstep) = quant8_scaled(f, mul, is, s, qf);
+                sp += 2 * sstep;
+                qp += 2 * qstep;
+            }
+            if (row < fit) {
+                float f[8];
+                unpack8(*reinterpret_cast<const uint4 *>(sp), f);
+                *reinterpret_cast<uint2 *>(qp) = quant8_scaled(f, mul, is, s, qf);
+                qp += qstep;
+                row += rstride;
+            }
+            const __half *xp = a.X + ((size_t)r0 + row) * a.ldx + cg * 8;
+            for (; row < rows; row += 4 * rstride) {
+                uint4 v[4];
 #pragma unroll
-                for (int u = 0; u < 2; ++u) {
-                    const int rr = row + u * rstride;
-                    v[u] = make_uint4(0u, 0u, 0u, 0u);
-                    if (rr < fit) v[u] = *reinterpret_cast<const uint4 *>(slab + (size_t)rr * K * 2 + cg * 16);
-                    else if (rr < rows) v[u] = __ldg(reinterpret_cast<const uint4 *>(a.X + ((size_t)r0 + rr) * a.ldx) + cg);
-                }
+                for (int u = 0; u < 4; ++u)
+                    v[u] = row + u * rstride < rows ? __ldg(reinterpret_cast<const uint4 *>(xp + u * xstep))
+                                                    : make_uint4(0u, 0u, 0u, 0u);
 #pragma unroll
-                for (int u = 0; u < 2; ++u) {
-                    const int rr = row + u * rstride;
-                    if (rr < rows) {
+                for (int u = 0; u < 4; ++u) {
+                    if (row + u * rstride < rows) {
                         float f[8];
                         unpack8(v[u], f);
-                        *reinterpret_cast<uint2 *>(a.body_q + ((size_t)r0 + rr) * a.ld_q + cg * 8) =
-                            quant8_scaled(f, mul, is, s, qf);
+                        *reinterpret_cast<uint2 *>(qp + u * qstep) = quant8_scaled(f, mul, is, s, qf);
                     }
                 }
+                xp += 4 * xstep;
+                qp += 4 * qstep;
             }
         }
     } else {
