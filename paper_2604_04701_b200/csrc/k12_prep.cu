@@ -72,6 +72,17 @@ __device__ __forceinline__ void load_chunk(const uint4 *src, int ch, const uint8
     }
 }
 
+// The exact form of Eq. 1 for one 8-channel chunk (mask: its outlier channels).  Kept out of line: it runs for
+// about one chunk in a thousand, and inlined at every use it costs the quantization loops their registers.
+__device__ __noinline__ uint2 codes_exact(uint4 v, uint32_t mask, float down, float s, float qf) {
+    float f[8];
+    unpack8(v, f);
+    uint32_t code[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) code[i] = (uint32_t)quant_exact((mask >> i) & 1u ? f[i] * down : f[i], s, qf);
+    return pack8(code);
+}
+
 __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, int rows_base, int rows_extra, int slab_bytes) {
     extern __shared__ __align__(16) uint8_t smem[];
     __shared__ float s_warp_max[kWarps];
@@ -103,23 +114,24 @@ __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, int rows_base,
         if (row_off < rstride) {
             __half2 m[4];
             m[0] = m[1] = m[2] = m[3] = __float2half2_rn(0.f);
-            const __half *px = a.X + (size_t)r0 * a.ldx + cg * 8;
-            uint8_t *ps = slab + cg * 16;
-            // up to 8 independent 16-byte loads in flight per thread
+            // up to 8 independent 16-byte loads in flight per thread; addresses advance by constant steps
+            const size_t xstep = (size_t)rstride * a.ldx;
+            const uint32_t sstep = (uint32_t)rstride * (uint32_t)K * 2u;
+            const __half *px = a.X + ((size_t)r0 + row_off) * a.ldx + cg * 8;
+            uint8_t *ps = slab + (size_t)row_off * K * 2 + cg * 16;
             for (int row = row_off; row < rows; row += 8 * rstride) {
                 uint4 v[8];
 #pragma unroll
-                for (int u = 0; u < 8; ++u) {
-                    const int rr = row + u * rstride;
-                    v[u] = rr < rows ? __ldg(reinterpret_cast<const uint4 *>(px + (size_t)rr * a.ldx))
-                                     : make_uint4(0u, 0u, 0u, 0u);
-                }
+                for (int u = 0; u < 8; ++u)
+                    v[u] = row + u * rstride < rows ? __ldg(reinterpret_cast<const uint4 *>(px + u * xstep))
+                                                    : make_uint4(0u, 0u, 0u, 0u);
 #pragma unroll
                 for (int u = 0; u < 8; ++u) {
                     absmax4(m, v[u]);
-                    const int rr = row + u * rstride;
-                    if (rr < fit) *reinterpret_cast<uint4 *>(ps + (size_t)rr * K * 2) = v[u];
+                    if (row + u * rstride < fit) *reinterpret_cast<uint4 *>(ps + u * sstep) = v[u];
                 }
+                px += 8 * xstep;
+                ps += 8 * sstep;
             }
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
@@ -189,23 +201,23 @@ __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, int rows_base,
     const int rstride = kT / G;
     const int cg = t % G, row_off = t / G;
     float mul[8];
+    uint32_t fmask = 0;  // bit i: channel 8*cg + i is an outlier channel
     {
         const float4 v0 = reinterpret_cast<const float4 *>(s_colmax)[2 * cg];
         const float4 v1 = reinterpret_cast<const float4 *>(s_colmax)[2 * cg + 1];
         const float cm[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
         float bmax = 0.0f;
-        uint32_t mask = 0;  // bit i: channel 8*cg + i is an outlier channel
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
             const bool flagged = cm[i] > a.tau;
             mul[i] = flagged ? down : 1.0f;
-            mask |= flagged ? (1u << i) : 0u;
+            fmask |= flagged ? (1u << i) : 0u;
             bmax = fmaxf(bmax, cm[i] * mul[i]);  // power-of-two scaling: exact
         }
         if (row_off == 0) {  // shared copies: the outlier listing below and the per-token path read them
             reinterpret_cast<float4 *>(s_colmul)[2 * cg] = make_float4(mul[0], mul[1], mul[2], mul[3]);
             reinterpret_cast<float4 *>(s_colmul)[2 * cg + 1] = make_float4(mul[4], mul[5], mul[6], mul[7]);
-            s_flag[cg] = (uint8_t)mask;
+            s_flag[cg] = (uint8_t)fmask;
         }
         bmax = warp_max(bmax);
         if (lane == 0) s_warp_max[warp] = bmax;
@@ -271,9 +283,22 @@ __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, int rows_base,
         // Per-tensor scale: the pass-1 mapping again (a thread owns 8 channels and walks down the
         // rows), so the channel factors stay in registers and consecutive lanes store consecutive codes.
         if (row_off < rstride) {
-            float is[8];
+            // brackets of 1/s with the channel factor folded in (power of two: exact)
+            float blo[8], bhi[8];
+            {
+                float lo, hi;
+                recip_bracket(inv_s, lo, hi);
 #pragma unroll
-            for (int i = 0; i < 8; ++i) is[i] = inv_s * mul[i];  // the channel factor folded into 1/s (power of two: exact)
+                for (int i = 0; i < 8; ++i) { blo[i] = lo * mul[i]; bhi[i] = hi * mul[i]; }
+            }
+            // 8 values of this thread's channel group -> 8 codes; the exact division only next to a tie
+            auto codes = [&](const uint4 &v) -> uint2 {
+                float f[8];
+                unpack8(v, f);
+                uint32_t code[8];
+                if (quant8_bracket(f, blo, bhi, code)) return codes_exact(v, fmask, down, s, qf);  // next to a tie: rare
+                return pack8(code);
+            };
             // Rows row_off, row_off + rstride, ...: first those held in the slab, two per iteration, then the
             // rest from global memory (normally L2), four loads in flight.  Addresses advance by constant steps.
             const uint32_t sstep = (uint32_t)rstride * (uint32_t)K * 2u;
@@ -284,18 +309,13 @@ __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, int rows_base,
             for (; row + rstride < fit; row += 2 * rstride) {
                 const uint4 v0 = *reinterpret_cast<const uint4 *>(sp);
                 const uint4 v1 = *reinterpret_cast<const uint4 *>(sp + sstep);
-                float f[8];
-                unpack8(v0, f);
-                *reinterpret_cast<uint2 *>(qp) = quant8_scaled(f, mul, is, s, qf);
-                unpack8(v1, f);
-                *reinterpret_cast<uint2 *>(qp + qstep) = quant8_scaled(f, mul, is, s, qf);
+                *reinterpret_cast<uint2 *>(qp) = codes(v0);
+                *reinterpret_cast<uint2 *>(qp + qstep) = codes(v1);
                 sp += 2 * sstep;
                 qp += 2 * qstep;
             }
             if (row < fit) {
-                float f[8];
-                unpack8(*reinterpret_cast<const uint4 *>(sp), f);
-                *reinterpret_cast<uint2 *>(qp) = quant8_scaled(f, mul, is, s, qf);
+                *reinterpret_cast<uint2 *>(qp) = codes(*reinterpret_cast<const uint4 *>(sp));
                 qp += qstep;
                 row += rstride;
             }
@@ -308,11 +328,7 @@ __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, int rows_base,
                                                     : make_uint4(0u, 0u, 0u, 0u);
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {
-                    if (row + u * rstride < rows) {
-                        float f[8];
-                        unpack8(v[u], f);
-                        *reinterpret_cast<uint2 *>(qp + u * qstep) = quant8_scaled(f, mul, is, s, qf);
-                    }
+                    if (row + u * rstride < rows) *reinterpret_cast<uint2 *>(qp + u * qstep) = codes(v[u]);
                 }
                 xp += 4 * xstep;
                 qp += 4 * qstep;
@@ -335,13 +351,19 @@ __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, int rows_base,
             }
             mx = warp_max(mx);
             const float sr = mx > 0.0f ? __fdiv_rn(mx, qf) : 1.0f;
-            const float inv_sr = __fdiv_rn(1.0f, sr);
+            float rlo, rhi;
+            recip_bracket(__frcp_rn(sr), rlo, rhi);
             if (lane == 0) a.s_x_rows[m] = sr;
             int8_t *q = a.body_q + m * a.ld_q;
             for (int ch = lane; ch < G; ch += 32) {
                 float f[8];
                 load_chunk(src, ch, s_flag, s_colmul, f);
-                *reinterpret_cast<uint2 *>(q + ch * 8) = quant8(f, sr, inv_sr, qf);
+                uint32_t code[8];
+                if (quant8_bracket(f, rlo, rhi, code)) {
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) code[i] = (uint32_t)quant_exact(f[i], sr, qf);
+                }
+                *reinterpret_cast<uint2 *>(q + ch * 8) = pack8(code);
             }
             if (a.aux_q) {
                 // shared scale: Aux_q[m, c*j + i] is the code Body_q[m, O_j] this warp has just written

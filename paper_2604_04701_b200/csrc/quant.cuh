@@ -60,24 +60,45 @@ __device__ __forceinline__ uint2 quant8(const float (&f)[8], float s, float inv_
     return make_uint2(__byte_perm(p01, p23, 0x5410), __byte_perm(p45, p67, 0x5410));
 }
 
-// The same for values whose power-of-two channel factors mul[i] are still to be applied, with
-// is[i] = (1/s) * mul[i] (exact), and for a scale s that was derived from these very values, so that
-// no code can leave [-q, q] and the range check is not needed.
-__device__ __forceinline__ uint2 quant8_scaled(const float (&f)[8], const float (&mul)[8], const float (&is)[8],
-                                               float s, float qf) {
+// Bracket form of the fast path, for a scale s that was derived from the values themselves (no code can leave
+// [-q, q]).  With inv = RN(1/s), the correctly rounded quotient RN(v/s) differs from the real product v * inv
+// by a relative 2^-23 (1 + 2^-23) at most, so it lies between v * lo and v * hi for lo / hi three units in the
+// last place below / above inv.  fma(v, lo, 1.5 * 2^23) and fma(v, hi, 1.5 * 2^23) round those two real products
+// to integers (half to even) exactly once each; rounding to an integer is monotone, so when both give the same
+// integer, round_half_even(RN(v/s)) is that integer too, and its two's-complement low byte sits in the low byte
+// of the float's bit pattern.  Power-of-two channel factors folded into lo / hi keep all of this exact.
+// Returns nonzero when some value sits too close to a tie for the bracket to decide; the caller then takes
+// the exact division for the chunk.  Three instructions per value (two fma, one logic op).
+__device__ __forceinline__ void recip_bracket(float inv_s, float &lo, float &hi) {
+    lo = __uint_as_float(__float_as_uint(inv_s) - 3u);  // inv_s is a positive normal number
+    hi = __uint_as_float(__float_as_uint(inv_s) + 3u);
+}
+
+__device__ __forceinline__ uint32_t quant8_bracket(const float (&f)[8], const float (&lo)[8], const float (&hi)[8],
+                                                   uint32_t (&b)[8]) {
     const float magic = 12582912.0f;  // 1.5 * 2^23
-    uint32_t b[8];
-    float dmax = 0.0f;
+    uint32_t diff = 0;
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
-        const float tm = fmaf(f[i], is[i], magic);
-        dmax = fmaxf(dmax, fabsf(fmaf(f[i], is[i], magic - tm)));
-        b[i] = __float_as_uint(tm);
+        b[i] = __float_as_uint(fmaf(f[i], hi[i], magic));
+        diff |= b[i] ^ __float_as_uint(fmaf(f[i], lo[i], magic));
     }
-    if (dmax > 0.4999f) {
+    return diff;
+}
+
+__device__ __forceinline__ uint32_t quant8_bracket(const float (&f)[8], float lo, float hi, uint32_t (&b)[8]) {
+    const float magic = 12582912.0f;
+    uint32_t diff = 0;
 #pragma unroll
-        for (int i = 0; i < 8; ++i) b[i] = (uint32_t)quant_exact(f[i] * mul[i], s, qf);
+    for (int i = 0; i < 8; ++i) {
+        b[i] = __float_as_uint(fmaf(f[i], hi, magic));
+        diff |= b[i] ^ __float_as_uint(fmaf(f[i], lo, magic));
     }
+    return diff;
+}
+
+// low bytes of 8 words -> 8 codes in a uint2
+__device__ __forceinline__ uint2 pack8(const uint32_t (&b)[8]) {
     const uint32_t p01 = __byte_perm(b[0], b[1], 0x0040), p23 = __byte_perm(b[2], b[3], 0x0040);
     const uint32_t p45 = __byte_perm(b[4], b[5], 0x0040), p67 = __byte_perm(b[6], b[7], 0x0040);
     return make_uint2(__byte_perm(p01, p23, 0x5410), __byte_perm(p45, p67, 0x5410));
