@@ -193,8 +193,8 @@ typedef struct muxq_ws_view {
     size_t n_outliers;  /* int32 [1] */
     size_t s_x;         /* float [1] or [M] */
     size_t body_q;      /* int8 [M, ld_body_q] */
-    size_t aux_q;       /* int8 [M, aux_cols] */
-    size_t w_aux;       /* int8 [N, aux_cols] */
+    size_t aux_q;       /* int8 [M, aux_cols]; written up to column round_up(c * r, 32): codes, then zeros */
+    size_t w_aux;       /* int8 [N, aux_cols]; likewise (the products read no column beyond that) */
     int ld_body_q;
     int aux_cols;
 } muxq_ws_view;

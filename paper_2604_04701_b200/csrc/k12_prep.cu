@@ -83,6 +83,9 @@ __device__ __noinline__ uint2 codes_exact(uint4 v, uint32_t mask, float down, fl
     return pack8(code);
 }
 
+// kAllFit: the host has sized the slab for every row of the largest CTA share, so the loops over rows that
+// live only in global memory are compiled out (and with them their registers).
+template <bool kAllFit>
 __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, int rows_base, int rows_extra, int slab_bytes) {
     extern __shared__ __align__(16) uint8_t smem[];
     __shared__ float s_warp_max[kWarps];
@@ -102,7 +105,7 @@ __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, int rows_base,
     const int b = blockIdx.x;
     const int r0 = b * rows_base + min(b, rows_extra);
     const int rows = rows_base + (b < rows_extra ? 1 : 0);
-    const int fit = min(rows, slab_bytes / (2 * K));
+    const int fit = kAllFit ? rows : min(rows, slab_bytes / (2 * K));
     if (b == 0 && t == 0 && a.dev_status) *a.dev_status = 0;
 
     // ---------------------------------------------------------------- pass 1: channel maxima
@@ -190,11 +193,9 @@ __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, int rows_base,
     __syncthreads();
     // This CTA holds its copy of the maxima.  The CTA that takes the last ticket knows that every CTA does
     // (and has therefore left the barrier), so it may put the accumulators and both counters back to zero for
-    // the next call; the ticket is fetched here and looked at only before the last phase, off the critical path.
+    // the next call; the ticket is taken by the last warp, which is off the critical path of the quantization.
     // (No fence: the loads above have returned their values, so stores issued after the last ticket was
     // taken cannot reach them.)
-    uint32_t ticket = 0;
-    if (t == 0) ticket = atomicAdd(&a.ctrl->readers, 1u);
     // Every thread derives the factors of the 8 channels it owns in both passes: 2^-e where the channel
     // holds an element above the threshold (strict), else 1.  (When more channels are flagged than the
     // capacity allows the call fails with MUXQ_ERR_CAPACITY and Y is unspecified, so no ordering is needed here.)
@@ -237,6 +238,8 @@ __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, int rows_base,
     // per-group flag masks; nothing needs the list before the Aux block.  It also fills the source channel
     // of every Aux column: column c*j + i mirrors channel O_j (Eq. 5), repeated c times for Eq. 7.
     if (warp == kWarps - 1) {
+        uint32_t ticket = 0;
+        if (lane == 0) ticket = atomicAdd(&a.ctrl->readers, 1u);  // every thread passed the barrier after the fetch
         int carry = 0;
         for (int base = 0; base < G; base += 32) {
             const int g = base + lane;
@@ -265,6 +268,7 @@ __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, int rows_base,
         const int ucols = c * min(carry, a.cap);
         for (int i = lane; i < ucols; i += 32) s_auxsrc[i] = (uint16_t)s_oidx[i / c];
         if (lane == 0) {
+            s_last = ticket == gridDim.x - 1 ? 1 : 0;
             s_r_true = carry;
             if (b == 0) {
                 a.ctrl->n_outliers = carry;
@@ -320,7 +324,7 @@ __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, int rows_base,
                 row += rstride;
             }
             const __half *xp = a.X + ((size_t)r0 + row) * a.ldx + cg * 8;
-            for (; row < rows; row += 4 * rstride) {
+            for (; !kAllFit && row < rows; row += 4 * rstride) {
                 uint4 v[4];
 #pragma unroll
                 for (int u = 0; u < 4; ++u)
@@ -336,7 +340,7 @@ __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, int rows_base,
         }
     } else {
         const int r = min(s_r_true, a.cap);
-        const int used_cols = c * r, used_words = (used_cols + 3) >> 2;
+        const int used_cols = c * r, pad_words = ((used_cols + 31) & ~31) >> 2;
         for (int row = warp; row < rows; row += kWarps) {
             const size_t m = (size_t)r0 + row;
             const uint4 *src = row < fit ? reinterpret_cast<const uint4 *>(slab + (size_t)row * K * 2)
@@ -368,14 +372,12 @@ __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, int rows_base,
             if (a.aux_q) {
                 // shared scale: Aux_q[m, c*j + i] is the code Body_q[m, O_j] this warp has just written
                 __syncwarp();
-                for (int w = lane; w < (a.aux_cols >> 2); w += 32) {
+                for (int w = lane; w < pad_words; w += 32) {
                     uint32_t packed = 0;
-                    if (w < used_words) {
 #pragma unroll
-                        for (int bb = 0; bb < 4; ++bb)
-                            if (w * 4 + bb < used_cols)
-                                packed |= (uint32_t)(uint8_t)q[s_auxsrc[w * 4 + bb]] << (8 * bb);
-                    }
+                    for (int bb = 0; bb < 4; ++bb)
+                        if (w * 4 + bb < used_cols)
+                            packed |= (uint32_t)(uint8_t)q[s_auxsrc[w * 4 + bb]] << (8 * bb);
                     *reinterpret_cast<uint32_t *>(a.aux_q + m * a.ld_aux + w * 4) = packed;
                 }
             }
@@ -383,32 +385,37 @@ __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, int rows_base,
     }
 
     // ---------------------------------------------------------------- Aux block (per tensor) and W_aux
-    if (t == 0) s_last = ticket == gridDim.x - 1 ? 1 : 0;
     __syncthreads();  // the last warp's outlier list and Aux sources are complete
     const int r = min(s_r_true, a.cap);
-    const int used_cols = c * r, used_words = (used_cols + 3) >> 2;
-    // Three independent jobs share the CTA's warps so that their latencies overlap instead of adding up:
-    // warps 0-15 the Aux codes, warps 16-23 the Aux zero fill, warps 24-31 the W_aux gather.
+    const int used_cols = c * r;
+    // The GEMM consumes the Aux columns in steps of 32, i.e. columns [0, pad_cols); an Aux column of zeros makes the
+    // matching W_aux column irrelevant and vice versa, so both blocks are written up to pad_cols only (codes, then
+    // zeros) and the columns behind are left as they are.
+    const int pad_words = ((used_cols + 31) & ~31) >> 2;
+    // Independent jobs share the CTA's warps so that their latencies overlap instead of adding up: warps 0-15 the
+    // Aux codes, warps 16-31 the W_aux gather (and, in one CTA per launch, the clean-up for the next call).
     const bool do_aux = a.aux_q && !a.per_token;
     if (warp < 16) {
         if (do_aux) {
             // Aux_q[m, c*j + i] = code of Body[m, O_j] (Eq. 5, shared scale), recomputed from the slab with the
-            // exact division, one (row, column) pair per thread; the tail of the last used word is zero.
-            const int bcols = used_words * 4;
-            for (int i = t; i < rows * bcols; i += 512) {
-                const int row = i / bcols, col = i - row * bcols;
+            // exact division, one 4-byte word per thread and round
+            for (int i = t; i < rows * pad_words; i += 512) {
+                const int row = i / pad_words, w = i - row * pad_words;
                 const size_t m = (size_t)r0 + row;
-                int code = 0;
-                if (col < used_cols) {
-                    const __half *xr = row < fit ? reinterpret_cast<const __half *>(slab + (size_t)row * K * 2)
-                                                 : a.X + m * a.ldx;
-                    code = quant_exact(__half2float(xr[s_auxsrc[col]]) * down, s, qf);
+                const __half *xr = row < fit ? reinterpret_cast<const __half *>(slab + (size_t)row * K * 2)
+                                             : a.X + m * a.ldx;
+                uint32_t packed = 0;
+#pragma unroll
+                for (int bb = 0; bb < 4; ++bb) {
+                    const int col = w * 4 + bb;
+                    if (col < used_cols)
+                        packed |= (uint32_t)(quant_exact(__half2float(xr[s_auxsrc[col]]) * down, s, qf) & 0xff) << (8 * bb);
                 }
-                a.aux_q[m * a.ld_aux + col] = (int8_t)code;
+                *reinterpret_cast<uint32_t *>(a.aux_q + m * a.ld_aux + w * 4) = packed;
             }
         }
-    } else if (warp < 24) {
-        if (s_last) {
+    } else {
+        if (s_last && warp < 24) {
             uint4 *rep4 = reinterpret_cast<uint4 *>(a.colmax_rep);
             for (int i = t - 512; i < kColmaxReplicas * (K >> 2); i += 256) rep4[i] = make_uint4(0u, 0u, 0u, 0u);
             if (t == 512) {
@@ -416,29 +423,18 @@ __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, int rows_base,
                 a.ctrl->readers = 0u;
             }
         }
-        if (do_aux) {
-            // whole words of the Aux block beyond the used ones
-            const int aux_words = a.aux_cols >> 2;
-            const int zwords = aux_words - used_words;
-            for (int i = t - 512; i < rows * zwords; i += 256) {
-                const int row = i / zwords, w = used_words + (i - row * zwords);
-                *reinterpret_cast<uint32_t *>(a.aux_q + ((size_t)r0 + row) * a.ld_aux + w * 4) = 0u;
-            }
-        }
-    } else if (a.w_aux) {
-        // W_aux[n, c*j + i] = W_q[n, O_j], one 4-byte word per thread and round, spread over the grid
-        const int words_per_row = a.aux_cols >> 2;
-        const int total = a.N * words_per_row;
-        for (int i = b * 256 + (t - 768); i < total; i += gridDim.x * 256) {
-            const int n = i / words_per_row, w = i - n * words_per_row;
-            uint32_t packed = 0;
-            if (w < used_words) {
+        if (a.w_aux) {
+            // W_aux[n, c*j + i] = W_q[n, O_j], one 4-byte word per thread and round, spread over the grid
+            const int total = a.N * pad_words;
+            for (int i = b * 512 + (t - 512); i < total; i += gridDim.x * 512) {
+                const int n = i / pad_words, w = i - n * pad_words;
+                uint32_t packed = 0;
 #pragma unroll
                 for (int bb = 0; bb < 4; ++bb)
                     if (w * 4 + bb < used_cols)
                         packed |= (uint32_t)(uint8_t)a.w_q[(size_t)n * a.ldw + s_auxsrc[w * 4 + bb]] << (8 * bb);
+                *reinterpret_cast<uint32_t *>(a.w_aux + (size_t)n * a.ld_waux + w * 4) = packed;
             }
-            *reinterpret_cast<uint32_t *>(a.w_aux + (size_t)n * a.ld_waux + w * 4) = packed;
         }
     }
 }
@@ -450,7 +446,9 @@ bool prep_supported(int M, int K) { return M >= 1 && K >= 8 && K % 8 == 0 && K <
 cudaError_t launch_prep(const PrepArgs &a, cudaStream_t s) {
     static bool attr_set = false;
     if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(k_prep, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem);
+        cudaError_t e = cudaFuncSetAttribute(k_prep<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(k_prep<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem);
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
@@ -464,8 +462,9 @@ cudaError_t launch_prep(const PrepArgs &a, cudaStream_t s) {
     slab_bytes &= ~15;
     PrepArgs args = a;
     void *params[] = {&args, &rows_base, &rows_extra, &slab_bytes};
-    return cudaLaunchCooperativeKernel(reinterpret_cast<const void *>(k_prep), dim3(grid), dim3(kT), params,
-                                       (size_t)(fixed + slab_bytes), s);
+    const bool all_fit = (long long)slab_bytes >= want;
+    const void *fn = all_fit ? reinterpret_cast<const void *>(k_prep<true>) : reinterpret_cast<const void *>(k_prep<false>);
+    return cudaLaunchCooperativeKernel(fn, dim3(grid), dim3(kT), params, (size_t)(fixed + slab_bytes), s);
 }
 
 }  // namespace muxq
