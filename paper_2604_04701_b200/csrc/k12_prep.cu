@@ -85,7 +85,9 @@ __device__ __noinline__ uint2 codes_exact(uint4 v, uint32_t mask, float down, fl
 
 // kAllFit: the host has sized the slab for every row of the largest CTA share, so the loops over rows that
 // live only in global memory are compiled out (and with them their registers).
-template <bool kAllFit>
+// kPerToken: per-token scales (one warp per row in pass 2) instead of the per-tensor scale; one instantiation
+// per granularity keeps the other one's code out of the kernel.
+template <bool kAllFit, bool kPerToken>
 __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, int rows_base, int rows_extra, int slab_bytes) {
     extern __shared__ __align__(16) uint8_t smem[];
     __shared__ float s_warp_max[kWarps];
@@ -276,14 +278,14 @@ __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, int rows_base,
             }
         }
     }
-    if (a.per_token) __syncthreads();  // the per-token path reads the shared factor copies and the Aux sources
+    if (kPerToken) __syncthreads();  // the per-token path reads the shared factor copies and the Aux sources
 
     // Let a kernel launched as a programmatic dependent (the GEMM) start its set-up on SMs as they free up;
     // it still waits for this whole grid to finish before it reads anything written here.
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     // ---------------------------------------------------------------- pass 2: Body_q and the Aux block
-    if (!a.per_token) {
+    if (!kPerToken) {
         // Per-tensor scale: the pass-1 mapping again (a thread owns 8 channels and walks down the
         // rows), so the channel factors stay in registers and consecutive lanes store consecutive codes.
         if (row_off < rstride) {
@@ -394,7 +396,7 @@ __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, int rows_base,
     const int pad_words = ((used_cols + 31) & ~31) >> 2;
     // Independent jobs share the CTA's warps so that their latencies overlap instead of adding up: warps 0-15 the
     // Aux codes, warps 16-31 the W_aux gather (and, in one CTA per launch, the clean-up for the next call).
-    const bool do_aux = a.aux_q && !a.per_token;
+    const bool do_aux = a.aux_q && !kPerToken;
     if (warp < 16) {
         if (do_aux) {
             // Aux_q[m, c*j + i] = code of Body[m, O_j] (Eq. 5, shared scale), recomputed from the slab with the
@@ -444,12 +446,15 @@ __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, int rows_base,
 bool prep_supported(int M, int K) { return M >= 1 && K >= 8 && K % 8 == 0 && K <= kMaxK; }
 
 cudaError_t launch_prep(const PrepArgs &a, cudaStream_t s) {
+    static const void *const fns[4] = {
+        reinterpret_cast<const void *>(k_prep<false, false>), reinterpret_cast<const void *>(k_prep<false, true>),
+        reinterpret_cast<const void *>(k_prep<true, false>), reinterpret_cast<const void *>(k_prep<true, true>)};
     static bool attr_set = false;
     if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(k_prep<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem);
-        if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(k_prep<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem);
-        if (e != cudaSuccess) return e;
+        for (const void *f : fns) {
+            cudaError_t e = cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem);
+            if (e != cudaSuccess) return e;
+        }
         attr_set = true;
     }
     int grid = num_sms();
@@ -463,7 +468,7 @@ cudaError_t launch_prep(const PrepArgs &a, cudaStream_t s) {
     PrepArgs args = a;
     void *params[] = {&args, &rows_base, &rows_extra, &slab_bytes};
     const bool all_fit = (long long)slab_bytes >= want;
-    const void *fn = all_fit ? reinterpret_cast<const void *>(k_prep<true>) : reinterpret_cast<const void *>(k_prep<false>);
+    const void *fn = fns[(all_fit ? 2 : 0) + (a.per_token ? 1 : 0)];
     return cudaLaunchCooperativeKernel(fn, dim3(grid), dim3(kT), params, (size_t)(fixed + slab_bytes), s);
 }
 
