@@ -78,6 +78,9 @@ __global__ void __launch_bounds__(kT, 1) k_decode_fused(const DecodeFusedArgs a,
     const float qf = (float)a.qmax;
     const bool first = blockIdx.x == 0;
 
+    // Let the next kernel in the stream (programmatic dependent launch) become resident as early as there is
+    // room for it: it fetches its own weights and then waits for this grid to finish before it touches X or Y.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     // The first tile's share of W_q does not depend on X: its loads go out before the prologue, so the
     // HBM latency of the stream overlaps the detection and quantization work.
     const int r = lane >> 2, q = lane & 3;
@@ -98,7 +101,6 @@ __global__ void __launch_bounds__(kT, 1) k_decode_fused(const DecodeFusedArgs a,
     // Everything below reads X or writes results: under programmatic dependent launch it must wait for the
     // kernel before this one in the stream; the weights above are constants and were fetched ahead of that.
     asm volatile("griddepcontrol.wait;" ::: "memory");
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     if (first && t == 0 && a.dev_status) *a.dev_status = 0;
     if (t < 16) s_rowmax[t] = 0u;
