@@ -44,8 +44,10 @@ struct Smem {
     int off_segflag;    // [K/64] segment holds an outlier channel
     int off_grpmask;    // [K/8] per-group flag bits
     int off_red;        // [2][kWarps][128] int32 partial tiles
+    int off_xs;         // [MT][K] fp16 copy of X between the two passes (only when it fits), else -1
     int total;
 };
+constexpr int kMaxSmem = 200 * 1024;
 __host__ __device__ inline Smem smem_layout(int MT, int K) {
     Smem s;
     s.pitch = K + ((64 - (K & 127)) & 127);
@@ -55,6 +57,11 @@ __host__ __device__ inline Smem smem_layout(int MT, int K) {
     s.off_grpmask = s.off_segflag + (((K >> 6) + 15) & ~15);
     s.off_red = (s.off_grpmask + (K >> 3) + 15) & ~15;
     s.total = s.off_red + 2 * kWarps * 128 * 4;
+    s.off_xs = -1;
+    if (MT == 8 && s.total + MT * K * 2 <= kMaxSmem) {
+        s.off_xs = s.total;
+        s.total += MT * K * 2;
+    }
     return s;
 }
 
@@ -74,6 +81,7 @@ __global__ void __launch_bounds__(kT, 1) k_decode_fused(const DecodeFusedArgs a,
     uint8_t *s_segflag = smem + L.off_segflag;
     uint8_t *s_grpmask = smem + L.off_grpmask;
     int *s_red = reinterpret_cast<int *>(smem + L.off_red);
+    uint8_t *xs = L.off_xs >= 0 ? smem + L.off_xs : nullptr;
     const float down = __int_as_float((127 - a.exp_factor) << 23);  // 2^-e
     const float qf = (float)a.qmax;
     const bool first = blockIdx.x == 0;
@@ -98,6 +106,7 @@ __global__ void __launch_bounds__(kT, 1) k_decode_fused(const DecodeFusedArgs a,
             wpre[u] = seg < nseg ? __ldg(reinterpret_cast<const uint4 *>(wrow + seg * 64)) : make_uint4(0u, 0u, 0u, 0u);
         }
     }
+    const float sw0 = __ldg(a.s_w);  // a constant of the layer like W_q (the per-tensor scale, or the first column's)
     // Everything below reads X or writes results: under programmatic dependent launch it must wait for the
     // kernel before this one in the stream; the weights above are constants and were fetched ahead of that.
     asm volatile("griddepcontrol.wait;" ::: "memory");
@@ -123,6 +132,11 @@ __global__ void __launch_bounds__(kT, 1) k_decode_fused(const DecodeFusedArgs a,
                 for (int u = 0; u < 4; ++u)
                     v[u] = m0 + u < M ? __ldg(reinterpret_cast<const uint4 *>(a.X + (size_t)(m0 + u) * a.ldx) + cg)
                                       : make_uint4(0u, 0u, 0u, 0u);
+                if (xs) {
+#pragma unroll
+                    for (int u = 0; u < 4; ++u)
+                        if (m0 + u < M) *reinterpret_cast<uint4 *>(xs + (size_t)(m0 + u) * K * 2 + cg * 16) = v[u];
+                }
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {
                     cm[0] = __hmax2(cm[0], __habs2(*reinterpret_cast<const __half2 *>(&v[u].x)));
@@ -163,7 +177,8 @@ __global__ void __launch_bounds__(kT, 1) k_decode_fused(const DecodeFusedArgs a,
             const int cg = t + it * kT;
             if (cg < G) {
                 for (int m = 0; m < M; ++m) {
-                    const uint4 v = __ldg(reinterpret_cast<const uint4 *>(a.X + (size_t)m * a.ldx) + cg);
+                    const uint4 v = xs ? *reinterpret_cast<const uint4 *>(xs + (size_t)m * K * 2 + cg * 16)
+                                       : __ldg(reinterpret_cast<const uint4 *>(a.X + (size_t)m * a.ldx) + cg);
                     float f[8];
                     unpack8(v, f);
                     float rm = 0.0f;
@@ -238,12 +253,17 @@ __global__ void __launch_bounds__(kT, 1) k_decode_fused(const DecodeFusedArgs a,
             float mul[8];
 #pragma unroll
             for (int i = 0; i < 8; ++i) mul[i] = (my_mask[it] >> i) & 1u ? down : 1.0f;
+            float lo = 0.0f, hi = 0.0f;
+            if (!a.per_vec) recip_bracket(__frcp_rn(s_rowscale[0]), lo, hi);
             for (int m0 = 0; m0 < MT; m0 += 4) {  // four independent row loads in flight
                 uint4 v[4];
 #pragma unroll
-                for (int u = 0; u < 4; ++u)
-                    v[u] = m0 + u < M ? __ldg(reinterpret_cast<const uint4 *>(a.X + (size_t)(m0 + u) * a.ldx) + cg)
-                                      : make_uint4(0u, 0u, 0u, 0u);
+                for (int u = 0; u < 4; ++u) {
+                    v[u] = make_uint4(0u, 0u, 0u, 0u);
+                    if (m0 + u < M)
+                        v[u] = xs ? *reinterpret_cast<const uint4 *>(xs + (size_t)(m0 + u) * K * 2 + cg * 16)
+                                  : __ldg(reinterpret_cast<const uint4 *>(a.X + (size_t)(m0 + u) * a.ldx) + cg);
+                }
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {
                     const int m = m0 + u;
@@ -254,7 +274,14 @@ __global__ void __launch_bounds__(kT, 1) k_decode_fused(const DecodeFusedArgs a,
 #pragma unroll
                         for (int i = 0; i < 8; ++i) f[i] *= mul[i];  // exact
                         const float s = s_rowscale[a.per_vec ? m : 0];
-                        code = quant8(f, s, __frcp_rn(s), qf);
+                        if (a.per_vec) recip_bracket(__frcp_rn(s), lo, hi);
+                        // the scale comes from these very values: no code can leave the range (bracket form)
+                        uint32_t cb[8];
+                        if (quant8_bracket(f, lo, hi, cb)) {
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) cb[i] = (uint32_t)quant_exact(f[i], s, qf);
+                        }
+                        code = pack8(cb);
                     }
                     *reinterpret_cast<uint2 *>(xq + m * L.pitch + cg * 8) = code;
                 }
@@ -271,7 +298,9 @@ __global__ void __launch_bounds__(kT, 1) k_decode_fused(const DecodeFusedArgs a,
     const int groups = (tiles + tpg - 1) / tpg;
     for (int group = blockIdx.x; group < groups; group += gridDim.x) {
         const int8_t *xlo = xq + r * L.pitch + q * 16;
-        int accb[4] = {0, 0, 0, 0}, acca[4] = {0, 0, 0, 0};
+        // two Body accumulators (the two halves of a 64-byte segment): consecutive mma.sync on one accumulator
+        // wait for each other, and that chain is what this loop's time consists of
+        int accb[4] = {0, 0, 0, 0}, accb2[4] = {0, 0, 0, 0}, acca[4] = {0, 0, 0, 0};
         // this warp's segments (at most kPre by the choice of tpg) are already in registers
 #pragma unroll
         for (int u = 0; u < kPre; ++u) {
@@ -281,7 +310,7 @@ __global__ void __launch_bounds__(kT, 1) k_decode_fused(const DecodeFusedArgs a,
                 uint4 ahi = make_uint4(0u, 0u, 0u, 0u);
                 if (MT == 16) ahi = *reinterpret_cast<const uint4 *>(xlo + 8 * L.pitch + seg * 64);
                 mma_s8(accb, alo.x, ahi.x, alo.y, ahi.y, wpre[u].x, wpre[u].y);
-                mma_s8(accb, alo.z, ahi.z, alo.w, ahi.w, wpre[u].z, wpre[u].w);
+                mma_s8(accb2, alo.z, ahi.z, alo.w, ahi.w, wpre[u].z, wpre[u].w);
                 if (s_segflag[seg]) {  // warp-uniform: Aux term on the outlier channels of this segment
                     const uint4 mk = *reinterpret_cast<const uint4 *>(s_mask + seg * 64 + q * 16);
                     mma_s8(acca, alo.x & mk.x, ahi.x & mk.x, alo.y & mk.y, ahi.y & mk.y, wpre[u].x, wpre[u].y);
@@ -302,10 +331,10 @@ __global__ void __launch_bounds__(kT, 1) k_decode_fused(const DecodeFusedArgs a,
         // acc = acc_b + c * acc_a (Eq. 7), partial over this warp's K segments; element (row, col) of the
         // 16 x 8 tile: this lane holds rows r and r+8, columns 2q and 2q+1
         int *red = s_red + warp * 128;
-        red[r * 8 + 2 * q] = accb[0] + a.c * acca[0];
-        red[r * 8 + 2 * q + 1] = accb[1] + a.c * acca[1];
-        red[(r + 8) * 8 + 2 * q] = accb[2] + a.c * acca[2];
-        red[(r + 8) * 8 + 2 * q + 1] = accb[3] + a.c * acca[3];
+        red[r * 8 + 2 * q] = accb[0] + accb2[0] + a.c * acca[0];
+        red[r * 8 + 2 * q + 1] = accb[1] + accb2[1] + a.c * acca[1];
+        red[(r + 8) * 8 + 2 * q] = accb[2] + accb2[2] + a.c * acca[2];
+        red[(r + 8) * 8 + 2 * q + 1] = accb[3] + accb2[3] + a.c * acca[3];
         __syncthreads();
         for (int e = t; e < 128 * tpg; e += kT) {
             const int j = e >> 7, el = e & 127;  // tile of the group, element of its 16 x 8 tile
@@ -318,7 +347,7 @@ __global__ void __launch_bounds__(kT, 1) k_decode_fused(const DecodeFusedArgs a,
                     reinterpret_cast<int32_t *>(a.Y)[o] = acc;
                 } else {
                     const float sx = s_rowscale[a.per_vec ? m : 0];
-                    const float sw = a.per_vec ? __ldg(a.s_w + nn) : __ldg(a.s_w);
+                    const float sw = a.per_vec ? __ldg(a.s_w + nn) : sw0;
                     const float y = __fmul_rn(__fmul_rn(sx, sw), __int2float_rn(acc));  // Eq. 3
                     if (a.out_kind == 1) reinterpret_cast<float *>(a.Y)[o] = y;
                     else reinterpret_cast<__half *>(a.Y)[o] = __float2half_rn(y);
@@ -339,16 +368,16 @@ cudaError_t launch_decode_fused(const DecodeFusedArgs &a, cudaStream_t s) {
     static bool attr8 = false, attr16 = false;
     cudaError_t e;
     if (MT == 8 && !attr8) {
-        e = cudaFuncSetAttribute(k_decode_fused<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+        e = cudaFuncSetAttribute(k_decode_fused<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
         if (e != cudaSuccess) return e;
         attr8 = true;
     }
     if (MT == 16 && !attr16) {
-        e = cudaFuncSetAttribute(k_decode_fused<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+        e = cudaFuncSetAttribute(k_decode_fused<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
         if (e != cudaSuccess) return e;
         attr16 = true;
     }
-    if (L.total > 200 * 1024) return cudaErrorInvalidValue;
+    if (L.total > kMaxSmem) return cudaErrorInvalidValue;
     // tiles per group: the smallest power of two that gives every warp at least 4 segments of 64 bytes
     const int nseg = a.K / 64, tiles = (a.N + 7) / 8;
     int tpg = 1;
