@@ -95,7 +95,9 @@ __global__ void __launch_bounds__(kT, 1) k_decode_fused(const DecodeFusedArgs a,
     const int nseg = K >> 6;
     const int tiles = (a.N + 7) >> 3;
     const int ws = kWarps / tpg;             // warps per team
-    const int team = warp / ws, wi = warp - team * ws;
+    const int team = warp / ws;
+    // (when tpg does not divide the warp count, the warps left over get no segment: wi = nseg)
+    const int wi = team < tpg ? warp - team * ws : nseg;
     uint4 wpre[kPre];
     {
         const int n = (blockIdx.x * tpg + team) * 8 + r;
@@ -380,8 +382,20 @@ cudaError_t launch_decode_fused(const DecodeFusedArgs &a, cudaStream_t s) {
     if (L.total > kMaxSmem) return cudaErrorInvalidValue;
     // tiles per group: the smallest power of two that gives every warp at least 4 segments of 64 bytes
     const int nseg = a.K / 64, tiles = (a.N + 7) / 8;
+    // A warp holds at most kPre segments in registers.  Among the team counts that respect this, take the one that
+    // needs the fewest rounds of groups over the SMs (a second round costs a CTA a whole extra stream-and-reduce
+    // latency), then one that gives every warp at least 4 segments, then the smallest.
     int tpg = 1;
-    while (tpg < kWarps && nseg * tpg < 4 * kWarps) tpg *= 2;
+    {
+        long best = -1;
+        for (int T = 1; T <= kWarps; ++T) {
+            const int wsT = kWarps / T, spw = (nseg + wsT - 1) / wsT;
+            if (spw > kPre) continue;
+            const int g = (tiles + T - 1) / T, rounds = (g + num_sms() - 1) / num_sms();
+            const long key = ((long)rounds << 16) | ((spw >= 4 ? 0L : 1L) << 8) | T;
+            if (best < 0 || key < best) { best = key; tpg = T; }
+        }
+    }
     const int groups = (tiles + tpg - 1) / tpg;
     // at most one CTA per SM, so that the kernel of the next layer in the stream can become resident beside
     // this one (programmatic dependent launch) and fetch its weights while this one finishes
