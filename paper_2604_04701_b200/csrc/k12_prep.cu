@@ -72,17 +72,6 @@ __device__ __forceinline__ void load_chunk(const uint4 *src, int ch, const uint8
     }
 }
 
-// The exact form of Eq. 1 for one 8-channel chunk (mask: its outlier channels).  Kept out of line: it runs for
-// about one chunk in a thousand, and inlined at every use it costs the quantization loops their registers.
-__device__ __noinline__ uint2 codes_exact(uint4 v, uint32_t mask, float down, float s, float qf) {
-    float f[8];
-    unpack8(v, f);
-    uint32_t code[8];
-#pragma unroll
-    for (int i = 0; i < 8; ++i) code[i] = (uint32_t)quant_exact((mask >> i) & 1u ? f[i] * down : f[i], s, qf);
-    return pack8(code);
-}
-
 // kAllFit: the host has sized the slab for every row of the largest CTA share, so the loops over rows that
 // live only in global memory are compiled out (and with them their registers).
 // kPerToken: per-token scales (one warp per row in pass 2) instead of the per-tensor scale; one instantiation

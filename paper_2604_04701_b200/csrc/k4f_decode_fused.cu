@@ -279,11 +279,8 @@ __global__ void __launch_bounds__(kT, 1) k_decode_fused(const DecodeFusedArgs a,
                         if (a.per_vec) recip_bracket(__frcp_rn(s), lo, hi);
                         // the scale comes from these very values: no code can leave the range (bracket form)
                         uint32_t cb[8];
-                        if (quant8_bracket(f, lo, hi, cb)) {
-#pragma unroll
-                            for (int i = 0; i < 8; ++i) cb[i] = (uint32_t)quant_exact(f[i], s, qf);
-                        }
-                        code = pack8(cb);
+                        if (quant8_bracket(f, lo, hi, cb)) code = codes_exact(v[u], my_mask[it], down, s, qf);  // rare
+                        else code = pack8(cb);
                     }
                     *reinterpret_cast<uint2 *>(xq + m * L.pitch + cg * 8) = code;
                 }

@@ -104,4 +104,15 @@ __device__ __forceinline__ uint2 pack8(const uint32_t (&b)[8]) {
     return make_uint2(__byte_perm(p01, p23, 0x5410), __byte_perm(p45, p67, 0x5410));
 }
 
+// The exact form of Eq. 1 for one 8-channel chunk (mask: its outlier channels).  Kept out of line: it runs for
+// about one chunk in a thousand, and inlined at every use it costs the quantization loops their registers.
+static __device__ __noinline__ uint2 codes_exact(uint4 v, uint32_t mask, float down, float s, float qf) {
+    float f[8];
+    unpack8(v, f);
+    uint32_t code[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) code[i] = (uint32_t)quant_exact((mask >> i) & 1u ? f[i] * down : f[i], s, qf);
+    return pack8(code);
+}
+
 }  // namespace muxq
