@@ -25,7 +25,8 @@ namespace {
 
 constexpr int kT = 512;
 constexpr int kWarps = kT / 32;
-constexpr int kPre = 8;               // 64-byte W segments per warp fetched ahead of the prologue
+constexpr int kPre = 8;               // 64-byte W segments per warp fetched ahead of the prologue into registers
+constexpr int kExtra = 4;             // ... and further ones into shared memory (asynchronous copies)
 constexpr int kMaxIter = 2;           // channel groups (8 channels) per thread: K <= 8 * kT * kMaxIter
 constexpr int kStatusCapacity = 5;    // MUXQ_ERR_CAPACITY
 
@@ -44,6 +45,7 @@ struct Smem {
     int off_segflag;    // [K/64] segment holds an outlier channel
     int off_grpmask;    // [K/8] per-group flag bits
     int off_red;        // [2][kWarps][128] int32 partial tiles
+    int off_wx;         // [kWarps][kExtra][32] 16-byte pieces of W_q beyond the kPre segments a warp keeps in registers
     int off_xs;         // [MT][K] fp16 copy of X between the two passes (only when it fits), else -1
     int total;
 };
@@ -56,7 +58,8 @@ __host__ __device__ inline Smem smem_layout(int MT, int K) {
     s.off_segflag = s.off_mask + K;
     s.off_grpmask = s.off_segflag + (((K >> 6) + 15) & ~15);
     s.off_red = (s.off_grpmask + (K >> 3) + 15) & ~15;
-    s.total = s.off_red + 2 * kWarps * 128 * 4;
+    s.off_wx = s.off_red + 2 * kWarps * 128 * 4;
+    s.total = s.off_wx + kWarps * kExtra * 32 * 16;
     s.off_xs = -1;
     if (MT == 8 && s.total + MT * K * 2 <= kMaxSmem) {
         s.off_xs = s.total;
@@ -82,6 +85,7 @@ __global__ void __launch_bounds__(kT, 1) k_decode_fused(const DecodeFusedArgs a,
     uint8_t *s_grpmask = smem + L.off_grpmask;
     int *s_red = reinterpret_cast<int *>(smem + L.off_red);
     uint8_t *xs = L.off_xs >= 0 ? smem + L.off_xs : nullptr;
+    uint4 *s_wx = reinterpret_cast<uint4 *>(smem + L.off_wx) + warp * (kExtra * 32) + lane;  // this lane's pieces
     const float down = __int_as_float((127 - a.exp_factor) << 23);  // 2^-e
     const float qf = (float)a.qmax;
     const bool first = blockIdx.x == 0;
@@ -107,11 +111,21 @@ __global__ void __launch_bounds__(kT, 1) k_decode_fused(const DecodeFusedArgs a,
             const int seg = wi + u * ws;
             wpre[u] = seg < nseg ? __ldg(reinterpret_cast<const uint4 *>(wrow + seg * 64)) : make_uint4(0u, 0u, 0u, 0u);
         }
+        // segments beyond kPre (the host allows them only when all groups fit one round): to shared memory
+#pragma unroll
+        for (int e = 0; e < kExtra; ++e) {
+            const int seg = wi + (kPre + e) * ws;
+            if (seg < nseg) {
+                const uint32_t d = (uint32_t)__cvta_generic_to_shared(s_wx + e * 32);
+                asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d), "l"(wrow + seg * 64) : "memory");
+            }
+        }
     }
     const float sw0 = __ldg(a.s_w);  // a constant of the layer like W_q (the per-tensor scale, or the first column's)
     // Everything below reads X or writes results: under programmatic dependent launch it must wait for the
     // kernel before this one in the stream; the weights above are constants and were fetched ahead of that.
     asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("cp.async.wait_all;" ::: "memory");  // a lane reads back only the pieces it copied itself
 
     if (first && t == 0 && a.dev_status) *a.dev_status = 0;
     if (t < 16) s_rowmax[t] = 0u;
@@ -298,24 +312,39 @@ __global__ void __launch_bounds__(kT, 1) k_decode_fused(const DecodeFusedArgs a,
     for (int group = blockIdx.x; group < groups; group += gridDim.x) {
         const int8_t *xlo = xq + r * L.pitch + q * 16;
         // two Body accumulators (the two halves of a 64-byte segment): consecutive mma.sync on one accumulator
-        // wait for each other, and that chain is what this loop's time consists of
+        // wait for each other
         int accb[4] = {0, 0, 0, 0}, accb2[4] = {0, 0, 0, 0}, acca[4] = {0, 0, 0, 0};
-        // this warp's segments (at most kPre by the choice of tpg) are already in registers
+        auto consume = [&](int seg, const uint4 &w) {
+            const uint4 alo = *reinterpret_cast<const uint4 *>(xlo + seg * 64);
+            uint4 ahi = make_uint4(0u, 0u, 0u, 0u);
+            if (MT == 16) ahi = *reinterpret_cast<const uint4 *>(xlo + 8 * L.pitch + seg * 64);
+            mma_s8(accb, alo.x, ahi.x, alo.y, ahi.y, w.x, w.y);
+            mma_s8(accb2, alo.z, ahi.z, alo.w, ahi.w, w.z, w.w);
+            if (s_segflag[seg]) {  // warp-uniform: Aux term on the outlier channels of this segment
+                const uint4 mk = *reinterpret_cast<const uint4 *>(s_mask + seg * 64 + q * 16);
+                mma_s8(acca, alo.x & mk.x, ahi.x & mk.x, alo.y & mk.y, ahi.y & mk.y, w.x, w.y);
+                mma_s8(acca, alo.z & mk.z, ahi.z & mk.z, alo.w & mk.w, ahi.w & mk.w, w.z, w.w);
+            }
+        };
+        // this warp's first kPre segments are already in registers
 #pragma unroll
         for (int u = 0; u < kPre; ++u) {
             const int seg = wi + u * ws;
-            if (seg < nseg) {
-                const uint4 alo = *reinterpret_cast<const uint4 *>(xlo + seg * 64);
-                uint4 ahi = make_uint4(0u, 0u, 0u, 0u);
-                if (MT == 16) ahi = *reinterpret_cast<const uint4 *>(xlo + 8 * L.pitch + seg * 64);
-                mma_s8(accb, alo.x, ahi.x, alo.y, ahi.y, wpre[u].x, wpre[u].y);
-                mma_s8(accb2, alo.z, ahi.z, alo.w, ahi.w, wpre[u].z, wpre[u].w);
-                if (s_segflag[seg]) {  // warp-uniform: Aux term on the outlier channels of this segment
-                    const uint4 mk = *reinterpret_cast<const uint4 *>(s_mask + seg * 64 + q * 16);
-                    mma_s8(acca, alo.x & mk.x, ahi.x & mk.x, alo.y & mk.y, ahi.y & mk.y, wpre[u].x, wpre[u].y);
-                    mma_s8(acca, alo.z & mk.z, ahi.z & mk.z, alo.w & mk.w, ahi.w & mk.w, wpre[u].z, wpre[u].w);
-                }
+            if (seg < nseg) consume(seg, wpre[u]);
+        }
+        // the others: from shared memory for the CTA's first group, else straight from global memory
+#pragma unroll 1
+        for (int e = 0; e < kExtra; ++e) {
+            const int seg = wi + (kPre + e) * ws;
+            if (seg >= nseg) break;
+            uint4 w;
+            if (group == (int)blockIdx.x) {
+                w = s_wx[e * 32];
+            } else {
+                const int n = (group * tpg + team) * 8 + r;
+                w = __ldg(reinterpret_cast<const uint4 *>(a.w_q + (size_t)min(n, a.N - 1) * a.ldw + q * 16 + seg * 64));
             }
+            consume(seg, w);
         }
         // fetch the next group's segments now; they arrive while this group is reduced and stored
         if (group + (int)gridDim.x < groups) {
@@ -379,17 +408,17 @@ cudaError_t launch_decode_fused(const DecodeFusedArgs &a, cudaStream_t s) {
     if (L.total > kMaxSmem) return cudaErrorInvalidValue;
     // tiles per group: the smallest power of two that gives every warp at least 4 segments of 64 bytes
     const int nseg = a.K / 64, tiles = (a.N + 7) / 8;
-    // A warp holds at most kPre segments in registers.  Among the team counts that respect this, take the one that
-    // needs the fewest rounds of groups over the SMs (a second round costs a CTA a whole extra stream-and-reduce
-    // latency), then one that gives every warp at least 4 segments, then the smallest.
+    // A warp holds kPre segments in registers and up to kExtra more in shared memory; the latter only pays when it
+    // saves a round of groups over the SMs (a second round costs a CTA a whole extra stream-and-reduce latency).
+    // Order of preference: fewest rounds; all segments in registers; at least 4 segments per warp; fewest tiles.
     int tpg = 1;
     {
         long best = -1;
         for (int T = 1; T <= kWarps; ++T) {
             const int wsT = kWarps / T, spw = (nseg + wsT - 1) / wsT;
-            if (spw > kPre) continue;
             const int g = (tiles + T - 1) / T, rounds = (g + num_sms() - 1) / num_sms();
-            const long key = ((long)rounds << 16) | ((spw >= 4 ? 0L : 1L) << 8) | T;
+            if (spw > kPre + kExtra || (spw > kPre && rounds > 1)) continue;
+            const long key = ((long)rounds << 24) | ((spw > kPre ? 1L : 0L) << 16) | ((spw >= 4 ? 0L : 1L) << 8) | T;
             if (best < 0 || key < best) { best = key; tpg = T; }
         }
     }
