@@ -133,11 +133,14 @@ __global__ void __launch_bounds__(kT, 1) k_decode_fused(const DecodeFusedArgs a,
     __syncthreads();
 
     // ---------------------------------------------------------------- pass A: channel maxima, flags, Body maxima
-    uint32_t my_mask[kMaxIter];
+    // The loops over a thread's channel groups are deliberately NOT unrolled: each copy of their bodies would be
+    // code this SM has not fetched yet, and instruction fetch is what these short phases wait for.  The groups'
+    // outlier flags share one register, a byte per group.
+    static_assert(kMaxIter <= 4, "one byte of my_masks per channel group of the thread");
+    uint32_t my_masks = 0;
     float bmax = 0.0f;
-#pragma unroll
+#pragma unroll 1
     for (int it = 0; it < kMaxIter; ++it) {
-        my_mask[it] = 0;
         const int cg = t + it * kT;
         if (cg < G) {
             __half2 cm[4];
@@ -171,7 +174,7 @@ __global__ void __launch_bounds__(kT, 1) k_decode_fused(const DecodeFusedArgs a,
                 mask |= flagged ? (1u << i) : 0u;
                 bmax = fmaxf(bmax, flagged ? c8[i] * down : c8[i]);
             }
-            my_mask[it] = mask;
+            my_masks |= mask << (8 * it);
             s_grpmask[cg] = (uint8_t)mask;
             if (mask) s_segflag[cg >> 3] = 1;
             uint2 mb;
@@ -188,7 +191,7 @@ __global__ void __launch_bounds__(kT, 1) k_decode_fused(const DecodeFusedArgs a,
     }
     if (a.per_vec) {
         // per-token scales: row maxima of Body (after the 2^-e), a second cheap sweep with the flags known
-#pragma unroll
+#pragma unroll 1
         for (int it = 0; it < kMaxIter; ++it) {
             const int cg = t + it * kT;
             if (cg < G) {
@@ -199,7 +202,7 @@ __global__ void __launch_bounds__(kT, 1) k_decode_fused(const DecodeFusedArgs a,
                     unpack8(v, f);
                     float rm = 0.0f;
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) rm = fmaxf(rm, fabsf((my_mask[it] >> i) & 1u ? f[i] * down : f[i]));
+                    for (int i = 0; i < 8; ++i) rm = fmaxf(rm, fabsf((my_masks >> (8 * it + i)) & 1u ? f[i] * down : f[i]));
                     if (rm > 0.0f) atomicMax(&s_rowmax[m], __float_as_uint(rm));
                 }
             }
@@ -262,13 +265,13 @@ __global__ void __launch_bounds__(kT, 1) k_decode_fused(const DecodeFusedArgs a,
     __syncthreads();
 
     // ---------------------------------------------------------------- pass B: codes of X into shared memory
-#pragma unroll
+#pragma unroll 1
     for (int it = 0; it < kMaxIter; ++it) {
         const int cg = t + it * kT;
         if (cg < G) {
             float mul[8];
 #pragma unroll
-            for (int i = 0; i < 8; ++i) mul[i] = (my_mask[it] >> i) & 1u ? down : 1.0f;
+            for (int i = 0; i < 8; ++i) mul[i] = (my_masks >> (8 * it + i)) & 1u ? down : 1.0f;
             float lo = 0.0f, hi = 0.0f;
             if (!a.per_vec) recip_bracket(__frcp_rn(s_rowscale[0]), lo, hi);
             for (int m0 = 0; m0 < MT; m0 += 4) {  // four independent row loads in flight
@@ -293,7 +296,7 @@ __global__ void __launch_bounds__(kT, 1) k_decode_fused(const DecodeFusedArgs a,
                         if (a.per_vec) recip_bracket(__frcp_rn(s), lo, hi);
                         // the scale comes from these very values: no code can leave the range (bracket form)
                         uint32_t cb[8];
-                        if (quant8_bracket(f, lo, hi, cb)) code = codes_exact(v[u], my_mask[it], down, s, qf);  // rare
+                        if (quant8_bracket(f, lo, hi, cb)) code = codes_exact(v[u], (my_masks >> (8 * it)) & 0xffu, down, s, qf);  // rare
                         else code = pack8(cb);
                     }
                     *reinterpret_cast<uint2 *>(xq + m * L.pitch + cg * 8) = code;
