@@ -68,7 +68,11 @@ __host__ __device__ inline Smem smem_layout(int MT, int K) {
     return s;
 }
 
-template <int MT>
+// kDotM > 0 (MT == 8, M <= kDotM <= 4): the products are 4-way byte dot products (dp4a) per token row instead of
+// mma.sync tiles.  The legacy mma.sync path issues an INT8 m16n8k32 only about every 32 cycles per SM sub-partition
+// on this part; for a single row the dot products cost less (measured: 5.3 against 5.7 us per layer at M = 1, but
+// 6.8 against 6.2 us at M = 4, so only kDotM = 1 is instantiated).
+template <int MT, int kDotM>
 __global__ void __launch_bounds__(kT, 1) k_decode_fused(const DecodeFusedArgs a, int tpg) {
     extern __shared__ __align__(16) uint8_t smem[];
     __shared__ uint32_t s_rowmax[16];  // bit patterns of non-negative floats (per-token row maxima of Body)
@@ -124,13 +128,13 @@ __global__ void __launch_bounds__(kT, 1) k_decode_fused(const DecodeFusedArgs a,
     const float sw0 = __ldg(a.s_w);  // a constant of the layer like W_q (the per-tensor scale, or the first column's)
     // Everything below reads X or writes results: under programmatic dependent launch it must wait for the
     // kernel before this one in the stream; the weights above are constants and were fetched ahead of that.
+    if (t < 16) s_rowmax[t] = 0u;
+    for (int i = t; i < (K >> 6); i += kT) s_segflag[i] = 0;
+    __syncthreads();  // (shared-memory set-up needs nothing from the predecessor either)
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("cp.async.wait_all;" ::: "memory");  // a lane reads back only the pieces it copied itself
 
     if (first && t == 0 && a.dev_status) *a.dev_status = 0;
-    if (t < 16) s_rowmax[t] = 0u;
-    for (int i = t; i < (K >> 6); i += kT) s_segflag[i] = 0;
-    __syncthreads();
 
     // ---------------------------------------------------------------- pass A: channel maxima, flags, Body maxima
     // The loops over a thread's channel groups are deliberately NOT unrolled: each copy of their bodies would be
@@ -318,6 +322,28 @@ __global__ void __launch_bounds__(kT, 1) k_decode_fused(const DecodeFusedArgs a,
         // wait for each other
         int accb[4] = {0, 0, 0, 0}, accb2[4] = {0, 0, 0, 0}, acca[4] = {0, 0, 0, 0};
         auto consume = [&](int seg, const uint4 &w) {
+            if constexpr (kDotM > 0) {
+                // lane (r, q) holds 16 bytes of W_q row r; the same 16 channels of token row m come from shared memory
+                // (the 8 lanes with equal q read one address).  accb[m] / acca[m]: Body and Aux sums of row m.
+                const bool fl = s_segflag[seg] != 0;  // warp-uniform
+                uint4 mk = make_uint4(0u, 0u, 0u, 0u);
+                if (fl) mk = *reinterpret_cast<const uint4 *>(s_mask + seg * 64 + q * 16);
+#pragma unroll
+                for (int m = 0; m < kDotM; ++m) {
+                    const uint4 x = *reinterpret_cast<const uint4 *>(xq + m * L.pitch + q * 16 + seg * 64);
+                    accb[m] = __dp4a((int)w.x, (int)x.x, accb[m]);
+                    accb[m] = __dp4a((int)w.y, (int)x.y, accb[m]);
+                    accb[m] = __dp4a((int)w.z, (int)x.z, accb[m]);
+                    accb[m] = __dp4a((int)w.w, (int)x.w, accb[m]);
+                    if (fl) {
+                        acca[m] = __dp4a((int)w.x, (int)(x.x & mk.x), acca[m]);
+                        acca[m] = __dp4a((int)w.y, (int)(x.y & mk.y), acca[m]);
+                        acca[m] = __dp4a((int)w.z, (int)(x.z & mk.z), acca[m]);
+                        acca[m] = __dp4a((int)w.w, (int)(x.w & mk.w), acca[m]);
+                    }
+                }
+                return;
+            }
             const uint4 alo = *reinterpret_cast<const uint4 *>(xlo + seg * 64);
             uint4 ahi = make_uint4(0u, 0u, 0u, 0u);
             if (MT == 16) ahi = *reinterpret_cast<const uint4 *>(xlo + 8 * L.pitch + seg * 64);
@@ -362,10 +388,21 @@ __global__ void __launch_bounds__(kT, 1) k_decode_fused(const DecodeFusedArgs a,
         // acc = acc_b + c * acc_a (Eq. 7), partial over this warp's K segments; element (row, col) of the
         // 16 x 8 tile: this lane holds rows r and r+8, columns 2q and 2q+1
         int *red = s_red + warp * 128;
-        red[r * 8 + 2 * q] = accb[0] + accb2[0] + a.c * acca[0];
-        red[r * 8 + 2 * q + 1] = accb[1] + accb2[1] + a.c * acca[1];
-        red[(r + 8) * 8 + 2 * q] = accb[2] + accb2[2] + a.c * acca[2];
-        red[(r + 8) * 8 + 2 * q + 1] = accb[3] + accb2[3] + a.c * acca[3];
+        if constexpr (kDotM > 0) {
+            // the four lanes of a W_q row add up; rows >= kDotM of the 16 x 8 tile are never stored (m < M below)
+#pragma unroll
+            for (int m = 0; m < kDotM; ++m) {
+                int v = accb[m] + a.c * acca[m];
+                v += __shfl_xor_sync(0xffffffffu, v, 1);
+                v += __shfl_xor_sync(0xffffffffu, v, 2);
+                if (q == 0) red[m * 8 + r] = v;
+            }
+        } else {
+            red[r * 8 + 2 * q] = accb[0] + accb2[0] + a.c * acca[0];
+            red[r * 8 + 2 * q + 1] = accb[1] + accb2[1] + a.c * acca[1];
+            red[(r + 8) * 8 + 2 * q] = accb[2] + accb2[2] + a.c * acca[2];
+            red[(r + 8) * 8 + 2 * q + 1] = accb[3] + accb2[3] + a.c * acca[3];
+        }
         __syncthreads();
         for (int e = t; e < 128 * tpg; e += kT) {
             const int j = e >> 7, el = e & 127;  // tile of the group, element of its 16 x 8 tile
@@ -396,17 +433,16 @@ bool decode_fused_supported(int M, int K) { return M >= 1 && M <= 16 && K % 64 =
 cudaError_t launch_decode_fused(const DecodeFusedArgs &a, cudaStream_t s) {
     const int MT = a.M <= 8 ? 8 : 16;
     const Smem L = smem_layout(MT, a.K);
-    static bool attr8 = false, attr16 = false;
-    cudaError_t e;
-    if (MT == 8 && !attr8) {
-        e = cudaFuncSetAttribute(k_decode_fused<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
-        if (e != cudaSuccess) return e;
-        attr8 = true;
-    }
-    if (MT == 16 && !attr16) {
-        e = cudaFuncSetAttribute(k_decode_fused<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
-        if (e != cudaSuccess) return e;
-        attr16 = true;
+    static bool attr_set = false;
+    if (!attr_set) {
+        const void *fns[3] = {reinterpret_cast<const void *>(k_decode_fused<8, 1>),
+                              reinterpret_cast<const void *>(k_decode_fused<8, 0>),
+                              reinterpret_cast<const void *>(k_decode_fused<16, 0>)};
+        for (const void *f : fns) {
+            cudaError_t e = cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
+            if (e != cudaSuccess) return e;
+        }
+        attr_set = true;
     }
     if (L.total > kMaxSmem) return cudaErrorInvalidValue;
     // tiles per group: the smallest power of two that gives every warp at least 4 segments of 64 bytes
@@ -439,8 +475,9 @@ cudaError_t launch_decode_fused(const DecodeFusedArgs &a, cudaStream_t s) {
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr; cfg.numAttrs = 1;
-    if (MT == 8) return cudaLaunchKernelEx(&cfg, k_decode_fused<8>, a, tpg);
-    return cudaLaunchKernelEx(&cfg, k_decode_fused<16>, a, tpg);
+    if (a.M == 1) return cudaLaunchKernelEx(&cfg, k_decode_fused<8, 1>, a, tpg);
+    if (MT == 8) return cudaLaunchKernelEx(&cfg, k_decode_fused<8, 0>, a, tpg);
+    return cudaLaunchKernelEx(&cfg, k_decode_fused<16, 0>, a, tpg);
 }
 
 }  // namespace muxq
