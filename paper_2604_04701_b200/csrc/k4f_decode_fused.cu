@@ -39,6 +39,14 @@ __device__ __forceinline__ void mma_s8(int (&d)[4], uint32_t a0, uint32_t a1, ui
         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
+// 16-byte read-only load as a volatile statement: a batch of them is issued back to back before the first use,
+// whatever the register allocator would rather do (under register pressure it serialises plain loads).
+__device__ __forceinline__ uint4 ld_nc_v4(const void *p) {
+    uint4 v;
+    asm volatile("ld.global.nc.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
+
 struct Smem {
     int pitch;          // bytes per row of X codes; pitch % 128 == 64 keeps the 8-row x 64-byte reads conflict free
     int off_mask;       // [K] 0xFF at outlier channels
@@ -61,7 +69,7 @@ __host__ __device__ inline Smem smem_layout(int MT, int K) {
     s.off_wx = s.off_red + 2 * kWarps * 128 * 4;
     s.total = s.off_wx + kWarps * kExtra * 32 * 16;
     s.off_xs = -1;
-    if (MT == 8 && s.total + MT * K * 2 <= kMaxSmem) {
+    if (s.total + MT * K * 2 <= kMaxSmem) {
         s.off_xs = s.total;
         s.total += MT * K * 2;
     }
@@ -153,7 +161,7 @@ __global__ void __launch_bounds__(kT, 1) k_decode_fused(const DecodeFusedArgs a,
                 uint4 v[4];
 #pragma unroll
                 for (int u = 0; u < 4; ++u)
-                    v[u] = m0 + u < M ? __ldg(reinterpret_cast<const uint4 *>(a.X + (size_t)(m0 + u) * a.ldx) + cg)
+                    v[u] = m0 + u < M ? ld_nc_v4(reinterpret_cast<const uint4 *>(a.X + (size_t)(m0 + u) * a.ldx) + cg)
                                       : make_uint4(0u, 0u, 0u, 0u);
                 if (xs) {
 #pragma unroll
@@ -269,42 +277,43 @@ __global__ void __launch_bounds__(kT, 1) k_decode_fused(const DecodeFusedArgs a,
     __syncthreads();
 
     // ---------------------------------------------------------------- pass B: codes of X into shared memory
+    // Work items are (channel group, batch of four rows), spread over all threads: with one thread per channel group
+    // the rows would be walked one after the other by a fraction of the CTA.  The flags come from shared memory.
+    {
+        float lo = 0.0f, hi = 0.0f;
+        if (!a.per_vec) recip_bracket(__frcp_rn(s_rowscale[0]), lo, hi);
 #pragma unroll 1
-    for (int it = 0; it < kMaxIter; ++it) {
-        const int cg = t + it * kT;
-        if (cg < G) {
+        for (int item = t; item < G * (MT / 4); item += kT) {
+            const int batch = item / G, cg = item - batch * G, m0 = 4 * batch;
+            const uint32_t gmask = s_grpmask[cg];
             float mul[8];
 #pragma unroll
-            for (int i = 0; i < 8; ++i) mul[i] = (my_masks >> (8 * it + i)) & 1u ? down : 1.0f;
-            float lo = 0.0f, hi = 0.0f;
-            if (!a.per_vec) recip_bracket(__frcp_rn(s_rowscale[0]), lo, hi);
-            for (int m0 = 0; m0 < MT; m0 += 4) {  // four independent row loads in flight
-                uint4 v[4];
+            for (int i = 0; i < 8; ++i) mul[i] = (gmask >> i) & 1u ? down : 1.0f;
+            uint4 v[4];  // four independent row loads in flight
 #pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    v[u] = make_uint4(0u, 0u, 0u, 0u);
-                    if (m0 + u < M)
-                        v[u] = xs ? *reinterpret_cast<const uint4 *>(xs + (size_t)(m0 + u) * K * 2 + cg * 16)
-                                  : __ldg(reinterpret_cast<const uint4 *>(a.X + (size_t)(m0 + u) * a.ldx) + cg);
+            for (int u = 0; u < 4; ++u) {
+                v[u] = make_uint4(0u, 0u, 0u, 0u);
+                if (m0 + u < M)
+                    v[u] = xs ? *reinterpret_cast<const uint4 *>(xs + (size_t)(m0 + u) * K * 2 + cg * 16)
+                              : ld_nc_v4(reinterpret_cast<const uint4 *>(a.X + (size_t)(m0 + u) * a.ldx) + cg);
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int m = m0 + u;
+                uint2 code = make_uint2(0u, 0u);
+                if (m < M) {
+                    float f[8];
+                    unpack8(v[u], f);
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) f[i] *= mul[i];  // exact
+                    const float s = s_rowscale[a.per_vec ? m : 0];
+                    if (a.per_vec) recip_bracket(__frcp_rn(s), lo, hi);
+                    // the scale comes from these very values: no code can leave the range (bracket form)
+                    uint32_t cb[8];
+                    if (quant8_bracket(f, lo, hi, cb)) code = codes_exact(v[u], gmask, down, s, qf);  // rare
+                    else code = pack8(cb);
                 }
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const int m = m0 + u;
-                    uint2 code = make_uint2(0u, 0u);
-                    if (m < M) {
-                        float f[8];
-                        unpack8(v[u], f);
-#pragma unroll
-                        for (int i = 0; i < 8; ++i) f[i] *= mul[i];  // exact
-                        const float s = s_rowscale[a.per_vec ? m : 0];
-                        if (a.per_vec) recip_bracket(__frcp_rn(s), lo, hi);
-                        // the scale comes from these very values: no code can leave the range (bracket form)
-                        uint32_t cb[8];
-                        if (quant8_bracket(f, lo, hi, cb)) code = codes_exact(v[u], (my_masks >> (8 * it)) & 0xffu, down, s, qf);  // rare
-                        else code = pack8(cb);
-                    }
-                    *reinterpret_cast<uint2 *>(xq + m * L.pitch + cg * 8) = code;
-                }
+                *reinterpret_cast<uint2 *>(xq + m * L.pitch + cg * 8) = code;
             }
         }
     }
