@@ -61,7 +61,7 @@ typedef struct muxq_params {
     int act_bits;     /* 2..8 (Eq. 1 uses 8) */
     int w_bits;       /* 2..8 (Eq. 2 uses 8) */
     int gran;         /* muxq_gran */
-    int aux_scale;    /* muxq_aux_scale; only MUXQ_AUX_SHARED runs on the GPU path */
+    int aux_scale;    /* muxq_aux_scale; MUXQ_AUX_OWN is taken by muxq_linear / _events / _host only */
     int max_outliers; /* capacity of O, 1..64 */
 } muxq_params;
 
@@ -168,6 +168,12 @@ int muxq_gemm(const int8_t *Body_q, int ld_a, const int8_t *Aux_q, int ld_aux, c
  * then unspecified but in bounds) or MUXQ_ERR_TIMEOUT.
  * Intermediates stay in the workspace afterwards; muxq_workspace_view locates them.  For M <= 16
  * only col_absmax, outlier_idx, n_outliers and s_x are left there (the codes never leave the SMs).
+ * params.aux_scale == MUXQ_AUX_OWN (the other reading of how Eq. 1 applies to Aux: its own abs-max
+ * scale s_A, per tensor or per token): Aux_q [M, r] is stored once per outlier channel and padded with
+ * zeros, Y = (s_X s_W) Body_q.W_q + (2^exp - 1) (s_A s_W) Aux_q.W_q[O,:] is formed from two separately
+ * dequantized fp32 products (two GEMM launches and one streaming sum, for every M; workspace grows by
+ * 8 M N bytes; out_kind MUXQ_OUT_ACC_I32 and K > 8192 are MUXQ_ERR_UNSUPPORTED).  Provided for
+ * completeness of the method, not tuned.
  */
 int muxq_linear(const void *X_f16, int M, int K, int ldx, const int8_t *W_q, int ldw,
                 const float *s_w, int N, const muxq_params *p, void *Y, int ldy, int out_kind,
@@ -195,6 +201,7 @@ typedef struct muxq_ws_view {
     size_t body_q;      /* int8 [M, ld_body_q] */
     size_t aux_q;       /* int8 [M, aux_cols]; written up to column round_up(c * r, 32): codes, then zeros */
     size_t w_aux;       /* int8 [N, aux_cols]; likewise (the products read no column beyond that) */
+    size_t s_a;         /* float [1] or [M]: the Aux scale(s), MUXQ_AUX_OWN only */
     int ld_body_q;
     int aux_cols;
 } muxq_ws_view;

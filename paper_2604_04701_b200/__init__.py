@@ -10,5 +10,5 @@ from .binding import (  # noqa: F401
     muxq_workspace_bytes, muxq_small_workspace_bytes, muxq_host_workspace_bytes, muxq_workspace_view,
     MUXQ_OK, MUXQ_ERR_INVALID_ARG, MUXQ_ERR_UNSUPPORTED, MUXQ_ERR_WORKSPACE, MUXQ_ERR_CUDA,
     MUXQ_ERR_CAPACITY, MUXQ_ERR_TIMEOUT, MUXQ_ERR_STATIC_LIMIT, MUXQ_PER_TENSOR, MUXQ_PER_VECTOR, MUXQ_OUT_F16,
-    MUXQ_OUT_F32, MUXQ_OUT_ACC_I32, MuxqError,
+    MUXQ_OUT_F32, MUXQ_OUT_ACC_I32, MUXQ_AUX_SHARED, MUXQ_AUX_OWN, MuxqError,
 )

@@ -42,8 +42,8 @@ class _CParams(ctypes.Structure):
 class _CWsView(ctypes.Structure):
     _fields_ = [("col_absmax", ctypes.c_size_t), ("outlier_idx", ctypes.c_size_t),
                 ("n_outliers", ctypes.c_size_t), ("s_x", ctypes.c_size_t), ("body_q", ctypes.c_size_t),
-                ("aux_q", ctypes.c_size_t), ("w_aux", ctypes.c_size_t), ("ld_body_q", ctypes.c_int),
-                ("aux_cols", ctypes.c_int)]
+                ("aux_q", ctypes.c_size_t), ("w_aux", ctypes.c_size_t), ("s_a", ctypes.c_size_t),
+                ("ld_body_q", ctypes.c_int), ("aux_cols", ctypes.c_int)]
 
 
 @dataclass

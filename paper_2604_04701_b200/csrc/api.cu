@@ -39,7 +39,7 @@ SmallWs small_ws(int cols) {
 // muxq_linear workspace: the small block, then per-token scales, Body_q, Aux_q, W_aux.
 struct LinearWs {
     SmallWs s;
-    size_t colmax_rep, sx_rows, body_q, aux_q, w_aux, total;
+    size_t colmax_rep, sx_rows, sa_rows, body_q, aux_q, w_aux, t1, t2, total;
     int ld_q, aux_cols;
 };
 LinearWs linear_ws(int M, int K, int N, const muxq_params *p) {
@@ -54,10 +54,18 @@ LinearWs linear_ws(int M, int K, int N, const muxq_params *p) {
     const size_t shift = align_up(w.colmax_rep + kPrepRepRegionBytes, 256) - w.s.colmax;
     w.s.colmax += shift; w.s.colmul += shift; w.s.grpflag += shift; w.s.oidx += shift; w.s.total += shift;
     w.sx_rows = w.s.total;
-    w.body_q = align_up(w.sx_rows + (size_t)M * 4, 1024);
+    w.sa_rows = align_up(w.sx_rows + (size_t)M * 4, 256);
+    w.body_q = align_up(w.sa_rows + (size_t)M * 4, 1024);
     w.aux_q = align_up(w.body_q + (size_t)M * w.ld_q, 1024);
     w.w_aux = align_up(w.aux_q + (size_t)M * w.aux_cols, 1024);
     w.total = align_up(w.w_aux + (size_t)N * w.aux_cols, 1024);
+    // own-scale reading: the two dequantized products, fp32 [M, N] each
+    w.t1 = w.t2 = 0;
+    if (p->aux_scale == MUXQ_AUX_OWN) {
+        w.t1 = w.total;
+        w.t2 = align_up(w.t1 + (size_t)M * N * 4, 1024);
+        w.total = align_up(w.t2 + (size_t)M * N * 4, 1024);
+    }
     return w;
 }
 
@@ -113,6 +121,7 @@ int muxq_workspace_view(int M, int K, int N, const muxq_params *p, muxq_ws_view 
     v->outlier_idx = w.s.oidx;
     v->n_outliers = offsetof(Ctrl, n_outliers);
     v->s_x = p->gran == MUXQ_PER_VECTOR ? w.sx_rows : offsetof(Ctrl, s_x);
+    v->s_a = p->gran == MUXQ_PER_VECTOR ? w.sa_rows : offsetof(Ctrl, s_a);
     v->body_q = w.body_q;
     v->aux_q = w.aux_q;
     v->w_aux = w.w_aux;
@@ -275,15 +284,18 @@ static int linear_impl(const void *X, int M, int K, int ldx, const int8_t *W_q, 
     if (K % 16 || ldx % 8 || ldw % 16 || N % 8 || ldy % yal || !aligned16(X) || !aligned16(W_q) ||
         !aligned16(Y) || !aligned16(workspace) || (p->gran == MUXQ_PER_VECTOR && !aligned16(s_w)))
         return MUXQ_ERR_UNSUPPORTED;
-    if (p->aux_scale != MUXQ_AUX_SHARED) return MUXQ_ERR_UNSUPPORTED;
+    const bool aux_own = p->aux_scale == MUXQ_AUX_OWN;
+    if (aux_own && out_kind == MUXQ_OUT_ACC_I32) return MUXQ_ERR_UNSUPPORTED;  // there is no common accumulator
     const LinearWs w = linear_ws(M, K, N, p);
     if (workspace_bytes < w.total) return MUXQ_ERR_WORKSPACE;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     uint8_t *ws = static_cast<uint8_t *>(workspace);
 
     const bool per_vec = p->gran == MUXQ_PER_VECTOR;
-    const bool decode = M <= 16;
+    // (the own-scale reading runs as separate products through the GEMM kernels for every M)
+    const bool decode = M <= 16 && !aux_own;
     const bool fused = prep_supported(M, K);
+    if (aux_own && !fused) return MUXQ_ERR_UNSUPPORTED;
     Ctrl *ctrl = reinterpret_cast<Ctrl *>(ws);
     // inside a stream capture the records become event-record nodes that every replay re-records
     cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
@@ -337,6 +349,8 @@ static int linear_impl(const void *X, int M, int K, int ldx, const int8_t *W_q, 
         f.M = M; f.K = K; f.ldx = ldx;
         f.tau = p->threshold; f.exp_factor = p->exp_factor; f.qmax = qmax_of(p->act_bits);
         f.cap = p->max_outliers; f.per_token = per_vec;
+        f.aux_own = aux_own ? 1 : 0;
+        f.s_a_rows = reinterpret_cast<float *>(ws + w.sa_rows);
         f.colmax_rep = reinterpret_cast<uint32_t *>(ws + w.colmax_rep);
         f.colmax_bits = reinterpret_cast<uint32_t *>(ws + w.s.colmax);
         f.ctrl = ctrl;
@@ -393,6 +407,31 @@ static int linear_impl(const void *X, int M, int K, int ldx, const int8_t *W_q, 
         k.s_w = s_w; k.s_w_per_col = per_vec;
         k.Y = Y; k.ldy = ldy; k.out_kind = out_kind;
         e = launch_decode(k, s);
+        mark(3);
+        return cuda_rc(e);
+    }
+    if (aux_own) {
+        // Y = (s_X s_W) Body_q.W_q + c (s_A s_W) Aux_q.W_aux: two dequantized products, then the sum
+        float *t1 = reinterpret_cast<float *>(ws + w.t1), *t2 = reinterpret_cast<float *>(ws + w.t2);
+        GemmArgs g{};
+        g.body_q = body_q; g.ld_a = w.ld_q;
+        g.w_q = W_q; g.ldw = ldw;
+        g.M = M; g.K = K; g.N = N; g.c = c; g.cap = p->max_outliers; g.aux_cols = w.aux_cols;
+        g.s_x = s_x; g.s_x_per_row = per_vec;
+        g.s_w = s_w; g.s_w_per_col = per_vec;
+        g.Y = t1; g.ldy = N; g.out_kind = MUXQ_OUT_F32;
+        g.dev_status = dev_status;
+        e = launch_gemm(g, s);
+        if (e != cudaSuccess) return MUXQ_ERR_CUDA;
+        g.body_q = aux_q; g.ld_a = w.aux_cols;  // zero beyond the r used columns
+        g.w_q = w_aux; g.ldw = w.aux_cols;
+        g.K = w.aux_cols;
+        g.s_x = per_vec ? reinterpret_cast<const float *>(ws + w.sa_rows) : &ctrl->s_a;
+        g.Y = t2;
+        e = launch_gemm(g, s);
+        if (e != cudaSuccess) return MUXQ_ERR_CUDA;
+        CombineArgs cb{t1, t2, M, N, c, Y, ldy, out_kind == MUXQ_OUT_F16 ? 1 : 0};
+        e = launch_combine(cb, s);
         mark(3);
         return cuda_rc(e);
     }

@@ -83,6 +83,7 @@ __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, int rows_base,
     __shared__ int s_r_true;
     __shared__ int s_fail;
     __shared__ int s_last;
+    __shared__ float s_aux_scale;  // per-tensor Aux scale (own-scale reading)
 
     const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
     const int K = a.K, G = K >> 3;
@@ -166,6 +167,9 @@ __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, int rows_base,
     const float down = __int_as_float((127 - a.exp_factor) << 23);  // 2^-e
     const float qf = (float)a.qmax;
     const int c = (1 << a.exp_factor) - 1;
+    // Aux layout: with the shared scale every Aux column is repeated c times (one accumulator serves Eq. 7); with its
+    // own scale Aux is a separate product and its columns are stored once
+    const int crep = a.aux_own ? 1 : c;
     // channel maxima = max over the replicas, fetched with coalesced 16-byte loads
     for (int k4 = t; k4 < (K >> 2); k4 += kT) {
         uint4 v[kColmaxReplicas];
@@ -256,12 +260,18 @@ __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, int rows_base,
             carry += __shfl_sync(0xffffffffu, incl, 31);
         }
         __syncwarp();
-        const int ucols = c * min(carry, a.cap);
-        for (int i = lane; i < ucols; i += 32) s_auxsrc[i] = (uint16_t)s_oidx[i / c];
+        const int ucols = crep * min(carry, a.cap);
+        for (int i = lane; i < ucols; i += 32) s_auxsrc[i] = (uint16_t)s_oidx[i / crep];
+        // own-scale reading, per tensor: max |Aux| = 2^-e times the largest maximum among the listed channels
+        float am = 0.0f;
+        for (int j = lane; j < min(carry, a.cap); j += 32) am = fmaxf(am, __uint_as_float(s_colmax[s_oidx[j]]) * down);
+        am = warp_max(am);
         if (lane == 0) {
             s_last = ticket == gridDim.x - 1 ? 1 : 0;
             s_r_true = carry;
+            s_aux_scale = am > 0.0f ? __fdiv_rn(am, qf) : 1.0f;
             if (b == 0) {
+                a.ctrl->s_a = s_aux_scale;
                 a.ctrl->n_outliers = carry;
                 if (carry > a.cap && a.dev_status) atomicMax(a.dev_status, kStatusCapacity);
             }
@@ -331,7 +341,7 @@ __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, int rows_base,
         }
     } else {
         const int r = min(s_r_true, a.cap);
-        const int used_cols = c * r, pad_words = ((used_cols + 31) & ~31) >> 2;
+        const int used_cols = crep * r, pad_words = a.aux_own ? a.aux_cols >> 2 : ((used_cols + 31) & ~31) >> 2;
         for (int row = warp; row < rows; row += kWarps) {
             const size_t m = (size_t)r0 + row;
             const uint4 *src = row < fit ? reinterpret_cast<const uint4 *>(slab + (size_t)row * K * 2)
@@ -360,7 +370,7 @@ __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, int rows_base,
                 }
                 *reinterpret_cast<uint2 *>(q + ch * 8) = pack8(code);
             }
-            if (a.aux_q) {
+            if (a.aux_q && !a.aux_own) {
                 // shared scale: Aux_q[m, c*j + i] is the code Body_q[m, O_j] this warp has just written
                 __syncwarp();
                 for (int w = lane; w < pad_words; w += 32) {
@@ -371,6 +381,23 @@ __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, int rows_base,
                             packed |= (uint32_t)(uint8_t)q[s_auxsrc[w * 4 + bb]] << (8 * bb);
                     *reinterpret_cast<uint32_t *>(a.aux_q + m * a.ld_aux + w * 4) = packed;
                 }
+            } else if (a.aux_q) {
+                // own scale per token: s_A[m] = max_j |Aux[m, j]| / q, then Eq. 1 on Aux[m, j] = X[m, O_j] * 2^-e
+                const __half *xr = reinterpret_cast<const __half *>(src);
+                float am = 0.0f;
+                for (int j = lane; j < used_cols; j += 32) am = fmaxf(am, fabsf(__half2float(xr[s_auxsrc[j]]) * down));
+                am = warp_max(am);
+                const float sa = am > 0.0f ? __fdiv_rn(am, qf) : 1.0f;
+                if (lane == 0) a.s_a_rows[m] = sa;
+                for (int w = lane; w < pad_words; w += 32) {
+                    uint32_t packed = 0;
+#pragma unroll
+                    for (int bb = 0; bb < 4; ++bb)
+                        if (w * 4 + bb < used_cols)
+                            packed |= (uint32_t)(quant_exact(__half2float(xr[s_auxsrc[w * 4 + bb]]) * down, sa, qf) & 0xff)
+                                      << (8 * bb);
+                    *reinterpret_cast<uint32_t *>(a.aux_q + m * a.ld_aux + w * 4) = packed;
+                }
             }
         }
     }
@@ -378,11 +405,13 @@ __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, int rows_base,
     // ---------------------------------------------------------------- Aux block (per tensor) and W_aux
     __syncthreads();  // the last warp's outlier list and Aux sources are complete
     const int r = min(s_r_true, a.cap);
-    const int used_cols = c * r;
+    const int used_cols = crep * r;
     // The GEMM consumes the Aux columns in steps of 32, i.e. columns [0, pad_cols); an Aux column of zeros makes the
     // matching W_aux column irrelevant and vice versa, so both blocks are written up to pad_cols only (codes, then
     // zeros) and the columns behind are left as they are.
-    const int pad_words = ((used_cols + 31) & ~31) >> 2;
+    // (With its own scale Aux is the A operand of a product over all aux_cols columns: zeros to the end.)
+    const int pad_words = a.aux_own ? a.aux_cols >> 2 : ((used_cols + 31) & ~31) >> 2;
+    const float s_codes = a.aux_own ? s_aux_scale : s;
     // Independent jobs share the CTA's warps so that their latencies overlap instead of adding up: warps 0-15 the
     // Aux codes, warps 16-31 the W_aux gather (and, in one CTA per launch, the clean-up for the next call).
     const bool do_aux = a.aux_q && !kPerToken;
@@ -400,7 +429,7 @@ __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, int rows_base,
                 for (int bb = 0; bb < 4; ++bb) {
                     const int col = w * 4 + bb;
                     if (col < used_cols)
-                        packed |= (uint32_t)(quant_exact(__half2float(xr[s_auxsrc[col]]) * down, s, qf) & 0xff) << (8 * bb);
+                        packed |= (uint32_t)(quant_exact(__half2float(xr[s_auxsrc[col]]) * down, s_codes, qf) & 0xff) << (8 * bb);
                 }
                 *reinterpret_cast<uint32_t *>(a.aux_q + m * a.ld_aux + w * 4) = packed;
             }

@@ -16,7 +16,8 @@ struct Ctrl {
     float inv_s_x;         // 1 / s_x, correctly rounded (used only to pre-screen the exact division)
     uint32_t arrived;      // fused prep kernel: CTAs that have reached the grid-wide barrier
     uint32_t readers;      // fused prep kernel: CTAs that have fetched the merged channel maxima
-    uint32_t reserved[58];
+    float s_a;             // per-tensor Aux scale when Aux has its own (Eq. 1 applied to Aux alone)
+    uint32_t reserved[57];
 };
 static_assert(sizeof(Ctrl) == 256, "Ctrl is one 256-byte block");
 
@@ -71,6 +72,8 @@ struct PrepArgs {
     int M, K, ldx;
     float tau;
     int exp_factor, qmax, cap, per_token;
+    int aux_own;             // Aux quantized with its own abs-max scale: columns not repeated, whole block padded with zeros
+    float *s_a_rows;         // [M] out when per_token && aux_own
     uint32_t *colmax_rep;    // [kPrepColmaxReplicas, K] accumulators: zero on entry, zeroed again before exit
     uint32_t *colmax_bits;   // [K] out: channel abs-max (bit patterns of non-negative floats)
     Ctrl *ctrl;              // arrived, readers: zero on entry, zero again on exit
@@ -82,6 +85,14 @@ struct PrepArgs {
     int8_t *w_aux; int ld_waux;
     int32_t *dev_status;     // set to 0 at kernel start, raised on r > cap or a barrier time-out
 };
+// Own-scale reading: Y = t1 + c * t2 (fp32 in, fp16 or fp32 out); t1, t2 dense [M, N].
+struct CombineArgs {
+    const float *t1, *t2;
+    int M, N, c;
+    void *Y; int ldy; int out_f16;
+};
+cudaError_t launch_combine(const CombineArgs &a, cudaStream_t s);
+
 // False when the shape does not fit the fused kernel (the caller then uses the separate kernels).
 bool prep_supported(int M, int K);
 cudaError_t launch_prep(const PrepArgs &a, cudaStream_t s);

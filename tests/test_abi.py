@@ -63,7 +63,8 @@ def test_argument_validation_without_gpu(L):
     assert lib.muxq_linear(odd, 128, 768, 768, fake, 768, fake, 768, ctypes.byref(p), fake, 768, 0, fake, big, fake, None) == 2
     assert lib.muxq_linear(fake, 128, 768, 768, fake, 768, fake, 772, ctypes.byref(p), fake, 772, 0, fake, big, fake, None) == 2
     own = L.MuxqParams(aux_scale=1).c()
-    assert lib.muxq_linear(fake, 128, 768, 768, fake, 768, fake, 768, ctypes.byref(own), fake, 768, 0, fake, big, fake, None) == 2
+    # the own-scale reading has no common integer accumulator to return
+    assert lib.muxq_linear(fake, 128, 768, 768, fake, 768, fake, 768, ctypes.byref(own), fake, 768, 2, fake, big, fake, None) == 2
     # workspace too small
     assert lib.muxq_linear(fake, 128, 768, 768, fake, 768, fake, 768, ctypes.byref(p), fake, 768, 0, fake, 1024, fake, None) == 3
     # other entry points

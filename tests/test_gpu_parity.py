@@ -355,7 +355,7 @@ def test_argument_errors(mx):
         mx.muxq_linear(x, w_q, s_w, mx.MuxqParams(exp_factor=5), ws)
     assert ei.value.status == mx.MUXQ_ERR_INVALID_ARG
     with pytest.raises(mx.MuxqError) as ei:
-        mx.muxq_linear(x, w_q, s_w, mx.MuxqParams(aux_scale=1), ws)
+        mx.muxq_linear(x, w_q, s_w, mx.MuxqParams(aux_scale=1), ws, mx.MUXQ_OUT_ACC_I32)
     assert ei.value.status == mx.MUXQ_ERR_UNSUPPORTED
 
 
@@ -496,3 +496,31 @@ def test_one_workspace_serves_a_sequence_of_shapes(mx):
         v = ws_views(mx, ws, M, K, N, p)
         assert v["n_outliers"] == res.r and np.array_equal(v["outlier_idx"][:res.r], res.O), (i, M, K, N)
         assert rel_err32(y.cpu().numpy(), res.y32) <= 1e-5, (i, M, K, N)
+
+
+# ------------------------------------------------------------------ own-scale reading of the Aux quantization
+@pytest.mark.parametrize("M,K,N,gran,e,n_out", [(300, 768, 256, 0, 2, 5), (300, 768, 256, 1, 2, 5), (8, 512, 128, 0, 2, 3),
+                                                 (1000, 1024, 264, 0, 3, 9), (520, 3072, 128, 1, 1, 6), (64, 256, 136, 0, 2, 0)])
+def test_aux_own_scale_layer_matches_oracle(mx, M, K, N, gran, e, n_out):
+    """Aux quantized with its own abs-max scale (the other reading of Eq. 1 for Aux): scales, Aux codes and
+    outputs against the oracle's aux_own path."""
+    p = mx.MuxqParams(gran=gran, exp_factor=e, aux_scale=mx.MUXQ_AUX_OWN)
+    x, w, _ = make_case(1200 + M + e, M, K, N, n_out=n_out)
+    wq, sw = oracle.quantize_weight(w, bits=p.w_bits, per_channel=gran == 1)
+    res = oracle.linear(x, wq, sw, tau=p.threshold, e=e, act_bits=p.act_bits, per_vector=gran == 1, aux_own=True,
+                        cap=p.max_outliers)
+    for out_kind in (mx.MUXQ_OUT_F32, mx.MUXQ_OUT_F16):
+        y, ws, st, _, _ = run_linear(mx, x, w, p, out_kind)
+        assert st == 0
+        v = ws_views(mx, ws, M, K, N, p)
+        view = mx.muxq_workspace_view(M, K, N, p)
+        b = ws.buf.cpu().numpy()
+        s_a = b[view.s_a: view.s_a + 4 * (M if gran == 1 else 1)].view(np.float32)
+        assert v["n_outliers"] == res.r and np.array_equal(v["outlier_idx"][:res.r], res.O)
+        assert np.array_equal(v["s_x"], res.s_x) and np.array_equal(s_a, res.s_a)
+        assert np.array_equal(v["body_q"], res.body_q)
+        assert np.array_equal(v["aux_q"][:, :res.r], res.aux_q) and not v["aux_q"][:, res.r:].any()
+        if out_kind == mx.MUXQ_OUT_F32:
+            assert rel_err32(y.cpu().numpy(), res.y32) <= 1e-5
+        else:
+            assert f16_ulp_diff(y.cpu().numpy(), res.y16).max() <= 1
