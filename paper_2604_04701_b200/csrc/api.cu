@@ -17,7 +17,7 @@ bool params_ok(const muxq_params *p) {
     return p && p->exp_factor >= 1 && p->exp_factor <= 3 && p->act_bits >= 2 && p->act_bits <= 8 &&
            p->w_bits >= 2 && p->w_bits <= 8 && (p->gran == MUXQ_PER_TENSOR || p->gran == MUXQ_PER_VECTOR) &&
            (p->aux_scale == MUXQ_AUX_SHARED || p->aux_scale == MUXQ_AUX_OWN) && p->max_outliers >= 1 &&
-           p->max_outliers <= 64 && isfinite(p->threshold) && p->threshold >= 0.0f;
+           p->max_outliers <= kMaxOutlierCap && isfinite(p->threshold) && p->threshold >= 0.0f;
 }
 inline int qmax_of(int bits) { return (1 << (bits - 1)) - 1; }
 
@@ -32,7 +32,7 @@ SmallWs small_ws(int cols) {
     w.colmul = align_up(w.colmax + (size_t)cols * 4, 256);
     w.grpflag = align_up(w.colmul + (size_t)cols * 4, 256);
     w.oidx = align_up(w.grpflag + (size_t)(cols + 7) / 8, 256);
-    w.total = align_up(w.oidx + 64 * 4, 256);
+    w.total = align_up(w.oidx + (size_t)kMaxOutlierCap * 4, 256);
     return w;
 }
 

@@ -32,18 +32,16 @@ constexpr int kT = 1024;  // the warp-group split of the last phase (512 + 256 +
 constexpr int kWarps = kT / 32;
 constexpr int kMaxK = 8 * kT;  // one group of 8 channels per thread
 static_assert(kMaxK == kPrepMaxK, "the accumulator region of the workspace is sized for kPrepMaxK channels");
-constexpr int kMaxOut = 64;
-constexpr int kMaxAuxCols = 512;  // (2^3 - 1) * 64 rounded up to 128
 constexpr int kColmaxReplicas = kPrepColmaxReplicas;
 constexpr int kStatusCapacity = 5;  // MUXQ_ERR_CAPACITY
 constexpr int kStatusTimeout = 6;   // MUXQ_ERR_TIMEOUT
 constexpr uint32_t kBarrierSpin = 1u << 21;
 constexpr int kMaxDynSmem = 227 * 1024 - 1024;
 
-__host__ __device__ inline int fixed_smem_bytes(int K) {
+__host__ __device__ inline int fixed_smem_bytes(int K, int cap, int aux_cols) {
     const int G = K >> 3;
-    // colmul | colmax | group flags | outlier indices | source channel of every Aux column
-    return 8 * K + ((G + 15) & ~15) + kMaxOut * 4 + kMaxAuxCols * 2;
+    // colmul | colmax | group flags | outlier indices [cap] | source channel of every Aux column [aux_cols]
+    return 8 * K + ((G + 15) & ~15) + ((cap + 3) & ~3) * 4 + ((aux_cols * 2 + 15) & ~15);
 }
 
 __device__ __forceinline__ uint32_t ld_acquire_u32(const uint32_t *p) {
@@ -91,8 +89,8 @@ __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, int rows_base,
     uint32_t *s_colmax = reinterpret_cast<uint32_t *>(smem + 4 * K);
     uint8_t *s_flag = smem + 8 * K;
     int32_t *s_oidx = reinterpret_cast<int32_t *>(smem + 8 * K + ((G + 15) & ~15));
-    uint16_t *s_auxsrc = reinterpret_cast<uint16_t *>(s_oidx + kMaxOut);
-    uint8_t *slab = smem + fixed_smem_bytes(K);
+    uint16_t *s_auxsrc = reinterpret_cast<uint16_t *>(s_oidx + ((a.cap + 3) & ~3));
+    uint8_t *slab = smem + fixed_smem_bytes(K, a.cap, a.aux_cols);
 
     const int b = blockIdx.x;
     const int r0 = b * rows_base + min(b, rows_extra);
@@ -260,7 +258,8 @@ __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, int rows_base,
             carry += __shfl_sync(0xffffffffu, incl, 31);
         }
         __syncwarp();
-        const int ucols = crep * min(carry, a.cap);
+        // (a.aux_cols == 0: no Aux block and no W_aux wanted, the list of sources has no room and no reader)
+        const int ucols = min(crep * min(carry, a.cap), a.aux_cols);
         for (int i = lane; i < ucols; i += 32) s_auxsrc[i] = (uint16_t)s_oidx[i / crep];
         // own-scale reading, per tensor: max |Aux| = 2^-e times the largest maximum among the listed channels
         float am = 0.0f;
@@ -479,7 +478,7 @@ cudaError_t launch_prep(const PrepArgs &a, cudaStream_t s) {
     if (grid > a.M) grid = a.M;
     int rows_base = a.M / grid, rows_extra = a.M % grid;
     const int rows_max = rows_base + (rows_extra ? 1 : 0);
-    const int fixed = fixed_smem_bytes(a.K);
+    const int fixed = fixed_smem_bytes(a.K, a.cap, a.aux_cols);
     const long long want = (long long)rows_max * a.K * 2;
     int slab_bytes = (int)(want < (long long)(kMaxDynSmem - fixed) ? want : (long long)(kMaxDynSmem - fixed));
     slab_bytes &= ~15;

@@ -524,3 +524,36 @@ def test_aux_own_scale_layer_matches_oracle(mx, M, K, N, gran, e, n_out):
             assert rel_err32(y.cpu().numpy(), res.y32) <= 1e-5
         else:
             assert f16_ulp_diff(y.cpu().numpy(), res.y16).max() <= 1
+
+
+# ------------------------------------------------------------------ many outlier channels (capacity up to 1024)
+@pytest.mark.parametrize("M,K,N,gran,own", [(300, 1024, 256, 0, 0), (300, 1024, 256, 1, 0), (8, 1024, 128, 0, 0),
+                                             (200, 512, 136, 0, 1)])
+def test_many_outlier_channels(mx, M, K, N, gran, own):
+    """Heavy-tailed activations at unit scale flag most channels (Section III-C detection on a Student-t bulk):
+    with max_outliers = 1024 the layer still matches the oracle code for code."""
+    p = mx.MuxqParams(gran=gran, max_outliers=1024, aux_scale=own)
+    # (a few rows need a wider bulk to push most channels over the threshold)
+    x, w, _ = make_case(1500 + M + gran, M, K, N, n_out=8, mult=60.0, bulk="t4", bulk_scale=1.0 if M > 16 else 4.0)
+    wq, sw = oracle.quantize_weight(w, bits=p.w_bits, per_channel=gran == 1)
+    res = oracle.linear(x, wq, sw, tau=p.threshold, e=p.exp_factor, act_bits=p.act_bits, per_vector=gran == 1,
+                        aux_own=bool(own), cap=1024)
+    assert res.r > 64  # beyond the default capacity
+    y, ws, st, _, _ = run_linear(mx, x, w, p, mx.MUXQ_OUT_F32)
+    assert st == 0
+    v = ws_views(mx, ws, M, K, N, p)
+    assert v["n_outliers"] == res.r and np.array_equal(v["outlier_idx"][:res.r], res.O)
+    assert np.array_equal(v["s_x"], res.s_x)
+    if M > 16:
+        assert np.array_equal(v["body_q"], res.body_q)
+        c = 1 if own else (1 << p.exp_factor) - 1
+        assert np.array_equal(v["aux_q"][:, 0:c * res.r:c], res.aux_q)
+    assert rel_err32(y.cpu().numpy(), res.y32) <= 1e-5
+    if not own:
+        acc = mx.muxq_linear(dev(x), *mx.muxq_quantize(dev(w), p, True, mx.Workspace(mx.muxq_small_workspace_bytes(N))),
+                             p, mx.Workspace(mx.muxq_workspace_bytes(M, K, N, p)), mx.MUXQ_OUT_ACC_I32)
+        assert np.array_equal(acc.cpu().numpy(), res.acc)
+    # the default capacity reports the overflow instead
+    p64 = mx.MuxqParams(gran=gran, aux_scale=own)
+    _, ws64, st64, _, _ = run_linear(mx, x, w, p64, mx.MUXQ_OUT_F32)
+    assert st64 == mx.MUXQ_ERR_CAPACITY
