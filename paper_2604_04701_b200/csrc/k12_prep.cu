@@ -75,7 +75,8 @@ __device__ __forceinline__ void load_chunk(const uint4 *src, int ch, const uint8
 // kPerToken: per-token scales (one warp per row in pass 2) instead of the per-tensor scale; one instantiation
 // per granularity keeps the other one's code out of the kernel.
 template <bool kAllFit, bool kPerToken>
-__global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, int rows_base, int rows_extra, int slab_bytes) {
+__global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, int rows_base, int rows_extra, int slab_bytes,
+                                                int rstride, uint32_t g_magic) {
     extern __shared__ __align__(16) uint8_t smem[];
     __shared__ float s_warp_max[kWarps];
     __shared__ int s_r_true;
@@ -102,8 +103,11 @@ __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, int rows_base,
     for (int k = t; k < K; k += kT) s_colmax[k] = 0u;
     __syncthreads();
     {
-        const int rstride = kT / G;  // G <= kT: thread = (row offset, channel group)
-        const int cg = t % G, row_off = t / G;
+        // thread = (row offset, channel group); rstride = kT / G row offsets are in use (G <= kT).  The division
+        // t / G is a multiplication by g_magic = ceil(2^20 / G), exact for t < 1024 (t * G < 2^20); both constants
+        // come from the host: with 32 warps per SM every instruction of per-thread set-up costs 8 cycles of SM time,
+        // and a 32-bit division is some 25 instructions
+        const int row_off = (int)(((uint32_t)t * g_magic) >> 20), cg = t - row_off * G;
         if (row_off < rstride) {
             __half2 m[4];
             m[0] = m[1] = m[2] = m[3] = __float2half2_rn(0.f);
@@ -192,8 +196,7 @@ __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, int rows_base,
     // Every thread derives the factors of the 8 channels it owns in both passes: 2^-e where the channel
     // holds an element above the threshold (strict), else 1.  (When more channels are flagged than the
     // capacity allows the call fails with MUXQ_ERR_CAPACITY and Y is unspecified, so no ordering is needed here.)
-    const int rstride = kT / G;
-    const int cg = t % G, row_off = t / G;
+    const int row_off = (int)(((uint32_t)t * g_magic) >> 20), cg = t - row_off * G;
     float mul[8];
     uint32_t fmask = 0;  // bit i: channel 8*cg + i is an outlier channel
     {
@@ -483,7 +486,10 @@ cudaError_t launch_prep(const PrepArgs &a, cudaStream_t s) {
     int slab_bytes = (int)(want < (long long)(kMaxDynSmem - fixed) ? want : (long long)(kMaxDynSmem - fixed));
     slab_bytes &= ~15;
     PrepArgs args = a;
-    void *params[] = {&args, &rows_base, &rows_extra, &slab_bytes};
+    const int G = a.K >> 3;
+    int rstride = kT / G;
+    uint32_t g_magic = ((1u << 20) + (uint32_t)G - 1u) / (uint32_t)G;
+    void *params[] = {&args, &rows_base, &rows_extra, &slab_bytes, &rstride, &g_magic};
     const bool all_fit = (long long)slab_bytes >= want;
     const void *fn = fns[(all_fit ? 2 : 0) + (a.per_token ? 1 : 0)];
     return cudaLaunchCooperativeKernel(fn, dim3(grid), dim3(kT), params, (size_t)(fixed + slab_bytes), s);
