@@ -78,6 +78,8 @@ def test_argument_validation_without_gpu(L):
     assert lib.muxq_gemm(fake, 768, None, 0, fake, 768, None, 0, None, 128, 768, 768, ctypes.byref(p), None, None, fake, 768, 0, fake, None) == 1
     assert lib.muxq_gemm(fake, 776, None, 0, fake, 768, None, 0, None, 128, 768, 768, ctypes.byref(p), fake, fake, fake, 768, 0, fake, None) == 2
     assert lib.muxq_read_status(None, None) == 1
+    assert lib.muxq_workspace_init(None, big, None) == 1
+    assert lib.muxq_workspace_init(fake, 128, None) == 1   # smaller than the control block
     assert lib.muxq_linear_host(None, 128, 768, fake, 768, fake, 768, ctypes.byref(p), fake, 0, fake, big, fake, None) == 1
     assert lib.muxq_linear_host(fake, 128, 768, fake, 768, fake, 768, ctypes.byref(p), fake, 0, fake, 4096, fake, None) == 3
 
