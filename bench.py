@@ -152,6 +152,22 @@ def run_reference(args, rank):
 
 
 # --------------------------------------------------------------------------- CUDA arm
+def max_over_ranks(ms: float, world: int, device) -> float:
+    """The slowest rank's time: what a replica run is charged (all-reduce MAX over the process group)."""
+    if world <= 1:
+        return ms
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_tops(world: int, ops_per_step: float, ms_per_step: float) -> float:
+    """Replicas only: every rank does the same work, the job's rate is the sum over ranks at the slowest rank's time."""
+    return world * ops_per_step / (ms_per_step * 1e-3) / 1e12
+
+
 def run_muxq(args, rank, world):
     import torch
     import torch.distributed as dist
@@ -222,13 +238,9 @@ def run_muxq(args, rank, world):
     torch.cuda.synchronize(); barrier()
     clocks = sampler.stop()
     check_status()
-    ms = e0.elapsed_time(e1)
-    if world > 1:
-        t = torch.tensor([ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = max_over_ranks(e0.elapsed_time(e1), world, dev)
     ms_per_step = ms / args.steps
-    value = world * ops_per_step / (ms_per_step * 1e-3) / 1e12
+    value = whole_job_tops(world, ops_per_step, ms_per_step)
 
     # ---- per-kernel durations: the same step captured with event-record nodes at the kernel
     # boundaries (same stream, same buffers), replayed and read back one replay at a time
@@ -346,12 +358,8 @@ def run_muxq(args, rank, world):
     h1.record()
     torch.cuda.synchronize(); barrier()
     check_status()
-    ems = h0.elapsed_time(h1)
-    if world > 1:
-        t = torch.tensor([ems], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ems = float(t.item())
-    e2e = {"value": world * ops_per_step / (ems / esteps * 1e-3) / 1e12, "unit": UNIT,
+    ems = max_over_ranks(h0.elapsed_time(h1), world, dev)
+    e2e = {"value": whole_job_tops(world, ops_per_step, ems / esteps), "unit": UNIT,
            "h2d_bytes_per_step": int(sum(xh.numel() * 2 for xh, _ in hosts)),
            "d2h_bytes_per_step": int(sum(yh.numel() * 2 for _, yh in hosts)), "steps": esteps,
            "ms_per_step": ems / esteps}
