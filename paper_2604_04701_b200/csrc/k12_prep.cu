@@ -344,25 +344,35 @@ __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, int rows_base,
     } else {
         const int r = min(s_r_true, a.cap);
         const int used_cols = crep * r, pad_words = a.aux_own ? a.aux_cols >> 2 : ((used_cols + 31) & ~31) >> 2;
-        for (int row = warp; row < rows; row += kWarps) {
+        // A row is walked by a whole warp, or by half a warp when the CTA has more rows than warps: two rounds of
+        // rows per warp would run every reduction, division and store latency of a row twice in sequence.
+        const int lpr = rows > kWarps ? 16 : 32;  // lanes per row
+        const int rpw = 32 / lpr, sub = lane / lpr, l = lane - sub * lpr;
+        auto part_max = [&](float v) {  // over the lanes of one row
+            for (int o = lpr >> 1; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+            return v;
+        };
+        for (int base = warp * rpw; base < rows; base += kWarps * rpw) {  // warp-uniform trip count
+            const int row = min(base + sub, rows - 1);
+            const bool live = base + sub < rows;  // the other half of the warp may have run out of rows
             const size_t m = (size_t)r0 + row;
             const uint4 *src = row < fit ? reinterpret_cast<const uint4 *>(slab + (size_t)row * K * 2)
                                          : reinterpret_cast<const uint4 *>(a.X + m * a.ldx);
             // per-token scale from Body's row (after the 2^-e redistribution)
             float mx = 0.0f;
-            for (int ch = lane; ch < G; ch += 32) {
+            for (int ch = l; ch < G; ch += lpr) {
                 float f[8];
                 load_chunk(src, ch, s_flag, s_colmul, f);
 #pragma unroll
                 for (int i = 0; i < 8; ++i) mx = fmaxf(mx, fabsf(f[i]));
             }
-            mx = warp_max(mx);
+            mx = part_max(mx);
             const float sr = mx > 0.0f ? __fdiv_rn(mx, qf) : 1.0f;
             float rlo, rhi;
             recip_bracket(__frcp_rn(sr), rlo, rhi);
-            if (lane == 0) a.s_x_rows[m] = sr;
+            if (l == 0 && live) a.s_x_rows[m] = sr;
             int8_t *q = a.body_q + m * a.ld_q;
-            for (int ch = lane; ch < G; ch += 32) {
+            for (int ch = l; ch < G && live; ch += lpr) {
                 float f[8];
                 load_chunk(src, ch, s_flag, s_colmul, f);
                 uint32_t code[8];
@@ -373,9 +383,9 @@ __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, int rows_base,
                 *reinterpret_cast<uint2 *>(q + ch * 8) = pack8(code);
             }
             if (a.aux_q && !a.aux_own) {
-                // shared scale: Aux_q[m, c*j + i] is the code Body_q[m, O_j] this warp has just written
+                // shared scale: Aux_q[m, c*j + i] is the code Body_q[m, O_j] these lanes have just written
                 __syncwarp();
-                for (int w = lane; w < pad_words; w += 32) {
+                for (int w = l; w < pad_words && live; w += lpr) {
                     uint32_t packed = 0;
 #pragma unroll
                     for (int bb = 0; bb < 4; ++bb)
@@ -387,11 +397,11 @@ __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, int rows_base,
                 // own scale per token: s_A[m] = max_j |Aux[m, j]| / q, then Eq. 1 on Aux[m, j] = X[m, O_j] * 2^-e
                 const __half *xr = reinterpret_cast<const __half *>(src);
                 float am = 0.0f;
-                for (int j = lane; j < used_cols; j += 32) am = fmaxf(am, fabsf(__half2float(xr[s_auxsrc[j]]) * down));
-                am = warp_max(am);
+                for (int j = l; j < used_cols; j += lpr) am = fmaxf(am, fabsf(__half2float(xr[s_auxsrc[j]]) * down));
+                am = part_max(am);
                 const float sa = am > 0.0f ? __fdiv_rn(am, qf) : 1.0f;
-                if (lane == 0) a.s_a_rows[m] = sa;
-                for (int w = lane; w < pad_words; w += 32) {
+                if (l == 0 && live) a.s_a_rows[m] = sa;
+                for (int w = l; w < pad_words && live; w += lpr) {
                     uint32_t packed = 0;
 #pragma unroll
                     for (int bb = 0; bb < 4; ++bb)
