@@ -93,11 +93,14 @@ k_gemm_i8_pair(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");  // a dependent still waits for this grid to finish
 
-    int aux_cols_used = 0;
-    if (p.has_aux) aux_cols_used = p.c * min(__ldg(p.n_outliers), p.cap);
-    aux_cols_used = __shfl_sync(0xffffffffu, aux_cols_used, 0);
-    const int aux_kb = (aux_cols_used + BK - 1) / BK;
-    const int total_kb = p.num_kb + aux_kb;
+    // r (and with it the number of Aux K blocks) lives in global memory.  It is fetched when a role first reaches the
+    // end of a tile's Body blocks, not here: the first operand loads need not wait for that round trip.
+    int aux_cols_used = p.has_aux ? -1 : 0, aux_kb = 0;
+    auto fetch_aux = [&]() {
+        int v = p.c * min(__ldg(p.n_outliers), p.cap);
+        aux_cols_used = __shfl_sync(0xffffffffu, v, 0);
+        aux_kb = (aux_cols_used + BK - 1) / BK;
+    };
     const int num_tiles = p.tiles_m * p.tiles_n;
     const int pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
 
@@ -108,7 +111,11 @@ k_gemm_i8_pair(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
         for (int tile = pair; tile < num_tiles && ok; tile += num_pairs) {
             const int m0 = (tile / p.tiles_n) * (2 * BM) + (int)rank * BM;
             const int n0 = (tile % p.tiles_n) * BN + (int)rank * (BN / 2);
-            for (int kb = 0; kb < total_kb; ++kb, ++it) {
+            for (int kb = 0;; ++kb, ++it) {
+                if (kb >= p.num_kb) {
+                    if (aux_cols_used < 0) fetch_aux();
+                    if (kb >= p.num_kb + aux_kb) break;
+                }
                 const uint32_t s = it % C::kStages, ph = (it / C::kStages) & 1u;
                 if (!mbar_wait_warp(&bar_empty[s], ph ^ 1u, abort_flag)) { ok = false; break; }
                 uint8_t *sa = smem_al + s * C::kStageBytes;
@@ -152,7 +159,11 @@ k_gemm_i8_pair(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                 if (!mbar_wait_warp_cluster(&bar_acc_empty[buf], aph ^ 1u, abort_flag)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + buf * BN;
-                for (int kb = 0; kb < total_kb; ++kb, ++it) {
+                for (int kb = 0;; ++kb, ++it) {
+                    if (kb >= p.num_kb) {
+                        if (aux_cols_used < 0) fetch_aux();
+                        if (kb >= p.num_kb + aux_kb) break;
+                    }
                     const uint32_t s = it % C::kStages, ph = (it / C::kStages) & 1u;
                     if (!mbar_wait_warp(&bar_full[s], ph, abort_flag)) { ok = false; break; }
                     tc_fence_after();
