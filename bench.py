@@ -462,6 +462,32 @@ def run_muxq(args, rank, world):
             gbs = wbytes / us / 1e3
             decode[f"M{Md}"] = {"us_per_layer": us / len(dlayers), "gb_per_s": gbs, "frac_of_measured_hbm": gbs / peaks["hbm_gbs"]}
             del g_dec
+            # one call on its own (nothing before it in the stream to overlap with, weights cold): the call is captured
+            # with event-record nodes at its boundaries and replayed 15 times, each after a write of 256 MB that
+            # pushes the weights out of L2; median device time between the records (includes their node overhead)
+            flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+            iso = {}
+            for li, (K, N, wq) in enumerate(dlayers[:4]):
+                ievs = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+                for e in ievs:
+                    e.record()
+                torch.cuda.synchronize()
+                with torch.cuda.stream(side):
+                    g_one = torch.cuda.CUDAGraph()
+                    with torch.cuda.graph(g_one, stream=side):
+                        mx.muxq_linear_events(dx[K], wq, sw1, p, dws[K], ievs, mx.MUXQ_OUT_F16, out=dy[N])
+                torch.cuda.synchronize()
+                ts = []
+                for _ in range(15):
+                    flush.fill_(li)
+                    torch.cuda.synchronize()
+                    g_one.replay()
+                    torch.cuda.synchronize()
+                    ts.append(ievs[0].elapsed_time(ievs[3]) * 1e3)
+                iso[f"{K}->{N}"] = statistics.median(ts)
+                del g_one
+            decode[f"M{Md}"]["isolated_call_us"] = iso
+            del flush
         del dlayers
 
     cpu_baseline = None
