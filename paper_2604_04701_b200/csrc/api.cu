@@ -446,6 +446,7 @@ static int linear_impl(const void *X, int M, int K, int ldx, const int8_t *W_q, 
     g.s_w = s_w; g.s_w_per_col = per_vec;
     g.Y = Y; g.ldy = ldy; g.out_kind = out_kind;
     g.dev_status = dev_status;
+    g.w_stable = 1;  // the kernel before this one in the stream is the preparation of X, which does not write W_q
     e = launch_gemm(g, s);
     mark(3);
     return cuda_rc(e);

@@ -26,6 +26,7 @@ struct GemmParams {
     const float *s_x;
     const float *s_w;
     int32_t *dev_status;
+    int w_stable;  // the B operand may be read before the programmatic predecessor has finished
 };
 
 // One 32-column chunk of one accumulator row: int32 -> fp32 (round to nearest even, exact below

@@ -88,6 +88,21 @@ k_gemm_i8_pair(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     const uint32_t tmem_base = __shfl_sync(0xffffffffu, s_tmem_base, 0);
     volatile uint32_t *abort_flag = &s_abort;
 
+    const int num_tiles = p.tiles_m * p.tiles_n;
+    const int pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
+    // The weights are constants of the layer: when the caller vouches for that, the producer fetches the B tiles of its
+    // first stages before waiting for the predecessor (the preparation of X), whose tail then hides their latency
+    // and the first pass through the producer's code.  The A tiles of those stages follow after the wait.
+    int pre = 0;
+    if (warp == 0 && p.w_stable && pair < num_tiles) {
+        pre = min(C::kStages, p.num_kb);
+        const int n0 = (pair % p.tiles_n) * BN + (int)rank * (BN / 2);
+        for (int kb = 0; kb < pre; ++kb) {
+            uint8_t *sb = smem_al + kb * C::kStageBytes + C::kABytes;
+            if (rank == 0) mbar_expect_tx_elect(&bar_full[kb], 2 * C::kStageBytes);
+            tma_load_2d_pair_elect(sb, &tm_b, map_to_cta(smem_u32(&bar_full[kb]), 0), kb * BK, n0);
+        }
+    }
     // Launched as a programmatic dependent of the kernel before it in the stream (the activation
     // preparation): the set-up above overlaps that kernel's tail; its results are read only from here on.
     asm volatile("griddepcontrol.wait;" ::: "memory");
@@ -101,8 +116,6 @@ k_gemm_i8_pair(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
         aux_cols_used = __shfl_sync(0xffffffffu, v, 0);
         aux_kb = (aux_cols_used + BK - 1) / BK;
     };
-    const int num_tiles = p.tiles_m * p.tiles_n;
-    const int pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
 
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer (both CTAs)
@@ -117,11 +130,15 @@ k_gemm_i8_pair(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                     if (kb >= p.num_kb + aux_kb) break;
                 }
                 const uint32_t s = it % C::kStages, ph = (it / C::kStages) & 1u;
-                if (!mbar_wait_warp(&bar_empty[s], ph ^ 1u, abort_flag)) { ok = false; break; }
                 uint8_t *sa = smem_al + s * C::kStageBytes;
                 uint8_t *sb = sa + C::kABytes;
-                if (rank == 0) mbar_expect_tx_elect(&bar_full[s], 2 * C::kStageBytes);
                 const uint32_t full_leader = map_to_cta(smem_u32(&bar_full[s]), 0);
+                if (it < (uint32_t)pre) {  // stage announced and its B tile already on the way (see above)
+                    tma_load_2d_pair_elect(sa, &tm_a, full_leader, kb * BK, m0);
+                    continue;
+                }
+                if (!mbar_wait_warp(&bar_empty[s], ph ^ 1u, abort_flag)) { ok = false; break; }
+                if (rank == 0) mbar_expect_tx_elect(&bar_full[s], 2 * C::kStageBytes);
                 if (kb < p.num_kb) {
                     tma_load_2d_pair_elect(sa, &tm_a, full_leader, kb * BK, m0);
                     tma_load_2d_pair_elect(sb, &tm_b, full_leader, kb * BK, n0);
@@ -313,6 +330,7 @@ cudaError_t launch_pair_inst(const GemmArgs &a, cudaStream_t s) {
     p.s_x = a.s_x;
     p.s_w = a.s_w;
     p.dev_status = a.dev_status;
+    p.w_stable = a.w_stable;
     int clusters = p.tiles_m * p.tiles_n;
     if (clusters > max_clusters) clusters = max_clusters;
     cudaLaunchConfig_t cfg{};

@@ -128,6 +128,7 @@ struct GemmArgs {
     const float *s_w; int s_w_per_col;
     void *Y; int ldy; int out_kind;
     int32_t *dev_status;
+    int w_stable;  // W_q is not written by the kernel before this one in the stream: its tiles may be fetched early
 };
 cudaError_t launch_gemm(const GemmArgs &a, cudaStream_t s);
 cudaError_t launch_gemm_pair(const GemmArgs &a, int bn, cudaStream_t s);  // two CTAs per 256-row tile
