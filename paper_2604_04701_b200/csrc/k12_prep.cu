@@ -424,6 +424,12 @@ __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, int rows_base,
     // (With its own scale Aux is the A operand of a product over all aux_cols columns: zeros to the end.)
     const int pad_words = a.aux_own ? a.aux_cols >> 2 : ((used_cols + 31) & ~31) >> 2;
     const float s_codes = a.aux_own ? s_aux_scale : s;
+    // i / pad_words below as a multiplication where the item counts are small (i < 2^22: the float holds i + 0.5
+    // exactly, and (i + 0.5) / pad_words is at least 0.5 / pad_words away from an integer, far more than the rounding
+    // of the product); a 32-bit division is some 25 instructions, and this phase is one or two items per thread
+    const float inv_pad = 1.0f / (float)max(pad_words, 1);
+    const bool small_counts = (long long)max(rows, a.N) * pad_words < (1ll << 22);
+    auto div_pad = [&](int i) { return small_counts ? (int)(((float)i + 0.5f) * inv_pad) : i / max(pad_words, 1); };
     // Independent jobs share the CTA's warps so that their latencies overlap instead of adding up: warps 0-15 the
     // Aux codes, warps 16-31 the W_aux gather (and, in one CTA per launch, the clean-up for the next call).
     const bool do_aux = a.aux_q && !kPerToken;
@@ -432,7 +438,7 @@ __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, int rows_base,
             // Aux_q[m, c*j + i] = code of Body[m, O_j] (Eq. 5, shared scale), recomputed from the slab with the
             // exact division, one 4-byte word per thread and round
             for (int i = t; i < rows * pad_words; i += 512) {
-                const int row = i / pad_words, w = i - row * pad_words;
+                const int row = div_pad(i), w = i - row * pad_words;
                 const size_t m = (size_t)r0 + row;
                 const __half *xr = row < fit ? reinterpret_cast<const __half *>(slab + (size_t)row * K * 2)
                                              : a.X + m * a.ldx;
@@ -459,7 +465,7 @@ __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, int rows_base,
             // W_aux[n, c*j + i] = W_q[n, O_j], one 4-byte word per thread and round, spread over the grid
             const int total = a.N * pad_words;
             for (int i = b * 512 + (t - 512); i < total; i += gridDim.x * 512) {
-                const int n = i / pad_words, w = i - n * pad_words;
+                const int n = div_pad(i), w = i - n * pad_words;
                 uint32_t packed = 0;
 #pragma unroll
                 for (int bb = 0; bb < 4; ++bb)
