@@ -133,8 +133,8 @@ __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, int rows_base,
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
                 const float lo = __low2float(m[i]), hi = __high2float(m[i]);
-                if (lo > 0.0f) atomicMax(&s_colmax[cg * 8 + 2 * i], __float_as_uint(lo));
-                if (hi > 0.0f) atomicMax(&s_colmax[cg * 8 + 2 * i + 1], __float_as_uint(hi));
+                atomicMax(&s_colmax[cg * 8 + 2 * i], __float_as_uint(lo));  // non-negative: bit patterns order like values
+                atomicMax(&s_colmax[cg * 8 + 2 * i + 1], __float_as_uint(hi));
             }
         }
     }
@@ -433,6 +433,11 @@ __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, int rows_base,
     // Independent jobs share the CTA's warps so that their latencies overlap instead of adding up: warps 0-15 the
     // Aux codes, warps 16-31 the W_aux gather (and, in one CTA per launch, the clean-up for the next call).
     const bool do_aux = a.aux_q && !kPerToken;
+    // Aux codes by the bracket test too (2^-e folded into the brackets), the exact division only next to a tie
+    float alo, ahi;
+    recip_bracket(__frcp_rn(s_codes), alo, ahi);
+    alo *= down;
+    ahi *= down;
     if (warp < 16) {
         if (do_aux) {
             // Aux_q[m, c*j + i] = code of Body[m, O_j] (Eq. 5, shared scale), recomputed from the slab with the
@@ -446,8 +451,13 @@ __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, int rows_base,
 #pragma unroll
                 for (int bb = 0; bb < 4; ++bb) {
                     const int col = w * 4 + bb;
-                    if (col < used_cols)
-                        packed |= (uint32_t)(quant_exact(__half2float(xr[s_auxsrc[col]]) * down, s_codes, qf) & 0xff) << (8 * bb);
+                    if (col < used_cols) {
+                        const float xv = __half2float(xr[s_auxsrc[col]]);
+                        const uint32_t ca = __float_as_uint(fmaf(xv, ahi, 12582912.0f));
+                        const uint32_t cb = __float_as_uint(fmaf(xv, alo, 12582912.0f));
+                        const uint32_t code = ca == cb ? ca : (uint32_t)quant_exact(xv * down, s_codes, qf);
+                        packed |= (code & 0xffu) << (8 * bb);
+                    }
                 }
                 *reinterpret_cast<uint32_t *>(a.aux_q + m * a.ld_aux + w * 4) = packed;
             }
