@@ -100,7 +100,12 @@ __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, int rows_base,
     if (b == 0 && t == 0 && a.dev_status) *a.dev_status = 0;
 
     // ---------------------------------------------------------------- pass 1: channel maxima
-    for (int k = t; k < K; k += kT) s_colmax[k] = 0u;
+    // CTA-wide maxima of pass 1 accumulate in s_part, laid out [channel within group][group] so that the lanes of a
+    // warp (consecutive groups) hit consecutive banks; with the natural [group][channel] layout every shared-memory
+    // atomic of a warp would be an 8-way bank conflict.  It shares its bytes with s_colmul, which is written only
+    // after the grid barrier.
+    uint32_t *s_part = reinterpret_cast<uint32_t *>(smem);
+    for (int k = t; k < K; k += kT) s_part[k] = 0u;
     __syncthreads();
     {
         // thread = (row offset, channel group); rstride = kT / G row offsets are in use (G <= kT).  The division
@@ -133,8 +138,8 @@ __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, int rows_base,
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
                 const float lo = __low2float(m[i]), hi = __high2float(m[i]);
-                atomicMax(&s_colmax[cg * 8 + 2 * i], __float_as_uint(lo));  // non-negative: bit patterns order like values
-                atomicMax(&s_colmax[cg * 8 + 2 * i + 1], __float_as_uint(hi));
+                atomicMax(&s_part[(2 * i) * G + cg], __float_as_uint(lo));  // non-negative: bit patterns order like values
+                atomicMax(&s_part[(2 * i + 1) * G + cg], __float_as_uint(hi));
             }
         }
     }
@@ -143,7 +148,7 @@ __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, int rows_base,
         uint32_t *rep = a.colmax_rep + (size_t)(b % kColmaxReplicas) * K;
         for (int k = t; k < K; k += kT) {
             // a warp's 32 consecutive channels travel as one 128-byte reduction request
-            const uint32_t v = s_colmax[k];
+            const uint32_t v = s_part[(k & 7) * G + (k >> 3)];
             if (v != 0u) atomicMax(rep + k, v);
         }
     }
