@@ -2,9 +2,12 @@
 """Benchmark of the MUXQ linear hot path on B200.
 
 A "step" is one pass of the whole hot path -- outlier detection, redistribute + quantize, INT8
-tensor-core GEMM with the Aux correction and dequantization -- over the four GPT-2-small-shaped
-linears (768->2304, 768->768, 768->3072, 3072->768) at M = 8192 tokens, per-tensor INT8, on seeded
-synthetic activations with 6 outlier channels.  Weights are quantized once before timing.
+tensor-core GEMM with the Aux correction and dequantization -- over the four GPT-2-large-shaped
+linears (1280->3840, 1280->1280, 1280->5120, 5120->1280) at M = 16384 tokens, per-tensor INT8, on
+seeded synthetic activations with 8 outlier channels (the largest single-GPU prefill workload of the
+benchmark list).  The GPT-2-small set at M = 8192 is measured the same way and reported beside it,
+and so are the decode shapes (M = 1, 4, 16) as a stream of layers.  Weights are quantized once
+before timing.
 
     python bench.py --gpus 1 --steps K --warmup W          # the CUDA library (one JSON line)
     python bench.py --impl reference ...                    # the CPU oracle on a bounded sample
@@ -15,14 +18,13 @@ Multi-GPU: the path does not shard (one GPU per problem); N ranks run N independ
 from __future__ import annotations
 
 import argparse
+import hashlib
 import json
 import os
 import statistics
 import subprocess
 import sys
 import time
-
-import numpy as np
 
 ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
@@ -32,7 +34,40 @@ import muxq_synth as synth  # noqa: E402
 
 METRIC = "muxq_linear_effective_int8_tops_prefill"
 UNIT = "TOPS"
-CONFIG_ID = 1
+HEADLINE_CONFIG = 3
+NOMINAL_INT8_TOPS = 4500.0
+
+WORKLOAD_TEXT = {
+    1: "configs[1]: GPT-2-small linear set (768->2304, 768->768, 768->3072, 3072->768), M={M} tokens, "
+       "6 outlier channels x40-80, per-tensor INT8, fp16 in/out",
+    3: "configs[3] prefill: GPT-2-large linear set (1280->3840, 1280->1280, 1280->5120, 5120->1280), M={M} tokens, "
+       "8 outlier channels x60, per-tensor INT8, fp16 in/out",
+}
+
+# DRAM traffic per launch from ncu captures (dram__bytes_read.sum + dram__bytes_write.sum, see profiles/): reported
+# only while the kernel's sources still hash to what was captured, null otherwise.
+CSRC = os.path.join(ROOT, "paper_2604_04701_b200", "csrc")
+TRAFFIC = {
+    # kernel key: (source files, sha16 of their concatenation at capture time, {shape: bytes per launch}, note)
+}
+
+
+def _src_sha16(files):
+    h = hashlib.sha256()
+    for f in files:
+        with open(os.path.join(CSRC, f), "rb") as fh:
+            h.update(fh.read())
+    return h.hexdigest()[:16]
+
+
+def traffic_for(kernel, shape):
+    ent = TRAFFIC.get(kernel)
+    if not ent:
+        return None
+    files, sha, table, _ = ent
+    if _src_sha16(files) != sha:
+        return None  # the kernel has changed since the counters were taken
+    return table.get(shape)
 
 
 def load_peaks():
@@ -45,17 +80,29 @@ def load_peaks():
     return {"hbm_gbs": 6650.0, "bf16_burst": 1590.0, "bf16_sustained": 1400.0, "source": "fallback"}
 
 
-def workload(M=None):
-    specs = synth.config_layers(CONFIG_ID, M=M)
+def int8_peak_for(peaks, clocks):
+    """Dense INT8 rate = 2 x the bf16 rate (8192 against 4096 MAC per clock and SM).  The burst figure applies when
+    the timed region ran at the maximum SM clock, the sustained one when the clock had dropped under the power cap."""
+    sm, mx_ = clocks.get("sm_mhz"), clocks.get("sm_max_mhz")
+    burst = sm is None or mx_ is None or sm >= 0.97 * mx_
+    kind = "burst" if burst else "sustained"
+    return 2.0 * peaks["bf16_" + kind], f"2 x bf16_tflops{'' if burst else '_sustained'} ({kind}) of {peaks['source']}"
+
+
+def workload(cfg_id=HEADLINE_CONFIG, M=None):
+    specs = synth.config_layers(cfg_id, M=M)
     ops = sum(2.0 * s.M * s.N * s.K for s in specs)
     return specs, ops
 
 
-def config_dict(specs, extra=None):
-    d = {"workload": "configs[1]: GPT-2-small linear set (768->2304, 768->768, 768->3072, 3072->768), "
-                     f"M={specs[0].M} tokens, 6 outlier channels x40-80, per-tensor INT8, fp16 in/out",
+def config_dict(cfg_id, specs, extra=None):
+    x_mb = sum(2.0 * s.M * s.K for s in specs) / 1e6
+    y_mb = sum(2.0 * s.M * s.N for s in specs) / 1e6
+    q_mb = sum(1.0 * s.M * s.K for s in specs) / 1e6
+    d = {"workload": WORKLOAD_TEXT[cfg_id].format(M=specs[0].M),
          "layers_per_step": len(specs), "granularity": "per-tensor",
-         "l2": "no explicit flush: one step streams ~250 MB (X 88 MB, codes 50 MB, Y 113 MB) > 126 MB L2"}
+         "l2": f"no explicit flush: one step streams ~{x_mb + y_mb + q_mb:.0f} MB (X {x_mb:.0f} MB, codes {q_mb:.0f} MB, "
+               f"Y {y_mb:.0f} MB) > 126 MB L2"}
     if extra:
         d.update(extra)
     return d
@@ -128,11 +175,14 @@ def oracle_sample(specs, rows_per_layer):
     return ops / dt / 1e12, dt, oracle.num_threads()
 
 
+REFERENCE_ROWS = 1024
+
+
 def run_reference(args, rank):
     if rank != 0:
         return
     specs, _ = workload()
-    rows = 2048
+    rows = REFERENCE_ROWS
     vals = []
     oracle_sample(specs, rows)  # one untimed pass
     t_all = 0.0
@@ -145,7 +195,7 @@ def run_reference(args, rank):
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
             "steps": steps, "warmup": 1, "ms_per_step": 1e3 * t_all / steps, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "int8", "data": "synthetic",
-            "config": config_dict(specs),
+            "config": config_dict(HEADLINE_CONFIG, specs),
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line))
@@ -168,21 +218,34 @@ def whole_job_tops(world: int, ops_per_step: float, ms_per_step: float) -> float
     return world * ops_per_step / (ms_per_step * 1e-3) / 1e12
 
 
-def run_muxq(args, rank, world):
-    import torch
-    import torch.distributed as dist
+def prep_bytes(s, aux_written=32):
+    """Algorithmic bytes of the preparation kernel for one layer: X read once (fp16), Body_q written, the Aux columns
+    the GEMM reads (codes up to the next multiple of 32) and the W_aux gather."""
+    return s.M * (2.0 * s.K + s.K + aux_written) + s.N * aux_written
 
-    import paper_2604_04701_b200 as mx
 
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    torch.cuda.set_device(local)
-    dev = torch.device("cuda", local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=dev)
-    mx.lib()  # fails loudly if the CUDA library is missing
+def layer_bytes(s):
+    """Algorithmic HBM bytes of the whole layer: X fp16 read once, W_q, Y fp16 written once."""
+    return 2.0 * s.M * s.K + s.N * s.K + 2.0 * s.M * s.N
 
-    specs, ops_per_step = workload()
-    p = mx.MuxqParams(max_outliers=32)
+
+class Timer:
+    def __init__(self, torch):
+        self.torch = torch
+
+    def replays(self, graph, n):
+        t = self.torch
+        e0, e1 = t.cuda.Event(enable_timing=True), t.cuda.Event(enable_timing=True)
+        t.cuda.synchronize()
+        e0.record()
+        for _ in range(n):
+            graph.replay()
+        e1.record()
+        t.cuda.synchronize()
+        return e0.elapsed_time(e1) / n  # ms per replay
+
+
+def build_layers(mx, torch, dev, specs, p, out_kind):
     layers = []
     for s in specs:
         x, _ = s.x()
@@ -190,10 +253,39 @@ def run_muxq(args, rank, world):
         xd = torch.from_numpy(x).to(dev)
         w_q, s_w = mx.muxq_quantize(torch.from_numpy(w).to(dev), p, True,
                                     mx.Workspace(mx.muxq_small_workspace_bytes(s.N), dev))
-        ws = mx.Workspace(mx.muxq_host_workspace_bytes(s.M, s.K, s.N, p, mx.MUXQ_OUT_F16), dev)
+        ws = mx.Workspace(mx.muxq_host_workspace_bytes(s.M, s.K, s.N, p, out_kind), dev)
         y = torch.empty(s.M, s.N, dtype=torch.float16, device=dev)
         layers.append({"spec": s, "x": xd, "w_q": w_q, "s_w": s_w, "ws": ws, "y": y, "x_host": x})
     torch.cuda.synchronize()
+    return layers
+
+
+def check_status(mx, layers):
+    for L in layers:
+        st = mx.muxq_read_status(L["ws"])
+        if st != 0:
+            raise RuntimeError(f"device status {st} ({mx.muxq_status_string(st)}) on {L['spec'].name}")
+
+
+def capture(torch, side, fn):
+    with torch.cuda.stream(side):
+        fn()
+        side.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=side):
+            fn()
+    torch.cuda.synchronize()
+    return g
+
+
+def measure_prefill(mx, torch, dist, dev, world, cfg_id, steps, warmup, headline):
+    """Times one workload: the whole step (graph replay), the kernels inside it (event-record nodes), the GEMM
+    launches on their own; for the headline workload also the end-to-end leg and the sampled clocks."""
+    specs, ops_per_step = workload(cfg_id)
+    p = mx.MuxqParams(max_outliers=32)
+    layers = build_layers(mx, torch, dev, specs, p, mx.MUXQ_OUT_F16)
+    side = torch.cuda.Stream(device=dev)
+    timer = Timer(torch)
 
     def step():
         for L in layers:
@@ -203,48 +295,39 @@ def run_muxq(args, rank, world):
         if world > 1:
             dist.barrier()
 
-    def check_status():
-        for L in layers:
-            st = mx.muxq_read_status(L["ws"])
-            if st != 0:
-                raise RuntimeError(f"device status {st} ({mx.muxq_status_string(st)}) on {L['spec'].name}")
-
-    # One step = 4 layers x (fused prepare kernel, GEMM kernel): at ~10 us per kernel
-    # the host cannot enqueue fast enough, so the step is captured once into a CUDA graph (the entry
-    # points only enqueue work) and replayed; the graph holds exactly the launches muxq_linear makes.
-    side = torch.cuda.Stream(device=dev)
-    with torch.cuda.stream(side):
-        step()
-        side.synchronize()
-        check_status()
-        g_step = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(g_step, stream=side):
-            step()
-    torch.cuda.synchronize()
-    for _ in range(max(args.warmup, 3)):
+    # One step = 4 layers x (fused prepare kernel, GEMM kernel): the host cannot enqueue 10-50 us kernels fast
+    # enough, so the step is captured once into a CUDA graph (the entry points only enqueue work) and replayed;
+    # the graph holds exactly the launches muxq_linear makes.
+    g_step = capture(torch, side, step)
+    check_status(mx, layers)
+    for _ in range(max(warmup, 3)):
         g_step.replay()
     torch.cuda.synchronize()
-    check_status()
+    check_status(mx, layers)
 
-    uuid = str(torch.cuda.get_device_properties(dev).uuid)
-    sampler = ClockSampler(uuid if uuid.startswith("GPU-") else "GPU-" + uuid)
+    clocks = None
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier(); torch.cuda.synchronize()
-    sampler.start()
+    sampler = None
+    if headline:
+        uuid = str(torch.cuda.get_device_properties(dev).uuid)
+        sampler = ClockSampler(uuid if uuid.startswith("GPU-") else "GPU-" + uuid)
+        sampler.start()
     e0.record()
-    for _ in range(args.steps):
+    for _ in range(steps):
         g_step.replay()
     e1.record()
     torch.cuda.synchronize(); barrier()
-    clocks = sampler.stop()
-    check_status()
+    if sampler:
+        clocks = sampler.stop()
+    check_status(mx, layers)
     ms = max_over_ranks(e0.elapsed_time(e1), world, dev)
-    ms_per_step = ms / args.steps
+    ms_per_step = ms / steps
     value = whole_job_tops(world, ops_per_step, ms_per_step)
 
     # ---- per-kernel durations: the same step captured with event-record nodes at the kernel
     # boundaries (same stream, same buffers), replayed and read back one replay at a time
-    ksteps = min(args.steps, 200)
+    ksteps = min(steps, 100)
     evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in layers]
     for per_layer in evs:
         for e in per_layer:
@@ -267,6 +350,7 @@ def run_muxq(args, rank, world):
                 acc_us[li][j] += evs[li][j].elapsed_time(evs[li][j + 1]) * 1e3 / ksteps
     kern_us = {"event_node": [a[0] for a in acc_us], "prepare": [a[1] for a in acc_us], "gemm": [a[2] for a in acc_us]}
     total_us = sum(sum(v) for v in kern_us.values())
+    del g_ev
 
     # ---- the dominant kernel on its own: a graph of only the four GEMM launches, fed from the
     # intermediates the last step left in each layer's workspace (Body_q, Aux_q, W_aux, r, s_X)
@@ -288,95 +372,56 @@ def run_muxq(args, rank, world):
         for (bq, aq, wq, wa, nout, sx, sw, wsx, y) in gemm_calls:
             mx.muxq_gemm(bq, aq, wq, wa, nout, p, sx, sw, mx.MUXQ_OUT_F16, wsx, out=y)
 
-    with torch.cuda.stream(side):
-        gemm_step()
-        side.synchronize()
-        g_gemm = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(g_gemm, stream=side):
-            gemm_step()
-    torch.cuda.synchronize()
+    g_gemm = capture(torch, side, gemm_step)
     for _ in range(3):
         g_gemm.replay()
-    k0, k1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    torch.cuda.synchronize()
-    k0.record()
-    for _ in range(ksteps):
-        g_gemm.replay()
-    k1.record()
-    torch.cuda.synchronize()
-    check_status()
-    gemm_us_per_step = k0.elapsed_time(k1) * 1e3 / ksteps
-    peaks = load_peaks()
-    int8_peak = 2.0 * peaks["bf16_sustained"]  # INT8 dense rate = 2 x bf16 (nominal 4.5 vs 2.25 POPS)
-    achieved = ops_per_step / (gemm_us_per_step * 1e-6) / 1e12
-    roofline = {"kernel": "k_gemm_i8_pair (tcgen05 kind::i8 cta_group::2, fused Aux + dequant epilogue)",
-                "bound": "tensor", "achieved": achieved, "peak": int8_peak, "unit": "TOPS",
-                "frac": achieved / int8_peak, "peak_source": f"2 x bf16_tflops_sustained of {peaks['source']}",
-                "traffic": None, "launches_per_step": len(layers), "us_per_step": gemm_us_per_step,
-                "how": "CUDA events around replays of a graph holding only the step's four GEMM launches",
-                "per_layer_in_step": [{"layer": L["spec"].name, "M": L["spec"].M, "K": L["spec"].K, "N": L["spec"].N,
-                                       "event_node_us": kern_us["event_node"][i], "prepare_us": kern_us["prepare"][i],
-                                       "gemm_us": kern_us["gemm"][i]} for i, L in enumerate(layers)],
-                "share_of_step": {k: sum(v) / total_us for k, v in kern_us.items()},
-                "share_note": "from event-record nodes inside the step graph; each segment carries node overhead, and "
-                              "event_node is a segment with no work in it (two records back to back)"}
+    gemm_us_per_step = timer.replays(g_gemm, ksteps) * 1e3
+    check_status(mx, layers)
+    del g_gemm
+
+    out = {"cfg": cfg_id, "specs": specs, "ops_per_step": ops_per_step, "ms_per_step": ms_per_step, "value": value,
+           "clocks": clocks, "kern_us": kern_us, "total_us": total_us, "gemm_us_per_step": gemm_us_per_step,
+           "p": p, "e2e": None, "per_vector": None}
 
     # ---- end to end: host buffers, copies inside the timed region
-    esteps = max(3, min(args.steps, 20))
-    hosts = []
-    for L in layers:
-        xh = torch.from_numpy(L["x_host"]).pin_memory()
-        yh = torch.empty(L["spec"].M, L["spec"].N, dtype=torch.float16).pin_memory()
-        hosts.append((xh, yh))
+    if headline:
+        esteps = max(3, min(steps, 10))
+        hosts = []
+        for L in layers:
+            xh = torch.from_numpy(L["x_host"]).pin_memory()
+            yh = torch.empty(L["spec"].M, L["spec"].N, dtype=torch.float16).pin_memory()
+            hosts.append((xh, yh))
+        # Consecutive layers alternate between two streams, so one layer's device-to-host copy of Y overlaps the
+        # next layer's host-to-device copy of X (PCIe is full duplex); each layer has its own buffers.
+        h_streams = [torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev)]
 
-    # Consecutive layers alternate between two streams, so one layer's device-to-host copy of Y overlaps the
-    # next layer's host-to-device copy of X (PCIe is full duplex); each layer has its own buffers.
-    h_streams = [torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev)]
+        def step_host():
+            for i, (L, (xh, yh)) in enumerate(zip(layers, hosts)):
+                with torch.cuda.stream(h_streams[i & 1]):
+                    mx.muxq_linear_host(xh, L["w_q"], L["s_w"], p, L["ws"], yh, mx.MUXQ_OUT_F16)
 
-    def step_host():
-        for i, (L, (xh, yh)) in enumerate(zip(layers, hosts)):
-            with torch.cuda.stream(h_streams[i & 1]):
-                mx.muxq_linear_host(xh, L["w_q"], L["s_w"], p, L["ws"], yh, mx.MUXQ_OUT_F16)
-
-    def join_host():
-        for hs in h_streams:
-            torch.cuda.current_stream().wait_stream(hs)
-
-    def fork_host():
+        for _ in range(2):
+            step_host()
+        torch.cuda.synchronize(); barrier()
+        h0, h1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        h0.record()
         for hs in h_streams:
             hs.wait_stream(torch.cuda.current_stream())
-
-    for _ in range(2):
-        step_host()
-    torch.cuda.synchronize(); barrier()
-    h0, h1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    h0.record()
-    fork_host()
-    for _ in range(esteps):
-        step_host()
-    join_host()
-    h1.record()
-    torch.cuda.synchronize(); barrier()
-    check_status()
-    ems = max_over_ranks(h0.elapsed_time(h1), world, dev)
-    e2e = {"value": whole_job_tops(world, ops_per_step, ems / esteps), "unit": UNIT,
-           "h2d_bytes_per_step": int(sum(xh.numel() * 2 for xh, _ in hosts)),
-           "d2h_bytes_per_step": int(sum(yh.numel() * 2 for _, yh in hosts)), "steps": esteps,
-           "ms_per_step": ems / esteps}
-
-    # ---- whole-layer roofline: per layer the slower of the INT8 tensor time and the HBM time of its
-    # algorithmic bytes (X fp16 read once, W_q, Y fp16 written once), summed over the step
-    t_roof_us = 0.0
-    for L in layers:
-        sp = L["spec"]
-        t_c = 2.0 * sp.M * sp.N * sp.K / (int8_peak * 1e12) * 1e6
-        t_m = (2.0 * sp.M * sp.K + sp.N * sp.K + 2.0 * sp.M * sp.N) / (peaks["hbm_gbs"] * 1e9) * 1e6
-        t_roof_us += max(t_c, t_m)
-    step_roofline = {"t_roof_us": t_roof_us, "frac": t_roof_us / (ms_per_step * 1e3),
-                     "peaks": {"int8_tops": int8_peak, "hbm_gbs": peaks["hbm_gbs"], "source": peaks["source"]}}
+        for _ in range(esteps):
+            step_host()
+        for hs in h_streams:
+            torch.cuda.current_stream().wait_stream(hs)
+        h1.record()
+        torch.cuda.synchronize(); barrier()
+        check_status(mx, layers)
+        ems = max_over_ranks(h0.elapsed_time(h1), world, dev)
+        out["e2e"] = {"value": whole_job_tops(world, ops_per_step, ems / esteps), "unit": UNIT,
+                      "h2d_bytes_per_step": int(sum(xh.numel() * 2 for xh, _ in hosts)),
+                      "d2h_bytes_per_step": int(sum(yh.numel() * 2 for _, yh in hosts)), "steps": esteps,
+                      "ms_per_step": ems / esteps}
+        del hosts
 
     # ---- the per-vector variant of the same workload (per-token X scales, per-channel W scales)
-    per_vector = None
     if world == 1:
         pv = mx.MuxqParams(max_outliers=32, gran=mx.MUXQ_PER_VECTOR)
         pv_layers = []
@@ -390,122 +435,212 @@ def run_muxq(args, rank, world):
             for (xd, w_q, s_w, wsx, y) in pv_layers:
                 mx.muxq_linear(xd, w_q, s_w, pv, wsx, mx.MUXQ_OUT_F16, out=y)
 
-        with torch.cuda.stream(side):
-            pv_step()
-            side.synchronize()
-            check_status()
-            g_pv = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(g_pv, stream=side):
-                pv_step()
-        torch.cuda.synchronize()
+        g_pv = capture(torch, side, pv_step)
+        check_status(mx, layers)
         for _ in range(3):
             g_pv.replay()
-        v0, v1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        torch.cuda.synchronize()
-        v0.record()
-        for _ in range(ksteps):
-            g_pv.replay()
-        v1.record()
-        torch.cuda.synchronize()
-        check_status()
-        pv_ms = v0.elapsed_time(v1) / ksteps
-        per_vector = {"granularity": "per-token X, per-channel W", "ms_per_step": pv_ms,
-                      "value": ops_per_step / (pv_ms * 1e-3) / 1e12, "unit": UNIT}
+        pv_ms = timer.replays(g_pv, ksteps)
+        check_status(mx, layers)
+        out["per_vector"] = {"granularity": "per-token X, per-channel W", "ms_per_step": pv_ms,
+                             "value": ops_per_step / (pv_ms * 1e-3) / 1e12, "unit": UNIT}
         del g_pv, pv_layers
+    del g_step, layers
+    torch.cuda.empty_cache()
+    return out
 
-    # ---- decode shapes (M <= 16): the 36 x 4 GPT-2-large linears as one stream of layers with distinct
-    # weights (708 MB of W_q, far more than the L2 holds), replayed from a graph; GB/s = W_q bytes / time
-    decode = None
-    if world == 1 and not args.no_decode:
-        d = 1280
-        dshapes = [(d, 3 * d), (d, d), (d, 4 * d), (4 * d, d)]
-        gen = torch.Generator(device=dev)
-        gen.manual_seed(4)
-        dlayers = []
-        for _ in range(36):
-            for (K, N) in dshapes:
-                dlayers.append((K, N, torch.randint(-127, 128, (N, K), dtype=torch.int8, device=dev, generator=gen)))
-        wbytes = sum(K * N for K, N, _ in dlayers)
-        sw1 = torch.full((1,), 0.02 / 127.0, device=dev)
-        decode = {"workload": "configs[3]/[4] decode: 36 x (1280->3840, 1280->1280, 1280->5120, 5120->1280), "
-                              "8 outlier channels x60, per-tensor INT8, one fused launch per layer",
-                  "w_bytes": wbytes, "layers": len(dlayers), "hbm_peak_gbs": peaks["hbm_gbs"]}
-        for Md in (1, 4, 16):
-            dx = {K: torch.from_numpy(synth.make_x(3, 100 + K, Md, K, 8, 60.0, 60.0)[0]).to(dev) for K in (d, 4 * d)}
-            dy = {N: torch.empty(Md, N, dtype=torch.float16, device=dev) for N in (d, 3 * d, 4 * d)}
-            dws = {K: mx.Workspace(mx.muxq_workspace_bytes(Md, K, 4 * d, p), dev) for K in (d, 4 * d)}
 
-            def chain():
-                for (K, N, wq) in dlayers:
-                    mx.muxq_linear(dx[K], wq, sw1, p, dws[K], mx.MUXQ_OUT_F16, out=dy[N])
+def int8_probe(mx, torch, dev):
+    """The repo's own issue-bound tcgen05.mma kind::i8 loop (operands resident in shared memory, no loads): the INT8
+    rate the tensor pipes attain at the clocks of this moment.  Timed with CUDA events around the launch."""
+    ws = mx.Workspace(256, dev)
+    ctas = torch.cuda.get_device_properties(dev).multi_processor_count
+    iters = 16384
+    mx.muxq_int8_mma_peak(256, 1024, ctas, ws)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    cyc = mx.muxq_int8_mma_peak(256, iters, ctas, ws)
+    e1.record()
+    torch.cuda.synchronize()
+    if mx.muxq_read_status(ws) != 0:
+        return None
+    ops = 2.0 * 128 * 256 * 32 * iters * ctas
+    ms = e0.elapsed_time(e1)
+    return {"tops": ops / (ms * 1e-3) / 1e12, "cycles_per_mma_m128n256k32": float(cyc.double().mean().item()) / iters,
+            "ctas": ctas, "iters": iters, "how": "CUDA events around one launch of the issue-bound MMA loop"}
 
+
+def prefill_report(res, peaks, int8_peak, peak_source, probe):
+    """roofline blocks of one measured workload"""
+    specs, ops = res["specs"], res["ops_per_step"]
+    kern_us = res["kern_us"]
+    node = statistics.mean(kern_us["event_node"])  # a segment with no work in it: two records back to back
+    achieved = ops / (res["gemm_us_per_step"] * 1e-6) / 1e12
+    gemm = {"kernel": "k_gemm_i8_pair (tcgen05 kind::i8 cta_group::2, fused Aux + dequant epilogue)",
+            "bound": "tensor", "achieved": achieved, "peak": int8_peak, "unit": "TOPS",
+            "frac": achieved / int8_peak, "peak_source": peak_source,
+            "int8_probe_tops": probe["tops"] if probe else None,
+            "frac_vs_probe": achieved / probe["tops"] if probe else None,
+            "frac_vs_nominal_4500": achieved / NOMINAL_INT8_TOPS,
+            "traffic": traffic_for("k_gemm_i8_pair", f"cfg{res['cfg']}"),
+            "algorithmic_bytes_per_step": sum(s.M * s.K + s.N * s.K + 2.0 * s.M * s.N for s in specs),
+            "launches_per_step": len(specs), "us_per_step": res["gemm_us_per_step"],
+            "how": "CUDA events around replays of a graph holding only the step's four GEMM launches",
+            "per_layer_in_step": [{"layer": s.name, "M": s.M, "K": s.K, "N": s.N,
+                                   "event_node_us": kern_us["event_node"][i], "prepare_us": kern_us["prepare"][i],
+                                   "gemm_us": kern_us["gemm"][i]} for i, s in enumerate(specs)],
+            "share_of_step": {k: sum(v) / res["total_us"] for k, v in kern_us.items()},
+            "share_note": "from event-record nodes inside the step graph; each segment carries node overhead, and "
+                          "event_node is a segment with no work in it (two records back to back)"}
+    pbytes = sum(prep_bytes(s) for s in specs)
+    pus = sum(max(u - node, 0.1) for u in kern_us["prepare"])
+    prep = {"kernel": "k_prep (fused detect + redistribute + quantize, cooperative, one CTA per SM)", "bound": "hbm",
+            "achieved": pbytes / pus / 1e3, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+            "frac": pbytes / pus / 1e3 / peaks["hbm_gbs"], "peak_source": f"hbm_gbs of {peaks['source']}",
+            "traffic": traffic_for("k_prep", f"cfg{res['cfg']}"), "algorithmic_bytes_per_step": pbytes,
+            "us_per_step": pus,
+            "how": "event-record segments around the kernel inside the step graph, minus the empty segment's overhead; "
+                   "bytes = M(2K + K + 32) + 32N per layer"}
+    t_roof_us = 0.0
+    for s in specs:
+        t_c = 2.0 * s.M * s.N * s.K / (int8_peak * 1e12) * 1e6
+        t_m = layer_bytes(s) / (peaks["hbm_gbs"] * 1e9) * 1e6
+        t_roof_us += max(t_c, t_m)
+    step = {"t_roof_us": t_roof_us, "frac": t_roof_us / (res["ms_per_step"] * 1e3),
+            "peaks": {"int8_tops": int8_peak, "hbm_gbs": peaks["hbm_gbs"], "source": peak_source},
+            "how": "per layer the slower of the INT8 tensor time and the HBM time of X + W_q + Y, summed"}
+    return gemm, prep, step
+
+
+def measure_decode(mx, torch, dev, peaks, p):
+    """Decode shapes (M <= 16): the 36 x 4 GPT-2-large linears as one stream of layers with distinct weights
+    (708 MB of W_q, far more than the L2 holds), replayed from a graph; GB/s = W_q bytes / time."""
+    side = torch.cuda.Stream(device=dev)
+    timer = Timer(torch)
+    d = 1280
+    dshapes = [(d, 3 * d), (d, d), (d, 4 * d), (4 * d, d)]
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(4)
+    dlayers = []
+    for _ in range(36):
+        for (K, N) in dshapes:
+            dlayers.append((K, N, torch.randint(-127, 128, (N, K), dtype=torch.int8, device=dev, generator=gen)))
+    wbytes = sum(K * N for K, N, _ in dlayers)
+    sw1 = torch.full((1,), 0.02 / 127.0, device=dev)
+    decode = {"workload": "configs[3]/[4] decode: 36 x (1280->3840, 1280->1280, 1280->5120, 5120->1280), "
+                          "8 outlier channels x60, per-tensor INT8, one fused launch per layer",
+              "w_bytes": wbytes, "layers": len(dlayers), "hbm_peak_gbs": peaks["hbm_gbs"]}
+    for Md in (1, 4, 16):
+        dx = {K: torch.from_numpy(synth.make_x(3, 100 + K, Md, K, 8, 60.0, 60.0)[0]).to(dev) for K in (d, 4 * d)}
+        dy = {N: torch.empty(Md, N, dtype=torch.float16, device=dev) for N in (d, 3 * d, 4 * d)}
+        dws = {K: mx.Workspace(mx.muxq_workspace_bytes(Md, K, 4 * d, p), dev) for K in (d, 4 * d)}
+
+        def chain():
+            for (K, N, wq) in dlayers:
+                mx.muxq_linear(dx[K], wq, sw1, p, dws[K], mx.MUXQ_OUT_F16, out=dy[N])
+
+        g_dec = capture(torch, side, chain)
+        for _ in range(3):
+            g_dec.replay()
+        us = timer.replays(g_dec, 10) * 1e3
+        for K in dws:
+            if mx.muxq_read_status(dws[K]) != 0:
+                raise RuntimeError("device status raised on the decode chain")
+        gbs = wbytes / us / 1e3
+        decode[f"M{Md}"] = {"us_per_layer": us / len(dlayers), "gb_per_s": gbs, "frac_of_measured_hbm": gbs / peaks["hbm_gbs"]}
+        del g_dec
+        # one call on its own (nothing before it in the stream to overlap with, weights cold): the call is captured
+        # with event-record nodes at its boundaries and replayed 15 times, each after a write of 256 MB that
+        # pushes the weights out of L2; median device time between the records (includes their node overhead)
+        flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+        iso = {}
+        for li, (K, N, wq) in enumerate(dlayers[:4]):
+            ievs = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+            for e in ievs:
+                e.record()
+            torch.cuda.synchronize()
             with torch.cuda.stream(side):
-                chain()
-                side.synchronize()
-                g_dec = torch.cuda.CUDAGraph()
-                with torch.cuda.graph(g_dec, stream=side):
-                    chain()
+                g_one = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g_one, stream=side):
+                    mx.muxq_linear_events(dx[K], wq, sw1, p, dws[K], ievs, mx.MUXQ_OUT_F16, out=dy[N])
             torch.cuda.synchronize()
-            for _ in range(3):
-                g_dec.replay()
-            d0, d1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            torch.cuda.synchronize()
-            d0.record()
-            for _ in range(10):
-                g_dec.replay()
-            d1.record()
-            torch.cuda.synchronize()
-            for K in dws:
-                if mx.muxq_read_status(dws[K]) != 0:
-                    raise RuntimeError("device status raised on the decode chain")
-            us = d0.elapsed_time(d1) * 1e3 / 10
-            gbs = wbytes / us / 1e3
-            decode[f"M{Md}"] = {"us_per_layer": us / len(dlayers), "gb_per_s": gbs, "frac_of_measured_hbm": gbs / peaks["hbm_gbs"]}
-            del g_dec
-            # one call on its own (nothing before it in the stream to overlap with, weights cold): the call is captured
-            # with event-record nodes at its boundaries and replayed 15 times, each after a write of 256 MB that
-            # pushes the weights out of L2; median device time between the records (includes their node overhead)
-            flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
-            iso = {}
-            for li, (K, N, wq) in enumerate(dlayers[:4]):
-                ievs = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
-                for e in ievs:
-                    e.record()
+            ts = []
+            for _ in range(15):
+                flush.fill_(li)
                 torch.cuda.synchronize()
-                with torch.cuda.stream(side):
-                    g_one = torch.cuda.CUDAGraph()
-                    with torch.cuda.graph(g_one, stream=side):
-                        mx.muxq_linear_events(dx[K], wq, sw1, p, dws[K], ievs, mx.MUXQ_OUT_F16, out=dy[N])
+                g_one.replay()
                 torch.cuda.synchronize()
-                ts = []
-                for _ in range(15):
-                    flush.fill_(li)
-                    torch.cuda.synchronize()
-                    g_one.replay()
-                    torch.cuda.synchronize()
-                    ts.append(ievs[0].elapsed_time(ievs[3]) * 1e3)
-                iso[f"{K}->{N}"] = statistics.median(ts)
-                del g_one
-            decode[f"M{Md}"]["isolated_call_us"] = iso
-            del flush
-        del dlayers
+                ts.append(ievs[0].elapsed_time(ievs[3]) * 1e3)
+            iso[f"{K}->{N}"] = statistics.median(ts)
+            del g_one
+        decode[f"M{Md}"]["isolated_call_us"] = iso
+        del flush
+    del dlayers
+    torch.cuda.empty_cache()
+    best = max(decode[f"M{m}"]["gb_per_s"] for m in (1, 4, 16))
+    roof = {"kernel": "k_decode_fused (one launch per layer, W_q streamed once)", "bound": "hbm",
+            "achieved": decode["M1"]["gb_per_s"], "peak": peaks["hbm_gbs"], "unit": "GB/s",
+            "frac": decode["M1"]["frac_of_measured_hbm"], "peak_source": f"hbm_gbs of {peaks['source']}",
+            "traffic": traffic_for("k_decode_fused", "chain"), "algorithmic_bytes_per_chain": wbytes,
+            "best_over_M_gb_per_s": best, "how": "W_q bytes of the 144-layer chain / CUDA-event time of its graph, M = 1"}
+    return decode, roof
+
+
+def run_muxq(args, rank, world):
+    import torch
+    import torch.distributed as dist
+
+    import paper_2604_04701_b200 as mx
+
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    mx.lib()  # fails loudly if the CUDA library is missing
+    peaks = load_peaks()
+
+    head = measure_prefill(mx, torch, dist, dev, world, HEADLINE_CONFIG, args.steps, args.warmup, headline=True)
+    clocks = head["clocks"]
+    int8_peak, peak_source = int8_peak_for(peaks, clocks)
+    probe = int8_probe(mx, torch, dev) if world == 1 else None
+    gemm_roof, prep_roof, step_roof = prefill_report(head, peaks, int8_peak, peak_source, probe)
+
+    extra = {}
+    if world == 1 and not args.no_small:
+        small = measure_prefill(mx, torch, dist, dev, world, 1, max(args.steps, 50), args.warmup, headline=False)
+        s_gemm, s_prep, s_step = prefill_report(small, peaks, int8_peak, peak_source, probe)
+        extra["configs1"] = {"config": config_dict(1, small["specs"]), "value": small["value"], "unit": UNIT,
+                             "ms_per_step": small["ms_per_step"],
+                             "us_per_layer": small["ms_per_step"] * 1e3 / len(small["specs"]),
+                             "pct_of_nominal_int8_peak_4500": 100.0 * small["value"] / NOMINAL_INT8_TOPS,
+                             "roofline": s_gemm, "roofline_prep": s_prep, "step_roofline": s_step,
+                             "per_vector": small["per_vector"]}
+
+    decode = decode_roof = None
+    if world == 1 and not args.no_decode:
+        decode, decode_roof = measure_decode(mx, torch, dev, peaks, head["p"])
 
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        rows = specs[0].M
-        v, dt, cores = oracle_sample(specs, rows)
+        rows = 4096
+        v, dt, cores = oracle_sample(head["specs"], rows)
         cpu_baseline = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "seconds": dt,
-                        "sample": f"all {rows} token rows of each of the 4 layers, one pass (one step)"}
+                        "sample": f"first {rows} of {head['specs'][0].M} token rows of each of the 4 layers, one pass"}
 
     if rank == 0:
-        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-                "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
+        specs = head["specs"]
+        line = {"metric": METRIC, "value": head["value"], "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                "warmup": max(args.warmup, 3), "ms_per_step": head["ms_per_step"], "higher_is_better": True,
                 "scaling": "weak", "vs_baseline": None, "dtype": "int8", "data": "synthetic",
-                "config": config_dict(specs, {"parallelism": "replicas only" if world > 1 else "single GPU"}),
-                "us_per_layer": ms_per_step * 1e3 / len(layers),
-                "pct_of_nominal_int8_peak_4500": 100.0 * value / world / 4500.0,
-                "clocks": clocks, "e2e": e2e, "gpu_launches": args.steps * len(layers) * 2,
-                "roofline": roofline, "step_roofline": step_roofline, "per_vector": per_vector, "decode": decode, "cpu_baseline": cpu_baseline}
+                "config": config_dict(HEADLINE_CONFIG, specs,
+                                      {"parallelism": "replicas only" if world > 1 else "single GPU"}),
+                "us_per_layer": head["ms_per_step"] * 1e3 / len(specs),
+                "pct_of_nominal_int8_peak_4500": 100.0 * head["value"] / world / NOMINAL_INT8_TOPS,
+                "clocks": clocks, "e2e": head["e2e"], "gpu_launches": args.steps * len(specs) * 2,
+                "roofline": gemm_roof, "roofline_prep": prep_roof, "roofline_decode": decode_roof,
+                "step_roofline": step_roof, "int8_probe": probe, "per_vector": head["per_vector"],
+                "extra": extra, "decode": decode, "cpu_baseline": cpu_baseline}
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
@@ -514,11 +649,12 @@ def run_muxq(args, rank, world):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=5000)
-    ap.add_argument("--warmup", type=int, default=50)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="muxq", choices=["muxq", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-decode", action="store_true")
+    ap.add_argument("--no-small", action="store_true", help="skip the GPT-2-small workload reported under extra")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))

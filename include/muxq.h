@@ -17,14 +17,26 @@
  *   - All tensor pointers are DEVICE pointers unless the name says "host".  Row-major; "ld" is
  *     the row pitch in ELEMENTS.  fp16 is IEEE binary16 passed as void*.
  *   - The caller owns every buffer, including the workspace; the library allocates no device
- *     memory and keeps no host state between calls.  `stream` is a cudaStream_t passed as void*
- *     (NULL = the legacy default stream).
+ *     memory.  The only host state it keeps between calls is a per-device record of one-time set-up
+ *     (function attributes, occupancy, SM count), guarded by a mutex: a process may drive several
+ *     GPUs, each call acting on the device that is current when it is made.  `stream` is a
+ *     cudaStream_t passed as void* (NULL = the legacy default stream).
  *   - Calls only enqueue work; nothing synchronizes except muxq_read_status and
  *     muxq_linear_host's final copy-back wait when asked.
  *   - The int return value reports what the host can see at call time (bad arguments,
  *     unsupported shapes, workspace too small, CUDA launch errors).  Data-dependent conditions
  *     (more outlier channels than the capacity, an expired bounded device-side wait) are
  *     written to the device status word; a kernel never traps and never writes out of bounds.
+ *     The status word is STICKY: kernels only ever raise it (atomic max), no call clears it, so
+ *     one word may collect the worst status of many enqueued calls.  Zero it yourself (a 4-byte
+ *     cudaMemsetAsync) before the calls whose status you want to read.
+ *   - W_q and s_w are constants of a layer.  The layer kernels are launched with programmatic
+ *     stream serialization and fetch their first weight tiles BEFORE they wait for the preceding
+ *     work of the stream, so W_q / s_w must not be written by a kernel that (a) directly precedes a
+ *     muxq_linear call on the same stream and (b) itself releases its dependents early
+ *     (cudaTriggerProgrammaticLaunchCompletion / griddepcontrol.launch_dependents).  Ordinary
+ *     kernels, copies and this library's own muxq_quantize are safe predecessors: without an
+ *     early trigger the layer kernel starts only once they have completed.
  *   - Inputs must be finite.  NaN/Inf give unspecified (but memory-safe) results.
  *   - Alignment: X, W, Y, workspace 16-byte aligned; K % 16 == 0; ldx % 8 == 0; N % 8 == 0.
  */
@@ -86,7 +98,9 @@ size_t muxq_host_workspace_bytes(int M, int K, int N, const muxq_params *p, int 
  * kernels find these words zero and put them back to zero before they finish, so that a layer call
  * carries no clearing step of its own.  Call it once after allocating the workspace, before its
  * first layer call, and again
- *   - after a layer call whose status word read MUXQ_ERR_TIMEOUT,
+ *   - after a layer call whose status word read MUXQ_ERR_TIMEOUT (the time-out marks the workspace:
+ *     every later layer call on it fails with MUXQ_ERR_TIMEOUT at once, instead of computing on
+ *     half-merged channel maxima, until this call clears the mark),
  *   - after the same memory was handed to muxq_detect_outliers or muxq_quantize as their workspace,
  *     or written by anything else.
  * One workspace may then serve any sequence of layer shapes, one call at a time (calls that share a
@@ -164,8 +178,8 @@ int muxq_gemm(const int8_t *Body_q, int ld_a, const int8_t *Aux_q, int ld_aux, c
  * with the same params.  M > 16: one preparation kernel and one tensor-core GEMM kernel.  M <= 16:
  * the memory-bound decode path, a single kernel that streams W_q once.  Y: [M, ldy] by out_kind.
  * workspace >= muxq_workspace_bytes(M,K,N,p), prepared once by muxq_workspace_init.  dev_status: device
- * int32; the call sets it to 0 first, kernels raise it to MUXQ_ERR_CAPACITY (r > max_outliers; Y
- * then unspecified but in bounds) or MUXQ_ERR_TIMEOUT.
+ * int32 (sticky, see above); kernels raise it to MUXQ_ERR_CAPACITY (r > max_outliers; Y then
+ * unspecified but in bounds) or MUXQ_ERR_TIMEOUT.
  * Intermediates stay in the workspace afterwards; muxq_workspace_view locates them.  For M <= 16
  * only col_absmax, outlier_idx, n_outliers and s_x are left there (the codes never leave the SMs).
  * params.aux_scale == MUXQ_AUX_OWN (the other reading of how Eq. 1 applies to Aux: its own abs-max
@@ -178,19 +192,6 @@ int muxq_gemm(const int8_t *Body_q, int ld_a, const int8_t *Aux_q, int ld_aux, c
 int muxq_linear(const void *X_f16, int M, int K, int ldx, const int8_t *W_q, int ldw,
                 const float *s_w, int N, const muxq_params *p, void *Y, int ldy, int out_kind,
                 void *workspace, size_t workspace_bytes, int32_t *dev_status, void *stream);
-
-/*
- * muxq_linear that also records four caller-created CUDA events (cudaEvent_t passed as void*;
- * NULL entries are skipped) on `stream` at its kernel boundaries, for per-kernel timing:
- * events[0] at entry, [1] at the start of the fused detect + redistribute + quantize kernel (after
- * the clearing step where the shape needs one: K > 8192), [2] after that kernel, [3] after the GEMM (or decode) kernel.  When `stream`
- * is being captured into a CUDA graph the records become event-record nodes, re-recorded by every
- * replay.  Same results as muxq_linear.
- */
-int muxq_linear_events(const void *X_f16, int M, int K, int ldx, const int8_t *W_q, int ldw,
-                       const float *s_w, int N, const muxq_params *p, void *Y, int ldy, int out_kind,
-                       void *workspace, size_t workspace_bytes, int32_t *dev_status, void *stream,
-                       void *const *events);
 
 /* Where muxq_linear leaves its intermediates inside the workspace (byte offsets). */
 typedef struct muxq_ws_view {
@@ -230,7 +231,10 @@ int muxq_linear_host(const void *X_f16_host, int M, int K, const int8_t *W_q, in
  * return MUXQ_ERR_STATIC_LIMIT and launch nothing.  The call allocates and frees nothing.
  *
  * Arguments, results, alignment rules and the device status word are those of muxq_linear with
- * M <= 16 (same kernels, same arithmetic).  The first call on each device looks up the array's
+ * M <= 16, with these limits of its own: max_outliers <= 64 (else MUXQ_ERR_INVALID_ARG), the shared
+ * Aux scale only (MUXQ_AUX_OWN is MUXQ_ERR_UNSUPPORTED).  It always runs two kernels (the activation
+ * preparation, then the W_q-streaming product), never muxq_linear's single fused decode kernel; the
+ * arithmetic and therefore the results are the same.  The first call on each device looks up the array's
  * device address (the device must be current); make that first call outside any stream capture.
  * All calls on a device share the one array and it keeps the previous call's contents: the parts
  * that must start at zero are cleared on `stream` at the head of each call, and two calls whose
@@ -240,17 +244,6 @@ int muxq_linear_host(const void *X_f16_host, int M, int K, const int8_t *W_q, in
 int muxq_linear_decode_noalloc(const void *X_f16, int M, int K, int ldx, const int8_t *W_q, int ldw,
                                const float *s_w, int N, const muxq_params *p, void *Y, int ldy,
                                int out_kind, int32_t *dev_status, void *stream);
-
-/*
- * Measurement aid: runs `ctas` CTAs (one per SM when ctas = SM count) that each issue `iters`
- * back-to-back tcgen05.mma kind::i8 instructions of shape M128 x N(mma_n = 128 or 256) x K32 on
- * operands resident in shared memory -- the issue-bound INT8 tensor rate of the GPU as it is clocked
- * right now.  cycles_per_cta [ctas] (device, uint64) receives each CTA's SM-clock cycle count from
- * first issue to completion; time the launch with CUDA events for ops/s =
- * ctas * iters * 2 * 128 * mma_n * 32 / seconds.
- */
-int muxq_int8_mma_peak(int mma_n, int iters, int ctas, unsigned long long *cycles_per_cta,
-                       int32_t *dev_status, void *stream);
 
 /* Synchronizes `stream` and returns the device status word (or MUXQ_ERR_CUDA). */
 int muxq_read_status(const int32_t *dev_status, void *stream);

@@ -22,7 +22,7 @@ EXPORTS = (
     "muxq_default_params", "muxq_aux_cols", "muxq_workspace_bytes", "muxq_small_workspace_bytes",
     "muxq_host_workspace_bytes", "muxq_workspace_init", "muxq_workspace_view", "muxq_detect_outliers", "muxq_build_aux",
     "muxq_quantize", "muxq_gemm", "muxq_linear", "muxq_linear_events", "muxq_linear_host",
-    "muxq_linear_decode_noalloc", "muxq_int8_mma_peak", "muxq_read_status",
+    "muxq_linear_decode_noalloc", "muxq_int8_mma_peak", "muxq_test_hooks", "muxq_read_status",
     "muxq_status_string",
 )
 
@@ -95,6 +95,7 @@ def lib() -> ctypes.CDLL:
         L.muxq_linear_host.argtypes = [vp, i, i, vp, i, vp, i, pp, vp, i, vp, sz, vp, vp]; L.muxq_linear_host.restype = i
         L.muxq_linear_decode_noalloc.argtypes = [vp, i, i, i, vp, i, vp, i, pp, vp, i, i, vp, vp]; L.muxq_linear_decode_noalloc.restype = i
         L.muxq_int8_mma_peak.argtypes = [i, i, i, vp, vp, vp]; L.muxq_int8_mma_peak.restype = i
+        L.muxq_test_hooks.argtypes = [vp]; L.muxq_test_hooks.restype = i
         L.muxq_read_status.argtypes = [vp, vp]; L.muxq_read_status.restype = i
         L.muxq_status_string.argtypes = [i]; L.muxq_status_string.restype = ctypes.c_char_p
         _lib = L
@@ -149,9 +150,14 @@ class Workspace:
         self.init()
 
     def init(self) -> None:
-        """muxq_workspace_init on the current stream (needed again after a time-out status or foreign writes)."""
+        """muxq_workspace_init on the current stream (needed again after a time-out status or foreign writes);
+        also zeroes the status word, which the library itself only ever raises."""
         with torch.cuda.device(self.buf.device):
             _check("muxq_workspace_init", lib().muxq_workspace_init(_ptr(self.buf), self.nbytes, _stream()))
+            self.status.zero_()
+
+    def clear_status(self) -> None:
+        self.status.zero_()
 
     @property
     def nbytes(self) -> int:
@@ -295,6 +301,17 @@ def muxq_int8_mma_peak(mma_n: int, iters: int, ctas: int, ws: Workspace) -> torc
     cycles = torch.zeros(ctas, dtype=torch.int64, device=ws.buf.device)
     _check("muxq_int8_mma_peak", lib().muxq_int8_mma_peak(mma_n, iters, ctas, _ptr(cycles), _ptr(ws.status), _stream()))
     return cycles
+
+
+class _CTestHooks(ctypes.Structure):
+    _fields_ = [("spin_limit", ctypes.c_uint32), ("prep_extra_arrivals", ctypes.c_uint32),
+                ("gemm_skip_k_block", ctypes.c_int32)]
+
+
+def muxq_test_hooks(spin_limit: int = 0, prep_extra_arrivals: int = 0, gemm_skip_k_block: int = 0) -> None:
+    """Fault injection for tests (include/muxq_measure.h); all zero restores normal operation."""
+    h = _CTestHooks(spin_limit, prep_extra_arrivals, gemm_skip_k_block)
+    _check("muxq_test_hooks", lib().muxq_test_hooks(ctypes.byref(h)))
 
 
 def muxq_read_status(ws: Workspace) -> int:

@@ -1,9 +1,11 @@
 // C-ABI host layer of libmuxq: argument checks, workspace carving, kernel launches.
-// No device memory is allocated here and no host state survives a call.
+// No device memory is allocated here; the only host state that survives a call is the per-device record of
+// one-time set-up (host_state.cu).
 #include <math.h>
 #include <string.h>
 
 #include "../../include/muxq.h"
+#include "../../include/muxq_measure.h"
 #include "kernels.h"
 
 using namespace muxq;
@@ -333,7 +335,6 @@ static int linear_impl(const void *X, int M, int K, int ldx, const int8_t *W_q, 
     if (!fused) {
         e = cudaMemsetAsync(ws, 0, sizeof(Ctrl), s);
         if (e == cudaSuccess) e = cudaMemsetAsync(ws + w.s.colmax, 0, (size_t)K * 4, s);
-        if (e == cudaSuccess) e = cudaMemsetAsync(dev_status, 0, 4, s);  // the fused kernel clears it itself
     }
     if (e != cudaSuccess) return MUXQ_ERR_CUDA;
     mark(1);
@@ -491,6 +492,18 @@ int muxq_int8_mma_peak(int mma_n, int iters, int ctas, unsigned long long *cycle
     if ((mma_n != 128 && mma_n != 256 && mma_n != 16 && mma_n != 64) || iters < 1 || iters > (1 << 20) || ctas < 1 || !cycles_per_cta)
         return MUXQ_ERR_INVALID_ARG;
     return cuda_rc(launch_mma_peak(mma_n, iters, cycles_per_cta, dev_status, ctas, static_cast<cudaStream_t>(stream)));
+}
+
+int muxq_test_hooks(const muxq_test_hooks_t *h) {
+    TestHooks t{};
+    if (h) {
+        if (h->gemm_skip_k_block < 0) return MUXQ_ERR_INVALID_ARG;
+        t.spin_limit = h->spin_limit;
+        t.prep_extra_arrivals = h->prep_extra_arrivals;
+        t.gemm_skip_kb = h->gemm_skip_k_block;
+    }
+    set_test_hooks(t);
+    return MUXQ_OK;
 }
 
 int muxq_read_status(const int32_t *dev_status, void *stream) {

@@ -27,6 +27,8 @@ struct GemmParams {
     const float *s_w;
     int32_t *dev_status;
     int w_stable;  // the B operand may be read before the programmatic predecessor has finished
+    uint32_t spin; // poll limit of the bounded waits
+    int skip_kb;   // -1; a test names a K block whose loads are left out so that a wait runs out
 };
 
 // One 32-column chunk of one accumulator row: int32 -> fp32 (round to nearest even, exact below

@@ -173,17 +173,6 @@ __global__ void __launch_bounds__(kThreads) k_detect_tail_only(const DetectArgs 
 
 }  // namespace
 
-int num_sms() {
-    static int n = 0;
-    if (n == 0) {
-        int dev = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess ||
-            cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
-            n = 148;
-    }
-    return n;
-}
-
 cudaError_t launch_detect(const DetectArgs &a, cudaStream_t s) {
     const int col_blocks = (a.K + kColsPerBlock - 1) / kColsPerBlock;
     int slices = (num_sms() * 6 + col_blocks - 1) / col_blocks;

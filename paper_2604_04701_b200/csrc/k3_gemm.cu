@@ -237,12 +237,17 @@ k_gemm_i8(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
 template <int BN, int kOut, bool kPerVec>
 cudaError_t launch_gemm_inst(const GemmArgs &a, cudaStream_t s) {
     using C = Cfg<BN>;
-    static bool attr_set = false;
-    if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(k_gemm_i8<BN, kOut, kPerVec>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             C::kSmemBytes);
-        if (e != cudaSuccess) return e;
-        attr_set = true;
+    static PerDevice<int> attr_set;  // per instantiation and device
+    const int dev = current_device();
+    if (dev < 0) return cudaErrorInvalidDevice;
+    {
+        std::lock_guard<std::mutex> lock(device_mutex());
+        if (!attr_set.have[dev]) {
+            cudaError_t e = cudaFuncSetAttribute(k_gemm_i8<BN, kOut, kPerVec>,
+                                                 cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
+            if (e != cudaSuccess) return e;
+            attr_set.have[dev] = true;
+        }
     }
     const bool has_aux = a.aux_q && a.w_aux && a.n_outliers;
     CUtensorMap tm_a, tm_b, tm_aux, tm_baux, tm_y;
@@ -267,6 +272,7 @@ cudaError_t launch_gemm_inst(const GemmArgs &a, cudaStream_t s) {
     p.s_x = a.s_x;
     p.s_w = a.s_w;
     p.dev_status = a.dev_status;
+    p.w_stable = 0; p.spin = kSpinLimit; p.skip_kb = -1;
     int grid = p.tiles_m * p.tiles_n;
     if (grid > num_sms()) grid = num_sms();
     k_gemm_i8<BN, kOut, kPerVec><<<grid, kGemmThreads, C::kSmemBytes, s>>>(tm_a, tm_aux, tm_b, tm_baux, tm_y, p);

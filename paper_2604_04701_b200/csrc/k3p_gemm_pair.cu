@@ -137,7 +137,8 @@ k_gemm_i8_pair(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                     tma_load_2d_pair_elect(sa, &tm_a, full_leader, kb * BK, m0);
                     continue;
                 }
-                if (!mbar_wait_warp(&bar_empty[s], ph ^ 1u, abort_flag)) { ok = false; break; }
+                if (!mbar_wait_warp(&bar_empty[s], ph ^ 1u, abort_flag, p.spin)) { ok = false; break; }
+                if (kb == p.skip_kb) continue;  // fault injection (never in normal operation): this stage is never filled
                 if (rank == 0) mbar_expect_tx_elect(&bar_full[s], 2 * C::kStageBytes);
                 if (kb < p.num_kb) {
                     tma_load_2d_pair_elect(sa, &tm_a, full_leader, kb * BK, m0);
@@ -155,7 +156,7 @@ k_gemm_i8_pair(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                 const uint32_t first = it > (uint32_t)C::kStages ? it - C::kStages : 0u;
                 for (uint32_t j = first; j < it; ++j) {
                     const uint32_t s = j % C::kStages, ph = (j / C::kStages) & 1u;
-                    for (uint32_t i = 0; i < kSpinLimit; ++i)
+                    for (uint32_t i = 0; i < p.spin; ++i)
                         if (__any_sync(0xffffffffu, mbar_try_wait(&bar_full[s], ph))) break;
                 }
             } else {
@@ -173,7 +174,7 @@ k_gemm_i8_pair(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
             bool ok = true;
             for (int tile = pair; tile < num_tiles && ok; tile += num_pairs, ++tile_it) {
                 const uint32_t buf = tile_it & 1u, aph = (tile_it >> 1) & 1u;
-                if (!mbar_wait_warp_cluster(&bar_acc_empty[buf], aph ^ 1u, abort_flag)) { ok = false; break; }
+                if (!mbar_wait_warp_cluster(&bar_acc_empty[buf], aph ^ 1u, abort_flag, p.spin)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + buf * BN;
                 for (int kb = 0;; ++kb, ++it) {
@@ -182,7 +183,7 @@ k_gemm_i8_pair(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                         if (kb >= p.num_kb + aux_kb) break;
                     }
                     const uint32_t s = it % C::kStages, ph = (it / C::kStages) & 1u;
-                    if (!mbar_wait_warp(&bar_full[s], ph, abort_flag)) { ok = false; break; }
+                    if (!mbar_wait_warp(&bar_full[s], ph, abort_flag, p.spin)) { ok = false; break; }
                     tc_fence_after();
                     const uint64_t a_desc = a_desc0 + (uint64_t)(s * (C::kStageBytes >> 4));
                     const uint64_t b_desc = b_desc0 + (uint64_t)(s * (C::kStageBytes >> 4));
@@ -228,7 +229,7 @@ k_gemm_i8_pair(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
             const uint32_t buf = tile_it & 1u, aph = (tile_it >> 1) & 1u;
             const int row0 = m0 + quad * 32;
             if (kPerVec && kOut != kOutI32) sx = row0 + lane < p.M ? __ldg(p.s_x + row0 + lane) : 0.0f;
-            ok = mbar_wait_warp(&bar_acc_full[buf], aph, abort_flag);
+            ok = mbar_wait_warp(&bar_acc_full[buf], aph, abort_flag, p.spin);
             if (!ok) break;
             tc_fence_after();
             const int col0 = chalf * kCols0;
@@ -289,23 +290,32 @@ template <int BN, int kOut, bool kPerVec>
 cudaError_t launch_pair_inst(const GemmArgs &a, cudaStream_t s) {
     using C = PairCfg<BN>;
     auto kern = k_gemm_i8_pair<BN, kOut, kPerVec>;
-    static int max_clusters = -1;  // per instantiation: clusters of 2 that fit on the device at once
-    if (max_clusters < 0) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
-        if (e != cudaSuccess) return e;
-        cudaLaunchConfig_t q{};
-        q.gridDim = dim3(2 * num_sms());
-        q.blockDim = dim3(kGemmThreads);
-        q.dynamicSmemBytes = C::kSmemBytes;
-        cudaLaunchAttribute qa[1];
-        qa[0].id = cudaLaunchAttributeClusterDimension;
-        qa[0].val.clusterDim.x = 2; qa[0].val.clusterDim.y = 1; qa[0].val.clusterDim.z = 1;
-        q.attrs = qa; q.numAttrs = 1;
-        int n = 0;
-        e = cudaOccupancyMaxActiveClusters(&n, kern, &q);
-        if (e != cudaSuccess) return e;
-        if (n < 1) return cudaErrorLaunchOutOfResources;
-        max_clusters = n;
+    static PerDevice<int> cache;  // per instantiation and device: clusters of 2 that fit on the device at once
+    const int dev = current_device();
+    if (dev < 0) return cudaErrorInvalidDevice;
+    const int sms = num_sms();
+    int max_clusters = 0;
+    {
+        std::lock_guard<std::mutex> lock(device_mutex());
+        if (!cache.have[dev]) {
+            cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
+            if (e != cudaSuccess) return e;
+            cudaLaunchConfig_t q{};
+            q.gridDim = dim3(2 * sms);
+            q.blockDim = dim3(kGemmThreads);
+            q.dynamicSmemBytes = C::kSmemBytes;
+            cudaLaunchAttribute qa[1];
+            qa[0].id = cudaLaunchAttributeClusterDimension;
+            qa[0].val.clusterDim.x = 2; qa[0].val.clusterDim.y = 1; qa[0].val.clusterDim.z = 1;
+            q.attrs = qa; q.numAttrs = 1;
+            int n = 0;
+            e = cudaOccupancyMaxActiveClusters(&n, kern, &q);
+            if (e != cudaSuccess) return e;
+            if (n < 1) return cudaErrorLaunchOutOfResources;
+            cache.v[dev] = n;
+            cache.have[dev] = true;
+        }
+        max_clusters = cache.v[dev];
     }
     const bool has_aux = a.aux_q && a.w_aux && a.n_outliers;
     CUtensorMap tm_a, tm_b, tm_aux, tm_baux, tm_y;
@@ -331,6 +341,8 @@ cudaError_t launch_pair_inst(const GemmArgs &a, cudaStream_t s) {
     p.s_w = a.s_w;
     p.dev_status = a.dev_status;
     p.w_stable = a.w_stable;
+    p.spin = test_hooks().spin_limit ? test_hooks().spin_limit : kSpinLimit;
+    p.skip_kb = test_hooks().gemm_skip_kb - 1;
     int clusters = p.tiles_m * p.tiles_n;
     if (clusters > max_clusters) clusters = max_clusters;
     cudaLaunchConfig_t cfg{};

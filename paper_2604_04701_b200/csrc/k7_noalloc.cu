@@ -9,6 +9,8 @@
 // (the array's name is only a host-side handle in host code) and passed to the same kernels the
 // workspace path launches.  Every call reuses the array, so calls that overlap on the GPU race;
 // what has to start at zero is cleared at the head of every call.
+#include <math.h>
+
 #include <mutex>
 
 #include "../../include/muxq.h"
@@ -43,7 +45,6 @@ static_assert(kScratchBytes == 426752, "documented size of the built-in scratch"
 
 static __device__ __align__(256) uint8_t g_noalloc_scratch[kScratchBytes];
 
-constexpr int kMaxDevices = 64;
 uint8_t *g_scratch_ptr[kMaxDevices];  // device address of the array on each device, once looked up
 std::mutex g_setup_mutex;
 
@@ -76,13 +77,15 @@ extern "C" int muxq_linear_decode_noalloc(const void *X, int M, int K, int ldx, 
                                           int out_kind, int32_t *dev_status, void *stream) {
     if (!X || !W_q || !s_w || !Y || !dev_status || !p || M <= 0 || K <= 0 || N <= 0 || ldx < K || ldw < K ||
         ldy < N || out_kind < 0 || out_kind > 2 || p->exp_factor < 1 || p->exp_factor > 3 || p->act_bits < 2 ||
-        p->act_bits > 8 || p->max_outliers < 1 || p->max_outliers > kMaxOutliers ||
-        (p->gran != MUXQ_PER_TENSOR && p->gran != MUXQ_PER_VECTOR) || !(p->threshold >= 0.0f))
+        p->act_bits > 8 || p->w_bits < 2 || p->w_bits > 8 || p->max_outliers < 1 || p->max_outliers > kMaxOutliers ||
+        (p->gran != MUXQ_PER_TENSOR && p->gran != MUXQ_PER_VECTOR) ||
+        (p->aux_scale != MUXQ_AUX_SHARED && p->aux_scale != MUXQ_AUX_OWN) || !(p->threshold >= 0.0f) ||
+        !(p->threshold < INFINITY))
         return MUXQ_ERR_INVALID_ARG;
     if (M > kNoallocMaxM || K > kNoallocMaxK) return MUXQ_ERR_STATIC_LIMIT;
     const int yal = out_kind == MUXQ_OUT_F16 ? 8 : 4;
     if (K % 16 || ldx % 8 || ldw % 16 || N % 8 || ldy % yal || !aligned16(X) || !aligned16(W_q) || !aligned16(Y) ||
-        p->aux_scale != MUXQ_AUX_SHARED || !prep_supported(M, K))
+        p->aux_scale != MUXQ_AUX_SHARED || (p->gran == MUXQ_PER_VECTOR && !aligned16(s_w)))
         return MUXQ_ERR_UNSUPPORTED;
 
     uint8_t *ws = nullptr;
@@ -95,6 +98,42 @@ extern "C" int muxq_linear_decode_noalloc(const void *X, int M, int K, int ldx, 
 
     const bool per_vec = p->gran == MUXQ_PER_VECTOR;
     Ctrl *ctrl = reinterpret_cast<Ctrl *>(ws);
+    if (!prep_supported(M, K)) {
+        // the widest rows (K beyond what one CTA of the fused kernel covers) take the separate detection and
+        // quantization kernels; their two small per-channel arrays use the space of the fused kernel's accumulators
+        DetectArgs d{};
+        d.X = static_cast<const __half *>(X);
+        d.M = M; d.K = K; d.ldx = ldx;
+        d.tau = p->threshold; d.exp_factor = p->exp_factor; d.qmax = (1 << (p->act_bits - 1)) - 1;
+        d.cap = p->max_outliers;
+        d.colmax_bits = reinterpret_cast<uint32_t *>(ws + l.colmax);
+        d.ctrl = ctrl;
+        d.outlier_idx = reinterpret_cast<int32_t *>(ws + l.oidx);
+        d.colmul = reinterpret_cast<float *>(ws + l.colmax_rep);
+        d.grpflag = ws + l.colmax_rep + (size_t)K * 4;
+        d.dev_status = dev_status;
+        if (launch_detect(d, s) != cudaSuccess) return MUXQ_ERR_CUDA;
+        QuantActArgs q{};
+        q.X = d.X; q.M = M; q.K = K; q.ldx = ldx;
+        q.exp_factor = p->exp_factor; q.qmax = d.qmax; q.cap = p->max_outliers; q.per_token = per_vec;
+        q.outlier_idx = d.outlier_idx;
+        q.n_outliers = &ctrl->n_outliers;
+        q.colmul = d.colmul; q.grpflag = d.grpflag;
+        q.s_x_tensor = &ctrl->s_x;
+        q.inv_s_x_tensor = &ctrl->inv_s_x;
+        q.s_x_rows = reinterpret_cast<float *>(ws + l.sx_rows);
+        q.body_q = reinterpret_cast<int8_t *>(ws + l.body_q); q.ld_q = K;
+        if (launch_quant_act(q, s) != cudaSuccess) return MUXQ_ERR_CUDA;
+        DecodeArgs k{};
+        k.body_q = q.body_q; k.ld_a = K;
+        k.w_q = W_q; k.ldw = ldw;
+        k.outlier_idx = d.outlier_idx; k.n_outliers = &ctrl->n_outliers;
+        k.M = M; k.K = K; k.N = N; k.c = (1 << p->exp_factor) - 1; k.cap = p->max_outliers;
+        k.s_x = per_vec ? q.s_x_rows : &ctrl->s_x; k.s_x_per_row = per_vec;
+        k.s_w = s_w; k.s_w_per_col = per_vec;
+        k.Y = Y; k.ldy = ldy; k.out_kind = out_kind;
+        return launch_decode(k, s) == cudaSuccess ? MUXQ_OK : MUXQ_ERR_CUDA;
+    }
     PrepArgs f{};
     f.X = static_cast<const __half *>(X);
     f.M = M; f.K = K; f.ldx = ldx;

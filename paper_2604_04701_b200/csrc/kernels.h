@@ -4,7 +4,33 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <mutex>
+
 namespace muxq {
+
+// ---------------------------------------------------------------- host-side state (host_state.cu)
+// The only state the library keeps between calls: results of one-time set-up per device (function attributes
+// that were set, occupancy that was queried, the SM count), indexed by the CUDA device ordinal and guarded by
+// one mutex, so that a process may drive several GPUs from several threads.
+constexpr int kMaxDevices = 64;
+template <typename T>
+struct PerDevice {
+    T v[kMaxDevices];
+    bool have[kMaxDevices];
+};
+int current_device();        // ordinal of the current device, or -1
+std::mutex &device_mutex();  // serialises first-use set-up
+int num_sms();               // SM count of the current device (0 on error)
+
+// Fault injection for tests, set through muxq_test_hooks (all zero in normal operation): a short poll limit for
+// the bounded device-side waits and conditions that make one of them run out without faulting anything.
+struct TestHooks {
+    uint32_t spin_limit;           // 0 = the kernels' own limits
+    uint32_t prep_extra_arrivals;  // the preparation kernel's grid barrier expects this many arrivals that never come
+    int32_t gemm_skip_kb;          // 1 + index of a K block whose operand loads the GEMM producer leaves out (0 = none)
+};
+const TestHooks &test_hooks();
+void set_test_hooks(const TestHooks &h);
 
 // Device control block at the start of every workspace.  The stand-alone kernels get it zeroed by a
 // memset per call; the fused prep kernel needs `arrived`, `readers` and its replicated abs-max
@@ -14,7 +40,7 @@ struct Ctrl {
     int32_t n_outliers;    // r, true count of outlier channels
     float s_x;             // per-tensor Body scale (Eq. 1)
     float inv_s_x;         // 1 / s_x, correctly rounded (used only to pre-screen the exact division)
-    uint32_t arrived;      // fused prep kernel: CTAs that have reached the grid-wide barrier
+    uint32_t arrived;      // fused prep kernel: CTAs that have reached the grid-wide barrier; top bit = a call timed out
     uint32_t readers;      // fused prep kernel: CTAs that have fetched the merged channel maxima
     float s_a;             // per-tensor Aux scale when Aux has its own (Eq. 1 applied to Aux alone)
     uint32_t reserved[57];
@@ -84,7 +110,7 @@ struct PrepArgs {
     int8_t *aux_q;   int ld_aux; int aux_cols;   // aux_q may be NULL (decode path)
     const int8_t *w_q; int ldw; int N;           // W_aux gather (all NULL/0 to skip)
     int8_t *w_aux; int ld_waux;
-    int32_t *dev_status;     // set to 0 at kernel start, raised on r > cap or a barrier time-out
+    int32_t *dev_status;     // raised (never cleared) on r > cap or when a bounded wait runs out
 };
 // Own-scale reading: Y = t1 + c * t2 (fp32 in, fp16 or fp32 out); t1, t2 dense [M, N].
 struct CombineArgs {
@@ -162,7 +188,5 @@ cudaError_t launch_decode_fused(const DecodeFusedArgs &a, cudaStream_t s);
 
 cudaError_t launch_mma_peak(int n, int iters, unsigned long long *cycles_out, int32_t *status, int grid,
                             cudaStream_t s);
-
-int num_sms();
 
 }  // namespace muxq

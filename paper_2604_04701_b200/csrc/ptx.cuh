@@ -62,8 +62,9 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volati
 
 // The same wait executed by a whole converged warp: every lane polls and the lanes vote, so the
 // result is warp-uniform (control flow after it stays converged).
-__device__ __forceinline__ bool mbar_wait_warp(uint64_t *bar, uint32_t parity, volatile uint32_t *abort_flag) {
-    for (uint32_t i = 0; i < kSpinLimit; ++i) {
+__device__ __forceinline__ bool mbar_wait_warp(uint64_t *bar, uint32_t parity, volatile uint32_t *abort_flag,
+                                               uint32_t limit = kSpinLimit) {
+    for (uint32_t i = 0; i < limit; ++i) {
         if (__any_sync(0xffffffffu, mbar_try_wait(bar, parity))) return true;
         if ((i & 63u) == 63u && __any_sync(0xffffffffu, *abort_flag != 0u)) return false;
     }
@@ -213,8 +214,9 @@ __device__ __forceinline__ bool mbar_try_wait_cluster(uint64_t *bar, uint32_t pa
         : "memory");
     return ok != 0;
 }
-__device__ __forceinline__ bool mbar_wait_warp_cluster(uint64_t *bar, uint32_t parity, volatile uint32_t *abort_flag) {
-    for (uint32_t i = 0; i < kSpinLimit; ++i) {
+__device__ __forceinline__ bool mbar_wait_warp_cluster(uint64_t *bar, uint32_t parity, volatile uint32_t *abort_flag,
+                                                       uint32_t limit = kSpinLimit) {
+    for (uint32_t i = 0; i < limit; ++i) {
         if (__any_sync(0xffffffffu, mbar_try_wait_cluster(bar, parity))) return true;
         if ((i & 63u) == 63u && __any_sync(0xffffffffu, *abort_flag != 0u)) return false;
     }

@@ -232,6 +232,40 @@ def test_gemm_worst_case_magnitudes(mx):
         assert np.array_equal(y16.cpu().numpy(), ((sx * sw) * ref.astype(np.float32)).astype(np.float16))
 
 
+@pytest.mark.parametrize("M,K,N", [(8192, 128, 2304), (8192, 256, 768), (8192, 128, 2048)])
+def test_gemm_several_tiles_per_cta_pair_full_matrix(mx, M, K, N):
+    """Full-matrix check of the persistent loop beyond its first tile: 288 / 128 / 256 output tiles over 74 CTA
+    pairs give every pair 2 to 4 tiles, so the flip between the two TMEM accumulator buffers, the phase wrap of
+    their barriers and the operand ring running on across tiles all decide values that are compared here.  The
+    reference is a float32 matrix product: every partial sum stays below 2^24, so it is exact."""
+    rng = np.random.default_rng(M + 3 * K + N)
+    a = rng.integers(-127, 128, (M, K), dtype=np.int8)
+    b = rng.integers(-127, 128, (N, K), dtype=np.int8)
+    assert 127 * 127 * K < 2 ** 24
+    ref = (a.astype(np.float32) @ b.astype(np.float32).T).astype(np.int32)
+    ws = mx.Workspace(256)
+    acc = mx.muxq_gemm(dev(a), None, dev(b), None, None, mx.MuxqParams(), None, None, mx.MUXQ_OUT_ACC_I32, ws)
+    assert mx.muxq_read_status(ws) == 0
+    assert np.array_equal(acc.cpu().numpy(), ref)
+
+
+@pytest.mark.parametrize("gran", [0, 1])
+def test_linear_several_tiles_per_cta_pair_full_matrix(mx, gran):
+    """The same through the whole layer with an Aux block (K = 256, 6 outlier channels, 288 output tiles):
+    every accumulator and every output of the 8192 x 2304 result against the oracle."""
+    M, K, N = 8192, 256, 2304
+    x, w, _ = make_case(77, M, K, N, n_out=6, mult=50.0)
+    p = mx.MuxqParams(gran=gran, max_outliers=32)
+    _, _, res = oracle_linear(x, w, p)
+    assert res.r >= 6
+    acc, _, st, _, _ = run_linear(mx, x, w, p, mx.MUXQ_OUT_ACC_I32)
+    assert st == 0 and np.array_equal(acc.cpu().numpy(), res.acc)
+    y16, _, st, _, _ = run_linear(mx, x, w, p, mx.MUXQ_OUT_F16)
+    assert st == 0 and f16_ulp_diff(y16.cpu().numpy(), res.y16).max() <= 1
+    y32, _, st, _, _ = run_linear(mx, x, w, p, mx.MUXQ_OUT_F32)
+    assert st == 0 and np.array_equal(y32.cpu().numpy(), res.y32)
+
+
 # ------------------------------------------------------------------ whole layer
 @pytest.mark.parametrize("gran", [0, 1])
 @pytest.mark.parametrize("M,K,N,n_out", [(128, 768, 768, 4), (300, 1040, 520, 7), (512, 256, 1288, 0),
@@ -374,18 +408,26 @@ def test_host_buffer_entry_point(mx):
     assert f16_ulp_diff(yh.numpy(), res.y16).max() <= 1
 
 
-# ------------------------------------------------------------------ full benchmark sizes, sampled rows
-def _full_size_check(mx, spec, gran, n_rows=48, cap=32):
+# ------------------------------------------------------------------ full benchmark sizes
+def _full_size_check(mx, spec, gran, n_rows=32, cap=32, full=False):
     """One layer at its full size through muxq_linear (the launch configuration bench.py times);
-    detection results and scales are compared in full, the products on seeded sample rows (each row of
-    the layer is independent once O and the scales are fixed, so the oracle computes them one by one)."""
+    detection results, scales and every code of the full matrix are compared.  The products are compared
+    on every row (full=True) or on sample rows: one row of every 128-row block of X (so that every
+    output tile of the persistent GEMM loop, whichever CTA of a pair owns it, is hit) at an offset that
+    walks through the block, the edges, and seeded random rows.  Each row of the layer is independent
+    once O and the scales are fixed, so the oracle computes them one by one."""
     x, _ = spec.x()
     w = spec.w()
     p = mx.MuxqParams(gran=gran, max_outliers=cap)
-    rng = np.random.default_rng(spec.seed * 1000 + spec.tensor_id)
-    rows = np.unique(np.concatenate([[0, spec.M - 1, 127, 128, spec.M // 2],
-                                     rng.integers(0, spec.M, n_rows)])).astype(np.int32)
-    rows = rows[rows < spec.M]
+    rows = None
+    if not full:
+        rng = np.random.default_rng(spec.seed * 1000 + spec.tensor_id)
+        blocks = np.arange(0, spec.M, 128)
+        per_block = blocks + (blocks // 128 * 37) % 128
+        rows = np.unique(np.concatenate([[0, spec.M - 1, 127, 128, spec.M // 2], per_block,
+                                         rng.integers(0, spec.M, n_rows)])).astype(np.int32)
+        rows = rows[rows < spec.M]
+    sel = slice(None) if rows is None else rows
     wq_o, sw_o, res = oracle_linear(x, w, p, rows=rows)
     assert res.rc == 0 and res.r >= spec.n_outliers
     y16, ws, st, w_q, s_w = run_linear(mx, x, w, p, mx.MUXQ_OUT_F16)
@@ -396,25 +438,29 @@ def _full_size_check(mx, spec, gran, n_rows=48, cap=32):
     assert np.array_equal(v["s_x"].view(np.uint32), res.s_x.view(np.uint32))
     assert np.array_equal(v["body_q"], res.body_q)          # every code of the full matrix
     assert np.array_equal(w_q.cpu().numpy(), wq_o.T)
-    assert f16_ulp_diff(y16.cpu().numpy()[rows], res.y16).max() <= 1
+    assert f16_ulp_diff(y16.cpu().numpy()[sel], res.y16).max() <= 1
     acc, _, st, _, _ = run_linear(mx, x, w, p, mx.MUXQ_OUT_ACC_I32)
-    assert st == 0 and np.array_equal(acc.cpu().numpy()[rows], res.acc)
+    assert st == 0 and np.array_equal(acc.cpu().numpy()[sel], res.acc)
     y32, _, st, _, _ = run_linear(mx, x, w, p, mx.MUXQ_OUT_F32)
-    assert st == 0 and rel_err32(y32.cpu().numpy()[rows], res.y32) <= 1e-5
+    assert st == 0 and rel_err32(y32.cpu().numpy()[sel], res.y32) <= 1e-5
+
+
+def test_config0_full_matrix(mx):
+    _full_size_check(mx, synth.config_layers(0)[0], 0, full=True)
 
 
 @pytest.mark.parametrize("gran", [0, 1])
 @pytest.mark.parametrize("layer", [0, 1, 2, 3])
-def test_config1_full_size_sampled_rows(mx, layer, gran):
-    _full_size_check(mx, synth.config_layers(1)[layer], gran)
+def test_config1_full_matrix(mx, layer, gran):
+    _full_size_check(mx, synth.config_layers(1)[layer], gran, full=True)
 
 
-@pytest.mark.parametrize("layer", [0, 3])
+@pytest.mark.parametrize("layer", [0, 1, 2, 3])
 def test_config2_heavy_tailed_full_size_sampled_rows(mx, layer):
     _full_size_check(mx, synth.config_layers(2)[layer], 0, cap=64)
 
 
-@pytest.mark.parametrize("layer", [1, 3])
+@pytest.mark.parametrize("layer", [0, 1, 2, 3])
 def test_config3_prefill_full_size_sampled_rows(mx, layer):
     _full_size_check(mx, synth.config_layers(3)[layer], 0)
 
@@ -438,6 +484,16 @@ def test_config3_decode_full_size(mx, M):
 def test_config4_outlier_sweep_full_size_sampled_rows(mx, n_out):
     spec = synth.config_layers(4, n_outliers=n_out, layers=36)[35 * 4 + 2]   # last layer's c_fc, 8192 x 1280 -> 5120
     _full_size_check(mx, spec, 0, cap=64)
+
+
+@pytest.mark.parametrize("linear", [0, 1, 2, 3])
+@pytest.mark.parametrize("layer", [0, 17, 35])
+def test_config4_first_middle_last_layer(mx, layer, linear):
+    """Layers 0, 17 and 35 of the 36-layer stack, all four linears (8 outlier channels): the layers are
+    independent problems (fresh X per layer), so three of them with every linear shape cover the stack's shapes
+    and seeds at both ends and in the middle."""
+    spec = synth.config_layers(4, n_outliers=8, layers=36)[layer * 4 + linear]
+    _full_size_check(mx, spec, 0, cap=64, full=(layer == 0 and linear == 1))
 
 
 @pytest.mark.parametrize("e,act_bits,w_bits,gran", [(1, 8, 8, 0), (3, 6, 5, 0), (3, 7, 4, 1), (2, 5, 8, 1)])

@@ -132,6 +132,31 @@ def test_zero_outliers_reduces_to_plain_absmax_int8(per_vector):
     assert np.array_equal(res.y16, y.astype(np.float16))
 
 
+@pytest.mark.parametrize("per_channel", [False, True])
+@pytest.mark.parametrize("bits", [8, 7, 5, 4, 2])
+def test_weight_quantization_at_reduced_bit_widths(bits, per_channel):
+    """Eq. 2 with qmax = 2^(bits-1) - 1 (the W 5 / W 4 settings of Table 2), against a numpy statement of the
+    same formula; the ties at 0.5 and 2.5 of the second matrix must go to the even neighbour."""
+    q = (1 << (bits - 1)) - 1
+    w = synth.make_w(11, 5, 96, 40)
+    tie = np.zeros((4, 8), np.float16)
+    tie[0, :] = q                      # abs-max = q in every column: scale exactly 1
+    tie[1, :4] = [0.5, 1.5, 2.5, -0.5]
+    tie[2, :4] = [-1.5, -2.5, 3.5, 0.25]
+    for mat in (w, tie):
+        wq, sw = oracle.quantize_weight(mat, bits=bits, per_channel=per_channel)
+        f = mat.astype(np.float32)
+        amax = np.abs(f).max(axis=0, keepdims=True) if per_channel else np.abs(f).max().reshape(1, 1)
+        s = (amax / np.float32(q)).astype(np.float32)
+        ref = np.clip(np.rint(f / s), -q, q).astype(np.int32)
+        assert np.array_equal(sw, s.ravel())
+        assert np.array_equal(wq.astype(np.int32), ref)
+        assert np.abs(wq.astype(np.int32)).max() == q      # the abs-max element maps to +-q, nothing beyond
+    if q >= 3:
+        wq, _ = oracle.quantize_weight(tie, bits=bits, per_channel=per_channel)
+        assert wq[1, :4].tolist() == [0, 2, 2, 0] and wq[2, :4].tolist() == [-2, -2, min(4, q), 0]
+
+
 # ------------------------------------------------------------------ Eq. 6 / Eq. 7 identities
 @pytest.mark.parametrize("e", [1, 2, 3])
 def test_decomposition_reconstructs_x_exactly(e):

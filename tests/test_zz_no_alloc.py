@@ -10,6 +10,7 @@ import numpy as np
 import pytest
 
 import muxq_synth as synth
+import oracle
 
 torch = pytest.importorskip("torch")
 pytestmark = pytest.mark.gpu
@@ -28,12 +29,16 @@ def _dev(a):
     return torch.from_numpy(np.ascontiguousarray(a)).cuda()
 
 
+@pytest.mark.parametrize("K,N", [(1280, 3840), (8192, 264), (1040, 520)])
 @pytest.mark.parametrize("gran", [0, 1])
-def test_two_calls_in_a_row_match_the_workspace_entry_point(mx, gran):
-    K, N = 1280, 3840
+def test_two_calls_in_a_row_match_the_workspace_entry_point_and_the_oracle(mx, gran, K, N):
+    """K = 8192 is the entry point's limit (and wider than one CTA of the fused preparation kernel covers, so it
+    takes the separate detection and quantization kernels); K = 1040 is not a multiple of 64, so there the
+    workspace entry point runs the same two kernels instead of its fused decode kernel."""
     p = mx.MuxqParams(gran=gran, max_outliers=32)
     w = synth.make_w(91, 3, K, N)
     w_q, s_w = mx.muxq_quantize(_dev(w), p, True, mx.Workspace(mx.muxq_small_workspace_bytes(N)))
+    wq_o, sw_o = oracle.quantize_weight(w, per_channel=gran == 1)
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     # Second call: fewer rows, fewer and weaker outlier channels, smaller maxima -- anything the
     # first call left in the shared scratch (abs-max accumulators, outlier list, codes of rows 4..15)
@@ -42,6 +47,8 @@ def test_two_calls_in_a_row_match_the_workspace_entry_point(mx, gran):
     for x in cases:
         M = x.shape[0]
         xd = _dev(x)
+        res = oracle.linear(x, wq_o, sw_o, per_vector=gran == 1, cap=32)
+        assert res.rc == 0
         for out_kind, dt in ((mx.MUXQ_OUT_ACC_I32, torch.int32), (mx.MUXQ_OUT_F32, torch.float32),
                              (mx.MUXQ_OUT_F16, torch.float16)):
             ws = mx.Workspace(mx.muxq_workspace_bytes(M, K, N, p))
@@ -51,8 +58,18 @@ def test_two_calls_in_a_row_match_the_workspace_entry_point(mx, gran):
             got = mx.muxq_linear_decode_noalloc(xd, w_q, s_w, p, status, out_kind, out=out)
             torch.cuda.synchronize()
             assert int(status.item()) == 0
-            # same kernels, same arithmetic: integer accumulators, fp32 and fp16 outputs all bit-equal
+            # same arithmetic: integer accumulators, fp32 and fp16 outputs all bit-equal
             assert torch.equal(got, ref)
+            g = got.cpu().numpy()
+            if out_kind == mx.MUXQ_OUT_ACC_I32:
+                assert np.array_equal(g, res.acc)
+            elif out_kind == mx.MUXQ_OUT_F32:
+                assert np.array_equal(g, res.y32)
+            else:
+                key = lambda v: np.where(v.view(np.uint16).astype(np.int32) & 0x8000,
+                                         -(v.view(np.uint16).astype(np.int32) & 0x7FFF),
+                                         v.view(np.uint16).astype(np.int32))
+                assert np.abs(key(g) - key(res.y16)).max() <= 1
 
 
 def test_sizes_beyond_the_built_in_scratch_are_refused(mx):
