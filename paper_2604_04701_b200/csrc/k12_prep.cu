@@ -1,89 +1,58 @@
 // Fused activation preparation for muxq_linear: per-channel abs-max and outlier detection
 // (Section III-C), the redistribution of Eq. 4-5 and the abs-max quantization of Eq. 1, in ONE
-// launch.
+// launch that reads X from HBM once.
 //
 // The per-tensor scale and the outlier set depend on every row of X, so the kernel has two passes
 // separated by a grid-wide barrier.  It is launched cooperatively with one CTA per SM; CTA b owns a
-// contiguous slab of token rows.  Both passes are built around one ring of row stripes in shared
-// memory that a producer warp fills with bulk asynchronous copies (one per token row, completion on an
-// mbarrier per stripe) while the other 31 warps consume:
-//   stripe   nrow = floor(992 / (K/8)) consecutive rows; consumer thread (row_off, cg) owns the 16-byte
-//            chunk of channels 8cg..8cg+7 of row row_off of every stripe, so its channel maxima (pass 1)
-//            and its channel factors (pass 2) stay in registers
-//   pass 1   stripes 0..T-1 stream through the ring (S slots); a thread folds its chunk into its 8
-//            running maxima.  The ring ends up holding the LAST S stripes.  Channel maxima are merged
-//            CTA-wide in shared memory and device-wide with integer atomicMax on the bit patterns
-//            (maxima of non-negative floats are order independent, so the result is exact), into
-//            accumulators replicated kColmaxReplicas times (CTA b uses copy b mod R: same-address
-//            atomics serialise in L2)
-//   barrier  bounded spin on an arrival counter; a time-out raises MUXQ_ERR_TIMEOUT, marks the workspace
-//            (the counter keeps its top bit until muxq_workspace_init clears it) and returns
-//   pass 2   every CTA derives the channel factors and s_X from the K maxima (cheap, redundant; the
-//            producer warp lists O meanwhile), then quantizes: first the stripes still resident, in
-//            place, then the evicted ones, which the producer fetches again in REVERSE order -- the most
-//            recently evicted stripe is the one most likely still in L2 -- into slots as they are
-//            freed.  A thread writes the 8 codes of its chunk to Body_q, and, where its chunk holds an
-//            outlier channel, the copies of those codes that make up the Aux block (Eq. 5).  Per-token
-//            scales take one warp per token row instead (rows not resident are read from global memory).
-//            The producer warp gathers this CTA's share of W_aux before it starts fetching.
-// The kernel expects the barrier counter, the reader counter and the replicated accumulators to be zero
-// and leaves them zero: once every CTA has fetched the merged maxima (each takes a ticket after doing so;
-// the holder of the last ticket knows), nothing reads them any more, and that CTA clears them at its end.
-// A call therefore needs no separate clearing step.
+// contiguous slab of token rows and keeps it in shared memory between the passes (a slab of
+// M/148 rows x K fp16 fits for the GPT-2 shapes; rows that do not fit are re-read, normally from L2):
+//   pass 1  stream the slab (128-bit loads, a thread owns 8 channels and walks down the rows),
+//           stash it in shared memory, merge channel maxima CTA-wide in shared memory and then
+//           device-wide with integer atomicMax on the bit patterns (maxima of non-negative floats
+//           are order independent, so the result is exact).  The device-wide accumulators are
+//           replicated kColmaxReplicas times (CTA b uses copy b mod R): same-address atomics
+//           serialise in L2, and one copy would take 148 of them per channel
+//   barrier bounded spin on an arrival counter; a time-out raises MUXQ_ERR_TIMEOUT, marks the workspace (the
+//           counter keeps its top bit until muxq_workspace_init clears it, and every later call that finds
+//           the mark fails at once instead of computing on half-merged maxima) and returns
+//   pass 2  every CTA derives the channel factors and s_X from the K maxima (cheap, redundant; warp 0
+//           lists O meanwhile), then quantizes its slab out of shared memory with the pass-1 thread
+//           mapping (per tensor) or one warp per token row (per token), writing Body_q, the Aux block
+//           and (spread over the grid) the gathered W_aux rows.
+// The kernel expects the barrier counter, the reader counter and the replicated accumulators to be zero and
+// leaves them zero: once every CTA has fetched the merged maxima (each takes a ticket after doing so; the
+// holder of the last ticket knows), nothing reads them any more, and that CTA clears them during the last phase.
+// A call therefore needs no separate clearing step; a barrier time-out leaves them dirty (and marked).
 #include <mutex>
 
 #include "kernels.h"
-#include "ptx.cuh"
 #include "quant.cuh"
 
 namespace muxq {
 
 namespace {
 
-constexpr int kT = 1024;
+constexpr int kT = 1024;  // the warp-group split of the last phase (512 + 256 + 256 threads) assumes this
 constexpr int kWarps = kT / 32;
-constexpr int kConsWarps = kWarps - 1;      // warp kWarps-1 is the producer
-constexpr int kConsThreads = 32 * kConsWarps;
-constexpr int kMaxG = kConsThreads;         // one group of 8 channels per consumer thread
-constexpr int kMaxSlots = 32;
+constexpr int kMaxK = 8 * kT;  // one group of 8 channels per thread
+static_assert(kMaxK == kPrepMaxK, "the accumulator region of the workspace is sized for kPrepMaxK channels");
 constexpr int kColmaxReplicas = kPrepColmaxReplicas;
 constexpr int kStatusCapacity = 5;  // MUXQ_ERR_CAPACITY
 constexpr int kStatusTimeout = 6;   // MUXQ_ERR_TIMEOUT
+constexpr uint32_t kBarrierSpin = 1u << 21;
 constexpr uint32_t kPoisonBit = 0x80000000u;  // in Ctrl::arrived: an earlier call on this workspace timed out
-constexpr int kMaxDynSmem = 227 * 1024 - 2048;
+constexpr int kMaxDynSmem = 227 * 1024 - 1024;
 
 __host__ __device__ inline int fixed_smem_bytes(int K, int cap, int aux_cols) {
     const int G = K >> 3;
-    // colmul | colmax | group flags | rank of each group's first outlier channel [G] u16 | outlier indices [cap] |
-    // source channel of every Aux column [aux_cols] u16; rounded so that the ring behind it is 128-byte aligned
-    const int n = 8 * K + ((G + 15) & ~15) + ((2 * G + 15) & ~15) + ((cap + 3) & ~3) * 4 + ((aux_cols * 2 + 15) & ~15);
-    return (n + 127) & ~127;
+    // colmul | colmax | group flags | outlier indices [cap] | source channel of every Aux column [aux_cols]
+    return 8 * K + ((G + 15) & ~15) + ((cap + 3) & ~3) * 4 + ((aux_cols * 2 + 15) & ~15);
 }
 
 __device__ __forceinline__ uint32_t ld_acquire_u32(const uint32_t *p) {
     uint32_t v;
     asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
     return v;
-}
-
-// One token row (or any 16-byte-aligned span) global -> shared, completion counted in bytes on an mbarrier.
-__device__ __forceinline__ void bulk_load(void *smem_dst, const void *gsrc, uint32_t bytes, uint64_t *bar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
-                     smem_u32(smem_dst)),
-                 "l"(gsrc), "r"(bytes), "r"(smem_u32(bar))
-                 : "memory");
-}
-
-// Bounded wait of a whole converged warp with a caller-chosen limit (the default limit is far above any
-// legitimate wait; a test shortens it to make a wait run out).
-__device__ __forceinline__ bool wait_warp(uint64_t *bar, uint32_t parity, volatile uint32_t *abort_flag,
-                                          uint32_t limit) {
-    for (uint32_t i = 0; i < limit; ++i) {
-        if (__any_sync(0xffffffffu, mbar_try_wait(bar, parity))) return true;
-        if ((i & 63u) == 63u && __any_sync(0xffffffffu, *abort_flag != 0u)) return false;
-    }
-    *abort_flag = 1u;
-    return false;
 }
 
 __device__ __forceinline__ void absmax4(__half2 (&m)[4], const uint4 &v) {
@@ -106,113 +75,70 @@ __device__ __forceinline__ void load_chunk(const uint4 *src, int ch, const uint8
     }
 }
 
-// Geometry of one launch, computed on the host.
-struct PrepGeom {
-    int rows_base, rows_extra;  // CTA b owns rows_base (+1 if b < rows_extra) rows
-    int nrow;                   // rows per stripe
-    int slots;                  // S: stripes the ring holds
-    uint32_t g_magic;           // ceil(2^20 / G): t / G as a multiplication, exact for t < 1024
-    uint32_t spin;              // poll limit of every bounded wait
-    uint32_t extra_arrivals;    // 0; a test sets it to make the grid barrier wait for arrivals that never come
-};
-
+// kAllFit: the host has sized the slab for every row of the largest CTA share, so the loops over rows that
+// live only in global memory are compiled out (and with them their registers).
 // kPerToken: per-token scales (one warp per row in pass 2) instead of the per-tensor scale; one instantiation
 // per granularity keeps the other one's code out of the kernel.
-template <bool kPerToken>
-__global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, const PrepGeom g) {
-    extern __shared__ __align__(128) uint8_t smem[];
-    __shared__ uint64_t bar_full[kMaxSlots], bar_empty[kMaxSlots];
+template <bool kAllFit, bool kPerToken>
+__global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, int rows_base, int rows_extra, int slab_bytes,
+                                                int rstride, uint32_t g_magic, uint32_t spin, uint32_t extra_arrivals) {
+    extern __shared__ __align__(16) uint8_t smem[];
     __shared__ float s_warp_max[kWarps];
     __shared__ int s_r_true;
-    __shared__ uint32_t s_abort;
+    __shared__ int s_fail;
     __shared__ int s_last;
-    __shared__ volatile int s_list_ready;
     __shared__ float s_aux_scale;  // per-tensor Aux scale (own-scale reading)
 
-    const int t = threadIdx.x, lane = t & 31;
-    const int warp = __shfl_sync(0xffffffffu, t >> 5, 0);  // warp-uniform by construction
+    const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
     const int K = a.K, G = K >> 3;
     float *s_colmul = reinterpret_cast<float *>(smem);
     uint32_t *s_colmax = reinterpret_cast<uint32_t *>(smem + 4 * K);
     uint8_t *s_flag = smem + 8 * K;
-    uint16_t *s_rank = reinterpret_cast<uint16_t *>(smem + 8 * K + ((G + 15) & ~15));
-    int32_t *s_oidx = reinterpret_cast<int32_t *>(reinterpret_cast<uint8_t *>(s_rank) + ((2 * G + 15) & ~15));
+    int32_t *s_oidx = reinterpret_cast<int32_t *>(smem + 8 * K + ((G + 15) & ~15));
     uint16_t *s_auxsrc = reinterpret_cast<uint16_t *>(s_oidx + ((a.cap + 3) & ~3));
-    uint8_t *ring = smem + fixed_smem_bytes(K, a.cap, a.aux_cols);
+    uint8_t *slab = smem + fixed_smem_bytes(K, a.cap, a.aux_cols);
 
     const int b = blockIdx.x;
-    const int r0 = b * g.rows_base + min(b, g.rows_extra);
-    const int rows = g.rows_base + (b < g.rows_extra ? 1 : 0);
-    const int nrow = g.nrow, S = g.slots;
-    const int T = (rows + nrow - 1) / nrow;          // stripes of this CTA
-    const int Sres = min(S, T);                      // stripes resident after pass 1
-    const uint32_t row_bytes = (uint32_t)K * 2u;
-    const uint32_t slot_bytes = (uint32_t)nrow * row_bytes;
-    volatile uint32_t *abort_flag = &s_abort;
-    const bool producer = warp == kWarps - 1;
-
-    // consumer thread = (row offset inside a stripe, channel group)
-    const int row_off = (int)(((uint32_t)t * g.g_magic) >> 20), cg = t - row_off * G;
-    const bool active = !producer && row_off < nrow;
-
-    // CTA-wide maxima of pass 1 accumulate in s_part, laid out [channel within group][group] so that the lanes of a
-    // warp (consecutive groups) hit consecutive banks.  It shares its bytes with s_colmul, written after the barrier.
-    uint32_t *s_part = reinterpret_cast<uint32_t *>(smem);
-    for (int k = t; k < K; k += kT) s_part[k] = 0u;
-    if (t == 0) {
-        for (int s = 0; s < S; ++s) {
-            mbar_init(&bar_full[s], 1);            // the producer's expect_tx arrival; bytes from the copies
-            mbar_init(&bar_empty[s], kConsWarps);  // one arrival per consumer warp
-        }
-        s_abort = 0u;
-        s_list_ready = 0;
-        fence_barrier_init();
-    }
-    __syncthreads();
-
-    // Fetch of stripe `stripe` (rows stripe*nrow ...) into ring position n % S, load number n of this CTA.
-    auto issue = [&](int n, int stripe) -> bool {
-        const int slot = n % S;
-        if (n >= S && !wait_warp(&bar_empty[slot], (uint32_t)((n / S) - 1) & 1u, abort_flag, g.spin)) return false;
-        const int first = stripe * nrow, cnt = min(nrow, rows - first);
-        if (lane == 0) mbar_expect_tx(&bar_full[slot], (uint32_t)cnt * row_bytes);
-        __syncwarp();
-        for (int i = lane; i < cnt; i += 32)
-            bulk_load(ring + (size_t)slot * slot_bytes + (size_t)i * row_bytes,
-                      a.X + ((size_t)r0 + first + i) * a.ldx, row_bytes, &bar_full[slot]);
-        return true;
-    };
-    // After a time-out the copies already issued must land before this CTA's shared memory is released.
-    auto drain = [&](int issued) {
-        for (int n = max(0, issued - S); n < issued; ++n) {
-            const int slot = n % S;
-            for (uint32_t i = 0; i < g.spin; ++i)
-                if (__any_sync(0xffffffffu, mbar_try_wait(&bar_full[slot], (uint32_t)(n / S) & 1u))) break;
-        }
-    };
+    const int r0 = b * rows_base + min(b, rows_extra);
+    const int rows = rows_base + (b < rows_extra ? 1 : 0);
+    const int fit = kAllFit ? rows : min(rows, slab_bytes / (2 * K));
 
     // ---------------------------------------------------------------- pass 1: channel maxima
-    int issued = 0;  // producer warp: loads issued so far (drained after a time-out)
-    if (producer) {
-        for (; issued < T; ++issued)
-            if (!issue(issued, issued)) break;
-    } else {
-        __half2 m[4];
-        m[0] = m[1] = m[2] = m[3] = __float2half2_rn(0.f);
-        const uint8_t *mine = ring + (size_t)row_off * row_bytes + cg * 16;
-        bool ok = true;
-        for (int n = 0; n < T && ok; ++n) {
-            const int slot = n % S;
-            ok = wait_warp(&bar_full[slot], (uint32_t)(n / S) & 1u, abort_flag, g.spin);
-            if (!ok) break;
-            if (active && n * nrow + row_off < rows)
-                absmax4(m, *reinterpret_cast<const uint4 *>(mine + (size_t)slot * slot_bytes));
-            if (n + S < T) {  // this position is fetched into again during pass 1
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&bar_empty[slot]);
+    // CTA-wide maxima of pass 1 accumulate in s_part, laid out [channel within group][group] so that the lanes of a
+    // warp (consecutive groups) hit consecutive banks; with the natural [group][channel] layout every shared-memory
+    // atomic of a warp would be an 8-way bank conflict.  It shares its bytes with s_colmul, which is written only
+    // after the grid barrier.
+    uint32_t *s_part = reinterpret_cast<uint32_t *>(smem);
+    for (int k = t; k < K; k += kT) s_part[k] = 0u;
+    __syncthreads();
+    {
+        // thread = (row offset, channel group); rstride = kT / G row offsets are in use (G <= kT).  The division
+        // t / G is a multiplication by g_magic = ceil(2^20 / G), exact for t < 1024 (t * G < 2^20); both constants
+        // come from the host: with 32 warps per SM every instruction of per-thread set-up costs 8 cycles of SM time,
+        // and a 32-bit division is some 25 instructions
+        const int row_off = (int)(((uint32_t)t * g_magic) >> 20), cg = t - row_off * G;
+        if (row_off < rstride) {
+            __half2 m[4];
+            m[0] = m[1] = m[2] = m[3] = __float2half2_rn(0.f);
+            // up to 8 independent 16-byte loads in flight per thread; addresses advance by constant steps
+            const size_t xstep = (size_t)rstride * a.ldx;
+            const uint32_t sstep = (uint32_t)rstride * (uint32_t)K * 2u;
+            const __half *px = a.X + ((size_t)r0 + row_off) * a.ldx + cg * 8;
+            uint8_t *ps = slab + (size_t)row_off * K * 2 + cg * 16;
+            for (int row = row_off; row < rows; row += 8 * rstride) {
+                uint4 v[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u)
+                    v[u] = row + u * rstride < rows ? __ldg(reinterpret_cast<const uint4 *>(px + u * xstep))
+                                                    : make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    absmax4(m, v[u]);
+                    if (row + u * rstride < fit) *reinterpret_cast<uint4 *>(ps + u * sstep) = v[u];
+                }
+                px += 8 * xstep;
+                ps += 8 * sstep;
             }
-        }
-        if (active) {
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
                 const float lo = __low2float(m[i]), hi = __high2float(m[i]);
@@ -222,15 +148,6 @@ __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, const PrepGeom
         }
     }
     __syncthreads();
-    if (s_abort) {  // a wait of pass 1 ran out: let the copies in flight land, mark the workspace, leave
-        if (producer) drain(issued);
-        __syncthreads();
-        if (t == 0) {
-            atomicOr(&a.ctrl->arrived, kPoisonBit);
-            if (a.dev_status) atomicMax(a.dev_status, kStatusTimeout);
-        }
-        return;
-    }
     {
         uint32_t *rep = a.colmax_rep + (size_t)(b % kColmaxReplicas) * K;
         for (int k = t; k < K; k += kT) {
@@ -246,23 +163,23 @@ __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, const PrepGeom
         __threadfence();  // cumulative: publishes the whole CTA's reductions, ordered before it by the barrier
         atomicAdd(&a.ctrl->arrived, 1u);
         bool ok = false;
-        const uint32_t want = gridDim.x + g.extra_arrivals;
+        const uint32_t want = gridDim.x + extra_arrivals;  // (extra arrivals: a test's way of making this wait run out)
         // acquire loads: once the full count is seen, the other CTAs' reductions (released before their
-        // arrivals) are visible to this thread, and through the barrier below to the whole CTA.  A set top
-        // bit means an earlier call on this workspace timed out and left the counters dirty.
-        for (uint32_t i = 0; i < g.spin; ++i) {
+        // arrivals) are visible to this thread, and through the barrier below to the whole CTA.  A set top bit
+        // means an earlier call on this workspace timed out and left the counters dirty.
+        for (uint32_t i = 0; i < spin; ++i) {
             const uint32_t v = ld_acquire_u32(&a.ctrl->arrived);
             if (v & kPoisonBit) break;
             if (v >= want) { ok = true; break; }
         }
+        s_fail = ok ? 0 : 1;
         if (!ok) {
-            s_abort = 1u;
             atomicOr(&a.ctrl->arrived, kPoisonBit);
             if (a.dev_status) atomicMax(a.dev_status, kStatusTimeout);
         }
     }
     __syncthreads();
-    if (s_abort) return;
+    if (s_fail) return;
 
     // ---------------------------------------------------------------- channel factors and s_X (every CTA)
     const float down = __int_as_float((127 - a.exp_factor) << 23);  // 2^-e
@@ -289,14 +206,16 @@ __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, const PrepGeom
     __syncthreads();
     // This CTA holds its copy of the maxima.  The CTA that takes the last ticket knows that every CTA does
     // (and has therefore left the barrier), so it may put the accumulators and both counters back to zero for
-    // the next call.  (No fence: the loads above have returned their values, so stores issued after the last
-    // ticket was taken cannot reach them.)
+    // the next call; the ticket is taken by the last warp, which is off the critical path of the quantization.
+    // (No fence: the loads above have returned their values, so stores issued after the last ticket was
+    // taken cannot reach them.)
     // Every thread derives the factors of the 8 channels it owns in both passes: 2^-e where the channel
-    // holds an element above the threshold (strict), else 1.
+    // holds an element above the threshold (strict), else 1.  (When more channels are flagged than the
+    // capacity allows the call fails with MUXQ_ERR_CAPACITY and Y is unspecified, so no ordering is needed here.)
+    const int row_off = (int)(((uint32_t)t * g_magic) >> 20), cg = t - row_off * G;
     float mul[8];
     uint32_t fmask = 0;  // bit i: channel 8*cg + i is an outlier channel
     {
-        // (every thread has a valid channel group; the copies held by threads beyond the stripe mapping are unused)
         const float4 v0 = reinterpret_cast<const float4 *>(s_colmax)[2 * cg];
         const float4 v1 = reinterpret_cast<const float4 *>(s_colmax)[2 * cg + 1];
         const float cm[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
@@ -308,8 +227,7 @@ __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, const PrepGeom
             fmask |= flagged ? (1u << i) : 0u;
             bmax = fmaxf(bmax, cm[i] * mul[i]);  // power-of-two scaling: exact
         }
-        if (row_off == 0) {  // shared copies: the outlier listing and the per-token path read them
-            // (s_part, which shares its bytes with s_colmul, was last read before the grid barrier)
+        if (row_off == 0) {  // shared copies: the outlier listing below and the per-token path read them
             reinterpret_cast<float4 *>(s_colmul)[2 * cg] = make_float4(mul[0], mul[1], mul[2], mul[3]);
             reinterpret_cast<float4 *>(s_colmul)[2 * cg + 1] = make_float4(mul[4], mul[5], mul[6], mul[7]);
             s_flag[cg] = (uint8_t)fmask;
@@ -328,48 +246,43 @@ __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, const PrepGeom
             a.ctrl->inv_s_x = inv_s;
         }
     }
-
-    // Let a kernel launched as a programmatic dependent (the GEMM) start its set-up on SMs as they free up;
-    // it still waits for this whole grid to finish before it reads anything written here.
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-
-    if (producer) {
-        // -------------------------------------------------------------- outlier list, Aux sources, W_aux, refetches
+    // The last warp (idle or lightly loaded in the quantization loop) lists O in ascending order from the
+    // per-group flag masks; nothing needs the list before the Aux block.  It also fills the source channel
+    // of every Aux column: column c*j + i mirrors channel O_j (Eq. 5), repeated c times for Eq. 7.
+    if (warp == kWarps - 1) {
         uint32_t ticket = 0;
         if (lane == 0) ticket = atomicAdd(&a.ctrl->readers, 1u);  // every thread passed the barrier after the fetch
         int carry = 0;
         for (int base = 0; base < G; base += 32) {
-            const int gi = base + lane;
-            uint32_t mk = gi < G ? s_flag[gi] : 0u;
-            if (!__any_sync(0xffffffffu, mk != 0u)) continue;
-            const int cnt = __popc(mk);
+            const int g = base + lane;
+            uint32_t m = g < G ? s_flag[g] : 0u;
+            if (!__any_sync(0xffffffffu, m != 0u)) continue;
+            const int cnt = __popc(m);
             int incl = cnt;
 #pragma unroll
             for (int o = 1; o < 32; o <<= 1) {
-                const int nn = __shfl_up_sync(0xffffffffu, incl, o);
-                if (lane >= o) incl += nn;
+                const int n = __shfl_up_sync(0xffffffffu, incl, o);
+                if (lane >= o) incl += n;
             }
             int pos = carry + incl - cnt;
-            if (mk) s_rank[gi] = (uint16_t)min(pos, 0xffff);  // rank in O of the group's first outlier channel
-            while (mk) {
-                const int i = __ffs(mk) - 1;
-                mk &= mk - 1;
+            while (m) {
+                const int i = __ffs(m) - 1;
+                m &= m - 1;
                 if (pos < a.cap) {
-                    s_oidx[pos] = 8 * gi + i;
-                    if (b == 0) a.outlier_idx[pos] = 8 * gi + i;
+                    s_oidx[pos] = 8 * g + i;
+                    if (b == 0) a.outlier_idx[pos] = 8 * g + i;
                 }
                 ++pos;
             }
             carry += __shfl_sync(0xffffffffu, incl, 31);
         }
         __syncwarp();
-        const int r = min(carry, a.cap);
         // (a.aux_cols == 0: no Aux block and no W_aux wanted, the list of sources has no room and no reader)
-        const int ucols = min(crep * r, a.aux_cols);
+        const int ucols = min(crep * min(carry, a.cap), a.aux_cols);
         for (int i = lane; i < ucols; i += 32) s_auxsrc[i] = (uint16_t)s_oidx[i / crep];
         // own-scale reading, per tensor: max |Aux| = 2^-e times the largest maximum among the listed channels
         float am = 0.0f;
-        for (int j = lane; j < r; j += 32) am = fmaxf(am, __uint_as_float(s_colmax[s_oidx[j]]) * down);
+        for (int j = lane; j < min(carry, a.cap); j += 32) am = fmaxf(am, __uint_as_float(s_colmax[s_oidx[j]]) * down);
         am = warp_max(am);
         if (lane == 0) {
             s_last = ticket == gridDim.x - 1 ? 1 : 0;
@@ -380,130 +293,81 @@ __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, const PrepGeom
                 a.ctrl->n_outliers = carry;
                 if (carry > a.cap && a.dev_status) atomicMax(a.dev_status, kStatusCapacity);
             }
-            __threadfence_block();
-            s_list_ready = 1;
-        }
-        __syncwarp();
-        if (kPerToken) __syncthreads();  // the per-token path reads the shared factor copies and the Aux sources
-        // W_aux[n, crep*j + i] = W_q[n, O_j]: this CTA's share, one 4-byte word per lane and round.  The GEMM consumes
-        // the Aux columns in steps of 32, i.e. columns [0, pad_cols); an Aux column of zeros makes the matching W_aux
-        // column irrelevant and vice versa, so both blocks are written up to pad_cols only (codes, then zeros).
-        // (With its own scale Aux is the A operand of a product over all aux_cols columns: zeros to the end.)
-        if (a.w_aux) {
-            const int used_cols = crep * r;
-            const int pad_words = a.aux_own ? a.aux_cols >> 2 : ((used_cols + 31) & ~31) >> 2;
-            const int total = a.N * pad_words;
-            for (int i = b * 32 + lane; i < total; i += gridDim.x * 32) {
-                const int n = i / pad_words, w = i - n * pad_words;
-                uint32_t packed = 0;
-#pragma unroll
-                for (int bb = 0; bb < 4; ++bb)
-                    if (w * 4 + bb < used_cols)
-                        packed |= (uint32_t)(uint8_t)a.w_q[(size_t)n * a.ldw + s_auxsrc[w * 4 + bb]] << (8 * bb);
-                *reinterpret_cast<uint32_t *>(a.w_aux + (size_t)n * a.ld_waux + w * 4) = packed;
-            }
-        }
-        if (!kPerToken) {
-            // evicted stripes again, newest first: load T + j fetches stripe T - S - 1 - j
-            for (int j = 0; j < T - Sres; ++j) {
-                if (!issue(T + j, T - Sres - 1 - j)) break;
-                issued = T + j + 1;
-            }
-        }
-    } else if (!kPerToken) {
-        // -------------------------------------------------------------- pass 2, per-tensor scale
-        // The pass-1 mapping again, so the channel factors stay in registers and consecutive lanes store
-        // consecutive codes.  Brackets of 1/s with the channel factor folded in (power of two: exact).
-        float blo[8], bhi[8];
-        {
-            float lo, hi;
-            recip_bracket(inv_s, lo, hi);
-#pragma unroll
-            for (int i = 0; i < 8; ++i) { blo[i] = lo * mul[i]; bhi[i] = hi * mul[i]; }
-        }
-        // 8 values of this thread's channel group -> 8 codes; the exact division only next to a tie
-        auto codes = [&](const uint4 &v) -> uint2 {
-            float f[8];
-            unpack8(v, f);
-            uint32_t code[8];
-            if (quant8_bracket(f, blo, bhi, code)) return codes_exact(v, fmask, down, s, qf);  // next to a tie: rare
-            return pack8(code);
-        };
-        // Threads that write Aux bytes (their chunk holds an outlier channel, or they own the last channel group and
-        // with it the row's zero padding) need the producer warp's listing: rank of their first outlier channel, r.
-        const bool aux_writer = a.aux_q && active && (fmask != 0u || cg == G - 1);
-        int my_rank = 0, r = 0;
-        float s_aux = 1.0f;
-        bool ok = true;
-        if (a.aux_q && __any_sync(0xffffffffu, aux_writer)) {
-            uint32_t i = 0;
-            while (!s_list_ready && ++i < g.spin) { if ((i & 63u) == 63u && *abort_flag) break; }
-            ok = __all_sync(0xffffffffu, s_list_ready != 0);
-            if (!ok) *abort_flag = 1u;
-            r = min(s_r_true, a.cap);
-            s_aux = s_aux_scale;
-            if (fmask) my_rank = s_rank[cg];
-        }
-        const int used_cols = crep * r;
-        const int pad_cols = a.aux_own ? a.aux_cols : (used_cols + 31) & ~31;
-        auto write_aux = [&](const uint4 &v, uint2 code, size_t m) {
-            int8_t *arow = a.aux_q + m * a.ld_aux;
-            if (fmask) {
-                int j = my_rank;
-                uint32_t mk = fmask;
-                const __half *h = reinterpret_cast<const __half *>(&v);
-                while (mk) {
-                    const int i = __ffs(mk) - 1;
-                    mk &= mk - 1;
-                    if (j < a.cap) {
-                        int8_t cb;
-                        if (a.aux_own) cb = (int8_t)quant_exact(__half2float(h[i]) * down, s_aux, qf);  // Eq. 1, own scale
-                        else cb = (int8_t)((i < 4 ? code.x >> (8 * i) : code.y >> (8 * (i - 4))) & 0xffu);
-                        for (int rep = 0; rep < crep; ++rep) arow[crep * j + rep] = cb;
-                    }
-                    ++j;
-                }
-            }
-            if (cg == G - 1)
-                for (int col = used_cols; col < pad_cols; ++col) arow[col] = 0;
-        };
-        const uint8_t *mine = ring + (size_t)row_off * row_bytes + cg * 16;
-        for (int q = 0; q < T && ok; ++q) {
-            // resident stripes first (load numbers T-Sres .. T-1), then the refetched ones (load T + q - Sres)
-            const int n = q < Sres ? T - Sres + q : T + q - Sres;
-            const int stripe = q < Sres ? n : T - 1 - q;
-            const int slot = n % S;
-            if (q >= Sres) {
-                ok = wait_warp(&bar_full[slot], (uint32_t)(n / S) & 1u, abort_flag, g.spin);
-                if (!ok) break;
-            }
-            const int row = stripe * nrow + row_off;
-            if (active && row < rows) {
-                const uint4 v = *reinterpret_cast<const uint4 *>(mine + (size_t)slot * slot_bytes);
-                const uint2 cd = codes(v);
-                const size_t m = (size_t)r0 + row;
-                *reinterpret_cast<uint2 *>(a.body_q + m * a.ld_q + cg * 8) = cd;
-                if (aux_writer) write_aux(v, cd, m);
-            }
-            if (q + Sres < T) {  // a refetch is waiting for this position
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&bar_empty[slot]);
-            }
         }
     }
+    if (kPerToken) __syncthreads();  // the per-token path reads the shared factor copies and the Aux sources
 
-    if (kPerToken) {
-        if (!producer) __syncthreads();  // matches the producer warp's barrier after its listing
+    // Let a kernel launched as a programmatic dependent (the GEMM) start its set-up on SMs as they free up;
+    // it still waits for this whole grid to finish before it reads anything written here.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+
+    // ---------------------------------------------------------------- pass 2: Body_q and the Aux block
+    if (!kPerToken) {
+        // Per-tensor scale: the pass-1 mapping again (a thread owns 8 channels and walks down the
+        // rows), so the channel factors stay in registers and consecutive lanes store consecutive codes.
+        if (row_off < rstride) {
+            // brackets of 1/s with the channel factor folded in (power of two: exact)
+            float blo[8], bhi[8];
+            {
+                float lo, hi;
+                recip_bracket(inv_s, lo, hi);
+#pragma unroll
+                for (int i = 0; i < 8; ++i) { blo[i] = lo * mul[i]; bhi[i] = hi * mul[i]; }
+            }
+            // 8 values of this thread's channel group -> 8 codes; the exact division only next to a tie
+            auto codes = [&](const uint4 &v) -> uint2 {
+                float f[8];
+                unpack8(v, f);
+                uint32_t code[8];
+                if (quant8_bracket(f, blo, bhi, code)) return codes_exact(v, fmask, down, s, qf);  // next to a tie: rare
+                return pack8(code);
+            };
+            // Rows row_off, row_off + rstride, ...: first those held in the slab, two per iteration, then the
+            // rest from global memory (normally L2), four loads in flight.  Addresses advance by constant steps.
+            const uint32_t sstep = (uint32_t)rstride * (uint32_t)K * 2u;
+            const size_t qstep = (size_t)rstride * a.ld_q, xstep = (size_t)rstride * a.ldx;
+            const uint8_t *sp = slab + (size_t)row_off * K * 2 + cg * 16;
+            int8_t *qp = a.body_q + ((size_t)r0 + row_off) * a.ld_q + cg * 8;
+            int row = row_off;
+            for (; row + rstride < fit; row += 2 * rstride) {
+                const uint4 v0 = *reinterpret_cast<const uint4 *>(sp);
+                const uint4 v1 = *reinterpret_cast<const uint4 *>(sp + sstep);
+                *reinterpret_cast<uint2 *>(qp) = codes(v0);
+                *reinterpret_cast<uint2 *>(qp + qstep) = codes(v1);
+                sp += 2 * sstep;
+                qp += 2 * qstep;
+            }
+            if (row < fit) {
+                *reinterpret_cast<uint2 *>(qp) = codes(*reinterpret_cast<const uint4 *>(sp));
+                qp += qstep;
+                row += rstride;
+            }
+            // The rows that did not fit the slab come from global memory again, LAST row first: pass 1 read them in
+            // ascending order, so the highest rows are the ones most likely still in L2 when X is larger than L2
+            // (the slab holds the lowest rows, the first to be evicted).  Four loads in flight; addresses step down
+            // by constant amounts.
+            if (!kAllFit && row < rows) {
+                const int cnt = (rows - row + rstride - 1) / rstride;  // rows of this thread outside the slab
+                const __half *xp = a.X + ((size_t)r0 + row) * a.ldx + cg * 8 + (size_t)(cnt - 1) * xstep;
+                qp += (size_t)(cnt - 1) * qstep;
+                for (int k = cnt - 1; k >= 0; k -= 4) {
+                    uint4 v[4];
+#pragma unroll
+                    for (int u = 0; u < 4; ++u)
+                        v[u] = k - u >= 0 ? __ldg(reinterpret_cast<const uint4 *>(xp - u * xstep))
+                                          : make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        if (k - u >= 0) *reinterpret_cast<uint2 *>(qp - u * qstep) = codes(v[u]);
+                    }
+                    xp -= 4 * xstep;
+                    qp -= 4 * qstep;
+                }
+            }
+        }
+    } else {
         const int r = min(s_r_true, a.cap);
         const int used_cols = crep * r, pad_words = a.aux_own ? a.aux_cols >> 2 : ((used_cols + 31) & ~31) >> 2;
-        // where a row lives: the last Sres stripes are resident in the ring, the others are read from global memory
-        auto row_src = [&](int row) -> const uint4 * {
-            const int stripe = row / nrow;
-            if (stripe >= T - Sres)
-                return reinterpret_cast<const uint4 *>(ring + (size_t)(stripe % S) * slot_bytes +
-                                                       (size_t)(row - stripe * nrow) * row_bytes);
-            return reinterpret_cast<const uint4 *>(a.X + ((size_t)r0 + row) * a.ldx);
-        };
         // A row is walked by a whole warp, or by half a warp when the CTA has more rows than warps: two rounds of
         // rows per warp would run every reduction, division and store latency of a row twice in sequence.
         const int lpr = rows > kWarps ? 16 : 32;  // lanes per row
@@ -516,7 +380,8 @@ __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, const PrepGeom
             const int row = min(base + sub, rows - 1);
             const bool live = base + sub < rows;  // the other half of the warp may have run out of rows
             const size_t m = (size_t)r0 + row;
-            const uint4 *src = row_src(row);
+            const uint4 *src = row < fit ? reinterpret_cast<const uint4 *>(slab + (size_t)row * K * 2)
+                                         : reinterpret_cast<const uint4 *>(a.X + m * a.ldx);
             // per-token scale from Body's row (after the 2^-e redistribution)
             float mx = 0.0f;
             for (int ch = l; ch < G; ch += lpr) {
@@ -573,34 +438,87 @@ __global__ void __launch_bounds__(kT, 1) k_prep(const PrepArgs a, const PrepGeom
         }
     }
 
-    // ---------------------------------------------------------------- end: status, clean-up for the next call
-    __syncthreads();
-    if (s_abort) {  // a wait of pass 2 ran out: let the copies in flight land, mark the workspace, leave
-        if (producer) drain(issued);
-        __syncthreads();
-        if (t == 0) {
-            atomicOr(&a.ctrl->arrived, kPoisonBit);
-            if (a.dev_status) atomicMax(a.dev_status, kStatusTimeout);
+    // ---------------------------------------------------------------- Aux block (per tensor) and W_aux
+    __syncthreads();  // the last warp's outlier list and Aux sources are complete
+    const int r = min(s_r_true, a.cap);
+    const int used_cols = crep * r;
+    // The GEMM consumes the Aux columns in steps of 32, i.e. columns [0, pad_cols); an Aux column of zeros makes the
+    // matching W_aux column irrelevant and vice versa, so both blocks are written up to pad_cols only (codes, then
+    // zeros) and the columns behind are left as they are.
+    // (With its own scale Aux is the A operand of a product over all aux_cols columns: zeros to the end.)
+    const int pad_words = a.aux_own ? a.aux_cols >> 2 : ((used_cols + 31) & ~31) >> 2;
+    const float s_codes = a.aux_own ? s_aux_scale : s;
+    // i / pad_words below as a multiplication where the item counts are small (i < 2^22: the float holds i + 0.5
+    // exactly, and (i + 0.5) / pad_words is at least 0.5 / pad_words away from an integer, far more than the rounding
+    // of the product); a 32-bit division is some 25 instructions, and this phase is one or two items per thread
+    const float inv_pad = 1.0f / (float)max(pad_words, 1);
+    const bool small_counts = (long long)max(rows, a.N) * pad_words < (1ll << 22);
+    auto div_pad = [&](int i) { return small_counts ? (int)(((float)i + 0.5f) * inv_pad) : i / max(pad_words, 1); };
+    // Independent jobs share the CTA's warps so that their latencies overlap instead of adding up: warps 0-15 the
+    // Aux codes, warps 16-31 the W_aux gather (and, in one CTA per launch, the clean-up for the next call).
+    const bool do_aux = a.aux_q && !kPerToken;
+    // Aux codes by the bracket test too (2^-e folded into the brackets), the exact division only next to a tie
+    float alo, ahi;
+    recip_bracket(__frcp_rn(s_codes), alo, ahi);
+    alo *= down;
+    ahi *= down;
+    if (warp < 16) {
+        if (do_aux) {
+            // Aux_q[m, c*j + i] = code of Body[m, O_j] (Eq. 5, shared scale), recomputed from the slab with the
+            // exact division, one 4-byte word per thread and round
+            for (int i = t; i < rows * pad_words; i += 512) {
+                const int row = div_pad(i), w = i - row * pad_words;
+                const size_t m = (size_t)r0 + row;
+                const __half *xr = row < fit ? reinterpret_cast<const __half *>(slab + (size_t)row * K * 2)
+                                             : a.X + m * a.ldx;
+                uint32_t packed = 0;
+#pragma unroll
+                for (int bb = 0; bb < 4; ++bb) {
+                    const int col = w * 4 + bb;
+                    if (col < used_cols) {
+                        const float xv = __half2float(xr[s_auxsrc[col]]);
+                        const uint32_t ca = __float_as_uint(fmaf(xv, ahi, 12582912.0f));
+                        const uint32_t cb = __float_as_uint(fmaf(xv, alo, 12582912.0f));
+                        const uint32_t code = ca == cb ? ca : (uint32_t)quant_exact(xv * down, s_codes, qf);
+                        packed |= (code & 0xffu) << (8 * bb);
+                    }
+                }
+                *reinterpret_cast<uint32_t *>(a.aux_q + m * a.ld_aux + w * 4) = packed;
+            }
         }
-        return;
-    }
-    if (s_last) {
-        uint4 *rep4 = reinterpret_cast<uint4 *>(a.colmax_rep);
-        for (int i = t; i < kColmaxReplicas * (K >> 2); i += kT) rep4[i] = make_uint4(0u, 0u, 0u, 0u);
-        if (t == 0) {
-            a.ctrl->arrived = 0u;
-            a.ctrl->readers = 0u;
+    } else {
+        if (s_last && warp < 24) {
+            uint4 *rep4 = reinterpret_cast<uint4 *>(a.colmax_rep);
+            for (int i = t - 512; i < kColmaxReplicas * (K >> 2); i += 256) rep4[i] = make_uint4(0u, 0u, 0u, 0u);
+            if (t == 512) {
+                a.ctrl->arrived = 0u;
+                a.ctrl->readers = 0u;
+            }
+        }
+        if (a.w_aux) {
+            // W_aux[n, c*j + i] = W_q[n, O_j], one 4-byte word per thread and round, spread over the grid
+            const int total = a.N * pad_words;
+            for (int i = b * 512 + (t - 512); i < total; i += gridDim.x * 512) {
+                const int n = div_pad(i), w = i - n * pad_words;
+                uint32_t packed = 0;
+#pragma unroll
+                for (int bb = 0; bb < 4; ++bb)
+                    if (w * 4 + bb < used_cols)
+                        packed |= (uint32_t)(uint8_t)a.w_q[(size_t)n * a.ldw + s_auxsrc[w * 4 + bb]] << (8 * bb);
+                *reinterpret_cast<uint32_t *>(a.w_aux + (size_t)n * a.ld_waux + w * 4) = packed;
+            }
         }
     }
 }
 
 }  // namespace
 
-bool prep_supported(int M, int K) { return M >= 1 && K >= 8 && K % 8 == 0 && (K >> 3) <= kMaxG; }
+bool prep_supported(int M, int K) { return M >= 1 && K >= 8 && K % 8 == 0 && K <= kMaxK; }
 
 cudaError_t launch_prep(const PrepArgs &a, cudaStream_t s) {
-    static const void *const fns[2] = {reinterpret_cast<const void *>(k_prep<false>),
-                                       reinterpret_cast<const void *>(k_prep<true>)};
+    static const void *const fns[4] = {
+        reinterpret_cast<const void *>(k_prep<false, false>), reinterpret_cast<const void *>(k_prep<false, true>),
+        reinterpret_cast<const void *>(k_prep<true, false>), reinterpret_cast<const void *>(k_prep<true, true>)};
     static PerDevice<int> attr_set;
     const int dev = current_device();
     if (dev < 0) return cudaErrorInvalidDevice;
@@ -617,29 +535,22 @@ cudaError_t launch_prep(const PrepArgs &a, cudaStream_t s) {
     int grid = num_sms();
     if (grid < 1) return cudaErrorInvalidDevice;
     if (grid > a.M) grid = a.M;
-    PrepGeom g{};
-    g.rows_base = a.M / grid;
-    g.rows_extra = a.M % grid;
-    const int rows_max = g.rows_base + (g.rows_extra ? 1 : 0);
-    const int G = a.K >> 3;
-    g.nrow = kConsThreads / G;
-    if (g.nrow > rows_max) g.nrow = rows_max;
+    int rows_base = a.M / grid, rows_extra = a.M % grid;
+    const int rows_max = rows_base + (rows_extra ? 1 : 0);
     const int fixed = fixed_smem_bytes(a.K, a.cap, a.aux_cols);
-    const long long slot_bytes = (long long)g.nrow * a.K * 2;
-    const int t_max = (rows_max + g.nrow - 1) / g.nrow;
-    long long slots = (kMaxDynSmem - fixed) / slot_bytes;
-    if (slots > kMaxSlots) slots = kMaxSlots;
-    if (slots > t_max) slots = t_max;
-    if (slots < 1) return cudaErrorInvalidValue;
-    g.slots = (int)slots;
-    g.g_magic = ((1u << 20) + (uint32_t)G - 1u) / (uint32_t)G;
-    const TestHooks &h = test_hooks();
-    g.spin = h.spin_limit ? h.spin_limit : (1u << 22);
-    g.extra_arrivals = h.prep_extra_arrivals;
+    const long long want = (long long)rows_max * a.K * 2;
+    int slab_bytes = (int)(want < (long long)(kMaxDynSmem - fixed) ? want : (long long)(kMaxDynSmem - fixed));
+    slab_bytes &= ~15;
     PrepArgs args = a;
-    void *params[] = {&args, &g};
-    const void *fn = fns[a.per_token ? 1 : 0];
-    return cudaLaunchCooperativeKernel(fn, dim3(grid), dim3(kT), params, (size_t)(fixed + g.slots * slot_bytes), s);
+    const int G = a.K >> 3;
+    int rstride = kT / G;
+    uint32_t g_magic = ((1u << 20) + (uint32_t)G - 1u) / (uint32_t)G;
+    uint32_t spin = test_hooks().spin_limit ? test_hooks().spin_limit : kBarrierSpin;
+    uint32_t extra_arrivals = test_hooks().prep_extra_arrivals;
+    void *params[] = {&args, &rows_base, &rows_extra, &slab_bytes, &rstride, &g_magic, &spin, &extra_arrivals};
+    const bool all_fit = (long long)slab_bytes >= want;
+    const void *fn = fns[(all_fit ? 2 : 0) + (a.per_token ? 1 : 0)];
+    return cudaLaunchCooperativeKernel(fn, dim3(grid), dim3(kT), params, (size_t)(fixed + slab_bytes), s);
 }
 
 }  // namespace muxq

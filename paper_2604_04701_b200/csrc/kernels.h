@@ -186,6 +186,43 @@ struct DecodeFusedArgs {
 bool decode_fused_supported(int M, int K);
 cudaError_t launch_decode_fused(const DecodeFusedArgs &a, cudaStream_t s);
 
+// A list of decode-shaped layers (M <= 16 rows each) in one persistent launch (k4s_decode_stream.cu).
+constexpr int kChainMaxLayers = 256;
+constexpr int kChainWaitPrev = 1;  // ChainLayer::flags: X of this layer is written by the layer before it
+struct ChainLayer {                // one entry of the device-resident layer table, 64 bytes
+    const __half *X;
+    const int8_t *w_q;
+    const float *s_w;
+    void *Y;
+    int ldx, ldw, ldy, K, N, flags;
+    int unit_off;  // filled by the host: unit u of this layer goes to CTA (unit_off + u) mod grid
+    int seg;       // filled by the host: bytes of each W_q row per ring stage (K / seg stages per unit of 8 rows)
+};
+static_assert(sizeof(ChainLayer) == 64, "layer table entry");
+struct ChainResult {               // per layer, written by CTA 0 (optional)
+    int32_t n_outliers;
+    int32_t status;                // 0 or MUXQ_ERR_CAPACITY
+    float s_x;                     // per-tensor scale (per-token: the first row's)
+    int32_t reserved;
+};
+struct ChainArgs {
+    const ChainLayer *layers;      // device table, or NULL: then `one` is the only layer
+    ChainLayer one;
+    int n_layers, M, kmax, grid;
+    float tau;
+    int exp_factor, qmax, cap, c, per_vec, out_kind;
+    ChainResult *results;          // [n_layers] or NULL
+    uint32_t *barrier;             // arrival counter of the grid-wide barriers, zero on entry (NULL: no layer waits)
+    int32_t *dev_status;
+    uint32_t spin;
+    int slots, slot_bytes;         // ring geometry
+    int pdl;                       // launched with programmatic stream serialization
+};
+// Fills unit_off / seg of every entry (host copy of the table), returns the widest K or -1 if a layer does not fit.
+int chain_plan(ChainLayer *layers, int n_layers, int grid, int slot_bytes);
+bool chain_layer_supported(int M, int K, int N);
+cudaError_t launch_decode_chain(const ChainArgs &a, bool cooperative, cudaStream_t s);
+
 cudaError_t launch_mma_peak(int n, int iters, unsigned long long *cycles_out, int32_t *status, int grid,
                             cudaStream_t s);
 
