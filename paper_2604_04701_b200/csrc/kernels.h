@@ -188,7 +188,8 @@ cudaError_t launch_decode_fused(const DecodeFusedArgs &a, cudaStream_t s);
 
 // A list of decode-shaped layers (M <= 16 rows each) in one persistent launch (k4s_decode_stream.cu).
 constexpr int kChainMaxLayers = 256;
-constexpr int kChainWaitPrev = 1;  // ChainLayer::flags: X of this layer is written by the layer before it
+constexpr int kChainWaitPrev = 1;  // ChainLayer::flags bit 0: X of this layer is written by the layer before it
+                                   // (bits 1..: the ordinal of this wait within the list, filled by chain_plan)
 struct ChainLayer {                // one entry of the device-resident layer table, 64 bytes
     const __half *X;
     const int8_t *w_q;
@@ -206,8 +207,7 @@ struct ChainResult {               // per layer, written by CTA 0 (optional)
     int32_t reserved;
 };
 struct ChainArgs {
-    const ChainLayer *layers;      // device table, or NULL: then `one` is the only layer
-    ChainLayer one;
+    const ChainLayer *layers;      // device table
     int n_layers, M, kmax, grid;
     float tau;
     int exp_factor, qmax, cap, c, per_vec, out_kind;
@@ -216,10 +216,13 @@ struct ChainArgs {
     int32_t *dev_status;
     uint32_t spin;
     int slots, slot_bytes;         // ring geometry
-    int pdl;                       // launched with programmatic stream serialization
+    int nbuf, pgroups;             // buffers of prepared X, groups of prepare warps (set by the launcher)
+    int stage_x;                   // the fp16 rows of X are staged in shared memory one layer ahead (set by the launcher)
 };
-// Fills unit_off / seg of every entry (host copy of the table), returns the widest K or -1 if a layer does not fit.
+// Fills unit_off / seg / wait ordinals of every entry (host copy of the table); returns the widest K, -1 if a layer
+// does not fit.
 int chain_plan(ChainLayer *layers, int n_layers, int grid, int slot_bytes);
+int chain_slot_bytes(int M);  // bytes of a ring stage for lists of M-row layers
 bool chain_layer_supported(int M, int K, int N);
 cudaError_t launch_decode_chain(const ChainArgs &a, bool cooperative, cudaStream_t s);
 
