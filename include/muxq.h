@@ -219,6 +219,52 @@ int muxq_linear_host(const void *X_f16_host, int M, int K, const int8_t *W_q, in
                      void *workspace, size_t workspace_bytes, int32_t *dev_status, void *stream);
 
 /*
+ * A list of decode-shaped layers (M <= 16 token rows each) in ONE persistent launch: the same computation as
+ * muxq_linear with M <= 16 for every entry (Section III-C, Eq. 1, Eq. 4-5, Eq. 7, Eq. 3), with the weight
+ * stream running on across layer boundaries -- what the projections of consecutive GPT-2 blocks (Section
+ * IV-C: c_attn, attention c_proj, c_fc, MLP c_proj) look like to the memory system at decode time.  A layer's
+ * W_q is fetched while the layers before it are still being computed; a one-layer call cannot do that.
+ *
+ * muxq_layer: X [M, ldx] fp16, W_q [N, ldw] int8 and s_w from muxq_quantize(is_weight = 1), Y [M, ldy] by the
+ * list's out_kind.  flags = MUXQ_LAYER_WAIT_PREV says that this layer's X is written by the layer before it
+ * in the list (its Y, or memory derived from nothing else): all CTAs then meet at a bounded grid-wide barrier
+ * before they read it.  Without the flag the layers are independent and no CTA ever waits for another.
+ * Limits: 1 <= n_layers <= 256, M <= 16, K a multiple of 64 up to 8192, N a multiple of 8, shared Aux scale;
+ * alignment as for muxq_linear.  One params / M / out_kind for the whole list.
+ *
+ * muxq_chain_build validates the list, derives the schedule (which CTA streams which rows of every W_q) into
+ * plan_host -- caller-owned HOST memory of muxq_chain_plan_bytes(n_layers) bytes, which must stay valid and
+ * unchanged as long as the plan is used -- and enqueues its copy to plan_dev (device memory of the same size,
+ * 16-byte aligned) on `stream`.  muxq_chain_run enqueues the launch.  results (device, n_layers entries, or
+ * NULL) receives r, the per-tensor scale and 0 / MUXQ_ERR_CAPACITY per layer; a layer whose r exceeds
+ * max_outliers leaves its Y unspecified (in bounds), raises the status word, and the list goes on.  The status
+ * word is sticky as everywhere.  Runs of one plan must not overlap on the GPU (the plan holds the barrier
+ * counter); runs of different plans may.  W_q and s_w are constants of the layers: they must not be written
+ * while a run that reads them may be in flight.
+ */
+#define MUXQ_LAYER_WAIT_PREV 1
+typedef struct muxq_layer {
+    const void *X_f16;
+    const int8_t *W_q;
+    const float *s_w;
+    void *Y;
+    int ldx, ldw, ldy;
+    int K, N;
+    int flags;
+} muxq_layer;
+typedef struct muxq_chain_result {
+    int32_t n_outliers; /* r of this layer's X */
+    int32_t status;     /* 0 or MUXQ_ERR_CAPACITY */
+    float s_x;          /* per-tensor scale (per token: the first row's) */
+    int32_t reserved;
+} muxq_chain_result;
+size_t muxq_chain_plan_bytes(int n_layers); /* 0 on n_layers outside 1..256 */
+int muxq_chain_build(const muxq_layer *layers_host, int n_layers, int M, const muxq_params *p, int out_kind,
+                     void *plan_host, void *plan_dev, size_t plan_bytes, void *stream);
+int muxq_chain_run(const void *plan_host, void *plan_dev, muxq_chain_result *results_or_null,
+                   int32_t *dev_status, void *stream);
+
+/*
  * The decode-shaped layer without a caller-provided workspace.  (The paper has no counterpart:
  * this entry point exists for the sake of callers, not of the method.)
  *

@@ -23,6 +23,7 @@ EXPORTS = (
     "muxq_host_workspace_bytes", "muxq_workspace_init", "muxq_workspace_view", "muxq_detect_outliers", "muxq_build_aux",
     "muxq_quantize", "muxq_gemm", "muxq_linear", "muxq_linear_events", "muxq_linear_host",
     "muxq_linear_decode_noalloc", "muxq_int8_mma_peak", "muxq_test_hooks", "muxq_read_status",
+    "muxq_chain_plan_bytes", "muxq_chain_build", "muxq_chain_run",
     "muxq_status_string",
 )
 
@@ -96,6 +97,9 @@ def lib() -> ctypes.CDLL:
         L.muxq_linear_decode_noalloc.argtypes = [vp, i, i, i, vp, i, vp, i, pp, vp, i, i, vp, vp]; L.muxq_linear_decode_noalloc.restype = i
         L.muxq_int8_mma_peak.argtypes = [i, i, i, vp, vp, vp]; L.muxq_int8_mma_peak.restype = i
         L.muxq_test_hooks.argtypes = [vp]; L.muxq_test_hooks.restype = i
+        L.muxq_chain_plan_bytes.argtypes = [i]; L.muxq_chain_plan_bytes.restype = sz
+        L.muxq_chain_build.argtypes = [vp, i, i, pp, i, vp, vp, sz, vp]; L.muxq_chain_build.restype = i
+        L.muxq_chain_run.argtypes = [vp, vp, vp, vp, vp]; L.muxq_chain_run.restype = i
         L.muxq_read_status.argtypes = [vp, vp]; L.muxq_read_status.restype = i
         L.muxq_status_string.argtypes = [i]; L.muxq_status_string.restype = ctypes.c_char_p
         _lib = L
@@ -301,6 +305,53 @@ def muxq_int8_mma_peak(mma_n: int, iters: int, ctas: int, ws: Workspace) -> torc
     cycles = torch.zeros(ctas, dtype=torch.int64, device=ws.buf.device)
     _check("muxq_int8_mma_peak", lib().muxq_int8_mma_peak(mma_n, iters, ctas, _ptr(cycles), _ptr(ws.status), _stream()))
     return cycles
+
+
+MUXQ_LAYER_WAIT_PREV = 1
+
+
+class _CLayer(ctypes.Structure):
+    _fields_ = [("X_f16", ctypes.c_void_p), ("W_q", ctypes.c_void_p), ("s_w", ctypes.c_void_p), ("Y", ctypes.c_void_p),
+                ("ldx", ctypes.c_int), ("ldw", ctypes.c_int), ("ldy", ctypes.c_int), ("K", ctypes.c_int),
+                ("N", ctypes.c_int), ("flags", ctypes.c_int)]
+
+
+class Chain:
+    """A list of decode-shaped layers run by one persistent launch (muxq_chain_build / muxq_chain_run).
+
+    layers: sequence of (X [M,K] f16, w_q [N,K] i8, s_w, Y [M,N], flags).  The tensors are kept alive by this
+    object; results (one row of [r, status, s_x bits, 0] per layer, int32) and the status word live on the device."""
+
+    def __init__(self, layers, p: MuxqParams, out_kind: int = MUXQ_OUT_F16):
+        n = len(layers)
+        self.layers = list(layers)
+        self.M = int(layers[0][0].shape[0])
+        dev = layers[0][0].device
+        arr = (_CLayer * n)()
+        for k, (X, w_q, s_w, Y, flags) in enumerate(layers):
+            assert X.is_cuda and X.dtype == torch.float16 and X.stride(1) == 1 and X.shape[0] == self.M
+            arr[k] = _CLayer(X.data_ptr(), w_q.data_ptr(), s_w.data_ptr(), Y.data_ptr(), X.stride(0), w_q.stride(0),
+                             Y.stride(0), X.shape[1], w_q.shape[0], int(flags))
+        nbytes = int(lib().muxq_chain_plan_bytes(n))
+        if nbytes == 0:
+            raise MuxqError("muxq_chain_plan_bytes", MUXQ_ERR_INVALID_ARG)
+        self.plan_host = (ctypes.c_uint8 * nbytes)()
+        self.plan_dev = torch.empty(nbytes, dtype=torch.uint8, device=dev)
+        self.results = torch.zeros(n, 4, dtype=torch.int32, device=dev)
+        self.status = torch.zeros(1, dtype=torch.int32, device=dev)
+        with torch.cuda.device(dev):
+            _check("muxq_chain_build",
+                   lib().muxq_chain_build(arr, n, self.M, ctypes.byref(p.c()), out_kind, self.plan_host,
+                                          _ptr(self.plan_dev), nbytes, _stream()))
+            torch.cuda.current_stream().synchronize()  # the copy has read plan_host
+
+    def run(self) -> None:
+        with torch.cuda.device(self.plan_dev.device):
+            _check("muxq_chain_run", lib().muxq_chain_run(self.plan_host, _ptr(self.plan_dev), _ptr(self.results),
+                                                          _ptr(self.status), _stream()))
+
+    def read_status(self) -> int:
+        return int(lib().muxq_read_status(_ptr(self.status), _stream()))
 
 
 class _CTestHooks(ctypes.Structure):

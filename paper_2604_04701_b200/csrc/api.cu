@@ -494,6 +494,89 @@ int muxq_int8_mma_peak(int mma_n, int iters, int ctas, unsigned long long *cycle
     return cuda_rc(launch_mma_peak(mma_n, iters, cycles_per_cta, dev_status, ctas, static_cast<cudaStream_t>(stream)));
 }
 
+// ---------------------------------------------------------------- a list of decode-shaped layers in one launch
+namespace {
+constexpr uint32_t kPlanMagic = 0x4d555851u;
+struct PlanHeader {           // first 128 bytes of a plan (host and device copy alike)
+    uint32_t magic;
+    int32_t n_layers, M, kmax, grid, any_wait, out_kind;
+    muxq_params params;
+    uint32_t barrier;         // device copy: arrival counter of the grid-wide barriers
+    uint32_t reserved[15];
+};
+static_assert(sizeof(PlanHeader) <= 128, "plan header");
+constexpr size_t kPlanTableOffset = 128;
+}  // namespace
+
+size_t muxq_chain_plan_bytes(int n_layers) {
+    if (n_layers < 1 || n_layers > kChainMaxLayers) return 0;
+    return kPlanTableOffset + (size_t)n_layers * sizeof(ChainLayer);
+}
+
+int muxq_chain_build(const muxq_layer *layers, int n_layers, int M, const muxq_params *p, int out_kind,
+                     void *plan_host, void *plan_dev, size_t plan_bytes, void *stream) {
+    if (!layers || !plan_host || !plan_dev || n_layers < 1 || M < 1 || !params_ok(p) || out_kind < 0 || out_kind > 2)
+        return MUXQ_ERR_INVALID_ARG;
+    if (n_layers > kChainMaxLayers || M > 16 || p->aux_scale != MUXQ_AUX_SHARED) return MUXQ_ERR_UNSUPPORTED;
+    if (plan_bytes < muxq_chain_plan_bytes(n_layers)) return MUXQ_ERR_WORKSPACE;
+    if (!aligned16(plan_dev)) return MUXQ_ERR_UNSUPPORTED;
+    const int grid = num_sms();
+    if (grid < 1) return MUXQ_ERR_CUDA;
+    PlanHeader *h = static_cast<PlanHeader *>(plan_host);
+    ChainLayer *tab = reinterpret_cast<ChainLayer *>(static_cast<uint8_t *>(plan_host) + kPlanTableOffset);
+    memset(h, 0, sizeof(PlanHeader));
+    const int yal = out_kind == MUXQ_OUT_F16 ? 8 : 4;
+    int any_wait = 0;
+    for (int l = 0; l < n_layers; ++l) {
+        const muxq_layer &in = layers[l];
+        if (!in.X_f16 || !in.W_q || !in.s_w || !in.Y || in.K <= 0 || in.N <= 0 || in.ldx < in.K || in.ldw < in.K ||
+            in.ldy < in.N || (in.flags & ~MUXQ_LAYER_WAIT_PREV) || (l == 0 && in.flags))
+            return MUXQ_ERR_INVALID_ARG;
+        if (!chain_layer_supported(M, in.K, in.N) || in.ldx % 8 || in.ldw % 16 || in.ldy % yal || !aligned16(in.X_f16) ||
+            !aligned16(in.W_q) || !aligned16(in.Y) || (p->gran == MUXQ_PER_VECTOR && !aligned16(in.s_w)))
+            return MUXQ_ERR_UNSUPPORTED;
+        ChainLayer &o = tab[l];
+        o.X = static_cast<const __half *>(in.X_f16);
+        o.w_q = in.W_q;
+        o.s_w = in.s_w;
+        o.Y = in.Y;
+        o.ldx = in.ldx; o.ldw = in.ldw; o.ldy = in.ldy; o.K = in.K; o.N = in.N;
+        o.flags = (in.flags & MUXQ_LAYER_WAIT_PREV) ? kChainWaitPrev : 0;
+        any_wait |= o.flags;
+    }
+    const int kmax = chain_plan(tab, n_layers, grid, chain_slot_bytes(M));
+    if (kmax < 0) return MUXQ_ERR_UNSUPPORTED;
+    h->magic = kPlanMagic;
+    h->n_layers = n_layers; h->M = M; h->kmax = kmax; h->grid = grid; h->any_wait = any_wait; h->out_kind = out_kind;
+    h->params = *p;
+    return cuda_rc(cudaMemcpyAsync(plan_dev, plan_host, muxq_chain_plan_bytes(n_layers), cudaMemcpyHostToDevice,
+                                   static_cast<cudaStream_t>(stream)));
+}
+
+int muxq_chain_run(const void *plan_host, void *plan_dev, muxq_chain_result *results, int32_t *dev_status,
+                   void *stream) {
+    if (!plan_host || !plan_dev || !dev_status) return MUXQ_ERR_INVALID_ARG;
+    const PlanHeader *h = static_cast<const PlanHeader *>(plan_host);
+    if (h->magic != kPlanMagic || h->grid != num_sms()) return MUXQ_ERR_INVALID_ARG;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    uint8_t *pd = static_cast<uint8_t *>(plan_dev);
+    ChainArgs a{};
+    a.layers = reinterpret_cast<const ChainLayer *>(pd + kPlanTableOffset);
+    a.n_layers = h->n_layers; a.M = h->M; a.kmax = h->kmax; a.grid = h->grid;
+    a.tau = h->params.threshold; a.exp_factor = h->params.exp_factor; a.qmax = qmax_of(h->params.act_bits);
+    a.cap = h->params.max_outliers; a.c = (1 << h->params.exp_factor) - 1;
+    a.per_vec = h->params.gran == MUXQ_PER_VECTOR; a.out_kind = h->out_kind;
+    a.results = reinterpret_cast<ChainResult *>(results);
+    a.dev_status = dev_status;
+    a.spin = test_hooks().spin_limit ? test_hooks().spin_limit : (1u << 22);
+    a.slot_bytes = chain_slot_bytes(h->M);
+    if (h->any_wait) {
+        a.barrier = reinterpret_cast<uint32_t *>(pd + offsetof(PlanHeader, barrier));
+        if (cudaMemsetAsync(a.barrier, 0, 4, s) != cudaSuccess) return MUXQ_ERR_CUDA;
+    }
+    return cuda_rc(launch_decode_chain(a, h->any_wait != 0, s));
+}
+
 int muxq_test_hooks(const muxq_test_hooks_t *h) {
     TestHooks t{};
     if (h) {
