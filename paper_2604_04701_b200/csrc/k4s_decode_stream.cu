@@ -4,7 +4,7 @@
 // cannot keep HBM busy: a layer moves 1.6-6.6 MB, less than a microsecond of HBM time.  Here the weight stream
 // never stops at a layer boundary:
 //   loader warps    walk the list of layers and, for every unit of 8 output channels that belongs to this CTA,
-//                   fetch the 8 rows of W_q with 16-byte asynchronous copies (cp.async, 64 threads) into a ring
+//                   fetch the 8 rows of W_q with 16-byte asynchronous copies (cp.async, 128 threads) into a ring
 //                   of shared-memory stages; every loader thread's copies report to the stage's mbarrier when
 //                   they have landed.  They depend on nothing but the ring's free slots, so they run several
 //                   layers ahead of the arithmetic.  (Bulk copies of the copy engine gave the same rate.)
@@ -34,7 +34,7 @@ namespace {
 
 constexpr int kUW = 8;                  // unit warps (warps 0..7)
 constexpr int kPW = 8;                  // prepare warps (warps 8..15)
-constexpr int kLW = 2;                  // loader warps (warps 16, 17)
+constexpr int kLW = 4;                  // loader warps (warps 16..19)
 constexpr int kLT = 32 * kLW;           // loader threads
 constexpr int kLoader0 = kUW + kPW;     // index of the first loader warp
 constexpr int kThreads = 32 * (kLoader0 + kLW);
@@ -195,8 +195,8 @@ __global__ void __launch_bounds__(kThreads, 1) k_decode_stream(const ChainArgs a
     if (warp >= kLoader0) {
         // ------------------------------------------------------------ loaders: W_q of every layer, in order.
         // The weights are constants of the layers: nothing here waits for X or a barrier.
-        // Thread (lr, lc) of the 64 copies row lr of a unit's 8 rows, 16-byte pieces lc, lc + 8, ...
-        const int tl = t - 32 * kLoader0, lr = tl >> 3, lc = tl & 7;
+        // Thread (lr, lc) of the 128 copies row lr of a unit's 8 rows, 16-byte pieces lc, lc + 16, ...
+        const int tl = t - 32 * kLoader0, lr = tl >> 4, lc = tl & 15;
         RingPos pos{0, 0u};
         int issued = 0;
         bool ok = true;
@@ -214,7 +214,7 @@ __global__ void __launch_bounds__(kThreads, 1) k_decode_stream(const ChainArgs a
                     if (tl == 0) s_issued = issued;  // the slot's previous use is over: its barrier may be waited on
                     uint8_t *dst = ring + (size_t)pos.slot * a.slot_bytes + lr * ly.seg + lc * 16;
                     const int8_t *src = wrow + (size_t)st * ly.seg;
-                    for (int c = lc; c < pieces; c += 8, dst += 128, src += 128) cp_async16(dst, src);
+                    for (int c = lc; c < pieces; c += 16, dst += 256, src += 256) cp_async16(dst, src);
                     cp_async_arrive(&bar_full[pos.slot]);
                     pos.advance(1, S);
                 }
@@ -223,7 +223,9 @@ __global__ void __launch_bounds__(kThreads, 1) k_decode_stream(const ChainArgs a
         asm volatile("cp.async.wait_all;" ::: "memory");  // nothing of this thread is in flight when the CTA ends
     } else if (warp >= kUW) {
         // ------------------------------------------------------------ prepare warps: X of layer l into buffer l mod NB
-        // PG groups of warps, group gi on layers gi, gi + PG, ...
+        // PG groups of warps.  Layer l belongs to group (l + l / PG) mod PG: every run of PG consecutive layers gives
+        // each group one layer, and the assignment shifts by one from run to run, so that a list with a period of
+        // PG layers (the four projections of a block) does not hand the same group the widest layer every time.
         const int wp = warp - kUW, wpg = kPW / PG, gi = wp / wpg, wg = wp - gi * wpg;
         const int GT = 32 * wpg, tp = t - 32 * (kUW + gi * wpg), bid = 1 + gi;
         const float down = __int_as_float((127 - a.exp_factor) << 23);  // 2^-e
@@ -231,25 +233,34 @@ __global__ void __launch_bounds__(kThreads, 1) k_decode_stream(const ChainArgs a
         const bool first_cta = cta == 0;
         uint32_t *rowmax = s_rowmax[gi];
         // asynchronous copy of the fp16 rows of a layer's X into one of this group's two staging copies
-        auto stage_x = [&](int l) {
+        auto group_of = [&](int l) { return (l + l / PG) % PG; };
+        auto next_mine = [&](int l) {  // the next layer of this group behind layer l (or n_layers)
+            for (++l; l < a.n_layers && group_of(l) != gi; ++l) {}
+            return l;
+        };
+        auto stage_x = [&](int l, int copy) {
             const ChainLayer &ly = tab[l];
-            uint8_t *dst = xbase + NB * L.buf_bytes + (2 * gi + ((l / PG) & 1)) * L.xs_bytes;
+            uint8_t *dst = xbase + NB * L.buf_bytes + (2 * gi + copy) * L.xs_bytes;
             const int G = ly.K >> 3;
             for (int cg = tp; cg < G; cg += GT)
                 for (int m = 0; m < M; ++m) cp_async16(dst + (size_t)m * ly.K * 2 + cg * 16, ly.X + (size_t)m * ly.ldx + cg * 8);
         };
         const bool staged = L.xs_bytes > 0;
         auto waits_for_prev = [&](int l) { return (tab[l].flags & kChainWaitPrev) && a.barrier; };
-        if (staged && gi < a.n_layers && !waits_for_prev(gi)) stage_x(gi);
+        int mine = 0;  // layers this group has prepared so far: parity selects the staging copy
+        {
+            const int l0 = next_mine(-1);
+            if (staged && l0 < a.n_layers && !waits_for_prev(l0)) stage_x(l0, 0);
+        }
         bool stop = false;
-        for (int l = gi; l < a.n_layers && !stop; l += PG) {
+        for (int l = next_mine(-1); l < a.n_layers && !stop; l = next_mine(l), ++mine) {
             const ChainLayer ly = tab[l];
             const int K = ly.K, G = K >> 3, b = l % NB, ph = l / NB;
             uint8_t *buf = xbase + b * L.buf_bytes;
             XHeader *hdr = reinterpret_cast<XHeader *>(buf);
             int8_t *xq = reinterpret_cast<int8_t *>(buf + L.off_xq);
             uint8_t *s_mask = buf + L.off_mask, *s_segflag = buf + L.off_segflag, *s_grpmask = buf + L.off_grpmask;
-            const uint8_t *xs = staged ? xbase + NB * L.buf_bytes + (2 * gi + ((l / PG) & 1)) * L.xs_bytes : nullptr;
+            const uint8_t *xs = staged ? xbase + NB * L.buf_bytes + (2 * gi + (mine & 1)) * L.xs_bytes : nullptr;
             const bool wait_prev = waits_for_prev(l);
             bool ok = true;
             // the buffer was last read for layer l - NB
@@ -270,13 +281,16 @@ __global__ void __launch_bounds__(kThreads, 1) k_decode_stream(const ChainArgs a
                     if (!seen) *abort_flag = 1u;
                 }
                 bar_prep(bid, GT);
-                if (staged) stage_x(l);  // could not be fetched ahead
+                if (staged) stage_x(l, mine & 1);  // could not be fetched ahead
             }
             if (tp < 16) rowmax[tp] = 0u;
             for (int i = tp; i < (K >> 6); i += GT) s_segflag[i] = 0;
             if (staged) asm volatile("cp.async.wait_all;" ::: "memory");
             bar_prep(bid, GT);  // this layer's staging copy is complete and visible; the group's other copy is free
-            if (staged && l + PG < a.n_layers && !waits_for_prev(l + PG)) stage_x(l + PG);
+            {
+                const int ln = next_mine(l);
+                if (staged && ln < a.n_layers && !waits_for_prev(ln)) stage_x(ln, (mine + 1) & 1);
+            }
             auto x_chunk = [&](int m, int cg) -> uint4 {
                 return xs ? *reinterpret_cast<const uint4 *>(xs + (size_t)m * K * 2 + cg * 16)
                           : __ldcg(reinterpret_cast<const uint4 *>(ly.X + (size_t)m * ly.ldx) + cg);
