@@ -644,6 +644,10 @@ def run_muxq(args, rank, world):
     mx.lib()  # fails loudly if the CUDA library is missing
     peaks = load_peaks()
 
+    if args.decode_only:  # profiling aid: only the decode section, printed as its own JSON line
+        decode, decode_roof = measure_decode(mx, torch, dev, peaks, mx.MuxqParams(max_outliers=32))
+        print(json.dumps({"decode": decode, "roofline_decode": decode_roof}))
+        return
     head = measure_prefill(mx, torch, dist, dev, world, HEADLINE_CONFIG, args.steps, args.warmup, headline=True)
     clocks = head["clocks"]
     int8_peak, peak_source = int8_peak_for(peaks, clocks)
@@ -699,6 +703,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-decode", action="store_true")
     ap.add_argument("--no-small", action="store_true", help="skip the GPT-2-small workload reported under extra")
+    ap.add_argument("--decode-only", action="store_true", help="run only the decode measurements (for profiling)")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
