@@ -331,6 +331,31 @@ def test_decode_matches_oracle(mx, M, K, N):
 
 
 # ------------------------------------------------------------------ edge cases
+@pytest.mark.parametrize("M", [1, 4, 16, 64])
+def test_layer_call_directly_after_its_weights_were_rewritten(mx, M):
+    """W_q and s_w are rewritten by ordinary kernels (the library's weight quantization, then a device copy into the
+    very buffers the layer reads) directly before the layer call on the same stream.  The layer kernels fetch weight
+    tiles ahead of their programmatic wait; predecessors that do not release their dependents early -- these -- must
+    still be seen in full.  Decode (M <= 16) and GEMM path."""
+    K, N = 1280, 1280
+    p = mx.MuxqParams(max_outliers=32)
+    x, _ = synth.make_x(21, 1, M, K, 6, 50.0, 50.0)
+    xd = dev(x)
+    ws = mx.Workspace(mx.muxq_workspace_bytes(M, K, N, p))
+    w1, w2 = synth.make_w(21, 1, K, N), synth.make_w(22, 2, K, N, sigma=0.05)
+    wsw = mx.Workspace(mx.muxq_small_workspace_bytes(N))
+    w_q, s_w = mx.muxq_quantize(dev(w1), p, True, wsw)
+    y1 = mx.muxq_linear(xd, w_q, s_w, p, ws, mx.MUXQ_OUT_F32)           # quantize -> layer, back to back
+    wq2, sw2 = mx.muxq_quantize(dev(w2), p, True, wsw)
+    for _ in range(3):
+        w_q.copy_(wq2); s_w.copy_(sw2)                                   # device copies into the buffers in use ...
+        y2 = mx.muxq_linear(xd, w_q, s_w, p, ws, mx.MUXQ_OUT_F32)       # ... directly followed by the layer
+    assert mx.muxq_read_status(ws) == 0
+    for w, y in ((w1, y1), (w2, y2)):
+        _, _, res = oracle_linear(x, w, p)
+        assert np.array_equal(y.cpu().numpy(), res.y32)
+
+
 def test_zero_outliers_equals_naive_int8(mx):
     x, w, _ = make_case(70, 256, 512, 256, n_out=0)
     p = mx.MuxqParams(threshold=1e4)
