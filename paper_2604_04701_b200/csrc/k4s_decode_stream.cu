@@ -4,10 +4,14 @@
 // cannot keep HBM busy: a layer moves 1.6-6.6 MB, less than a microsecond of HBM time.  Here the weight stream
 // never stops at a layer boundary:
 //   loader warps    walk the list of layers and, for every unit of 8 output channels that belongs to this CTA,
-//                   fetch the 8 rows of W_q with 16-byte asynchronous copies (cp.async, 128 threads) into a ring
-//                   of shared-memory stages; every loader thread's copies report to the stage's mbarrier when
-//                   they have landed.  They depend on nothing but the ring's free slots, so they run several
-//                   layers ahead of the arithmetic.  (Bulk copies of the copy engine gave the same rate.)
+//                   fetch the 8 rows of W_q with bulk asynchronous copies (cp.async.bulk, no multicast) into a
+//                   ring of shared-memory stages; the copies report their bytes to the stage's mbarrier.  They
+//                   depend on nothing but the ring's free slots, so they run several layers ahead of the
+//                   arithmetic.  Each loader warp takes every fourth stage on its own: one loop over the stages
+//                   (wait for the slot, issue, next) costs a single warp several hundred cycles per stage however
+//                   the bytes are moved (measured: 10 KB per 0.3 us, 4.4 TB/s over 148 SMs, with one loop of 128
+//                   threads making 16-byte copies; 6.7-7 TB/s with four independent loops), and with one bulk
+//                   copy per stage or per row the loop is a few dozen instructions.
 //   prepare warps   per layer: derive the channel maxima, the outlier flags, the scale(s) and the INT8 codes of X
 //                   into a shared-memory buffer (redundant per CTA, no grid-wide exchange).  The phases of one
 //                   layer are short serial chains with barriers in between, so for small M several groups of
@@ -35,7 +39,6 @@ namespace {
 constexpr int kUW = 8;                  // unit warps (warps 0..7)
 constexpr int kPW = 8;                  // prepare warps (warps 8..15)
 constexpr int kLW = 4;                  // loader warps (warps 16..19)
-constexpr int kLT = 32 * kLW;           // loader threads
 constexpr int kLoader0 = kUW + kPW;     // index of the first loader warp
 constexpr int kThreads = 32 * (kLoader0 + kLW);
 constexpr int kMaxK = 8192;             // widest layer: 1024 channel groups of 8
@@ -55,13 +58,17 @@ __device__ __forceinline__ void mma_s8(int (&d)[4], uint32_t a0, uint32_t a1, ui
         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
-// 16 bytes global -> shared, asynchronously; cp_async_arrive makes the executing thread's copies issued so far
-// count as ONE arrival on the mbarrier once they have all landed (the barrier's count includes every loader thread).
+// 16 bytes global -> shared, asynchronously (the fp16 rows of X; completion through cp.async.wait_all)
 __device__ __forceinline__ void cp_async16(void *smem_dst, const void *gsrc) {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(smem_dst)), "l"(gsrc) : "memory");
 }
-__device__ __forceinline__ void cp_async_arrive(uint64_t *bar) {
-    asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+// `bytes` (a multiple of 16, both addresses 16-byte aligned) global -> shared by the copy engine; the bytes are
+// reported to the mbarrier as they land
+__device__ __forceinline__ void bulk_load(void *smem_dst, const void *gsrc, uint32_t bytes, uint64_t *bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                     smem_u32(smem_dst)),
+                 "l"(gsrc), "r"(bytes), "r"(smem_u32(bar))
+                 : "memory");
 }
 
 // Bounded wait of a whole converged warp that backs off between polls: the warps of this kernel spend most of
@@ -152,7 +159,7 @@ __global__ void __launch_bounds__(kThreads, 1) k_decode_stream(const ChainArgs a
     __shared__ uint32_t s_rowmax[kMaxGroups][16];   // bit patterns of non-negative floats (row maxima of Body)
     __shared__ float s_wmax[kPW];
     __shared__ uint32_t s_abort;
-    __shared__ volatile int s_issued;               // stages the loaders have begun to fill so far
+    __shared__ volatile uint32_t s_begun[kMaxSlots];  // uses of a slot the loaders have begun to fill so far
 
     const int t = threadIdx.x, lane = t & 31;
     const int warp = __shfl_sync(0xffffffffu, t >> 5, 0);  // warp-uniform by construction
@@ -172,15 +179,15 @@ __global__ void __launch_bounds__(kThreads, 1) k_decode_stream(const ChainArgs a
     }
     if (t == 0) {
         for (int s = 0; s < S; ++s) {
-            mbar_init(&bar_full[s], kLT);  // every loader thread, once its copies into the stage have landed
+            mbar_init(&bar_full[s], 1);    // the loader's arrival that announces the stage's bytes; the copies report them
             mbar_init(&bar_empty[s], 1);   // the one unit warp that took the stage
+            s_begun[s] = 0u;
         }
         for (int b = 0; b < kMaxBufs; ++b) {
             mbar_init(&bar_ready[b], 1);   // one prepare thread, after its group's barrier
             mbar_init(&bar_free[b], kUW);  // every unit warp, once per layer
         }
         s_abort = 0u;
-        s_issued = 0;
         fence_barrier_init();
     }
     __syncthreads();
@@ -194,33 +201,59 @@ __global__ void __launch_bounds__(kThreads, 1) k_decode_stream(const ChainArgs a
 
     if (warp >= kLoader0) {
         // ------------------------------------------------------------ loaders: W_q of every layer, in order.
-        // The weights are constants of the layers: nothing here waits for X or a barrier.
-        // Thread (lr, lc) of the 128 copies row lr of a unit's 8 rows, 16-byte pieces lc, lc + 16, ...
-        const int tl = t - 32 * kLoader0, lr = tl >> 4, lc = tl & 15;
-        RingPos pos{0, 0u};
-        int issued = 0;
-        bool ok = true;
+        // The weights are constants of the layers: nothing here waits for X or a barrier.  Loader warp g fills
+        // the stages of this CTA whose running number is g modulo the number of loader warps in use, which
+        // divides the number of slots: a slot is always refilled by the warp that filled it before (a warp that
+        // met another warp's slot could mistake an older phase of its barrier).
+        // A stage is 8 rows of `seg` bytes, stored row after row: one copy when the rows are contiguous in W_q
+        // (seg == K == ldw), else one copy per row, issued by 8 lanes.
+        const int wl = warp - kLoader0, LG = a.lgroups;
+        uint32_t lseq = 0;  // number of this CTA's stages before the current layer
+        bool ok = wl < LG;
         for (int l = 0; l < a.n_layers && ok; ++l) {
             const ChainLayer ly = tab[l];
-            const int units = ly.N >> 3, nst = ly.K / ly.seg, pieces = ly.seg >> 4;
-            for (int u = first_unit(ly); u < units && ok; u += grid) {
-                const int8_t *wrow = ly.w_q + ((size_t)u * 8 + lr) * ly.ldw + lc * 16;
-                for (int st = 0; st < nst; ++st) {
-                    if (pos.use > 0 && !wait_sleep(&bar_empty[pos.slot], (pos.use - 1u) & 1u, abort_flag, a.spin)) {
-                        ok = false;
-                        break;
-                    }
-                    ++issued;
-                    if (tl == 0) s_issued = issued;  // the slot's previous use is over: its barrier may be waited on
-                    uint8_t *dst = ring + (size_t)pos.slot * a.slot_bytes + lr * ly.seg + lc * 16;
-                    const int8_t *src = wrow + (size_t)st * ly.seg;
-                    for (int c = lc; c < pieces; c += 16, dst += 256, src += 256) cp_async16(dst, src);
-                    cp_async_arrive(&bar_full[pos.slot]);
-                    pos.advance(1, S);
+            const int units = ly.N >> 3, nst = ly.K / ly.seg;
+            const int first = first_unit(ly);
+            const int cnt = first < units ? (units - first + grid - 1) / grid : 0;
+            const uint32_t nstage = (uint32_t)(cnt * nst);
+            const bool flat = ly.seg == ly.ldw;
+            uint32_t j = (uint32_t)(wl + LG - (int)(lseq % (uint32_t)LG)) % (uint32_t)LG;  // first stage of the layer that is this warp's
+            int i = (int)j / nst, st = (int)j - i * nst;                                    // its unit and K slice
+            for (; j < nstage; j += LG) {
+                const uint32_t seq = lseq + j;
+                const int slot = (int)(seq % (uint32_t)S);
+                const uint32_t use = seq / (uint32_t)S;
+                if (use > 0 && !wait_sleep(&bar_empty[slot], (use - 1u) & 1u, abort_flag, a.spin)) {
+                    ok = false;
+                    break;
+                }
+                uint8_t *dst = ring + (size_t)slot * a.slot_bytes;
+                const int8_t *src = ly.w_q + (size_t)(first + i * grid) * 8 * ly.ldw + (size_t)st * ly.seg;
+                if (lane == 0) {
+                    s_begun[slot] = use + 1u;  // the slot's previous use is over: its barrier may be waited on
+                    mbar_expect_tx(&bar_full[slot], 8u * (uint32_t)ly.seg);
+                }
+                __syncwarp();
+                if (flat) {
+                    if (lane == 0) bulk_load(dst, src, 8u * (uint32_t)ly.seg, &bar_full[slot]);
+                } else if (lane < 8) {
+                    bulk_load(dst + lane * ly.seg, src + (size_t)lane * ly.ldw, (uint32_t)ly.seg, &bar_full[slot]);
+                }
+                st += LG;
+                while (st >= nst) { st -= nst; ++i; }
+            }
+            lseq += nstage;
+        }
+        // This warp leaves only when the copies it has issued have landed (they all have when the list was walked
+        // to its end, since a unit warp has waited for each; after a time-out some may still be on their way).
+        if (wl < LG)
+            for (int slot = wl; slot < S; slot += LG) {
+                const uint32_t begun = s_begun[slot];
+                if (begun > 0u) {
+                    bool landed = false;
+                    for (uint32_t k = 0; k < a.spin && !landed; ++k) landed = mbar_try_wait(&bar_full[slot], (begun - 1u) & 1u);
                 }
             }
-        }
-        asm volatile("cp.async.wait_all;" ::: "memory");  // nothing of this thread is in flight when the CTA ends
     } else if (warp >= kUW) {
         // ------------------------------------------------------------ prepare warps: X of layer l into buffer l mod NB
         // PG groups of warps.  Layer l belongs to group (l + l / PG) mod PG: every run of PG consecutive layers gives
@@ -474,11 +507,11 @@ __global__ void __launch_bounds__(kThreads, 1) k_decode_stream(const ChainArgs a
                     // that far ahead.
                     {
                         uint32_t spins = 0;
-                        while (s_issued <= seq0 + st && ++spins < a.spin) {
+                        while (s_begun[pos.slot] <= pos.use && ++spins < a.spin) {
                             __nanosleep(40);
                             if ((spins & 15u) == 15u && *abort_flag) break;
                         }
-                        got = __all_sync(0xffffffffu, s_issued > seq0 + st);
+                        got = __all_sync(0xffffffffu, s_begun[pos.slot] > pos.use);
                         if (!got) *abort_flag = 1u;
                     }
                     got = got && wait_sleep(&bar_full[pos.slot], pos.use & 1u, abort_flag, a.spin);
@@ -656,6 +689,8 @@ cudaError_t launch_inst(ChainArgs a, bool cooperative, cudaStream_t s) {
     }
     if (slots > kMaxSlots) slots = kMaxSlots;
     if (slots < 2) return cudaErrorInvalidValue;
+    a.lgroups = slots >= kLW ? kLW : 2;
+    slots -= slots % a.lgroups;  // a slot keeps its loader warp
     a.slots = slots;
     const size_t smem = (size_t)slots * a.slot_bytes + fixed;
     if (cooperative) {

@@ -218,6 +218,7 @@ struct ChainArgs {
     int slots, slot_bytes;         // ring geometry
     int nbuf, pgroups;             // buffers of prepared X, groups of prepare warps (set by the launcher)
     int stage_x;                   // the fp16 rows of X are staged in shared memory one layer ahead (set by the launcher)
+    int lgroups;                   // loader warps in use; divides slots (set by the launcher)
 };
 // Fills unit_off / seg / wait ordinals of every entry (host copy of the table); returns the widest K, -1 if a layer
 // does not fit.
