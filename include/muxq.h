@@ -227,20 +227,27 @@ int muxq_linear_host(const void *X_f16_host, int M, int K, const int8_t *W_q, in
  *
  * muxq_layer: X [M, ldx] fp16, W_q [N, ldw] int8 and s_w from muxq_quantize(is_weight = 1), Y [M, ldy] by the
  * list's out_kind.  flags = MUXQ_LAYER_WAIT_PREV says that this layer's X is written by the layer before it
- * in the list (its Y, or memory derived from nothing else): all CTAs then meet at a bounded grid-wide barrier
- * before they read it.  Without the flag the layers are independent and no CTA ever waits for another.
+ * in the list (its Y, or memory derived from nothing else): the layer's activation work then starts only when
+ * every CTA has counted its part of that Y as stored (bounded waits on counters in the plan's device memory).
+ * Without the flag the layers are independent.  The activation work of a layer (Section III-C, Eq. 4, Eq. 1) is
+ * done once for the grid, in slices of 64 channels, and handed to all CTAs through the plan's device memory.
  * Limits: 1 <= n_layers <= 256, M <= 16, K a multiple of 64 up to 8192, N a multiple of 8, shared Aux scale;
- * alignment as for muxq_linear.  One params / M / out_kind for the whole list.
+ * alignment as for muxq_linear.  One params / M / out_kind for the whole list.  The launch is cooperative.
  *
- * muxq_chain_build validates the list, derives the schedule (which CTA streams which rows of every W_q) into
- * plan_host -- caller-owned HOST memory of muxq_chain_plan_bytes(n_layers) bytes, which must stay valid and
- * unchanged as long as the plan is used -- and enqueues its copy to plan_dev (device memory of the same size,
- * 16-byte aligned) on `stream`.  muxq_chain_run enqueues the launch.  results (device, n_layers entries, or
- * NULL) receives r, the per-tensor scale and 0 / MUXQ_ERR_CAPACITY per layer; a layer whose r exceeds
- * max_outliers leaves its Y unspecified (in bounds), raises the status word, and the list goes on.  The status
- * word is sticky as everywhere.  Runs of one plan must not overlap on the GPU (the plan holds the barrier
- * counter); runs of different plans may.  W_q and s_w are constants of the layers: they must not be written
- * while a run that reads them may be in flight.
+ * muxq_chain_build validates the list, derives the schedule (which CTA streams which rows of every W_q, which
+ * warp prepares which slice of every X) into plan_host -- caller-owned HOST memory of
+ * muxq_chain_plan_bytes(n_layers) bytes, which must stay valid and unchanged as long as the plan is used --
+ * and enqueues the copy of it to plan_dev on `stream`.  plan_dev is caller-owned device memory, 16-byte
+ * aligned, of muxq_chain_device_bytes(layers, n_layers, M) bytes (0: a K that is not a positive multiple of 64,
+ * n_layers or M out of range): the table, 128 bytes of counters per layer and, per layer, the codes, the
+ * outlier mask and the flags of its X (about (M + 1) K bytes).  Too small a buffer is MUXQ_ERR_WORKSPACE.
+ * muxq_chain_run clears the counters and enqueues the launch.  results (device, n_layers entries, or NULL)
+ * receives r, the per-tensor scale and 0 / MUXQ_ERR_CAPACITY per layer; a layer whose r exceeds max_outliers
+ * leaves its Y unspecified (in bounds), raises the status word, and the list goes on.  The status word is
+ * sticky as everywhere.  Runs of one plan must not overlap on the GPU (the plan holds the counters and the
+ * prepared activations); runs of different plans may, as far as the device can hold their CTAs at the same
+ * time.  W_q and s_w are constants of the layers: they must not be written while a run that reads them may be
+ * in flight.
  */
 #define MUXQ_LAYER_WAIT_PREV 1
 typedef struct muxq_layer {
@@ -258,9 +265,10 @@ typedef struct muxq_chain_result {
     float s_x;          /* per-tensor scale (per token: the first row's) */
     int32_t reserved;
 } muxq_chain_result;
-size_t muxq_chain_plan_bytes(int n_layers); /* 0 on n_layers outside 1..256 */
+size_t muxq_chain_plan_bytes(int n_layers); /* host copy; 0 on n_layers outside 1..256 */
+size_t muxq_chain_device_bytes(const muxq_layer *layers_host, int n_layers, int M);
 int muxq_chain_build(const muxq_layer *layers_host, int n_layers, int M, const muxq_params *p, int out_kind,
-                     void *plan_host, void *plan_dev, size_t plan_bytes, void *stream);
+                     void *plan_host, size_t plan_host_bytes, void *plan_dev, size_t plan_dev_bytes, void *stream);
 int muxq_chain_run(const void *plan_host, void *plan_dev, muxq_chain_result *results_or_null,
                    int32_t *dev_status, void *stream);
 

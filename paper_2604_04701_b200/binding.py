@@ -23,7 +23,7 @@ EXPORTS = (
     "muxq_host_workspace_bytes", "muxq_workspace_init", "muxq_workspace_view", "muxq_detect_outliers", "muxq_build_aux",
     "muxq_quantize", "muxq_gemm", "muxq_linear", "muxq_linear_events", "muxq_linear_host",
     "muxq_linear_decode_noalloc", "muxq_int8_mma_peak", "muxq_test_hooks", "muxq_read_status",
-    "muxq_chain_plan_bytes", "muxq_chain_build", "muxq_chain_run",
+    "muxq_chain_plan_bytes", "muxq_chain_device_bytes", "muxq_chain_build", "muxq_chain_run",
     "muxq_status_string",
 )
 
@@ -98,7 +98,8 @@ def lib() -> ctypes.CDLL:
         L.muxq_int8_mma_peak.argtypes = [i, i, i, vp, vp, vp]; L.muxq_int8_mma_peak.restype = i
         L.muxq_test_hooks.argtypes = [vp]; L.muxq_test_hooks.restype = i
         L.muxq_chain_plan_bytes.argtypes = [i]; L.muxq_chain_plan_bytes.restype = sz
-        L.muxq_chain_build.argtypes = [vp, i, i, pp, i, vp, vp, sz, vp]; L.muxq_chain_build.restype = i
+        L.muxq_chain_device_bytes.argtypes = [vp, i, i]; L.muxq_chain_device_bytes.restype = sz
+        L.muxq_chain_build.argtypes = [vp, i, i, pp, i, vp, sz, vp, sz, vp]; L.muxq_chain_build.restype = i
         L.muxq_chain_run.argtypes = [vp, vp, vp, vp, vp]; L.muxq_chain_run.restype = i
         L.muxq_read_status.argtypes = [vp, vp]; L.muxq_read_status.restype = i
         L.muxq_status_string.argtypes = [i]; L.muxq_status_string.restype = ctypes.c_char_p
@@ -335,14 +336,17 @@ class Chain:
         nbytes = int(lib().muxq_chain_plan_bytes(n))
         if nbytes == 0:
             raise MuxqError("muxq_chain_plan_bytes", MUXQ_ERR_INVALID_ARG)
+        dbytes = int(lib().muxq_chain_device_bytes(arr, n, self.M))
+        if dbytes == 0:
+            raise MuxqError("muxq_chain_device_bytes", MUXQ_ERR_UNSUPPORTED)
         self.plan_host = (ctypes.c_uint8 * nbytes)()
-        self.plan_dev = torch.empty(nbytes, dtype=torch.uint8, device=dev)
+        self.plan_dev = torch.empty(dbytes, dtype=torch.uint8, device=dev)
         self.results = torch.zeros(n, 4, dtype=torch.int32, device=dev)
         self.status = torch.zeros(1, dtype=torch.int32, device=dev)
         with torch.cuda.device(dev):
             _check("muxq_chain_build",
-                   lib().muxq_chain_build(arr, n, self.M, ctypes.byref(p.c()), out_kind, self.plan_host,
-                                          _ptr(self.plan_dev), nbytes, _stream()))
+                   lib().muxq_chain_build(arr, n, self.M, ctypes.byref(p.c()), out_kind, self.plan_host, nbytes,
+                                          _ptr(self.plan_dev), dbytes, _stream()))
             torch.cuda.current_stream().synchronize()  # the copy has read plan_host
 
     def run(self) -> None:

@@ -499,13 +499,14 @@ namespace {
 constexpr uint32_t kPlanMagic = 0x4d555851u;
 struct PlanHeader {           // first 128 bytes of a plan (host and device copy alike)
     uint32_t magic;
-    int32_t n_layers, M, kmax, grid, any_wait, out_kind;
+    int32_t n_layers, M, kmax, grid, out_kind;
     muxq_params params;
-    uint32_t barrier;         // device copy: arrival counter of the grid-wide barriers
-    uint32_t reserved[15];
+    uint64_t sync_off, scratch_off, device_bytes;  // layout of the device copy behind the table
+    uint32_t reserved[8];
 };
 static_assert(sizeof(PlanHeader) <= 128, "plan header");
 constexpr size_t kPlanTableOffset = 128;
+size_t plan_sync_offset(int n_layers) { return align_up(kPlanTableOffset + (size_t)n_layers * sizeof(ChainLayer), 128); }
 }  // namespace
 
 size_t muxq_chain_plan_bytes(int n_layers) {
@@ -513,12 +514,24 @@ size_t muxq_chain_plan_bytes(int n_layers) {
     return kPlanTableOffset + (size_t)n_layers * sizeof(ChainLayer);
 }
 
+size_t muxq_chain_device_bytes(const muxq_layer *layers, int n_layers, int M) {
+    if (!layers || n_layers < 1 || n_layers > kChainMaxLayers || M < 1 || M > 16) return 0;
+    size_t scratch = 0;
+    for (int l = 0; l < n_layers; ++l) {
+        if (layers[l].K <= 0 || layers[l].K % 64) return 0;
+        ChainLayer one{};
+        one.K = layers[l].K;
+        scratch += chain_scratch_bytes(&one, 1, M);
+    }
+    return plan_sync_offset(n_layers) + chain_sync_bytes(n_layers) + scratch;
+}
+
 int muxq_chain_build(const muxq_layer *layers, int n_layers, int M, const muxq_params *p, int out_kind,
-                     void *plan_host, void *plan_dev, size_t plan_bytes, void *stream) {
+                     void *plan_host, size_t plan_host_bytes, void *plan_dev, size_t plan_dev_bytes, void *stream) {
     if (!layers || !plan_host || !plan_dev || n_layers < 1 || M < 1 || !params_ok(p) || out_kind < 0 || out_kind > 2)
         return MUXQ_ERR_INVALID_ARG;
     if (n_layers > kChainMaxLayers || M > 16 || p->aux_scale != MUXQ_AUX_SHARED) return MUXQ_ERR_UNSUPPORTED;
-    if (plan_bytes < muxq_chain_plan_bytes(n_layers)) return MUXQ_ERR_WORKSPACE;
+    if (plan_host_bytes < muxq_chain_plan_bytes(n_layers)) return MUXQ_ERR_WORKSPACE;
     if (!aligned16(plan_dev)) return MUXQ_ERR_UNSUPPORTED;
     const int grid = num_sms();
     if (grid < 1) return MUXQ_ERR_CUDA;
@@ -526,7 +539,6 @@ int muxq_chain_build(const muxq_layer *layers, int n_layers, int M, const muxq_p
     ChainLayer *tab = reinterpret_cast<ChainLayer *>(static_cast<uint8_t *>(plan_host) + kPlanTableOffset);
     memset(h, 0, sizeof(PlanHeader));
     const int yal = out_kind == MUXQ_OUT_F16 ? 8 : 4;
-    int any_wait = 0;
     for (int l = 0; l < n_layers; ++l) {
         const muxq_layer &in = layers[l];
         if (!in.X_f16 || !in.W_q || !in.s_w || !in.Y || in.K <= 0 || in.N <= 0 || in.ldx < in.K || in.ldw < in.K ||
@@ -542,12 +554,15 @@ int muxq_chain_build(const muxq_layer *layers, int n_layers, int M, const muxq_p
         o.Y = in.Y;
         o.ldx = in.ldx; o.ldw = in.ldw; o.ldy = in.ldy; o.K = in.K; o.N = in.N;
         o.flags = (in.flags & MUXQ_LAYER_WAIT_PREV) ? kChainWaitPrev : 0;
-        any_wait |= o.flags;
     }
     const int kmax = chain_plan(tab, n_layers, grid, chain_slot_bytes(M));
     if (kmax < 0) return MUXQ_ERR_UNSUPPORTED;
+    h->sync_off = plan_sync_offset(n_layers);
+    h->scratch_off = h->sync_off + chain_sync_bytes(n_layers);
+    h->device_bytes = h->scratch_off + chain_scratch_bytes(tab, n_layers, M);
+    if (plan_dev_bytes < h->device_bytes) return MUXQ_ERR_WORKSPACE;
     h->magic = kPlanMagic;
-    h->n_layers = n_layers; h->M = M; h->kmax = kmax; h->grid = grid; h->any_wait = any_wait; h->out_kind = out_kind;
+    h->n_layers = n_layers; h->M = M; h->kmax = kmax; h->grid = grid; h->out_kind = out_kind;
     h->params = *p;
     return cuda_rc(cudaMemcpyAsync(plan_dev, plan_host, muxq_chain_plan_bytes(n_layers), cudaMemcpyHostToDevice,
                                    static_cast<cudaStream_t>(stream)));
@@ -570,11 +585,11 @@ int muxq_chain_run(const void *plan_host, void *plan_dev, muxq_chain_result *res
     a.dev_status = dev_status;
     a.spin = test_hooks().spin_limit ? test_hooks().spin_limit : (1u << 22);
     a.slot_bytes = chain_slot_bytes(h->M);
-    if (h->any_wait) {
-        a.barrier = reinterpret_cast<uint32_t *>(pd + offsetof(PlanHeader, barrier));
-        if (cudaMemsetAsync(a.barrier, 0, 4, s) != cudaSuccess) return MUXQ_ERR_CUDA;
-    }
-    return cuda_rc(launch_decode_chain(a, h->any_wait != 0, s));
+    a.sync = pd + h->sync_off;
+    a.scratch = pd + h->scratch_off;
+    // the per-layer counters and maxima start every run at zero
+    if (cudaMemsetAsync(a.sync, 0, chain_sync_bytes(h->n_layers), s) != cudaSuccess) return MUXQ_ERR_CUDA;
+    return cuda_rc(launch_decode_chain(a, s));
 }
 
 int muxq_test_hooks(const muxq_test_hooks_t *h) {

@@ -2,7 +2,7 @@
 // each; Section III-C, Eq. 1, Eq. 4-5, Eq. 7, Eq. 3 per layer, exactly as the one-layer decode kernel computes
 // them).  At these sizes a layer is a stream over its W_q (N*K bytes) and little else, and one launch per layer
 // cannot keep HBM busy: a layer moves 1.6-6.6 MB, less than a microsecond of HBM time.  Here the weight stream
-// never stops at a layer boundary:
+// never stops at a layer boundary, and the activation work of a layer is done once for the whole grid:
 //   loader warps    walk the list of layers and, for every unit of 8 output channels that belongs to this CTA,
 //                   fetch the 8 rows of W_q with bulk asynchronous copies (cp.async.bulk, no multicast) into a
 //                   ring of shared-memory stages; the copies report their bytes to the stage's mbarrier.  They
@@ -12,20 +12,27 @@
 //                   the bytes are moved (measured: 10 KB per 0.3 us, 4.4 TB/s over 148 SMs, with one loop of 128
 //                   threads making 16-byte copies; 6.7-7 TB/s with four independent loops), and with one bulk
 //                   copy per stage or per row the loop is a few dozen instructions.
-//   prepare warps   per layer: derive the channel maxima, the outlier flags, the scale(s) and the INT8 codes of X
-//                   into a shared-memory buffer (redundant per CTA, no grid-wide exchange).  The phases of one
-//                   layer are short serial chains with barriers in between, so for small M several groups of
-//                   warps work on different layers at once (one buffer more than groups), and the fp16 rows
-//                   of X are fetched a layer ahead with asynchronous copies.
+//   slice warps     X of a layer is cut into slices of 64 input channels; every slice belongs to one warp of the
+//                   grid (round-robin over CTAs, with an offset that keeps running through the list).  Its warp
+//                   derives the slice's channel maxima and outlier flags (Section III-C) and merges the maxima of
+//                   Body (Eq. 4) into the layer's words in global memory; when all slices of the layer have done so
+//                   (a counter), the scale(s) of Eq. 1 are known and the warp writes its slice's INT8 codes and
+//                   its outlier mask to the layer's scratch area in global memory and counts itself done.
+//                   Every CTA used to do all of this for itself, which cost more than the weight stream.
+//   fetch warp      per layer, in order: waits until all slices are done, builds the list of flagged 64-byte
+//                   segments and the header (scales, r) in one of the CTA's buffers in shared memory and has the
+//                   copy engine bring the codes and the mask there.
 //   unit warps      per layer: each unit is taken by ONE warp, which accumulates the unit's 8 x M outputs over all
 //                   of K in registers (4-way byte dot products for M <= 4, mma.sync m16n8k32 above), adds the Aux
 //                   term of Eq. 7 for the 64-byte segments that hold an outlier channel, dequantizes and stores.
 // Units go to CTAs round-robin with an offset that keeps running from layer to layer, so that the bytes a CTA
 // streams even out over a few layers although a single layer rarely divides evenly.
 // Layers are independent unless a layer's flags say that its X is written by the layer before it: then the
-// prepare warps first wait for this CTA's unit warps to finish that layer and pass a bounded grid-wide barrier
-// (the launch is cooperative); the loaders do not wait.
-// All waits are bounded; a wait that runs out raises MUXQ_ERR_TIMEOUT and every role leaves.
+// slice warps of that layer first wait until every CTA has counted its units of the layer before as stored.
+// A warp never waits for a condition that needs one of its own later steps: slices are taken in list order, no
+// warp owns two slices of a layer, and the fetch and unit warps only ever wait for earlier layers or for the
+// slice warps.  All CTAs are resident (cooperative launch, one CTA per SM).  All waits are bounded; a wait that
+// runs out raises MUXQ_ERR_TIMEOUT, tells the other CTAs through a word in global memory, and every role leaves.
 #include <mutex>
 
 #include "kernels.h"
@@ -37,13 +44,13 @@ namespace muxq {
 namespace {
 
 constexpr int kUW = 8;                  // unit warps (warps 0..7)
-constexpr int kPW = 8;                  // prepare warps (warps 8..15)
+constexpr int kFetch = kUW;             // the fetch warp
+constexpr int kSW = kChainSliceWarps;   // slice warps per CTA (warps 9..15)
 constexpr int kLW = 4;                  // loader warps (warps 16..19)
-constexpr int kLoader0 = kUW + kPW;     // index of the first loader warp
+constexpr int kLoader0 = kUW + 1 + kSW; // index of the first loader warp
 constexpr int kThreads = 32 * (kLoader0 + kLW);
-constexpr int kMaxK = 8192;             // widest layer: 1024 channel groups of 8
-constexpr int kMaxGroups = 4;           // groups of prepare warps, each on a layer of its own
-constexpr int kMaxBufs = kMaxGroups + 1;
+constexpr int kMaxK = 8192;             // widest layer: 128 slices
+constexpr int kMaxBufs = 4;             // buffers of prepared X per CTA
 constexpr int kMaxSlots = 24;
 constexpr int kStatusCapacity = 5;      // MUXQ_ERR_CAPACITY
 constexpr int kStatusTimeout = 6;       // MUXQ_ERR_TIMEOUT
@@ -58,10 +65,6 @@ __device__ __forceinline__ void mma_s8(int (&d)[4], uint32_t a0, uint32_t a1, ui
         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
-// 16 bytes global -> shared, asynchronously (the fp16 rows of X; completion through cp.async.wait_all)
-__device__ __forceinline__ void cp_async16(void *smem_dst, const void *gsrc) {
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(smem_dst)), "l"(gsrc) : "memory");
-}
 // `bytes` (a multiple of 16, both addresses 16-byte aligned) global -> shared by the copy engine; the bytes are
 // reported to the mbarrier as they land
 __device__ __forceinline__ void bulk_load(void *smem_dst, const void *gsrc, uint32_t bytes, uint64_t *bar) {
@@ -70,6 +73,9 @@ __device__ __forceinline__ void bulk_load(void *smem_dst, const void *gsrc, uint
                  "l"(gsrc), "r"(bytes), "r"(smem_u32(bar))
                  : "memory");
 }
+// orders this thread's earlier accesses through ordinary loads and stores (made visible to it by an acquire)
+// before its later copies through the copy engine, global memory included
+__device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
 
 // Bounded wait of a whole converged warp that backs off between polls: the warps of this kernel spend most of
 // their time waiting for each other, and a warp that polls without pause takes issue slots from the few that work.
@@ -83,54 +89,73 @@ __device__ __forceinline__ bool wait_sleep(uint64_t *bar, uint32_t parity, volat
     return false;
 }
 
-// named barrier `id` over `nthreads` threads (one per group of prepare warps)
-__device__ __forceinline__ void bar_prep(int id, int nthreads) {
-    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
-}
-// the same barrier, which also tells every one of its threads whether any of them has seen `flag`
-__device__ __forceinline__ bool bar_prep_or(int id, int nthreads, bool flag) {
-    uint32_t r;
-    asm volatile(
-        "{\n\t.reg .pred p, q;\n\t"
-        "setp.ne.u32 q, %1, 0;\n\t"
-        "bar.red.or.pred p, %2, %3, q;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}\n"
-        : "=r"(r)
-        : "r"((uint32_t)flag), "r"(id), "r"(nthreads)
-        : "memory");
-    return r != 0;
-}
-
 __device__ __forceinline__ uint32_t ld_acquire_u32(const uint32_t *p) {
     uint32_t v;
     asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
     return v;
 }
+__device__ __forceinline__ uint32_t ld_relaxed_u32(const uint32_t *p) {
+    uint32_t v;
+    asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
 
-// A buffer that holds a layer's prepared X (sized for the widest K of the list).
+// Bounded wait of a whole converged warp for a counter in global memory to reach `want` (lane 0 polls, with an
+// acquire; the warp's later loads are ordered behind it by the shuffle).  A time-out here or anywhere else in the
+// grid (the word *g_abort) ends the wait; the first kind also raises both abort flags.
+__device__ __forceinline__ bool wait_count(const uint32_t *ctr, uint32_t want, volatile uint32_t *abort_flag,
+                                           uint32_t *g_abort, uint32_t limit) {
+    int ok = 0;
+    if ((threadIdx.x & 31) == 0) {
+        bool stopped = false;
+        for (uint32_t i = 0; i < limit && !ok && !stopped; ++i) {
+            if (ld_acquire_u32(ctr) >= want) ok = 1;
+            else {
+                __nanosleep(i < 8 ? 100 : 400);
+                if ((i & 7u) == 7u) stopped = *abort_flag != 0u || ld_relaxed_u32(g_abort) != 0u;
+            }
+        }
+        if (!ok) {
+            *abort_flag = 1u;
+            if (!stopped) atomicExch(g_abort, 1u);
+        }
+    }
+    return __shfl_sync(0xffffffffu, ok, 0) != 0;
+}
+
+// Per layer, in global memory (zero when the launch starts): the counters and maxima the slice warps share.
+struct LayerSync {
+    uint32_t merged;      // slices whose maxima and outlier counts are in
+    uint32_t coded;       // slices whose codes and mask are written
+    uint32_t r;           // outlier channels found so far
+    uint32_t stored;      // CTAs whose units of this layer are stored (counted only when the next layer waits)
+    uint32_t bmax[16];    // bit patterns of the row maxima of Body (per tensor: word 0 only)
+    uint32_t pad[12];
+};
+static_assert(sizeof(LayerSync) == 128, "per-layer words");
+
+// A layer's scratch area in global memory: codes [M][K], mask [K] (0xFF at outlier channels), segflag [K / 64].
+__host__ __device__ inline size_t scratch_codes_bytes(int M, int K) { return ((size_t)M * K + 127) & ~(size_t)127; }
+__host__ __device__ inline size_t scratch_layer_bytes(int M, int K) {
+    return scratch_codes_bytes(M, K) + (size_t)K + (size_t)(((K >> 6) + 127) & ~127);
+}
+
+// A buffer in shared memory that holds a layer's prepared X (sized for the widest K of the list).
 struct XLayout {
     int pitch;          // bytes per row of X codes; pitch % 128 == 64 keeps the 8-row x 64-byte reads conflict free
     int off_xq;         // [rows][pitch] INT8 codes (behind a 128-byte header: 16 row scales, r, list length)
     int off_mask;       // [K] 0xFF at outlier channels
-    int off_segflag;    // [K/64] segment holds an outlier channel
-    int off_grpmask;    // [K/8] per-group flag bits
     int off_flaglist;   // [K/64] u16: the segments that hold an outlier channel, ascending
     int buf_bytes;
-    int xs_bytes;       // bytes of one fp16 staging copy of X ([M][K]); 0 when X is not staged
-    int total;          // the buffers + two staging copies per group of prepare warps
 };
-__host__ __device__ inline XLayout x_layout(int rows, int M, int K, bool stage_x, int nbuf, int groups) {
+__host__ __device__ inline XLayout x_layout(int rows, int K) {
     XLayout s;
     s.pitch = K + ((64 - (K & 127)) & 127);
     if ((s.pitch & 127) != 64) s.pitch += 64;
     s.off_xq = 128;
     s.off_mask = s.off_xq + rows * s.pitch;
-    s.off_segflag = s.off_mask + K;
-    s.off_grpmask = s.off_segflag + (((K >> 6) + 15) & ~15);
-    s.off_flaglist = (s.off_grpmask + (K >> 3) + 15) & ~15;
+    s.off_flaglist = s.off_mask + K;
     s.buf_bytes = (s.off_flaglist + 2 * (K >> 6) + 127) & ~127;
-    s.xs_bytes = stage_x ? M * K * 2 : 0;
-    s.total = nbuf * s.buf_bytes + 2 * groups * s.xs_bytes;
     return s;
 }
 struct XHeader {        // first bytes of a buffer
@@ -156,26 +181,31 @@ __global__ void __launch_bounds__(kThreads, 1) k_decode_stream(const ChainArgs a
     extern __shared__ __align__(128) uint8_t smem[];
     __shared__ uint64_t bar_full[kMaxSlots], bar_empty[kMaxSlots];
     __shared__ uint64_t bar_ready[kMaxBufs], bar_free[kMaxBufs];  // a buffer of prepared X: filled / no longer read
-    __shared__ uint32_t s_rowmax[kMaxGroups][16];   // bit patterns of non-negative floats (row maxima of Body)
-    __shared__ float s_wmax[kPW];
     __shared__ uint32_t s_abort;
     __shared__ volatile uint32_t s_begun[kMaxSlots];  // uses of a slot the loaders have begun to fill so far
+    __shared__ uint32_t s_unitdone[kMaxBufs];         // unit warps that have stored their part of the buffer's layer
 
     const int t = threadIdx.x, lane = t & 31;
     const int warp = __shfl_sync(0xffffffffu, t >> 5, 0);  // warp-uniform by construction
-    const int S = a.slots, M = a.M, NB = a.nbuf, PG = a.pgroups;
+    const int S = a.slots, M = a.M, NB = a.nbuf;
     const int grid = (int)gridDim.x, cta = (int)blockIdx.x;
     uint8_t *ring = smem;
     ChainLayer *tab = reinterpret_cast<ChainLayer *>(smem + (size_t)S * a.slot_bytes);
     uint8_t *xbase = reinterpret_cast<uint8_t *>(tab + a.n_layers);
-    const XLayout L = x_layout(kRows, M, a.kmax, a.stage_x != 0, NB, PG);
+    const XLayout L = x_layout(kRows, a.kmax);
     volatile uint32_t *abort_flag = &s_abort;
+    LayerSync *sync = reinterpret_cast<LayerSync *>(a.sync);
+    uint32_t *g_abort = reinterpret_cast<uint32_t *>(sync + a.n_layers);
 
-    // the layer table into shared memory (16-byte pieces), barriers
+    // the layer table into shared memory (16-byte pieces), zero codes in the buffers (rows M.. of a buffer are
+    // read by the products and never written again), barriers
     {
         const uint4 *src = reinterpret_cast<const uint4 *>(a.layers);
         uint4 *dst = reinterpret_cast<uint4 *>(tab);
         for (int i = t; i < a.n_layers * 4; i += kThreads) dst[i] = __ldg(src + i);
+        uint4 *xz = reinterpret_cast<uint4 *>(xbase);
+        for (int i = t; i < NB * (L.buf_bytes >> 4); i += kThreads) xz[i] = make_uint4(0u, 0u, 0u, 0u);
+        fence_proxy_async();  // the copy engine writes the same bytes later
     }
     if (t == 0) {
         for (int s = 0; s < S; ++s) {
@@ -184,8 +214,9 @@ __global__ void __launch_bounds__(kThreads, 1) k_decode_stream(const ChainArgs a
             s_begun[s] = 0u;
         }
         for (int b = 0; b < kMaxBufs; ++b) {
-            mbar_init(&bar_ready[b], 1);   // one prepare thread, after its group's barrier
+            mbar_init(&bar_ready[b], 1);   // the fetch warp's arrival that announces the bytes; the copies report them
             mbar_init(&bar_free[b], kUW);  // every unit warp, once per layer
+            s_unitdone[b] = 0u;
         }
         s_abort = 0u;
         fence_barrier_init();
@@ -194,7 +225,7 @@ __global__ void __launch_bounds__(kThreads, 1) k_decode_stream(const ChainArgs a
 
     // the units of a layer that belong to this CTA: first, first + grid, ... below N / 8
     auto first_unit = [&](const ChainLayer &ly) {
-        int f = cta - ly.unit_off;
+        int f = cta - (int)ly.unit_off;
         if (f < 0) f += grid;
         return f;
     };
@@ -212,11 +243,11 @@ __global__ void __launch_bounds__(kThreads, 1) k_decode_stream(const ChainArgs a
         bool ok = wl < LG;
         for (int l = 0; l < a.n_layers && ok; ++l) {
             const ChainLayer ly = tab[l];
-            const int units = ly.N >> 3, nst = ly.K / ly.seg;
+            const int seg = (int)ly.seg, units = ly.N >> 3, nst = ly.K / seg;
             const int first = first_unit(ly);
             const int cnt = first < units ? (units - first + grid - 1) / grid : 0;
             const uint32_t nstage = (uint32_t)(cnt * nst);
-            const bool flat = ly.seg == ly.ldw;
+            const bool flat = seg == ly.ldw;
             uint32_t j = (uint32_t)(wl + LG - (int)(lseq % (uint32_t)LG)) % (uint32_t)LG;  // first stage of the layer that is this warp's
             int i = (int)j / nst, st = (int)j - i * nst;                                    // its unit and K slice
             for (; j < nstage; j += LG) {
@@ -228,16 +259,16 @@ __global__ void __launch_bounds__(kThreads, 1) k_decode_stream(const ChainArgs a
                     break;
                 }
                 uint8_t *dst = ring + (size_t)slot * a.slot_bytes;
-                const int8_t *src = ly.w_q + (size_t)(first + i * grid) * 8 * ly.ldw + (size_t)st * ly.seg;
+                const int8_t *src = ly.w_q + (size_t)(first + i * grid) * 8 * ly.ldw + (size_t)st * seg;
                 if (lane == 0) {
                     s_begun[slot] = use + 1u;  // the slot's previous use is over: its barrier may be waited on
-                    mbar_expect_tx(&bar_full[slot], 8u * (uint32_t)ly.seg);
+                    mbar_expect_tx(&bar_full[slot], 8u * (uint32_t)seg);
                 }
                 __syncwarp();
                 if (flat) {
-                    if (lane == 0) bulk_load(dst, src, 8u * (uint32_t)ly.seg, &bar_full[slot]);
+                    if (lane == 0) bulk_load(dst, src, 8u * (uint32_t)seg, &bar_full[slot]);
                 } else if (lane < 8) {
-                    bulk_load(dst + lane * ly.seg, src + (size_t)lane * ly.ldw, (uint32_t)ly.seg, &bar_full[slot]);
+                    bulk_load(dst + lane * seg, src + (size_t)lane * ly.ldw, (uint32_t)seg, &bar_full[slot]);
                 }
                 st += LG;
                 while (st >= nst) { st -= nst; ++i; }
@@ -254,221 +285,211 @@ __global__ void __launch_bounds__(kThreads, 1) k_decode_stream(const ChainArgs a
                     for (uint32_t k = 0; k < a.spin && !landed; ++k) landed = mbar_try_wait(&bar_full[slot], (begun - 1u) & 1u);
                 }
             }
-    } else if (warp >= kUW) {
-        // ------------------------------------------------------------ prepare warps: X of layer l into buffer l mod NB
-        // PG groups of warps.  Layer l belongs to group (l + l / PG) mod PG: every run of PG consecutive layers gives
-        // each group one layer, and the assignment shifts by one from run to run, so that a list with a period of
-        // PG layers (the four projections of a block) does not hand the same group the widest layer every time.
-        const int wp = warp - kUW, wpg = kPW / PG, gi = wp / wpg, wg = wp - gi * wpg;
-        const int GT = 32 * wpg, tp = t - 32 * (kUW + gi * wpg), bid = 1 + gi;
-        const float down = __int_as_float((127 - a.exp_factor) << 23);  // 2^-e
+    } else if (warp == kFetch) {
+        // ------------------------------------------------------------ fetch warp: prepared X of layer l into buffer l mod NB
         const float qf = (float)a.qmax;
-        const bool first_cta = cta == 0;
-        uint32_t *rowmax = s_rowmax[gi];
-        // asynchronous copy of the fp16 rows of a layer's X into one of this group's two staging copies
-        auto group_of = [&](int l) { return (l + l / PG) % PG; };
-        auto next_mine = [&](int l) {  // the next layer of this group behind layer l (or n_layers)
-            for (++l; l < a.n_layers && group_of(l) != gi; ++l) {}
-            return l;
-        };
-        auto stage_x = [&](int l, int copy) {
-            const ChainLayer &ly = tab[l];
-            uint8_t *dst = xbase + NB * L.buf_bytes + (2 * gi + copy) * L.xs_bytes;
-            const int G = ly.K >> 3;
-            for (int cg = tp; cg < G; cg += GT)
-                for (int m = 0; m < M; ++m) cp_async16(dst + (size_t)m * ly.K * 2 + cg * 16, ly.X + (size_t)m * ly.ldx + cg * 8);
-        };
-        const bool staged = L.xs_bytes > 0;
-        auto waits_for_prev = [&](int l) { return (tab[l].flags & kChainWaitPrev) && a.barrier; };
-        int mine = 0;  // layers this group has prepared so far: parity selects the staging copy
-        {
-            const int l0 = next_mine(-1);
-            if (staged && l0 < a.n_layers && !waits_for_prev(l0)) stage_x(l0, 0);
-        }
-        bool stop = false;
-        for (int l = next_mine(-1); l < a.n_layers && !stop; l = next_mine(l), ++mine) {
+        size_t scr = 0;  // offset of the layer's scratch area
+        uint32_t last_bytes = 0;
+        int last_buf = -1;
+        uint32_t last_phase = 0;
+        for (int l = 0; l < a.n_layers; ++l) {
             const ChainLayer ly = tab[l];
-            const int K = ly.K, G = K >> 3, b = l % NB, ph = l / NB;
+            const int K = ly.K, ns = K >> 6, b = l % NB, ph = l / NB;
             uint8_t *buf = xbase + b * L.buf_bytes;
             XHeader *hdr = reinterpret_cast<XHeader *>(buf);
-            int8_t *xq = reinterpret_cast<int8_t *>(buf + L.off_xq);
-            uint8_t *s_mask = buf + L.off_mask, *s_segflag = buf + L.off_segflag, *s_grpmask = buf + L.off_grpmask;
-            const uint8_t *xs = staged ? xbase + NB * L.buf_bytes + (2 * gi + (mine & 1)) * L.xs_bytes : nullptr;
-            const bool wait_prev = waits_for_prev(l);
-            bool ok = true;
-            // the buffer was last read for layer l - NB
-            if (l >= NB) ok = wait_sleep(&bar_free[b], (uint32_t)(ph - 1) & 1u, abort_flag, a.spin);
-            if (wait_prev) {
-                // X of this layer is Y of the layer before it: this CTA's unit warps must have stored theirs (they
-                // arrive on the buffer's barrier after their stores), then every CTA's must be visible.  The flags
-                // carry the ordinal of this wait, which gives the arrival count to wait for.
-                ok = ok && wait_sleep(&bar_free[(l - 1) % NB], (uint32_t)((l - 1) / NB) & 1u, abort_flag, a.spin);
-                bar_prep(bid, GT);
-                if (tp == 0) {
-                    __threadfence();
-                    atomicAdd(a.barrier, 1u);
-                    const uint32_t want = (uint32_t)(ly.flags >> 1) * (uint32_t)grid;
-                    bool seen = false;
-                    for (uint32_t i = 0; i < a.spin; ++i)
-                        if (ld_acquire_u32(a.barrier) >= want) { seen = true; break; }
-                    if (!seen) *abort_flag = 1u;
-                }
-                bar_prep(bid, GT);
-                if (staged) stage_x(l, mine & 1);  // could not be fetched ahead
+            const uint8_t *g_codes = a.scratch + scr;
+            const uint8_t *g_mask = g_codes + scratch_codes_bytes(M, K);
+            const uint8_t *g_segflag = g_mask + K;
+            scr += scratch_layer_bytes(M, K);
+            // the buffer was last read for layer l - NB; then all slices of this layer must be coded
+            if (l >= NB && !wait_sleep(&bar_free[b], (uint32_t)(ph - 1) & 1u, abort_flag, a.spin)) break;
+            if (!wait_count(&sync[l].coded, (uint32_t)ns, abort_flag, g_abort, a.spin)) break;
+            const int r = (int)__ldcg(&sync[l].r);
+            const bool over = r > a.cap;  // MUXQ_ERR_CAPACITY: no codes were written, Y of this layer is unspecified
+            if (lane < 16) {
+                const float mx = __uint_as_float(__ldcg(&sync[l].bmax[a.per_vec ? lane : 0]));
+                hdr->rowscale[lane] = mx > 0.0f ? __fdiv_rn(mx, qf) : 1.0f;
             }
-            if (tp < 16) rowmax[tp] = 0u;
-            for (int i = tp; i < (K >> 6); i += GT) s_segflag[i] = 0;
-            if (staged) asm volatile("cp.async.wait_all;" ::: "memory");
-            bar_prep(bid, GT);  // this layer's staging copy is complete and visible; the group's other copy is free
-            {
-                const int ln = next_mine(l);
-                if (staged && ln < a.n_layers && !waits_for_prev(ln)) stage_x(ln, (mine + 1) & 1);
-            }
-            auto x_chunk = [&](int m, int cg) -> uint4 {
-                return xs ? *reinterpret_cast<const uint4 *>(xs + (size_t)m * K * 2 + cg * 16)
-                          : __ldcg(reinterpret_cast<const uint4 *>(ly.X + (size_t)m * ly.ldx) + cg);
-            };
-
-            // ---------------------------------------------------------- pass A: channel maxima, flags, Body maxima
-            float bmax = 0.0f;
-#pragma unroll 2
-            for (int cg = tp; cg < G; cg += GT) {
-                __half2 cm[4];
-                cm[0] = cm[1] = cm[2] = cm[3] = __float2half2_rn(0.f);
-                for (int m0 = 0; m0 < M; m0 += 4) {  // four independent row loads in flight
-                    uint4 v[4];
-#pragma unroll
-                    for (int u = 0; u < 4; ++u) v[u] = m0 + u < M ? x_chunk(m0 + u, cg) : make_uint4(0u, 0u, 0u, 0u);
-#pragma unroll
-                    for (int u = 0; u < 4; ++u) {
-                        cm[0] = __hmax2(cm[0], __habs2(*reinterpret_cast<const __half2 *>(&v[u].x)));
-                        cm[1] = __hmax2(cm[1], __habs2(*reinterpret_cast<const __half2 *>(&v[u].y)));
-                        cm[2] = __hmax2(cm[2], __habs2(*reinterpret_cast<const __half2 *>(&v[u].z)));
-                        cm[3] = __hmax2(cm[3], __habs2(*reinterpret_cast<const __half2 *>(&v[u].w)));
-                    }
-                }
-                float c8[8];
-#pragma unroll
-                for (int i = 0; i < 4; ++i) { c8[2 * i] = __low2float(cm[i]); c8[2 * i + 1] = __high2float(cm[i]); }
-                uint32_t mask = 0;
-#pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                    const bool flagged = c8[i] > a.tau;  // strict
-                    mask |= flagged ? (1u << i) : 0u;
-                    bmax = fmaxf(bmax, flagged ? c8[i] * down : c8[i]);
-                }
-                s_grpmask[cg] = (uint8_t)mask;
-                if (mask) s_segflag[cg >> 3] = 1;
-                uint2 mb;
-                mb.x = ((mask & 1) ? 0xFFu : 0u) | ((mask & 2) ? 0xFF00u : 0u) | ((mask & 4) ? 0xFF0000u : 0u) |
-                       ((mask & 8) ? 0xFF000000u : 0u);
-                mb.y = ((mask & 16) ? 0xFFu : 0u) | ((mask & 32) ? 0xFF00u : 0u) | ((mask & 64) ? 0xFF0000u : 0u) |
-                       ((mask & 128) ? 0xFF000000u : 0u);
-                *reinterpret_cast<uint2 *>(s_mask + cg * 8) = mb;
-            }
-            if (a.per_vec) {
-                // per-token scales: row maxima of Body (after the 2^-e), a second cheap sweep with the flags known
-#pragma unroll 1
-                for (int cg = tp; cg < G; cg += GT) {
-                    const uint32_t gmask = s_grpmask[cg];  // this thread's own store
-                    for (int m = 0; m < M; ++m) {
-                        float f[8];
-                        unpack8(x_chunk(m, cg), f);
-                        float rm = 0.0f;
-#pragma unroll
-                        for (int i = 0; i < 8; ++i) rm = fmaxf(rm, fabsf((gmask >> i) & 1u ? f[i] * down : f[i]));
-                        if (rm > 0.0f) atomicMax(&rowmax[m], __float_as_uint(rm));
-                    }
-                }
-            }
-            bmax = warp_max(bmax);
-            if (lane == 0) s_wmax[wp] = bmax;
-            bar_prep(bid, GT);
-            // ---------------------------------------------------------- scales (Eq. 1), outlier count, flagged segments
-            if (tp < 16) {
-                float sc;
-                if (a.per_vec) {
-                    const float mx = __uint_as_float(rowmax[tp]);
-                    sc = mx > 0.0f ? __fdiv_rn(mx, qf) : 1.0f;
-                } else {
-                    float mx = 0.0f;
-                    for (int w = 0; w < wpg; ++w) mx = fmaxf(mx, s_wmax[gi * wpg + w]);
-                    sc = mx > 0.0f ? __fdiv_rn(mx, qf) : 1.0f;
-                }
-                hdr->rowscale[tp] = sc;
-            }
-            if (wg == wpg - 1) {
-                int cnt = 0;
-                for (int gj = lane; gj < G; gj += 32) cnt += __popc((uint32_t)s_grpmask[gj]);
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
-                if (lane == 0) {
-                    hdr->r = cnt;
-                    if (cnt > a.cap && first_cta && a.dev_status) atomicMax(a.dev_status, kStatusCapacity);
-                }
-                // the flagged 64-byte segments, compacted in ascending order
-                uint16_t *flaglist = reinterpret_cast<uint16_t *>(buf + L.off_flaglist);
-                int nf = 0;
-                for (int base = 0; base < (K >> 6); base += 32) {
-                    const bool f = base + lane < (K >> 6) && s_segflag[base + lane] != 0;
+            // the flagged 64-byte segments, compacted in ascending order
+            uint16_t *flaglist = reinterpret_cast<uint16_t *>(buf + L.off_flaglist);
+            int nf = 0;
+            if (!over)
+                for (int base = 0; base < ns; base += 32) {
+                    const bool f = base + lane < ns && __ldcg(g_segflag + base + lane) != 0;
                     const uint32_t bal = __ballot_sync(0xffffffffu, f);
                     if (f) flaglist[nf + __popc(bal & ((1u << lane) - 1u))] = (uint16_t)(base + lane);
                     nf += __popc(bal);
                 }
-                if (lane == 0) hdr->nflag = nf;
-            }
-            bar_prep(bid, GT);
-            const int r = hdr->r;
-            if (first_cta && tp == 0 && a.results) {
-                ChainResult rr;
-                rr.n_outliers = r;
-                rr.status = r > a.cap ? kStatusCapacity : 0;
-                rr.s_x = hdr->rowscale[0];
-                rr.reserved = 0;
-                a.results[l] = rr;
-            }
-            // ---------------------------------------------------------- pass B: codes of X into the buffer
-            // (r beyond the capacity: Y of this layer is unspecified, no codes are needed)
-            if (r <= a.cap) {
-                float lo = 0.0f, hi = 0.0f;
-                if (!a.per_vec) recip_bracket(__frcp_rn(hdr->rowscale[0]), lo, hi);
-                // items = channel group x batch of four rows
-                constexpr int kBatches = kRows / 4 > 0 ? kRows / 4 : 1;
-#pragma unroll 2
-                for (int item = tp; item < G * kBatches; item += GT) {
-                    int batch = 0, cg = item;
-                    if (kBatches > 1) { batch = item / G; cg = item - batch * G; }
-                    const int m0 = 4 * batch;
-                    const uint32_t gmask = s_grpmask[cg];
-                    float mul[8];
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) mul[i] = (gmask >> i) & 1u ? down : 1.0f;
-                    uint4 v[4];  // four independent row loads in flight
-#pragma unroll
-                    for (int u = 0; u < 4; ++u) v[u] = (u < kRows && m0 + u < M) ? x_chunk(m0 + u, cg) : make_uint4(0u, 0u, 0u, 0u);
-#pragma unroll
-                    for (int u = 0; u < 4; ++u) {
-                        const int m = m0 + u;
-                        if (u >= kRows) break;
-                        uint2 code = make_uint2(0u, 0u);
-                        if (m < M) {
-                            float f[8];
-                            unpack8(v[u], f);
-#pragma unroll
-                            for (int i = 0; i < 8; ++i) f[i] *= mul[i];  // exact
-                            const float sc = hdr->rowscale[a.per_vec ? m : 0];
-                            if (a.per_vec) recip_bracket(__frcp_rn(sc), lo, hi);
-                            uint32_t cb[8];
-                            if (quant8_bracket(f, lo, hi, cb)) code = codes_exact(v[u], gmask, down, sc, qf);  // rare
-                            else code = pack8(cb);
-                        }
-                        *reinterpret_cast<uint2 *>(xq + m * L.pitch + cg * 8) = code;
+            if (lane == 0) {
+                hdr->r = r;
+                hdr->nflag = nf;
+                if (cta == 0) {
+                    if (over && a.dev_status) atomicMax(a.dev_status, kStatusCapacity);
+                    if (a.results) {
+                        ChainResult rr;
+                        rr.n_outliers = r;
+                        rr.status = over ? kStatusCapacity : 0;
+                        rr.s_x = hdr->rowscale[0];
+                        rr.reserved = 0;
+                        a.results[l] = rr;
                     }
                 }
             }
-            // every prepare thread's writes are ordered before the one arrival that hands the buffer to the unit warps
-            stop = bar_prep_or(bid, GT, !ok || *abort_flag != 0u);
-            if (tp == 0 && !stop) mbar_arrive(&bar_ready[b]);
+            // the header and the list are ordered before the arrival that announces the bytes; the codes and the mask,
+            // written by other SMs and made visible by the acquire above, are ordered before the copy engine reads them
+            const uint32_t bytes = over ? 0u : (uint32_t)(M * K + K);
+            fence_proxy_async_all();
+            __syncwarp();
+            if (lane == 0) mbar_expect_tx(&bar_ready[b], bytes);
+            __syncwarp();
+            if (!over) {
+                int8_t *xq = reinterpret_cast<int8_t *>(buf + L.off_xq);
+                if (lane < M) bulk_load(xq + (size_t)lane * L.pitch, g_codes + (size_t)lane * K, (uint32_t)K, &bar_ready[b]);
+                if (lane == 31) bulk_load(buf + L.off_mask, g_mask, (uint32_t)K, &bar_ready[b]);
+            }
+            last_bytes = bytes; last_buf = b; last_phase = (uint32_t)ph & 1u;
+        }
+        // the copies of the last layer fetched have landed before this warp leaves (see the loaders)
+        if (last_buf >= 0 && last_bytes > 0u) {
+            bool landed = false;
+            for (uint32_t k = 0; k < a.spin && !landed; ++k) landed = mbar_try_wait(&bar_ready[last_buf], last_phase);
+        }
+    } else if (warp > kFetch) {
+        // ------------------------------------------------------------ slice warps
+        // Warp number w = (warp index among the slice warps) * grid + cta of the grid's kSW * grid slice warps takes
+        // slice s of layer l when (slice_off(l) + s) mod (kSW * grid) == w: consecutive slices go to different CTAs.
+        const int NW = kSW * grid, myw = (warp - kFetch - 1) * grid + cta;
+        const int rg = lane >> 3, cg = lane & 7;  // this lane: rows rg, rg + 4, rg + 8, rg + 12; channels 8 cg .. 8 cg + 7 of the slice
+        const float down = __int_as_float((127 - a.exp_factor) << 23);  // 2^-e
+        const float qf = (float)a.qmax;
+        size_t scr = 0;
+        for (int l = 0; l < a.n_layers; ++l) {
+            const ChainLayer ly = tab[l];
+            const int K = ly.K, ns = K >> 6;
+            uint8_t *g_codes = a.scratch + scr;
+            uint8_t *g_mask = g_codes + scratch_codes_bytes(M, K);
+            uint8_t *g_segflag = g_mask + K;
+            scr += scratch_layer_bytes(M, K);
+            int s = myw - (int)ly.slice_off;
+            if (s < 0) s += NW;
+            if (s >= ns) continue;
+            // X of this layer is Y of the layer before it: every CTA must have stored its part
+            if ((ly.flags & kChainWaitPrev) && !wait_count(&sync[l - 1].stored, (uint32_t)grid, abort_flag, g_abort, a.spin)) break;
+            const int ch = s * 64 + cg * 8;
+            uint4 v[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int m = rg + 4 * u;
+                v[u] = m < M ? __ldcg(reinterpret_cast<const uint4 *>(ly.X + (size_t)m * ly.ldx + ch)) : make_uint4(0u, 0u, 0u, 0u);
+            }
+            // channel maxima over the rows (Section III-C): this lane's rows, then the lanes that hold the other rows
+            __half2 cm[4];
+            cm[0] = cm[1] = cm[2] = cm[3] = __float2half2_rn(0.f);
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                cm[0] = __hmax2(cm[0], __habs2(*reinterpret_cast<const __half2 *>(&v[u].x)));
+                cm[1] = __hmax2(cm[1], __habs2(*reinterpret_cast<const __half2 *>(&v[u].y)));
+                cm[2] = __hmax2(cm[2], __habs2(*reinterpret_cast<const __half2 *>(&v[u].z)));
+                cm[3] = __hmax2(cm[3], __habs2(*reinterpret_cast<const __half2 *>(&v[u].w)));
+            }
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                uint32_t w = *reinterpret_cast<uint32_t *>(&cm[i]);
+                uint32_t o = __shfl_xor_sync(0xffffffffu, w, 8);
+                cm[i] = __hmax2(cm[i], *reinterpret_cast<__half2 *>(&o));
+                w = *reinterpret_cast<uint32_t *>(&cm[i]);
+                o = __shfl_xor_sync(0xffffffffu, w, 16);
+                cm[i] = __hmax2(cm[i], *reinterpret_cast<__half2 *>(&o));
+            }
+            uint32_t mask = 0;
+            float mul[8];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const float c0 = __low2float(cm[i]), c1 = __high2float(cm[i]);
+                if (c0 > a.tau) mask |= 1u << (2 * i);  // strict
+                if (c1 > a.tau) mask |= 2u << (2 * i);
+            }
+#pragma unroll
+            for (int i = 0; i < 8; ++i) mul[i] = (mask >> i) & 1u ? down : 1.0f;
+            // maxima of Body (Eq. 4: outlier channels times 2^-e) per row, over the slice's 64 channels
+            float rm[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                float f[8];
+                unpack8(v[u], f);
+                float x = 0.0f;
+#pragma unroll
+                for (int i = 0; i < 8; ++i) x = fmaxf(x, fabsf(f[i] * mul[i]));
+                rm[u] = x;
+            }
+            if (!a.per_vec) rm[0] = fmaxf(fmaxf(rm[0], rm[1]), fmaxf(rm[2], rm[3]));
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                if (u > 0 && !a.per_vec) break;
+                rm[u] = fmaxf(rm[u], __shfl_xor_sync(0xffffffffu, rm[u], 1));
+                rm[u] = fmaxf(rm[u], __shfl_xor_sync(0xffffffffu, rm[u], 2));
+                rm[u] = fmaxf(rm[u], __shfl_xor_sync(0xffffffffu, rm[u], 4));
+            }
+            if (a.per_vec) {
+                if (cg == 0)
+#pragma unroll
+                    for (int u = 0; u < 4; ++u)
+                        if (rg + 4 * u < M && rm[u] > 0.0f) atomicMax(&sync[l].bmax[rg + 4 * u], __float_as_uint(rm[u]));
+            } else {
+                rm[0] = fmaxf(rm[0], __shfl_xor_sync(0xffffffffu, rm[0], 8));
+                rm[0] = fmaxf(rm[0], __shfl_xor_sync(0xffffffffu, rm[0], 16));
+                if (lane == 0 && rm[0] > 0.0f) atomicMax(&sync[l].bmax[0], __float_as_uint(rm[0]));
+            }
+            {
+                int cnt = rg == 0 ? __popc(mask) : 0;
+                cnt += __shfl_xor_sync(0xffffffffu, cnt, 1);
+                cnt += __shfl_xor_sync(0xffffffffu, cnt, 2);
+                cnt += __shfl_xor_sync(0xffffffffu, cnt, 4);
+                if (lane == 0 && cnt > 0) atomicAdd(&sync[l].r, (uint32_t)cnt);
+            }
+            __syncwarp();
+            if (lane == 0) {
+                __threadfence();
+                atomicAdd(&sync[l].merged, 1u);
+            }
+            // ---- all slices merged: the scale(s) of Eq. 1 are final; codes of this slice
+            if (!wait_count(&sync[l].merged, (uint32_t)ns, abort_flag, g_abort, a.spin)) break;
+            const int r = (int)__ldcg(&sync[l].r);
+            if (r <= a.cap) {
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int m = rg + 4 * u;
+                    if (m >= M) break;
+                    const float mx = __uint_as_float(__ldcg(&sync[l].bmax[a.per_vec ? m : 0]));
+                    const float sc = mx > 0.0f ? __fdiv_rn(mx, qf) : 1.0f;
+                    float lo, hi;
+                    recip_bracket(__frcp_rn(sc), lo, hi);
+                    float f[8];
+                    unpack8(v[u], f);
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) f[i] *= mul[i];  // exact
+                    uint32_t cb[8];
+                    uint2 code;
+                    if (quant8_bracket(f, lo, hi, cb)) code = codes_exact(v[u], mask, down, sc, qf);  // rare
+                    else code = pack8(cb);
+                    *reinterpret_cast<uint2 *>(g_codes + (size_t)m * K + ch) = code;
+                }
+                if (rg == 0) {
+                    uint2 mb;
+                    mb.x = ((mask & 1) ? 0xFFu : 0u) | ((mask & 2) ? 0xFF00u : 0u) | ((mask & 4) ? 0xFF0000u : 0u) |
+                           ((mask & 8) ? 0xFF000000u : 0u);
+                    mb.y = ((mask & 16) ? 0xFFu : 0u) | ((mask & 32) ? 0xFF00u : 0u) | ((mask & 64) ? 0xFF0000u : 0u) |
+                           ((mask & 128) ? 0xFF000000u : 0u);
+                    *reinterpret_cast<uint2 *>(g_mask + ch) = mb;
+                }
+                const uint32_t any = __ballot_sync(0xffffffffu, mask != 0u);
+                if (lane == 0) g_segflag[s] = any ? 1 : 0;
+            }
+            __syncwarp();
+            if (lane == 0) {
+                __threadfence();
+                atomicAdd(&sync[l].coded, 1u);
+            }
         }
     } else {
         // ------------------------------------------------------------ unit warps: the products of layer l
@@ -483,7 +504,7 @@ __global__ void __launch_bounds__(kThreads, 1) k_decode_stream(const ChainArgs a
             const int8_t *xq = reinterpret_cast<const int8_t *>(buf + L.off_xq);
             const uint8_t *s_mask = buf + L.off_mask;
             const uint16_t *flaglist = reinterpret_cast<const uint16_t *>(buf + L.off_flaglist);
-            const int units = ly.N >> 3, nst = K / ly.seg, segs = ly.seg >> 6;
+            const int seg = (int)ly.seg, units = ly.N >> 3, nst = K / seg, segs = seg >> 6;
             const int first = first_unit(ly);
             const int cnt = first < units ? (units - first + grid - 1) / grid : 0;
             const float sw0 = a.per_vec ? 0.0f : __ldg(ly.s_w);
@@ -522,7 +543,7 @@ __global__ void __launch_bounds__(kThreads, 1) k_decode_stream(const ChainArgs a
                         // for both operands, which a dot product does not notice.  Segments go in batches whose loads
                         // are all issued before the first product (one warp walks a whole unit), with no test of the
                         // outlier flags:
-                        const uint8_t *wrow = ring + (size_t)pos.slot * a.slot_bytes + g * ly.seg + q * 16;
+                        const uint8_t *wrow = ring + (size_t)pos.slot * a.slot_bytes + g * seg + q * 16;
                         const int seg0 = st * segs;
                         constexpr int kB = kDotM == 1 ? 4 : 2;
                         auto body = [&](const uint4 &w, const int8_t *xp, int par) {
@@ -618,9 +639,21 @@ __global__ void __launch_bounds__(kThreads, 1) k_decode_stream(const ChainArgs a
             }
             ucount += cnt;
             lseq += cnt * nst;
-            // this warp is done with the layer's buffer (and has made its stores): one of the kUW arrivals
+            // this warp is done with the layer's buffer (and has made its stores).  When the next layer reads these
+            // stores, the last unit warp of the CTA to get here counts the CTA in (each warp's stores are ordered
+            // before its own count by a fence, and all of them before the CTA's by the last warp's).
             __syncwarp();
-            if (lane == 0) mbar_arrive(&bar_free[b]);
+            if (lane == 0) {
+                if (l + 1 < a.n_layers && (tab[l + 1].flags & kChainWaitPrev)) {
+                    __threadfence();
+                    if (atomicAdd(&s_unitdone[b], 1u) == (uint32_t)(kUW - 1)) {
+                        s_unitdone[b] = 0u;
+                        __threadfence();
+                        atomicAdd(&sync[l].stored, 1u);
+                    }
+                }
+                mbar_arrive(&bar_free[b]);  // one of the kUW arrivals
+            }
             if (*abort_flag) break;
         }
     }
@@ -638,17 +671,28 @@ bool chain_layer_supported(int M, int K, int N) {
 
 int chain_slot_bytes(int) { return 10 * 1024; }
 
+size_t chain_sync_bytes(int n_layers) { return (size_t)(n_layers + 1) * sizeof(LayerSync); }
+
+size_t chain_scratch_bytes(const ChainLayer *layers, int n_layers, int M) {
+    size_t b = 0;
+    for (int l = 0; l < n_layers; ++l) b += scratch_layer_bytes(M, layers[l].K);
+    return b;
+}
+
 int chain_plan(ChainLayer *layers, int n_layers, int grid, int slot_bytes) {
-    int kmax = 0, off = 0, waits = 0;
+    if (kSW * grid < kMaxK / 64) return -1;  // a warp would own two slices of one layer
+    int kmax = 0, off = 0, soff = 0;
     for (int l = 0; l < n_layers; ++l) {
         ChainLayer &ly = layers[l];
-        if (ly.flags & kChainWaitPrev) ly.flags = kChainWaitPrev | (++waits << 1);  // the ordinal of this wait
         int nst = 1;
         while (nst <= ly.K / 64 && !(ly.K % nst == 0 && (ly.K / nst) % 64 == 0 && 8 * (ly.K / nst) <= slot_bytes)) ++nst;
         if (nst > ly.K / 64) return -1;
-        ly.seg = ly.K / nst;
-        ly.unit_off = off;
+        ly.seg = (uint16_t)(ly.K / nst);
+        ly.unit_off = (uint16_t)off;
+        ly.slice_off = (uint16_t)soff;
+        ly.reserved = 0;
         off = (off + (ly.N >> 3)) % grid;
+        soff = (soff + (ly.K >> 6)) % (kSW * grid);
         if (ly.K > kmax) kmax = ly.K;
     }
     return kmax;
@@ -657,7 +701,7 @@ int chain_plan(ChainLayer *layers, int n_layers, int grid, int slot_bytes) {
 namespace {
 
 template <int MT, int kDotM>
-cudaError_t launch_inst(ChainArgs a, bool cooperative, cudaStream_t s) {
+cudaError_t launch_inst(ChainArgs a, cudaStream_t s) {
     constexpr int kRows = kDotM > 0 ? kDotM : MT;
     auto kern = k_decode_stream<MT, kDotM>;
     static PerDevice<int> attr_set;
@@ -671,43 +715,31 @@ cudaError_t launch_inst(ChainArgs a, bool cooperative, cudaStream_t s) {
             attr_set.have[dev] = true;
         }
     }
-    // the fp16 rows of X are staged in shared memory one layer ahead when they are few (two copies per group)
-    a.stage_x = (kDotM > 0 && a.M <= 2) ? 1 : 0;
-    // Small M: several groups of prepare warps, each on a layer of its own (one buffer more than groups); else one
-    // group and two buffers when that leaves the ring four stages, one buffer otherwise.
-    int slots = 0, fixed = 0;
-    int pg = a.n_layers < 2 ? 1 : a.M <= 2 ? 4 : a.M <= 4 ? 2 : 1;
-    for (; pg >= 1 && slots < 2; pg >>= 1) {
-        for (int nbuf = pg > 1 ? pg + 1 : 2; nbuf >= (pg > 1 ? pg + 1 : 1) && slots < 2; --nbuf) {
-            const XLayout L = x_layout(kRows, a.M, a.kmax, a.stage_x != 0, nbuf, pg);
-            fixed = a.n_layers * (int)sizeof(ChainLayer) + L.total;
-            slots = (kMaxSmem - fixed) / a.slot_bytes;
-            if (slots < (nbuf >= 2 ? 4 : 2)) slots = 0;
-            a.nbuf = nbuf;
-            a.pgroups = pg;
-        }
-    }
+    // As many buffers of prepared X (up to kMaxBufs) as leave the ring eight stages; at least one, and then at
+    // least two stages.
+    const XLayout L = x_layout(kRows, a.kmax);
+    const int table = a.n_layers * (int)sizeof(ChainLayer);
+    int nbuf = kMaxBufs;
+    while (nbuf > 1 && (kMaxSmem - table - nbuf * L.buf_bytes) / a.slot_bytes < 8) --nbuf;
+    int slots = (kMaxSmem - table - nbuf * L.buf_bytes) / a.slot_bytes;
     if (slots > kMaxSlots) slots = kMaxSlots;
     if (slots < 2) return cudaErrorInvalidValue;
+    a.nbuf = nbuf;
     a.lgroups = slots >= kLW ? kLW : 2;
     slots -= slots % a.lgroups;  // a slot keeps its loader warp
     a.slots = slots;
-    const size_t smem = (size_t)slots * a.slot_bytes + fixed;
-    if (cooperative) {
-        void *params[] = {&a};
-        return cudaLaunchCooperativeKernel(reinterpret_cast<const void *>(kern), dim3(a.grid), dim3(kThreads), params, smem, s);
-    }
-    kern<<<a.grid, kThreads, smem, s>>>(a);
-    return cudaGetLastError();
+    const size_t smem = (size_t)slots * a.slot_bytes + table + (size_t)nbuf * L.buf_bytes;
+    void *params[] = {&a};
+    return cudaLaunchCooperativeKernel(reinterpret_cast<const void *>(kern), dim3(a.grid), dim3(kThreads), params, smem, s);
 }
 
 }  // namespace
 
-cudaError_t launch_decode_chain(const ChainArgs &a, bool cooperative, cudaStream_t s) {
-    if (a.M == 1) return launch_inst<8, 1>(a, cooperative, s);
-    if (a.M <= 4) return launch_inst<8, 4>(a, cooperative, s);
-    if (a.M <= 8) return launch_inst<8, 0>(a, cooperative, s);
-    return launch_inst<16, 0>(a, cooperative, s);
+cudaError_t launch_decode_chain(const ChainArgs &a, cudaStream_t s) {
+    if (a.M == 1) return launch_inst<8, 1>(a, s);
+    if (a.M <= 4) return launch_inst<8, 4>(a, s);
+    if (a.M <= 8) return launch_inst<8, 0>(a, s);
+    return launch_inst<16, 0>(a, s);
 }
 
 }  // namespace muxq

@@ -188,16 +188,19 @@ cudaError_t launch_decode_fused(const DecodeFusedArgs &a, cudaStream_t s);
 
 // A list of decode-shaped layers (M <= 16 rows each) in one persistent launch (k4s_decode_stream.cu).
 constexpr int kChainMaxLayers = 256;
-constexpr int kChainWaitPrev = 1;  // ChainLayer::flags bit 0: X of this layer is written by the layer before it
-                                   // (bits 1..: the ordinal of this wait within the list, filled by chain_plan)
-struct ChainLayer {                // one entry of the device-resident layer table, 64 bytes
+constexpr int kChainSliceWarps = 7;  // warps per CTA that prepare slices of X for the whole grid
+constexpr int kChainWaitPrev = 1;    // ChainLayer::flags bit 0: X of this layer is written by the layer before it
+struct ChainLayer {                  // one entry of the device-resident layer table, 64 bytes
     const __half *X;
     const int8_t *w_q;
     const float *s_w;
     void *Y;
     int ldx, ldw, ldy, K, N, flags;
-    int unit_off;  // filled by the host: unit u of this layer goes to CTA (unit_off + u) mod grid
-    int seg;       // filled by the host: bytes of each W_q row per ring stage (K / seg stages per unit of 8 rows)
+    // filled by the host (chain_plan):
+    uint16_t unit_off;   // unit u of this layer goes to CTA (unit_off + u) mod grid
+    uint16_t seg;        // bytes of each W_q row per ring stage (K / seg stages per unit of 8 rows)
+    uint16_t slice_off;  // slice s of this layer's X goes to slice warp (slice_off + s) mod (kChainSliceWarps * grid)
+    uint16_t reserved;
 };
 static_assert(sizeof(ChainLayer) == 64, "layer table entry");
 struct ChainResult {               // per layer, written by CTA 0 (optional)
@@ -212,20 +215,22 @@ struct ChainArgs {
     float tau;
     int exp_factor, qmax, cap, c, per_vec, out_kind;
     ChainResult *results;          // [n_layers] or NULL
-    uint32_t *barrier;             // arrival counter of the grid-wide barriers, zero on entry (NULL: no layer waits)
+    uint8_t *sync;                 // chain_sync_bytes(n_layers) of device memory, zero on entry: per-layer counters and maxima
+    uint8_t *scratch;              // chain_scratch_bytes(...) of device memory: per-layer codes, masks, segment flags
     int32_t *dev_status;
     uint32_t spin;
     int slots, slot_bytes;         // ring geometry
-    int nbuf, pgroups;             // buffers of prepared X, groups of prepare warps (set by the launcher)
-    int stage_x;                   // the fp16 rows of X are staged in shared memory one layer ahead (set by the launcher)
+    int nbuf;                      // buffers of prepared X per CTA (set by the launcher)
     int lgroups;                   // loader warps in use; divides slots (set by the launcher)
 };
-// Fills unit_off / seg / wait ordinals of every entry (host copy of the table); returns the widest K, -1 if a layer
-// does not fit.
+// Fills unit_off / seg / slice_off of every entry (host copy of the table); returns the widest K, -1 if a layer
+// does not fit (or the grid is too small for the slice scheme).
 int chain_plan(ChainLayer *layers, int n_layers, int grid, int slot_bytes);
 int chain_slot_bytes(int M);  // bytes of a ring stage for lists of M-row layers
+size_t chain_sync_bytes(int n_layers);
+size_t chain_scratch_bytes(const ChainLayer *layers, int n_layers, int M);
 bool chain_layer_supported(int M, int K, int N);
-cudaError_t launch_decode_chain(const ChainArgs &a, bool cooperative, cudaStream_t s);
+cudaError_t launch_decode_chain(const ChainArgs &a, cudaStream_t s);  // cooperative launch, a.grid CTAs
 
 cudaError_t launch_mma_peak(int n, int iters, unsigned long long *cycles_out, int32_t *status, int grid,
                             cudaStream_t s);
