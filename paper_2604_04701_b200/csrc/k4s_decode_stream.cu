@@ -17,11 +17,12 @@
 //                   derives the slice's channel maxima and outlier flags (Section III-C) and merges the maxima of
 //                   Body (Eq. 4) into the layer's words in global memory; when all slices of the layer have done so
 //                   (a counter), the scale(s) of Eq. 1 are known and the warp writes its slice's INT8 codes and
-//                   its outlier mask to the layer's scratch area in global memory and counts itself done.
+//                   its outlier mask to the layer's scratch area in global memory and counts itself done; the
+//                   last one to do so also writes the layer's header (scales, r, the list of 64-byte segments
+//                   that hold an outlier channel) and raises the layer's ready word.
 //                   Every CTA used to do all of this for itself, which cost more than the weight stream.
-//   fetch warp      per layer, in order: waits until all slices are done, builds the list of flagged 64-byte
-//                   segments and the header (scales, r) in one of the CTA's buffers in shared memory and has the
-//                   copy engine bring the codes and the mask there.
+//   fetch warp      per layer, in order: once the layer is ready (one poll looks 32 layers ahead) and one of the
+//                   CTA's buffers in shared memory is free, has the copy engine bring header, codes and mask there.
 //   unit warps      per layer: each unit is taken by ONE warp, which accumulates the unit's 8 x M outputs over all
 //                   of K in registers (4-way byte dot products for M <= 4, mma.sync m16n8k32 above), adds the Aux
 //                   term of Eq. 7 for the 64-byte segments that hold an outlier channel, dequantizes and stores.
@@ -130,35 +131,38 @@ struct LayerSync {
     uint32_t r;           // outlier channels found so far
     uint32_t stored;      // CTAs whose units of this layer are stored (counted only when the next layer waits)
     uint32_t bmax[16];    // bit patterns of the row maxima of Body (per tensor: word 0 only)
-    uint32_t pad[12];
+    uint32_t ready;       // the layer's header, codes and mask are complete
+    uint32_t pad[11];
 };
 static_assert(sizeof(LayerSync) == 128, "per-layer words");
 
-// A layer's scratch area in global memory: codes [M][K], mask [K] (0xFF at outlier channels), segflag [K / 64].
+// A layer's scratch area in global memory: header block (XHeader, then the list of flagged segments),
+// codes [M][K], mask [K] (0xFF at outlier channels), segflag [K / 64].
+constexpr int kHeaderBytes = 128, kFlagListBytes = 2 * (kMaxK / 64), kHeadBlock = kHeaderBytes + kFlagListBytes;
 __host__ __device__ inline size_t scratch_codes_bytes(int M, int K) { return ((size_t)M * K + 127) & ~(size_t)127; }
 __host__ __device__ inline size_t scratch_layer_bytes(int M, int K) {
-    return scratch_codes_bytes(M, K) + (size_t)K + (size_t)(((K >> 6) + 127) & ~127);
+    return (size_t)kHeadBlock + scratch_codes_bytes(M, K) + (size_t)K + (size_t)(((K >> 6) + 127) & ~127);
 }
 
 // A buffer in shared memory that holds a layer's prepared X (sized for the widest K of the list).
 struct XLayout {
     int pitch;          // bytes per row of X codes; pitch % 128 == 64 keeps the 8-row x 64-byte reads conflict free
-    int off_xq;         // [rows][pitch] INT8 codes (behind a 128-byte header: 16 row scales, r, list length)
+    int off_flaglist;   // [K/64] u16 behind the 128-byte header: the segments that hold an outlier channel, ascending
+    int off_xq;         // [rows][pitch] INT8 codes
     int off_mask;       // [K] 0xFF at outlier channels
-    int off_flaglist;   // [K/64] u16: the segments that hold an outlier channel, ascending
     int buf_bytes;
 };
 __host__ __device__ inline XLayout x_layout(int rows, int K) {
     XLayout s;
     s.pitch = K + ((64 - (K & 127)) & 127);
     if ((s.pitch & 127) != 64) s.pitch += 64;
-    s.off_xq = 128;
+    s.off_flaglist = kHeaderBytes;
+    s.off_xq = kHeadBlock;
     s.off_mask = s.off_xq + rows * s.pitch;
-    s.off_flaglist = s.off_mask + K;
-    s.buf_bytes = (s.off_flaglist + 2 * (K >> 6) + 127) & ~127;
+    s.buf_bytes = (s.off_mask + K + 127) & ~127;
     return s;
 }
-struct XHeader {        // first bytes of a buffer
+struct XHeader {        // first bytes of a buffer and of a layer's scratch area
     float rowscale[16];
     int r;              // outlier channels of this layer's X
     int nflag;          // entries of the list of flagged segments
@@ -287,70 +291,56 @@ __global__ void __launch_bounds__(kThreads, 1) k_decode_stream(const ChainArgs a
             }
     } else if (warp == kFetch) {
         // ------------------------------------------------------------ fetch warp: prepared X of layer l into buffer l mod NB
-        const float qf = (float)a.qmax;
         size_t scr = 0;  // offset of the layer's scratch area
-        uint32_t last_bytes = 0;
+        int ready_upto = 0;  // layers below this one are known to be ready
         int last_buf = -1;
         uint32_t last_phase = 0;
         for (int l = 0; l < a.n_layers; ++l) {
             const ChainLayer ly = tab[l];
-            const int K = ly.K, ns = K >> 6, b = l % NB, ph = l / NB;
+            const int K = ly.K, b = l % NB, ph = l / NB;
             uint8_t *buf = xbase + b * L.buf_bytes;
-            XHeader *hdr = reinterpret_cast<XHeader *>(buf);
-            const uint8_t *g_codes = a.scratch + scr;
+            const uint8_t *g_head = a.scratch + scr;
+            const uint8_t *g_codes = g_head + kHeadBlock;
             const uint8_t *g_mask = g_codes + scratch_codes_bytes(M, K);
-            const uint8_t *g_segflag = g_mask + K;
             scr += scratch_layer_bytes(M, K);
-            // the buffer was last read for layer l - NB; then all slices of this layer must be coded
+            // the buffer was last read for layer l - NB
             if (l >= NB && !wait_sleep(&bar_free[b], (uint32_t)(ph - 1) & 1u, abort_flag, a.spin)) break;
-            if (!wait_count(&sync[l].coded, (uint32_t)ns, abort_flag, g_abort, a.spin)) break;
-            const int r = (int)__ldcg(&sync[l].r);
-            const bool over = r > a.cap;  // MUXQ_ERR_CAPACITY: no codes were written, Y of this layer is unspecified
-            if (lane < 16) {
-                const float mx = __uint_as_float(__ldcg(&sync[l].bmax[a.per_vec ? lane : 0]));
-                hdr->rowscale[lane] = mx > 0.0f ? __fdiv_rn(mx, qf) : 1.0f;
-            }
-            // the flagged 64-byte segments, compacted in ascending order
-            uint16_t *flaglist = reinterpret_cast<uint16_t *>(buf + L.off_flaglist);
-            int nf = 0;
-            if (!over)
-                for (int base = 0; base < ns; base += 32) {
-                    const bool f = base + lane < ns && __ldcg(g_segflag + base + lane) != 0;
-                    const uint32_t bal = __ballot_sync(0xffffffffu, f);
-                    if (f) flaglist[nf + __popc(bal & ((1u << lane) - 1u))] = (uint16_t)(base + lane);
-                    nf += __popc(bal);
-                }
-            if (lane == 0) {
-                hdr->r = r;
-                hdr->nflag = nf;
-                if (cta == 0) {
-                    if (over && a.dev_status) atomicMax(a.dev_status, kStatusCapacity);
-                    if (a.results) {
-                        ChainResult rr;
-                        rr.n_outliers = r;
-                        rr.status = over ? kStatusCapacity : 0;
-                        rr.s_x = hdr->rowscale[0];
-                        rr.reserved = 0;
-                        a.results[l] = rr;
+            if (l >= ready_upto) {
+                // lane i looks at layer l + i: in a list of independent layers most are ready long before their turn
+                bool ok = false, stopped = false;
+                for (uint32_t i = 0; i < a.spin && !ok && !stopped; ++i) {
+                    const bool rdy = l + lane < a.n_layers && ld_acquire_u32(&sync[l + lane].ready) != 0u;
+                    const uint32_t bal = __ballot_sync(0xffffffffu, rdy);
+                    const int n = __ffs((int)~bal) - 1;  // consecutive ready layers from l on (-1: all 32)
+                    if (n != 0) {
+                        ready_upto = l + (n < 0 ? 32 : n);
+                        ok = true;
+                    } else {
+                        __nanosleep(i < 8 ? 100 : 400);
+                        if ((i & 7u) == 7u)
+                            stopped = __any_sync(0xffffffffu, *abort_flag != 0u || ld_relaxed_u32(g_abort) != 0u);
                     }
                 }
+                if (!ok) {
+                    if (lane == 0) {
+                        *abort_flag = 1u;
+                        if (!stopped) atomicExch(g_abort, 1u);
+                    }
+                    break;
+                }
             }
-            // the header and the list are ordered before the arrival that announces the bytes; the codes and the mask,
-            // written by other SMs and made visible by the acquire above, are ordered before the copy engine reads them
-            const uint32_t bytes = over ? 0u : (uint32_t)(M * K + K);
+            // header, codes and mask, written by other SMs and made visible by the acquire, are ordered before the
+            // copy engine reads them
             fence_proxy_async_all();
+            if (lane == 0) mbar_expect_tx(&bar_ready[b], (uint32_t)(kHeadBlock + M * K + K));
             __syncwarp();
-            if (lane == 0) mbar_expect_tx(&bar_ready[b], bytes);
-            __syncwarp();
-            if (!over) {
-                int8_t *xq = reinterpret_cast<int8_t *>(buf + L.off_xq);
-                if (lane < M) bulk_load(xq + (size_t)lane * L.pitch, g_codes + (size_t)lane * K, (uint32_t)K, &bar_ready[b]);
-                if (lane == 31) bulk_load(buf + L.off_mask, g_mask, (uint32_t)K, &bar_ready[b]);
-            }
-            last_bytes = bytes; last_buf = b; last_phase = (uint32_t)ph & 1u;
+            if (lane < M) bulk_load(buf + L.off_xq + (size_t)lane * L.pitch, g_codes + (size_t)lane * K, (uint32_t)K, &bar_ready[b]);
+            if (lane == 30) bulk_load(buf, g_head, (uint32_t)kHeadBlock, &bar_ready[b]);
+            if (lane == 31) bulk_load(buf + L.off_mask, g_mask, (uint32_t)K, &bar_ready[b]);
+            last_buf = b; last_phase = (uint32_t)ph & 1u;
         }
         // the copies of the last layer fetched have landed before this warp leaves (see the loaders)
-        if (last_buf >= 0 && last_bytes > 0u) {
+        if (last_buf >= 0) {
             bool landed = false;
             for (uint32_t k = 0; k < a.spin && !landed; ++k) landed = mbar_try_wait(&bar_ready[last_buf], last_phase);
         }
@@ -366,7 +356,8 @@ __global__ void __launch_bounds__(kThreads, 1) k_decode_stream(const ChainArgs a
         for (int l = 0; l < a.n_layers; ++l) {
             const ChainLayer ly = tab[l];
             const int K = ly.K, ns = K >> 6;
-            uint8_t *g_codes = a.scratch + scr;
+            uint8_t *g_head = a.scratch + scr;
+            uint8_t *g_codes = g_head + kHeadBlock;
             uint8_t *g_mask = g_codes + scratch_codes_bytes(M, K);
             uint8_t *g_segflag = g_mask + K;
             scr += scratch_layer_bytes(M, K);
@@ -486,9 +477,61 @@ __global__ void __launch_bounds__(kThreads, 1) k_decode_stream(const ChainArgs a
                 if (lane == 0) g_segflag[s] = any ? 1 : 0;
             }
             __syncwarp();
+            uint32_t before = 0;
             if (lane == 0) {
                 __threadfence();
-                atomicAdd(&sync[l].coded, 1u);
+                before = atomicAdd(&sync[l].coded, 1u);
+            }
+            before = __shfl_sync(0xffffffffu, before, 0);
+            if (before + 1u == (uint32_t)ns) {
+                // ---- the last slice of the layer: header block (scales, r, flagged 64-byte segments in ascending
+                // order), per-layer result, then the ready word
+                __threadfence();
+                const bool over = r > a.cap;  // MUXQ_ERR_CAPACITY: no codes were written, Y of this layer is unspecified
+                XHeader *hdr = reinterpret_cast<XHeader *>(g_head);
+                uint16_t *flaglist = reinterpret_cast<uint16_t *>(g_head + kHeaderBytes);
+                float sc0 = 1.0f;
+                if (lane < 16) {
+                    const float mx = __uint_as_float(__ldcg(&sync[l].bmax[a.per_vec ? lane : 0]));
+                    sc0 = mx > 0.0f ? __fdiv_rn(mx, qf) : 1.0f;
+                    hdr->rowscale[lane] = sc0;
+                }
+                uint32_t bits = 0;  // this lane: segments 4 lane .. 4 lane + 3
+                if (!over) {
+                    const uint32_t w = __ldcg(reinterpret_cast<const uint32_t *>(g_segflag) + lane);
+#pragma unroll
+                    for (int j = 0; j < 4; ++j)
+                        if (4 * lane + j < ns && ((w >> (8 * j)) & 0xFFu)) bits |= 1u << j;
+                }
+                int pre = __popc(bits);  // inclusive prefix count over the lanes
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const int n = __shfl_up_sync(0xffffffffu, pre, o);
+                    if (lane >= o) pre += n;
+                }
+                const int nf = __shfl_sync(0xffffffffu, pre, 31);
+                int at = pre - __popc(bits);
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+                    if ((bits >> j) & 1u) flaglist[at++] = (uint16_t)(4 * lane + j);
+                if (lane == 0) {
+                    hdr->r = r;
+                    hdr->nflag = nf;
+                    if (over && a.dev_status) atomicMax(a.dev_status, kStatusCapacity);
+                    if (a.results) {
+                        ChainResult rr;
+                        rr.n_outliers = r;
+                        rr.status = over ? kStatusCapacity : 0;
+                        rr.s_x = sc0;
+                        rr.reserved = 0;
+                        a.results[l] = rr;
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) {
+                    __threadfence();
+                    atomicExch(&sync[l].ready, 1u);
+                }
             }
         }
     } else {
