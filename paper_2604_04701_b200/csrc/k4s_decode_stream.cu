@@ -51,7 +51,7 @@ constexpr int kLW = 4;                  // loader warps (warps 16..19)
 constexpr int kLoader0 = kUW + 1 + kSW; // index of the first loader warp
 constexpr int kThreads = 32 * (kLoader0 + kLW);
 constexpr int kMaxK = 8192;             // widest layer: 128 slices
-constexpr int kMaxBufs = 4;             // buffers of prepared X per CTA
+constexpr int kMaxBufs = 8;             // buffers of prepared X per CTA
 constexpr int kMaxSlots = 24;
 constexpr int kStatusCapacity = 5;      // MUXQ_ERR_CAPACITY
 constexpr int kStatusTimeout = 6;       // MUXQ_ERR_TIMEOUT
@@ -136,9 +136,12 @@ struct LayerSync {
 };
 static_assert(sizeof(LayerSync) == 128, "per-layer words");
 
-// A layer's scratch area in global memory: header block (XHeader, then the list of flagged segments),
-// codes [M][K], mask [K] (0xFF at outlier channels), segflag [K / 64].
-constexpr int kHeaderBytes = 128, kFlagListBytes = 2 * (kMaxK / 64), kHeadBlock = kHeaderBytes + kFlagListBytes;
+// A layer's scratch area in global memory: header block (XHeader, the list of flagged segments, the list of the
+// first kChList outlier channels in no particular order), codes [M][K], mask [K] (0xFF at outlier channels),
+// segflag [K / 64].
+constexpr int kChList = 64;
+constexpr int kHeaderBytes = 128, kFlagListBytes = 2 * (kMaxK / 64);
+constexpr int kHeadBlock = kHeaderBytes + kFlagListBytes + 2 * kChList;
 __host__ __device__ inline size_t scratch_codes_bytes(int M, int K) { return ((size_t)M * K + 127) & ~(size_t)127; }
 __host__ __device__ inline size_t scratch_layer_bytes(int M, int K) {
     return (size_t)kHeadBlock + scratch_codes_bytes(M, K) + (size_t)K + (size_t)(((K >> 6) + 127) & ~127);
@@ -148,6 +151,7 @@ __host__ __device__ inline size_t scratch_layer_bytes(int M, int K) {
 struct XLayout {
     int pitch;          // bytes per row of X codes; pitch % 128 == 64 keeps the 8-row x 64-byte reads conflict free
     int off_flaglist;   // [K/64] u16 behind the 128-byte header: the segments that hold an outlier channel, ascending
+    int off_chlist;     // [kChList] u16: outlier channels (all of them when r <= kChList)
     int off_xq;         // [rows][pitch] INT8 codes
     int off_mask;       // [K] 0xFF at outlier channels
     int buf_bytes;
@@ -157,6 +161,7 @@ __host__ __device__ inline XLayout x_layout(int rows, int K) {
     s.pitch = K + ((64 - (K & 127)) & 127);
     if ((s.pitch & 127) != 64) s.pitch += 64;
     s.off_flaglist = kHeaderBytes;
+    s.off_chlist = kHeaderBytes + kFlagListBytes;
     s.off_xq = kHeadBlock;
     s.off_mask = s.off_xq + rows * s.pitch;
     s.buf_bytes = (s.off_mask + K + 127) & ~127;
@@ -328,10 +333,10 @@ __global__ void __launch_bounds__(kThreads, 1) k_decode_stream(const ChainArgs a
                     }
                     break;
                 }
+                // headers, codes and masks of the layers found ready, written by other SMs and made visible by the
+                // acquire, are ordered before the copy engine reads them
+                fence_proxy_async_all();
             }
-            // header, codes and mask, written by other SMs and made visible by the acquire, are ordered before the
-            // copy engine reads them
-            fence_proxy_async_all();
             if (lane == 0) mbar_expect_tx(&bar_ready[b], (uint32_t)(kHeadBlock + M * K + K));
             __syncwarp();
             if (lane < M) bulk_load(buf + L.off_xq + (size_t)lane * L.pitch, g_codes + (size_t)lane * K, (uint32_t)K, &bar_ready[b]);
@@ -432,11 +437,29 @@ __global__ void __launch_bounds__(kThreads, 1) k_decode_stream(const ChainArgs a
                 if (lane == 0 && rm[0] > 0.0f) atomicMax(&sync[l].bmax[0], __float_as_uint(rm[0]));
             }
             {
-                int cnt = rg == 0 ? __popc(mask) : 0;
-                cnt += __shfl_xor_sync(0xffffffffu, cnt, 1);
-                cnt += __shfl_xor_sync(0xffffffffu, cnt, 2);
-                cnt += __shfl_xor_sync(0xffffffffu, cnt, 4);
-                if (lane == 0 && cnt > 0) atomicAdd(&sync[l].r, (uint32_t)cnt);
+                // outlier count of the layer; the channels also go to the layer's list, at the places the count
+                // hands out (lanes 0..7 hold the slice's eight channel groups)
+                const int mine = rg == 0 ? __popc(mask) : 0;
+                int pre = mine;
+#pragma unroll
+                for (int o = 1; o < 8; o <<= 1) {
+                    const int n = __shfl_up_sync(0xffffffffu, pre, o);
+                    if (cg >= o) pre += n;
+                }
+                const int total = __shfl_sync(0xffffffffu, pre, 7);
+                uint32_t base = 0;
+                if (lane == 0 && total > 0) base = atomicAdd(&sync[l].r, (uint32_t)total);
+                base = __shfl_sync(0xffffffffu, base, 0);
+                if (rg == 0 && mine > 0) {
+                    uint16_t *chl = reinterpret_cast<uint16_t *>(g_head + kHeaderBytes + kFlagListBytes);
+                    int at = (int)base + pre - mine;
+#pragma unroll
+                    for (int i = 0; i < 8; ++i)
+                        if ((mask >> i) & 1u) {
+                            if (at < kChList) chl[at] = (uint16_t)(ch + i);
+                            ++at;
+                        }
+                }
             }
             __syncwarp();
             if (lane == 0) {
@@ -538,7 +561,12 @@ __global__ void __launch_bounds__(kThreads, 1) k_decode_stream(const ChainArgs a
         // ------------------------------------------------------------ unit warps: the products of layer l
         const int g = lane >> 2, q = lane & 3;
         int lseq = 0;    // number of this CTA's stages before the current layer
-        int ucount = 0;  // units of this CTA before the current layer
+        int ucount = 0;  // units of this CTA before the current layer, modulo kUW
+        // M <= 4: lane (g, q) reads 16 bytes of W_q row 8u + g per 64-byte segment and the matching 16 bytes of the
+        // codes of X.  Segments are taken in pairs, rows with odd g second segment first, so that the eight lanes
+        // that shared memory serves together touch all 32 banks (a row is a multiple of 128 bytes long); the K order
+        // is permuted the same way for both operands, which a dot product does not notice.
+        const int oa = (g & 1) * 64 + q * 16, ob = (1 - (g & 1)) * 64 + q * 16;
         for (int l = 0; l < a.n_layers; ++l) {
             const ChainLayer ly = tab[l];
             const int K = ly.K, b = l % NB, ph = l / NB;
@@ -547,140 +575,214 @@ __global__ void __launch_bounds__(kThreads, 1) k_decode_stream(const ChainArgs a
             const int8_t *xq = reinterpret_cast<const int8_t *>(buf + L.off_xq);
             const uint8_t *s_mask = buf + L.off_mask;
             const uint16_t *flaglist = reinterpret_cast<const uint16_t *>(buf + L.off_flaglist);
+            const uint16_t *chlist = reinterpret_cast<const uint16_t *>(buf + L.off_chlist);
             const int seg = (int)ly.seg, units = ly.N >> 3, nst = K / seg, segs = seg >> 6;
             const int first = first_unit(ly);
             const int cnt = first < units ? (units - first + grid - 1) / grid : 0;
-            const float sw0 = a.per_vec ? 0.0f : __ldg(ly.s_w);
+            const int i0 = (warp - ucount) & (kUW - 1);  // unit number ucount + i goes to warp (ucount + i) mod kUW
             if (!wait_sleep(&bar_ready[b], (uint32_t)ph & 1u, abort_flag, a.spin)) break;
-            const int nflag = hdr->nflag;
-            const bool skip = hdr->r > a.cap;  // MUXQ_ERR_CAPACITY: Y of this layer is unspecified; its weights still drain
-            for (int i = (warp - ucount) & (kUW - 1); i < cnt; i += kUW) {  // unit number ucount + i goes to warp (ucount + i) mod kUW
-                const int u = first + i * grid;
-                const int seq0 = lseq + i * nst;
-                RingPos pos;
-                pos.slot = seq0 % S;
-                pos.use = (uint32_t)(seq0 / S);
-                // Body accumulators (two: consecutive products on one accumulator wait for each other) and the Aux
-                // accumulator over the outlier channels (Aux_q == Body_q[:, O], Eq. 5)
-                int accb[4] = {0, 0, 0, 0}, accb2[4] = {0, 0, 0, 0}, acca[4] = {0, 0, 0, 0};
-                bool got = true;
-                for (int st = 0; st < nst; ++st) {
-                    // A barrier phase is told from the one two uses earlier only by its parity, so a warp must not wait
-                    // for a stage before the loaders have begun to fill it (by then the slot's previous use has been
-                    // consumed and its phase is complete).  With more units per layer than ring slots a warp can get
-                    // that far ahead.
-                    {
-                        uint32_t spins = 0;
-                        while (s_begun[pos.slot] <= pos.use && ++spins < a.spin) {
-                            __nanosleep(40);
-                            if ((spins & 15u) == 15u && *abort_flag) break;
-                        }
-                        got = __all_sync(0xffffffffu, s_begun[pos.slot] > pos.use);
-                        if (!got) *abort_flag = 1u;
-                    }
-                    got = got && wait_sleep(&bar_full[pos.slot], pos.use & 1u, abort_flag, a.spin);
-                    if (!got) break;
-                    if (!skip) {
-                        // lane (g, q) reads 16 bytes of W_q row 8u + g per 64-byte segment; the matching 16 bytes of the
-                        // codes of X come from shared memory.  The K order inside a segment is permuted the same way
-                        // for both operands, which a dot product does not notice.  Segments go in batches whose loads
-                        // are all issued before the first product (one warp walks a whole unit), with no test of the
-                        // outlier flags:
-                        const uint8_t *wrow = ring + (size_t)pos.slot * a.slot_bytes + g * seg + q * 16;
-                        const int seg0 = st * segs;
-                        constexpr int kB = kDotM == 1 ? 4 : 2;
-                        auto body = [&](const uint4 &w, const int8_t *xp, int par) {
-                            if constexpr (kDotM > 0) {
+            if (i0 < cnt) {
+                const float sw0 = a.per_vec ? 0.0f : __ldg(ly.s_w);
+                const int r = hdr->r, nflag = hdr->nflag;
+                const bool skip = r > a.cap;     // MUXQ_ERR_CAPACITY: Y of this layer is unspecified; its weights still drain
+                const bool listed = r <= kChList;  // every outlier channel is in the list
+                for (int i = i0; i < cnt; i += kUW) {
+                    const int u = first + i * grid;
+                    const int seq0 = lseq + i * nst;
+                    RingPos pos;
+                    pos.slot = seq0 % S;
+                    pos.use = (uint32_t)(seq0 / S);
+                    // Body accumulators (several: consecutive products on one accumulator wait for each other) and the
+                    // Aux accumulator over the outlier channels (Aux_q == Body_q[:, O], Eq. 5)
+                    constexpr int kAcc = kDotM == 1 ? 4 : 2;
+                    int accb[kAcc][4], acca[4] = {0, 0, 0, 0};
 #pragma unroll
-                                for (int m = 0; m < kDotM; ++m) {
-                                    const uint4 x = *reinterpret_cast<const uint4 *>(xp + m * L.pitch);
-                                    int &acc = par ? accb2[m] : accb[m];
-                                    acc = __dp4a((int)w.x, (int)x.x, acc);
-                                    acc = __dp4a((int)w.y, (int)x.y, acc);
-                                    acc = __dp4a((int)w.z, (int)x.z, acc);
-                                    acc = __dp4a((int)w.w, (int)x.w, acc);
+                    for (int j = 0; j < kAcc; ++j) accb[j][0] = accb[j][1] = accb[j][2] = accb[j][3] = 0;
+                    bool got = true;
+                    for (int st = 0; st < nst; ++st) {
+                        // A barrier phase is told from the one two uses earlier only by its parity, so a warp must not
+                        // wait for a stage before the loaders have begun to fill it (by then the slot's previous use has
+                        // been consumed and its phase is complete).  With more units per layer than ring slots a warp
+                        // can get that far ahead.
+                        {
+                            uint32_t spins = 0;
+                            while (s_begun[pos.slot] <= pos.use && ++spins < a.spin) {
+                                __nanosleep(40);
+                                if ((spins & 15u) == 15u && *abort_flag) break;
+                            }
+                            got = __all_sync(0xffffffffu, s_begun[pos.slot] > pos.use);
+                            if (!got) *abort_flag = 1u;
+                        }
+                        got = got && wait_sleep(&bar_full[pos.slot], pos.use & 1u, abort_flag, a.spin);
+                        if (!got) break;
+                        if (!skip) {
+                            const uint8_t *wst = ring + (size_t)pos.slot * a.slot_bytes;  // the stage: 8 rows of seg bytes
+                            const uint8_t *wrow = wst + g * seg;
+                            const int k0 = st * seg;
+                            const int8_t *xseg = xq + k0;
+                            if constexpr (kDotM > 0) {
+                                constexpr int kP = kAcc / 2;  // pairs of segments per batch: all loads, then all products
+                                int sgi = 0;
+                                for (; sgi + 2 * kP <= segs; sgi += 2 * kP) {
+                                    uint4 w[2 * kP], x[2 * kP][kDotM];
+#pragma unroll
+                                    for (int j = 0; j < 2 * kP; ++j) {
+                                        const int o = (sgi + (j & ~1)) * 64 + ((j & 1) ? ob : oa);
+                                        w[j] = *reinterpret_cast<const uint4 *>(wrow + o);
+#pragma unroll
+                                        for (int m = 0; m < kDotM; ++m) x[j][m] = *reinterpret_cast<const uint4 *>(xseg + m * L.pitch + o);
+                                    }
+#pragma unroll
+                                    for (int j = 0; j < 2 * kP; ++j)
+#pragma unroll
+                                        for (int m = 0; m < kDotM; ++m) {
+                                            int acc = accb[j][m];
+                                            acc = __dp4a((int)w[j].x, (int)x[j][m].x, acc);
+                                            acc = __dp4a((int)w[j].y, (int)x[j][m].y, acc);
+                                            acc = __dp4a((int)w[j].z, (int)x[j][m].z, acc);
+                                            acc = __dp4a((int)w[j].w, (int)x[j][m].w, acc);
+                                            accb[j][m] = acc;
+                                        }
+                                }
+                                for (; sgi < segs; ++sgi) {  // what is left, segment by segment in plain order
+                                    const int o = sgi * 64 + q * 16;
+                                    const uint4 w = *reinterpret_cast<const uint4 *>(wrow + o);
+#pragma unroll
+                                    for (int m = 0; m < kDotM; ++m) {
+                                        const uint4 x = *reinterpret_cast<const uint4 *>(xseg + m * L.pitch + o);
+                                        int acc = accb[0][m];
+                                        acc = __dp4a((int)w.x, (int)x.x, acc);
+                                        acc = __dp4a((int)w.y, (int)x.y, acc);
+                                        acc = __dp4a((int)w.z, (int)x.z, acc);
+                                        acc = __dp4a((int)w.w, (int)x.w, acc);
+                                        accb[0][m] = acc;
+                                    }
                                 }
                             } else {
-                                const uint4 alo = *reinterpret_cast<const uint4 *>(xp + g * L.pitch);
-                                uint4 ahi = make_uint4(0u, 0u, 0u, 0u);
-                                if (MT == 16) ahi = *reinterpret_cast<const uint4 *>(xp + (g + 8) * L.pitch);
-                                mma_s8(accb, alo.x, ahi.x, alo.y, ahi.y, w.x, w.y);
-                                mma_s8(accb2, alo.z, ahi.z, alo.w, ahi.w, w.z, w.w);
+                                // mma.sync tiles: lane (g, q) supplies 16 bytes of token rows g and g + 8 and of W_q row
+                                // 8u + g per segment (the K order inside a segment permuted alike for both operands)
+                                int sgi = 0;
+                                for (; sgi + 2 <= segs; sgi += 2) {
+                                    uint4 w[2], alo[2], ahi[2];
+#pragma unroll
+                                    for (int j = 0; j < 2; ++j) {
+                                        const int o = (sgi + j) * 64 + q * 16;
+                                        w[j] = *reinterpret_cast<const uint4 *>(wrow + o);
+                                        alo[j] = *reinterpret_cast<const uint4 *>(xseg + g * L.pitch + o);
+                                        ahi[j] = MT == 16 ? *reinterpret_cast<const uint4 *>(xseg + (g + 8) * L.pitch + o) : make_uint4(0u, 0u, 0u, 0u);
+                                    }
+#pragma unroll
+                                    for (int j = 0; j < 2; ++j) {
+                                        mma_s8(accb[0], alo[j].x, ahi[j].x, alo[j].y, ahi[j].y, w[j].x, w[j].y);
+                                        mma_s8(accb[1], alo[j].z, ahi[j].z, alo[j].w, ahi[j].w, w[j].z, w[j].w);
+                                    }
+                                }
+                                for (; sgi < segs; ++sgi) {
+                                    const int o = sgi * 64 + q * 16;
+                                    const uint4 w = *reinterpret_cast<const uint4 *>(wrow + o);
+                                    const uint4 alo = *reinterpret_cast<const uint4 *>(xseg + g * L.pitch + o);
+                                    const uint4 ahi = MT == 16 ? *reinterpret_cast<const uint4 *>(xseg + (g + 8) * L.pitch + o) : make_uint4(0u, 0u, 0u, 0u);
+                                    mma_s8(accb[0], alo.x, ahi.x, alo.y, ahi.y, w.x, w.y);
+                                    mma_s8(accb[1], alo.z, ahi.z, alo.w, ahi.w, w.z, w.w);
+                                }
                             }
-                        };
-                        const int8_t *xseg = xq + (size_t)seg0 * 64 + q * 16;
-                        int sgi = 0;
-                        for (; sgi + kB <= segs; sgi += kB) {
-                            uint4 w[kB];
+                            // ... then the Aux term (Eq. 7) over the outlier channels that fall into this stage
+                            if (listed) {
+                                // from the channel list: single products W_q[n][k] * X_q[m][k]
+                                if constexpr (kDotM > 0) {
+                                    // lane (g, q): output channel 8u + g, every fourth list entry (the four lanes add up below)
+                                    for (int o = q; o < r; o += 4) {
+                                        const int kk = (int)chlist[o] - k0;
+                                        if ((unsigned)kk < (unsigned)seg) {
+                                            const int w = (int)(int8_t)wrow[kk];
 #pragma unroll
-                            for (int j = 0; j < kB; ++j) w[j] = *reinterpret_cast<const uint4 *>(wrow + (sgi + j) * 64);
-#pragma unroll
-                            for (int j = 0; j < kB; ++j) body(w[j], xseg + (sgi + j) * 64, j & 1);
-                        }
-                        for (; sgi < segs; ++sgi) body(*reinterpret_cast<const uint4 *>(wrow + sgi * 64), xseg + sgi * 64, 0);
-                        // ... then the Aux term (Eq. 7) for the few segments of this stage that hold an outlier channel,
-                        // from the list the prepare warps made: the same products with X masked to those channels
-                        for (int j = 0; j < nflag; ++j) {
-                            const int fs = (int)flaglist[j] - seg0;
-                            if (fs < 0 || fs >= segs) continue;  // warp-uniform
-                            const uint4 w = *reinterpret_cast<const uint4 *>(wrow + fs * 64);
-                            const uint4 mk = *reinterpret_cast<const uint4 *>(s_mask + (size_t)(seg0 + fs) * 64 + q * 16);
-                            const int8_t *xp = xseg + fs * 64;
-                            if constexpr (kDotM > 0) {
-#pragma unroll
-                                for (int m = 0; m < kDotM; ++m) {
-                                    const uint4 x = *reinterpret_cast<const uint4 *>(xp + m * L.pitch);
-                                    acca[m] = __dp4a((int)w.x, (int)(x.x & mk.x), acca[m]);
-                                    acca[m] = __dp4a((int)w.y, (int)(x.y & mk.y), acca[m]);
-                                    acca[m] = __dp4a((int)w.z, (int)(x.z & mk.z), acca[m]);
-                                    acca[m] = __dp4a((int)w.w, (int)(x.w & mk.w), acca[m]);
+                                            for (int m = 0; m < kDotM; ++m) acca[m] += w * (int)xseg[m * L.pitch + kk];
+                                        }
+                                    }
+                                } else {
+                                    // lane (g, q): token rows g, g + 8; output channels 8u + 2q, 8u + 2q + 1; every entry
+                                    for (int o = 0; o < r; ++o) {
+                                        const int kk = (int)chlist[o] - k0;
+                                        if ((unsigned)kk < (unsigned)seg) {
+                                            const int w0 = (int)(int8_t)wst[(2 * q) * seg + kk], w1 = (int)(int8_t)wst[(2 * q + 1) * seg + kk];
+                                            const int x0 = (int)xseg[g * L.pitch + kk];
+                                            const int x1 = MT == 16 ? (int)xseg[(g + 8) * L.pitch + kk] : 0;
+                                            acca[0] += w0 * x0;
+                                            acca[1] += w1 * x0;
+                                            acca[2] += w0 * x1;
+                                            acca[3] += w1 * x1;
+                                        }
+                                    }
                                 }
                             } else {
-                                const uint4 alo = *reinterpret_cast<const uint4 *>(xp + g * L.pitch);
-                                uint4 ahi = make_uint4(0u, 0u, 0u, 0u);
-                                if (MT == 16) ahi = *reinterpret_cast<const uint4 *>(xp + (g + 8) * L.pitch);
-                                mma_s8(acca, alo.x & mk.x, ahi.x & mk.x, alo.y & mk.y, ahi.y & mk.y, w.x, w.y);
-                                mma_s8(acca, alo.z & mk.z, ahi.z & mk.z, alo.w & mk.w, ahi.w & mk.w, w.z, w.w);
+                                // many outlier channels: per flagged 64-byte segment, the same products as for Body with X
+                                // masked to the outlier channels
+                                const int seg0 = st * segs;
+                                for (int j = 0; j < nflag; ++j) {
+                                    const int fs = (int)flaglist[j] - seg0;
+                                    if (fs < 0 || fs >= segs) continue;  // warp-uniform
+                                    const int o = fs * 64 + q * 16;
+                                    const uint4 w = *reinterpret_cast<const uint4 *>(wrow + o);
+                                    const uint4 mk = *reinterpret_cast<const uint4 *>(s_mask + k0 + o);
+                                    if constexpr (kDotM > 0) {
+#pragma unroll
+                                        for (int m = 0; m < kDotM; ++m) {
+                                            const uint4 x = *reinterpret_cast<const uint4 *>(xseg + m * L.pitch + o);
+                                            acca[m] = __dp4a((int)w.x, (int)(x.x & mk.x), acca[m]);
+                                            acca[m] = __dp4a((int)w.y, (int)(x.y & mk.y), acca[m]);
+                                            acca[m] = __dp4a((int)w.z, (int)(x.z & mk.z), acca[m]);
+                                            acca[m] = __dp4a((int)w.w, (int)(x.w & mk.w), acca[m]);
+                                        }
+                                    } else {
+                                        const uint4 alo = *reinterpret_cast<const uint4 *>(xseg + g * L.pitch + o);
+                                        uint4 ahi = make_uint4(0u, 0u, 0u, 0u);
+                                        if (MT == 16) ahi = *reinterpret_cast<const uint4 *>(xseg + (g + 8) * L.pitch + o);
+                                        mma_s8(acca, alo.x & mk.x, ahi.x & mk.x, alo.y & mk.y, ahi.y & mk.y, w.x, w.y);
+                                        mma_s8(acca, alo.z & mk.z, ahi.z & mk.z, alo.w & mk.w, ahi.w & mk.w, w.z, w.w);
+                                    }
+                                }
                             }
                         }
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(&bar_empty[pos.slot]);  // the stage may be fetched into again
+                        pos.advance(1, S);
                     }
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(&bar_empty[pos.slot]);  // the stage may be fetched into again
-                    pos.advance(1, S);
-                }
-                if (!got || skip) continue;
-                // acc = acc_b + c * acc_a (Eq. 7), dequantization (Eq. 3), store
-                auto emit = [&](int m, int n, int acc) {
-                    if (m >= M) return;
-                    const size_t o = (size_t)m * ly.ldy + n;
-                    if (a.out_kind == 2) {
-                        reinterpret_cast<int32_t *>(ly.Y)[o] = acc;
+                    if (!got || skip) continue;
+                    // acc = acc_b + c * acc_a (Eq. 7), dequantization (Eq. 3), store
+                    auto emit = [&](int m, int n, int acc) {
+                        if (m >= M) return;
+                        const size_t o = (size_t)m * ly.ldy + n;
+                        if (a.out_kind == 2) {
+                            reinterpret_cast<int32_t *>(ly.Y)[o] = acc;
+                        } else {
+                            const float sx = hdr->rowscale[a.per_vec ? m : 0];
+                            const float sw = a.per_vec ? __ldg(ly.s_w + n) : sw0;
+                            const float y = __fmul_rn(__fmul_rn(sx, sw), __int2float_rn(acc));
+                            if (a.out_kind == 1) reinterpret_cast<float *>(ly.Y)[o] = y;
+                            else reinterpret_cast<__half *>(ly.Y)[o] = __float2half_rn(y);
+                        }
+                    };
+                    if constexpr (kDotM > 0) {
+                        // the four lanes of a W_q row add up; lane q == 0 of row g holds output channel 8u + g
+#pragma unroll
+                        for (int m = 0; m < kDotM; ++m) {
+                            int v = a.c * acca[m];
+#pragma unroll
+                            for (int j = 0; j < kAcc; ++j) v += accb[j][m];
+                            v += __shfl_xor_sync(0xffffffffu, v, 1);
+                            v += __shfl_xor_sync(0xffffffffu, v, 2);
+                            if (q == 0) emit(m, u * 8 + g, v);
+                        }
                     } else {
-                        const float sx = hdr->rowscale[a.per_vec ? m : 0];
-                        const float sw = a.per_vec ? __ldg(ly.s_w + n) : sw0;
-                        const float y = __fmul_rn(__fmul_rn(sx, sw), __int2float_rn(acc));
-                        if (a.out_kind == 1) reinterpret_cast<float *>(ly.Y)[o] = y;
-                        else reinterpret_cast<__half *>(ly.Y)[o] = __float2half_rn(y);
+                        // this lane holds token rows g and g + 8, output channels 8u + 2q and 8u + 2q + 1
+                        emit(g, u * 8 + 2 * q, accb[0][0] + accb[1][0] + a.c * acca[0]);
+                        emit(g, u * 8 + 2 * q + 1, accb[0][1] + accb[1][1] + a.c * acca[1]);
+                        emit(g + 8, u * 8 + 2 * q, accb[0][2] + accb[1][2] + a.c * acca[2]);
+                        emit(g + 8, u * 8 + 2 * q + 1, accb[0][3] + accb[1][3] + a.c * acca[3]);
                     }
-                };
-                if constexpr (kDotM > 0) {
-                    // the four lanes of a W_q row add up; lane q == 0 of row g holds output channel 8u + g
-#pragma unroll
-                    for (int m = 0; m < kDotM; ++m) {
-                        int v = accb[m] + accb2[m] + a.c * acca[m];
-                        v += __shfl_xor_sync(0xffffffffu, v, 1);
-                        v += __shfl_xor_sync(0xffffffffu, v, 2);
-                        if (q == 0) emit(m, u * 8 + g, v);
-                    }
-                } else {
-                    // this lane holds token rows g and g + 8, output channels 8u + 2q and 8u + 2q + 1
-                    emit(g, u * 8 + 2 * q, accb[0] + accb2[0] + a.c * acca[0]);
-                    emit(g, u * 8 + 2 * q + 1, accb[1] + accb2[1] + a.c * acca[1]);
-                    emit(g + 8, u * 8 + 2 * q, accb[2] + accb2[2] + a.c * acca[2]);
-                    emit(g + 8, u * 8 + 2 * q + 1, accb[3] + accb2[3] + a.c * acca[3]);
                 }
             }
-            ucount += cnt;
+            ucount = (ucount + cnt) & (kUW - 1);
             lseq += cnt * nst;
             // this warp is done with the layer's buffer (and has made its stores).  When the next layer reads these
             // stores, the last unit warp of the CTA to get here counts the CTA in (each warp's stores are ordered
