@@ -55,7 +55,7 @@ constexpr int kMaxBufs = 8;             // buffers of prepared X per CTA
 constexpr int kMaxSlots = 24;
 constexpr int kStatusCapacity = 5;      // MUXQ_ERR_CAPACITY
 constexpr int kStatusTimeout = 6;       // MUXQ_ERR_TIMEOUT
-constexpr int kMaxSmem = 227 * 1024 - 1024;
+constexpr int kMaxSmem = 227 * 1024 - 3072;  // dynamic part; the static arrays take about 2.5 KB
 
 __device__ __forceinline__ void mma_s8(int (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
                                        uint32_t b1) {
@@ -90,6 +90,9 @@ __device__ __forceinline__ bool wait_sleep(uint64_t *bar, uint32_t parity, volat
     return false;
 }
 
+__device__ __forceinline__ void mbar_arrive_n(uint64_t *bar, uint32_t n) {  // n arrivals at once
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(n) : "memory");
+}
 __device__ __forceinline__ uint32_t ld_acquire_u32(const uint32_t *p) {
     uint32_t v;
     asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
@@ -193,6 +196,11 @@ __global__ void __launch_bounds__(kThreads, 1) k_decode_stream(const ChainArgs a
     __shared__ uint32_t s_abort;
     __shared__ volatile uint32_t s_begun[kMaxSlots];  // uses of a slot the loaders have begun to fill so far
     __shared__ uint32_t s_unitdone[kMaxBufs];         // unit warps that have stored their part of the buffer's layer
+    __shared__ volatile uint32_t s_fetched[kMaxBufs]; // fetches into a buffer begun so far
+    // per layer, for this CTA: its units, the number of its units before the layer modulo kUW, its stages before the layer
+    __shared__ uint16_t s_cnt[kChainMaxLayers];
+    __shared__ uint8_t s_uc[kChainMaxLayers];
+    __shared__ uint32_t s_lseq[kChainMaxLayers];
 
     const int t = threadIdx.x, lane = t & 31;
     const int warp = __shfl_sync(0xffffffffu, t >> 5, 0);  // warp-uniform by construction
@@ -226,6 +234,7 @@ __global__ void __launch_bounds__(kThreads, 1) k_decode_stream(const ChainArgs a
             mbar_init(&bar_ready[b], 1);   // the fetch warp's arrival that announces the bytes; the copies report them
             mbar_init(&bar_free[b], kUW);  // every unit warp, once per layer
             s_unitdone[b] = 0u;
+            s_fetched[b] = 0u;
         }
         s_abort = 0u;
         fence_barrier_init();
@@ -238,6 +247,36 @@ __global__ void __launch_bounds__(kThreads, 1) k_decode_stream(const ChainArgs a
         if (f < 0) f += grid;
         return f;
     };
+    // How many there are per layer, and the running counts in front of every layer: the warps that have nothing to
+    // do in a layer pass it by with two loads.
+    for (int l = t; l < a.n_layers; l += kThreads) {
+        const ChainLayer &ly = tab[l];
+        const int units = ly.N >> 3, first = first_unit(ly);
+        const int cnt = first < units ? (units - first + grid - 1) / grid : 0;
+        s_cnt[l] = (uint16_t)cnt;
+        s_lseq[l] = (uint32_t)(cnt * (ly.K / (int)ly.seg));
+    }
+    __syncthreads();
+    if (warp == 0) {
+        uint32_t carry_u = 0, carry_s = 0;
+        for (int base = 0; base < a.n_layers; base += 32) {
+            const int l = base + lane;
+            const uint32_t c = l < a.n_layers ? s_cnt[l] : 0u, st = l < a.n_layers ? s_lseq[l] : 0u;
+            uint32_t pc = c, ps = st;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const uint32_t nc = __shfl_up_sync(0xffffffffu, pc, o), nsx = __shfl_up_sync(0xffffffffu, ps, o);
+                if (lane >= o) { pc += nc; ps += nsx; }
+            }
+            if (l < a.n_layers) {
+                s_uc[l] = (uint8_t)((carry_u + pc - c) & (kUW - 1));
+                s_lseq[l] = carry_s + ps - st;
+            }
+            carry_u += __shfl_sync(0xffffffffu, pc, 31);
+            carry_s += __shfl_sync(0xffffffffu, ps, 31);
+        }
+    }
+    __syncthreads();
 
     if (warp >= kLoader0) {
         // ------------------------------------------------------------ loaders: W_q of every layer, in order.
@@ -248,13 +287,14 @@ __global__ void __launch_bounds__(kThreads, 1) k_decode_stream(const ChainArgs a
         // A stage is 8 rows of `seg` bytes, stored row after row: one copy when the rows are contiguous in W_q
         // (seg == K == ldw), else one copy per row, issued by 8 lanes.
         const int wl = warp - kLoader0, LG = a.lgroups;
-        uint32_t lseq = 0;  // number of this CTA's stages before the current layer
         bool ok = wl < LG;
         for (int l = 0; l < a.n_layers && ok; ++l) {
+            const int cnt = (int)s_cnt[l];
+            if (cnt == 0) continue;
+            const uint32_t lseq = s_lseq[l];  // number of this CTA's stages before the layer
             const ChainLayer ly = tab[l];
-            const int seg = (int)ly.seg, units = ly.N >> 3, nst = ly.K / seg;
+            const int seg = (int)ly.seg, nst = ly.K / seg;
             const int first = first_unit(ly);
-            const int cnt = first < units ? (units - first + grid - 1) / grid : 0;
             const uint32_t nstage = (uint32_t)(cnt * nst);
             const bool flat = seg == ly.ldw;
             uint32_t j = (uint32_t)(wl + LG - (int)(lseq % (uint32_t)LG)) % (uint32_t)LG;  // first stage of the layer that is this warp's
@@ -282,7 +322,6 @@ __global__ void __launch_bounds__(kThreads, 1) k_decode_stream(const ChainArgs a
                 st += LG;
                 while (st >= nst) { st -= nst; ++i; }
             }
-            lseq += nstage;
         }
         // This warp leaves only when the copies it has issued have landed (they all have when the list was walked
         // to its end, since a unit warp has waited for each; after a time-out some may still be on their way).
@@ -308,8 +347,11 @@ __global__ void __launch_bounds__(kThreads, 1) k_decode_stream(const ChainArgs a
             const uint8_t *g_codes = g_head + kHeadBlock;
             const uint8_t *g_mask = g_codes + scratch_codes_bytes(M, K);
             scr += scratch_layer_bytes(M, K);
-            // the buffer was last read for layer l - NB
-            if (l >= NB && !wait_sleep(&bar_free[b], (uint32_t)(ph - 1) & 1u, abort_flag, a.spin)) break;
+            // the buffer was last read for layer l - NB; that layer's copies have landed (if no unit warp had a unit
+            // in it, nobody has waited for them yet)
+            if (l >= NB && !(wait_sleep(&bar_free[b], (uint32_t)(ph - 1) & 1u, abort_flag, a.spin) &&
+                             wait_sleep(&bar_ready[b], (uint32_t)(ph - 1) & 1u, abort_flag, a.spin)))
+                break;
             if (l >= ready_upto) {
                 // lane i looks at layer l + i: in a list of independent layers most are ready long before their turn
                 bool ok = false, stopped = false;
@@ -337,11 +379,18 @@ __global__ void __launch_bounds__(kThreads, 1) k_decode_stream(const ChainArgs a
                 // acquire, are ordered before the copy engine reads them
                 fence_proxy_async_all();
             }
-            if (lane == 0) mbar_expect_tx(&bar_ready[b], (uint32_t)(kHeadBlock + M * K + K));
+            if (lane == 0) {
+                s_fetched[b] = (uint32_t)ph + 1u;  // the barrier is in this layer's phase: it may be waited on
+                mbar_expect_tx(&bar_ready[b], (uint32_t)(kHeadBlock + M * K + K));
+            }
             __syncwarp();
             if (lane < M) bulk_load(buf + L.off_xq + (size_t)lane * L.pitch, g_codes + (size_t)lane * K, (uint32_t)K, &bar_ready[b]);
             if (lane == 30) bulk_load(buf, g_head, (uint32_t)kHeadBlock, &bar_ready[b]);
             if (lane == 31) bulk_load(buf + L.off_mask, g_mask, (uint32_t)K, &bar_ready[b]);
+            // the unit warps without a unit in this layer pass it by: their arrivals on the buffer's barrier are made here
+            // (the barrier is in this layer's phase: the one before was waited for above)
+            const int idle = kUW - min((int)s_cnt[l], kUW);
+            if (lane == 0 && idle > 0) mbar_arrive_n(&bar_free[b], (uint32_t)idle);
             last_buf = b; last_phase = (uint32_t)ph & 1u;
         }
         // the copies of the last layer fetched have landed before this warp leaves (see the loaders)
@@ -369,8 +418,10 @@ __global__ void __launch_bounds__(kThreads, 1) k_decode_stream(const ChainArgs a
             int s = myw - (int)ly.slice_off;
             if (s < 0) s += NW;
             if (s >= ns) continue;
-            // X of this layer is Y of the layer before it: every CTA must have stored its part
-            if ((ly.flags & kChainWaitPrev) && !wait_count(&sync[l - 1].stored, (uint32_t)grid, abort_flag, g_abort, a.spin)) break;
+            // X of this layer is Y of the layer before it: every CTA that has units of it must have stored its part
+            if ((ly.flags & kChainWaitPrev) &&
+                !wait_count(&sync[l - 1].stored, (uint32_t)min(tab[l - 1].N >> 3, grid), abort_flag, g_abort, a.spin))
+                break;
             const int ch = s * 64 + cg * 8;
             uint4 v[4];
 #pragma unroll
@@ -560,14 +611,16 @@ __global__ void __launch_bounds__(kThreads, 1) k_decode_stream(const ChainArgs a
     } else {
         // ------------------------------------------------------------ unit warps: the products of layer l
         const int g = lane >> 2, q = lane & 3;
-        int lseq = 0;    // number of this CTA's stages before the current layer
-        int ucount = 0;  // units of this CTA before the current layer, modulo kUW
         // M <= 4: lane (g, q) reads 16 bytes of W_q row 8u + g per 64-byte segment and the matching 16 bytes of the
         // codes of X.  Segments are taken in pairs, rows with odd g second segment first, so that the eight lanes
         // that shared memory serves together touch all 32 banks (a row is a multiple of 128 bytes long); the K order
         // is permuted the same way for both operands, which a dot product does not notice.
         const int oa = (g & 1) * 64 + q * 16, ob = (1 - (g & 1)) * 64 + q * 16;
         for (int l = 0; l < a.n_layers; ++l) {
+            const int cnt = (int)s_cnt[l];
+            const int i0 = (warp - (int)s_uc[l]) & (kUW - 1);  // unit number ucount + i of the CTA goes to warp (ucount + i) mod kUW
+            if (i0 >= cnt) continue;                             // nothing for this warp in this layer
+            const int lseq = (int)s_lseq[l];                     // number of this CTA's stages before the layer
             const ChainLayer ly = tab[l];
             const int K = ly.K, b = l % NB, ph = l / NB;
             const uint8_t *buf = xbase + b * L.buf_bytes;
@@ -576,12 +629,22 @@ __global__ void __launch_bounds__(kThreads, 1) k_decode_stream(const ChainArgs a
             const uint8_t *s_mask = buf + L.off_mask;
             const uint16_t *flaglist = reinterpret_cast<const uint16_t *>(buf + L.off_flaglist);
             const uint16_t *chlist = reinterpret_cast<const uint16_t *>(buf + L.off_chlist);
-            const int seg = (int)ly.seg, units = ly.N >> 3, nst = K / seg, segs = seg >> 6;
+            const int seg = (int)ly.seg, nst = K / seg, segs = seg >> 6;
             const int first = first_unit(ly);
-            const int cnt = first < units ? (units - first + grid - 1) / grid : 0;
-            const int i0 = (warp - ucount) & (kUW - 1);  // unit number ucount + i goes to warp (ucount + i) mod kUW
+            // (a warp that has passed layers by must not take an older phase of the barrier for this one)
+            {
+                uint32_t spins = 0;
+                while (s_fetched[b] <= (uint32_t)ph && ++spins < a.spin) {
+                    __nanosleep(100);
+                    if ((spins & 15u) == 15u && *abort_flag) break;
+                }
+                if (!__all_sync(0xffffffffu, s_fetched[b] > (uint32_t)ph)) {
+                    *abort_flag = 1u;
+                    break;
+                }
+            }
             if (!wait_sleep(&bar_ready[b], (uint32_t)ph & 1u, abort_flag, a.spin)) break;
-            if (i0 < cnt) {
+            {
                 const float sw0 = a.per_vec ? 0.0f : __ldg(ly.s_w);
                 const int r = hdr->r, nflag = hdr->nflag;
                 const bool skip = r > a.cap;     // MUXQ_ERR_CAPACITY: Y of this layer is unspecified; its weights still drain
@@ -782,22 +845,21 @@ __global__ void __launch_bounds__(kThreads, 1) k_decode_stream(const ChainArgs a
                     }
                 }
             }
-            ucount = (ucount + cnt) & (kUW - 1);
-            lseq += cnt * nst;
             // this warp is done with the layer's buffer (and has made its stores).  When the next layer reads these
-            // stores, the last unit warp of the CTA to get here counts the CTA in (each warp's stores are ordered
-            // before its own count by a fence, and all of them before the CTA's by the last warp's).
+            // stores, the last of the CTA's unit warps with a unit in this layer to get here counts the CTA in (each
+            // warp's stores are ordered before its own count by a fence, and all of them before the CTA's by the last
+            // warp's).
             __syncwarp();
             if (lane == 0) {
                 if (l + 1 < a.n_layers && (tab[l + 1].flags & kChainWaitPrev)) {
                     __threadfence();
-                    if (atomicAdd(&s_unitdone[b], 1u) == (uint32_t)(kUW - 1)) {
+                    if (atomicAdd(&s_unitdone[b], 1u) == (uint32_t)(min(cnt, kUW) - 1)) {
                         s_unitdone[b] = 0u;
                         __threadfence();
                         atomicAdd(&sync[l].stored, 1u);
                     }
                 }
-                mbar_arrive(&bar_free[b]);  // one of the kUW arrivals
+                mbar_arrive(&bar_free[b]);  // one of the kUW arrivals (the fetch warp has made those of the warps without a unit)
             }
             if (*abort_flag) break;
         }
