@@ -22,7 +22,7 @@
 //                   that hold an outlier channel) and raises the layer's ready word.
 //                   Every CTA used to do all of this for itself, which cost more than the weight stream.
 //   fetch warp      per layer, in order: once the layer is ready (one poll looks 32 layers ahead) and one of the
-//                   CTA's buffers in shared memory is free, has the copy engine bring header, codes and mask there.
+//                   CTA's buffers in shared memory is free, has the copy engine bring header and codes there.
 //   unit warps      per layer: each unit is taken by ONE warp, which accumulates the unit's 8 x M outputs over all
 //                   of K in registers (4-way byte dot products for M <= 4, mma.sync m16n8k32 above), adds the Aux
 //                   term of Eq. 7 for the 64-byte segments that hold an outlier channel, dequantizes and stores.
@@ -55,7 +55,7 @@ constexpr int kMaxBufs = 8;             // buffers of prepared X per CTA
 constexpr int kMaxSlots = 24;
 constexpr int kStatusCapacity = 5;      // MUXQ_ERR_CAPACITY
 constexpr int kStatusTimeout = 6;       // MUXQ_ERR_TIMEOUT
-constexpr int kMaxSmem = 227 * 1024 - 3072;  // dynamic part; the static arrays take about 2.5 KB
+constexpr int kMaxSmem = 227 * 1024 - 4096;  // dynamic part; the static arrays take about 3.6 KB
 
 __device__ __forceinline__ void mma_s8(int (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
                                        uint32_t b1) {
@@ -150,13 +150,13 @@ __host__ __device__ inline size_t scratch_layer_bytes(int M, int K) {
     return (size_t)kHeadBlock + scratch_codes_bytes(M, K) + (size_t)K + (size_t)(((K >> 6) + 127) & ~127);
 }
 
-// A buffer in shared memory that holds a layer's prepared X (sized for the widest K of the list).
+// A buffer in shared memory that holds a layer's prepared X (sized for the widest K of the list).  The outlier
+// mask stays in global memory: only a layer with more than kChList outlier channels reads it.
 struct XLayout {
     int pitch;          // bytes per row of X codes; pitch % 128 == 64 keeps the 8-row x 64-byte reads conflict free
     int off_flaglist;   // [K/64] u16 behind the 128-byte header: the segments that hold an outlier channel, ascending
     int off_chlist;     // [kChList] u16: outlier channels (all of them when r <= kChList)
     int off_xq;         // [rows][pitch] INT8 codes
-    int off_mask;       // [K] 0xFF at outlier channels
     int buf_bytes;
 };
 __host__ __device__ inline XLayout x_layout(int rows, int K) {
@@ -166,8 +166,7 @@ __host__ __device__ inline XLayout x_layout(int rows, int K) {
     s.off_flaglist = kHeaderBytes;
     s.off_chlist = kHeaderBytes + kFlagListBytes;
     s.off_xq = kHeadBlock;
-    s.off_mask = s.off_xq + rows * s.pitch;
-    s.buf_bytes = (s.off_mask + K + 127) & ~127;
+    s.buf_bytes = (s.off_xq + rows * s.pitch + 127) & ~127;
     return s;
 }
 struct XHeader {        // first bytes of a buffer and of a layer's scratch area
@@ -201,6 +200,7 @@ __global__ void __launch_bounds__(kThreads, 1) k_decode_stream(const ChainArgs a
     __shared__ uint16_t s_cnt[kChainMaxLayers];
     __shared__ uint8_t s_uc[kChainMaxLayers];
     __shared__ uint32_t s_lseq[kChainMaxLayers];
+    __shared__ uint32_t s_scr[kChainMaxLayers];       // offset of the layer's scratch area
 
     const int t = threadIdx.x, lane = t & 31;
     const int warp = __shfl_sync(0xffffffffu, t >> 5, 0);  // warp-uniform by construction
@@ -255,25 +255,30 @@ __global__ void __launch_bounds__(kThreads, 1) k_decode_stream(const ChainArgs a
         const int cnt = first < units ? (units - first + grid - 1) / grid : 0;
         s_cnt[l] = (uint16_t)cnt;
         s_lseq[l] = (uint32_t)(cnt * (ly.K / (int)ly.seg));
+        s_scr[l] = (uint32_t)scratch_layer_bytes(M, ly.K);
     }
     __syncthreads();
     if (warp == 0) {
-        uint32_t carry_u = 0, carry_s = 0;
+        uint32_t carry_u = 0, carry_s = 0, carry_b = 0;
         for (int base = 0; base < a.n_layers; base += 32) {
             const int l = base + lane;
-            const uint32_t c = l < a.n_layers ? s_cnt[l] : 0u, st = l < a.n_layers ? s_lseq[l] : 0u;
-            uint32_t pc = c, ps = st;
+            const bool in = l < a.n_layers;
+            const uint32_t c = in ? s_cnt[l] : 0u, st = in ? s_lseq[l] : 0u, sb = in ? s_scr[l] : 0u;
+            uint32_t pc = c, ps = st, pb = sb;
 #pragma unroll
             for (int o = 1; o < 32; o <<= 1) {
                 const uint32_t nc = __shfl_up_sync(0xffffffffu, pc, o), nsx = __shfl_up_sync(0xffffffffu, ps, o);
-                if (lane >= o) { pc += nc; ps += nsx; }
+                const uint32_t nb = __shfl_up_sync(0xffffffffu, pb, o);
+                if (lane >= o) { pc += nc; ps += nsx; pb += nb; }
             }
-            if (l < a.n_layers) {
+            if (in) {
                 s_uc[l] = (uint8_t)((carry_u + pc - c) & (kUW - 1));
                 s_lseq[l] = carry_s + ps - st;
+                s_scr[l] = carry_b + pb - sb;
             }
             carry_u += __shfl_sync(0xffffffffu, pc, 31);
             carry_s += __shfl_sync(0xffffffffu, ps, 31);
+            carry_b += __shfl_sync(0xffffffffu, pb, 31);
         }
     }
     __syncthreads();
@@ -345,7 +350,6 @@ __global__ void __launch_bounds__(kThreads, 1) k_decode_stream(const ChainArgs a
             uint8_t *buf = xbase + b * L.buf_bytes;
             const uint8_t *g_head = a.scratch + scr;
             const uint8_t *g_codes = g_head + kHeadBlock;
-            const uint8_t *g_mask = g_codes + scratch_codes_bytes(M, K);
             scr += scratch_layer_bytes(M, K);
             // the buffer was last read for layer l - NB; that layer's copies have landed (if no unit warp had a unit
             // in it, nobody has waited for them yet)
@@ -381,12 +385,11 @@ __global__ void __launch_bounds__(kThreads, 1) k_decode_stream(const ChainArgs a
             }
             if (lane == 0) {
                 s_fetched[b] = (uint32_t)ph + 1u;  // the barrier is in this layer's phase: it may be waited on
-                mbar_expect_tx(&bar_ready[b], (uint32_t)(kHeadBlock + M * K + K));
+                mbar_expect_tx(&bar_ready[b], (uint32_t)(kHeadBlock + M * K));
             }
             __syncwarp();
             if (lane < M) bulk_load(buf + L.off_xq + (size_t)lane * L.pitch, g_codes + (size_t)lane * K, (uint32_t)K, &bar_ready[b]);
             if (lane == 30) bulk_load(buf, g_head, (uint32_t)kHeadBlock, &bar_ready[b]);
-            if (lane == 31) bulk_load(buf + L.off_mask, g_mask, (uint32_t)K, &bar_ready[b]);
             // the unit warps without a unit in this layer pass it by: their arrivals on the buffer's barrier are made here
             // (the barrier is in this layer's phase: the one before was waited for above)
             const int idle = kUW - min((int)s_cnt[l], kUW);
@@ -626,7 +629,8 @@ __global__ void __launch_bounds__(kThreads, 1) k_decode_stream(const ChainArgs a
             const uint8_t *buf = xbase + b * L.buf_bytes;
             const XHeader *hdr = reinterpret_cast<const XHeader *>(buf);
             const int8_t *xq = reinterpret_cast<const int8_t *>(buf + L.off_xq);
-            const uint8_t *s_mask = buf + L.off_mask;
+            // (written in this launch by other SMs: read through L2; visible by way of the ready word and the buffer's barrier)
+            const uint8_t *g_mask = a.scratch + s_scr[l] + kHeadBlock + scratch_codes_bytes(M, ly.K);
             const uint16_t *flaglist = reinterpret_cast<const uint16_t *>(buf + L.off_flaglist);
             const uint16_t *chlist = reinterpret_cast<const uint16_t *>(buf + L.off_chlist);
             const int seg = (int)ly.seg, nst = K / seg, segs = seg >> 6;
@@ -645,7 +649,7 @@ __global__ void __launch_bounds__(kThreads, 1) k_decode_stream(const ChainArgs a
             }
             if (!wait_sleep(&bar_ready[b], (uint32_t)ph & 1u, abort_flag, a.spin)) break;
             {
-                const float sw0 = a.per_vec ? 0.0f : __ldg(ly.s_w);
+                const float ssw0 = a.per_vec ? 0.0f : __fmul_rn(hdr->rowscale[0], __ldg(ly.s_w));  // s_X * s_W (Eq. 3)
                 const int r = hdr->r, nflag = hdr->nflag;
                 const bool skip = r > a.cap;     // MUXQ_ERR_CAPACITY: Y of this layer is unspecified; its weights still drain
                 const bool listed = r <= kChList;  // every outlier channel is in the list
@@ -752,28 +756,47 @@ __global__ void __launch_bounds__(kThreads, 1) k_decode_stream(const ChainArgs a
                             // ... then the Aux term (Eq. 7) over the outlier channels that fall into this stage
                             if (listed) {
                                 // from the channel list: single products W_q[n][k] * X_q[m][k]
+                                // (entries in groups of four: the loads of a group do not depend on each other; an entry
+                                // outside this stage or past the end of the list reads offset 0 and counts as zero)
                                 if constexpr (kDotM > 0) {
-                                    // lane (g, q): output channel 8u + g, every fourth list entry (the four lanes add up below)
-                                    for (int o = q; o < r; o += 4) {
-                                        const int kk = (int)chlist[o] - k0;
-                                        if ((unsigned)kk < (unsigned)seg) {
-                                            const int w = (int)(int8_t)wrow[kk];
+                                    // lane (g, q): output channel 8u + g, entries q, q + 4, ... (the four lanes add up below)
+                                    for (int o0 = 0; o0 < r; o0 += 16) {
+                                        int kk[4], w[4];
 #pragma unroll
-                                            for (int m = 0; m < kDotM; ++m) acca[m] += w * (int)xseg[m * L.pitch + kk];
+                                        for (int j = 0; j < 4; ++j) {
+                                            const int o = o0 + 4 * j + q;
+                                            const int k = (int)chlist[o < kChList ? o : 0] - k0;
+                                            const bool in = o < r && (unsigned)k < (unsigned)seg;
+                                            kk[j] = in ? k : 0;
+                                            w[j] = in ? (int)(int8_t)wrow[kk[j]] : 0;
                                         }
+#pragma unroll
+                                        for (int j = 0; j < 4; ++j)
+#pragma unroll
+                                            for (int m = 0; m < kDotM; ++m) acca[m] += w[j] * (int)xseg[m * L.pitch + kk[j]];
                                     }
                                 } else {
                                     // lane (g, q): token rows g, g + 8; output channels 8u + 2q, 8u + 2q + 1; every entry
-                                    for (int o = 0; o < r; ++o) {
-                                        const int kk = (int)chlist[o] - k0;
-                                        if ((unsigned)kk < (unsigned)seg) {
-                                            const int w0 = (int)(int8_t)wst[(2 * q) * seg + kk], w1 = (int)(int8_t)wst[(2 * q + 1) * seg + kk];
-                                            const int x0 = (int)xseg[g * L.pitch + kk];
-                                            const int x1 = MT == 16 ? (int)xseg[(g + 8) * L.pitch + kk] : 0;
-                                            acca[0] += w0 * x0;
-                                            acca[1] += w1 * x0;
-                                            acca[2] += w0 * x1;
-                                            acca[3] += w1 * x1;
+                                    for (int o0 = 0; o0 < r; o0 += 4) {
+                                        const uint2 c4 = *reinterpret_cast<const uint2 *>(chlist + o0);
+                                        const int ch[4] = {(int)(c4.x & 0xFFFFu), (int)(c4.x >> 16), (int)(c4.y & 0xFFFFu), (int)(c4.y >> 16)};
+                                        int kk[4], w0[4], w1[4];
+#pragma unroll
+                                        for (int j = 0; j < 4; ++j) {
+                                            const int k = ch[j] - k0;
+                                            const bool in = o0 + j < r && (unsigned)k < (unsigned)seg;
+                                            kk[j] = in ? k : 0;
+                                            w0[j] = in ? (int)(int8_t)wst[(2 * q) * seg + kk[j]] : 0;
+                                            w1[j] = in ? (int)(int8_t)wst[(2 * q + 1) * seg + kk[j]] : 0;
+                                        }
+#pragma unroll
+                                        for (int j = 0; j < 4; ++j) {
+                                            const int x0 = (int)xseg[g * L.pitch + kk[j]];
+                                            const int x1 = MT == 16 ? (int)xseg[(g + 8) * L.pitch + kk[j]] : 0;
+                                            acca[0] += w0[j] * x0;
+                                            acca[1] += w1[j] * x0;
+                                            acca[2] += w0[j] * x1;
+                                            acca[3] += w1[j] * x1;
                                         }
                                     }
                                 }
@@ -786,7 +809,7 @@ __global__ void __launch_bounds__(kThreads, 1) k_decode_stream(const ChainArgs a
                                     if (fs < 0 || fs >= segs) continue;  // warp-uniform
                                     const int o = fs * 64 + q * 16;
                                     const uint4 w = *reinterpret_cast<const uint4 *>(wrow + o);
-                                    const uint4 mk = *reinterpret_cast<const uint4 *>(s_mask + k0 + o);
+                                    const uint4 mk = __ldcg(reinterpret_cast<const uint4 *>(g_mask + k0 + o));
                                     if constexpr (kDotM > 0) {
 #pragma unroll
                                         for (int m = 0; m < kDotM; ++m) {
@@ -818,9 +841,8 @@ __global__ void __launch_bounds__(kThreads, 1) k_decode_stream(const ChainArgs a
                         if (a.out_kind == 2) {
                             reinterpret_cast<int32_t *>(ly.Y)[o] = acc;
                         } else {
-                            const float sx = hdr->rowscale[a.per_vec ? m : 0];
-                            const float sw = a.per_vec ? __ldg(ly.s_w + n) : sw0;
-                            const float y = __fmul_rn(__fmul_rn(sx, sw), __int2float_rn(acc));
+                            const float ss = a.per_vec ? __fmul_rn(hdr->rowscale[m], __ldg(ly.s_w + n)) : ssw0;
+                            const float y = __fmul_rn(ss, __int2float_rn(acc));
                             if (a.out_kind == 1) reinterpret_cast<float *>(ly.Y)[o] = y;
                             else reinterpret_cast<__half *>(ly.Y)[o] = __float2half_rn(y);
                         }
@@ -922,12 +944,13 @@ cudaError_t launch_inst(ChainArgs a, cudaStream_t s) {
             attr_set.have[dev] = true;
         }
     }
-    // As many buffers of prepared X (up to kMaxBufs) as leave the ring eight stages; at least one, and then at
-    // least two stages.
+    // As many buffers of prepared X (up to kMaxBufs) as leave the ring eight stages; two if that leaves it four
+    // (while one layer's products run, the next layer's X arrives); else one, and then at least two stages.
     const XLayout L = x_layout(kRows, a.kmax);
     const int table = a.n_layers * (int)sizeof(ChainLayer);
     int nbuf = kMaxBufs;
-    while (nbuf > 1 && (kMaxSmem - table - nbuf * L.buf_bytes) / a.slot_bytes < 8) --nbuf;
+    while (nbuf > 2 && (kMaxSmem - table - nbuf * L.buf_bytes) / a.slot_bytes < 8) --nbuf;
+    if (nbuf == 2 && (kMaxSmem - table - 2 * L.buf_bytes) / a.slot_bytes < 4) nbuf = 1;
     int slots = (kMaxSmem - table - nbuf * L.buf_bytes) / a.slot_bytes;
     if (slots > kMaxSlots) slots = kMaxSlots;
     if (slots < 2) return cudaErrorInvalidValue;
