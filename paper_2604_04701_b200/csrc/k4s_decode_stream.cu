@@ -46,7 +46,7 @@ namespace {
 
 constexpr int kUW = 8;                  // unit warps (warps 0..7)
 constexpr int kFetch = kUW;             // the fetch warp
-constexpr int kSW = kChainSliceWarps;   // slice warps per CTA (warps 9..15)
+constexpr int kSW = kChainSliceWarps;   // slice warps per CTA (the warps behind the fetch warp)
 constexpr int kLW = 4;                  // loader warps (warps 16..19)
 constexpr int kLoader0 = kUW + 1 + kSW; // index of the first loader warp
 constexpr int kThreads = 32 * (kLoader0 + kLW);
@@ -661,7 +661,7 @@ __global__ void __launch_bounds__(kThreads, 1) k_decode_stream(const ChainArgs a
                     pos.use = (uint32_t)(seq0 / S);
                     // Body accumulators (several: consecutive products on one accumulator wait for each other) and the
                     // Aux accumulator over the outlier channels (Aux_q == Body_q[:, O], Eq. 5)
-                    constexpr int kAcc = kDotM == 1 ? 4 : 2;
+                    constexpr int kAcc = (kDotM == 1 || kDotM == 2) ? 4 : 2;
                     int accb[kAcc][4], acca[4] = {0, 0, 0, 0};
 #pragma unroll
                     for (int j = 0; j < kAcc; ++j) accb[j][0] = accb[j][1] = accb[j][2] = accb[j][3] = 0;
@@ -944,12 +944,14 @@ cudaError_t launch_inst(ChainArgs a, cudaStream_t s) {
             attr_set.have[dev] = true;
         }
     }
-    // As many buffers of prepared X (up to kMaxBufs) as leave the ring eight stages; two if that leaves it four
-    // (while one layer's products run, the next layer's X arrives); else one, and then at least two stages.
+    // As many buffers of prepared X (up to kMaxBufs) as leave the ring two stages per unit warp (with one, the stage
+    // a warp has just released is refilled with that very warp's next unit, and the warp sees the whole memory
+    // latency on every unit); two buffers if that leaves four stages (while one layer's products run, the next
+    // layer's X arrives); else one, and then at least two stages.
     const XLayout L = x_layout(kRows, a.kmax);
     const int table = a.n_layers * (int)sizeof(ChainLayer);
     int nbuf = kMaxBufs;
-    while (nbuf > 2 && (kMaxSmem - table - nbuf * L.buf_bytes) / a.slot_bytes < 8) --nbuf;
+    while (nbuf > 2 && (kMaxSmem - table - nbuf * L.buf_bytes) / a.slot_bytes < 2 * kUW) --nbuf;
     if (nbuf == 2 && (kMaxSmem - table - 2 * L.buf_bytes) / a.slot_bytes < 4) nbuf = 1;
     int slots = (kMaxSmem - table - nbuf * L.buf_bytes) / a.slot_bytes;
     if (slots > kMaxSlots) slots = kMaxSlots;
@@ -967,6 +969,7 @@ cudaError_t launch_inst(ChainArgs a, cudaStream_t s) {
 
 cudaError_t launch_decode_chain(const ChainArgs &a, cudaStream_t s) {
     if (a.M == 1) return launch_inst<8, 1>(a, s);
+    if (a.M == 2) return launch_inst<8, 2>(a, s);
     if (a.M <= 4) return launch_inst<8, 4>(a, s);
     if (a.M <= 8) return launch_inst<8, 0>(a, s);
     return launch_inst<16, 0>(a, s);
