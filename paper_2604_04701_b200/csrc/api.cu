@@ -501,17 +501,20 @@ struct PlanHeader {           // first 128 bytes of a plan (host and device copy
     uint32_t magic;
     int32_t n_layers, M, kmax, grid, out_kind;
     muxq_params params;
-    uint64_t sync_off, scratch_off, device_bytes;  // layout of the device copy behind the table
-    uint32_t reserved[8];
+    uint64_t sync_off, scratch_off, device_bytes;  // layout of the device copy behind the two tables
+    int32_t slots, lgroups, xregion;               // shared-memory geometry (chain_geometry)
+    uint32_t reserved[5];
 };
 static_assert(sizeof(PlanHeader) <= 128, "plan header");
 constexpr size_t kPlanTableOffset = 128;
-size_t plan_sync_offset(int n_layers) { return align_up(kPlanTableOffset + (size_t)n_layers * sizeof(ChainLayer), 128); }
+// behind the header: the layer table, then one word per layer (its place in shared memory), then counters and scratch
+size_t plan_place_offset(int n_layers) { return kPlanTableOffset + (size_t)n_layers * sizeof(ChainLayer); }
+size_t plan_sync_offset(int n_layers) { return align_up(plan_place_offset(n_layers) + (size_t)n_layers * 4, 128); }
 }  // namespace
 
 size_t muxq_chain_plan_bytes(int n_layers) {
     if (n_layers < 1 || n_layers > kChainMaxLayers) return 0;
-    return kPlanTableOffset + (size_t)n_layers * sizeof(ChainLayer);
+    return plan_sync_offset(n_layers);
 }
 
 size_t muxq_chain_device_bytes(const muxq_layer *layers, int n_layers, int M) {
@@ -561,11 +564,19 @@ int muxq_chain_build(const muxq_layer *layers, int n_layers, int M, const muxq_p
     h->scratch_off = h->sync_off + chain_sync_bytes(n_layers);
     h->device_bytes = h->scratch_off + chain_scratch_bytes(tab, n_layers, M);
     if (plan_dev_bytes < h->device_bytes) return MUXQ_ERR_WORKSPACE;
+    ChainGeometry geo{};
+    if (!chain_geometry(tab, n_layers, M, chain_slot_bytes(M), &geo,
+                        reinterpret_cast<uint32_t *>(static_cast<uint8_t *>(plan_host) + plan_place_offset(n_layers))))
+        return MUXQ_ERR_UNSUPPORTED;
+    h->slots = geo.slots; h->lgroups = geo.lgroups; h->xregion = geo.xregion;
     h->magic = kPlanMagic;
     h->n_layers = n_layers; h->M = M; h->kmax = kmax; h->grid = grid; h->out_kind = out_kind;
     h->params = *p;
-    return cuda_rc(cudaMemcpyAsync(plan_dev, plan_host, muxq_chain_plan_bytes(n_layers), cudaMemcpyHostToDevice,
-                                   static_cast<cudaStream_t>(stream)));
+    // the rows of codes beyond M in the scratch areas are read (as zero) and never written
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (cudaMemsetAsync(static_cast<uint8_t *>(plan_dev) + h->scratch_off, 0, h->device_bytes - h->scratch_off, s) != cudaSuccess)
+        return MUXQ_ERR_CUDA;
+    return cuda_rc(cudaMemcpyAsync(plan_dev, plan_host, muxq_chain_plan_bytes(n_layers), cudaMemcpyHostToDevice, s));
 }
 
 int muxq_chain_run(const void *plan_host, void *plan_dev, muxq_chain_result *results, int32_t *dev_status,
@@ -587,6 +598,8 @@ int muxq_chain_run(const void *plan_host, void *plan_dev, muxq_chain_result *res
     a.slot_bytes = chain_slot_bytes(h->M);
     a.sync = pd + h->sync_off;
     a.scratch = pd + h->scratch_off;
+    a.slots = h->slots; a.lgroups = h->lgroups; a.xregion = h->xregion;
+    a.place = reinterpret_cast<const uint32_t *>(pd + plan_place_offset(h->n_layers));
     // the per-layer counters and maxima start every run at zero
     if (cudaMemsetAsync(a.sync, 0, chain_sync_bytes(h->n_layers), s) != cudaSuccess) return MUXQ_ERR_CUDA;
     return cuda_rc(launch_decode_chain(a, s));

@@ -51,11 +51,11 @@ constexpr int kLW = 4;                  // loader warps (warps 16..19)
 constexpr int kLoader0 = kUW + 1 + kSW; // index of the first loader warp
 constexpr int kThreads = 32 * (kLoader0 + kLW);
 constexpr int kMaxK = 8192;             // widest layer: 128 slices
-constexpr int kMaxBufs = 8;             // buffers of prepared X per CTA
+constexpr int kDesc = 16;               // layers whose prepared X can be in shared memory at a time
 constexpr int kMaxSlots = 24;
 constexpr int kStatusCapacity = 5;      // MUXQ_ERR_CAPACITY
 constexpr int kStatusTimeout = 6;       // MUXQ_ERR_TIMEOUT
-constexpr int kMaxSmem = 227 * 1024 - 4096;  // dynamic part; the static arrays take about 3.6 KB
+constexpr int kMaxSmem = 227 * 1024 - 5120;  // dynamic part; the static arrays take about 4.8 KB
 
 __device__ __forceinline__ void mma_s8(int (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
                                        uint32_t b1) {
@@ -150,8 +150,10 @@ __host__ __device__ inline size_t scratch_layer_bytes(int M, int K) {
     return (size_t)kHeadBlock + scratch_codes_bytes(M, K) + (size_t)K + (size_t)(((K >> 6) + 127) & ~127);
 }
 
-// A buffer in shared memory that holds a layer's prepared X (sized for the widest K of the list).  The outlier
-// mask stays in global memory: only a layer with more than kChList outlier channels reads it.
+// A layer's prepared X in shared memory.  The outlier mask stays in global memory: only a layer with more than
+// kChList outlier channels reads it.  The layers' buffers are cut from one region like from a ring, each as large as
+// its own K needs, by the host (chain_geometry): place[l] says where layer l's buffer starts and which earlier layers
+// must have been released before it may be filled.
 struct XLayout {
     int pitch;          // bytes per row of X codes; pitch % 128 == 64 keeps the 8-row x 64-byte reads conflict free
     int off_flaglist;   // [K/64] u16 behind the 128-byte header: the segments that hold an outlier channel, ascending
@@ -191,38 +193,35 @@ __global__ void __launch_bounds__(kThreads, 1) k_decode_stream(const ChainArgs a
     constexpr int kRows = kDotM > 0 ? kDotM : MT;  // rows of codes a buffer holds
     extern __shared__ __align__(128) uint8_t smem[];
     __shared__ uint64_t bar_full[kMaxSlots], bar_empty[kMaxSlots];
-    __shared__ uint64_t bar_ready[kMaxBufs], bar_free[kMaxBufs];  // a buffer of prepared X: filled / no longer read
+    __shared__ uint64_t bar_ready[kDesc], bar_free[kDesc];  // prepared X of layer l (barriers l mod kDesc): filled / no longer read
     __shared__ uint32_t s_abort;
     __shared__ volatile uint32_t s_begun[kMaxSlots];  // uses of a slot the loaders have begun to fill so far
-    __shared__ uint32_t s_unitdone[kMaxBufs];         // unit warps that have stored their part of the buffer's layer
-    __shared__ volatile uint32_t s_fetched[kMaxBufs]; // fetches into a buffer begun so far
+    __shared__ uint32_t s_unitdone[kDesc];            // unit warps that have stored their part of the layer
+    __shared__ volatile uint32_t s_fetched[kDesc];    // fetches begun so far for the layers with these barriers
     // per layer, for this CTA: its units, the number of its units before the layer modulo kUW, its stages before the layer
     __shared__ uint16_t s_cnt[kChainMaxLayers];
     __shared__ uint8_t s_uc[kChainMaxLayers];
     __shared__ uint32_t s_lseq[kChainMaxLayers];
     __shared__ uint32_t s_scr[kChainMaxLayers];       // offset of the layer's scratch area
+    __shared__ uint32_t s_place[kChainMaxLayers];     // bits 0..15: start of the layer's buffer in 128-byte units; 16..: layers below this one released first
 
     const int t = threadIdx.x, lane = t & 31;
     const int warp = __shfl_sync(0xffffffffu, t >> 5, 0);  // warp-uniform by construction
-    const int S = a.slots, M = a.M, NB = a.nbuf;
+    const int S = a.slots, M = a.M;
     const int grid = (int)gridDim.x, cta = (int)blockIdx.x;
     uint8_t *ring = smem;
     ChainLayer *tab = reinterpret_cast<ChainLayer *>(smem + (size_t)S * a.slot_bytes);
     uint8_t *xbase = reinterpret_cast<uint8_t *>(tab + a.n_layers);
-    const XLayout L = x_layout(kRows, a.kmax);
     volatile uint32_t *abort_flag = &s_abort;
     LayerSync *sync = reinterpret_cast<LayerSync *>(a.sync);
     uint32_t *g_abort = reinterpret_cast<uint32_t *>(sync + a.n_layers);
 
-    // the layer table into shared memory (16-byte pieces), zero codes in the buffers (rows M.. of a buffer are
-    // read by the products and never written again), barriers
+    // the layer table into shared memory (16-byte pieces), barriers
     {
         const uint4 *src = reinterpret_cast<const uint4 *>(a.layers);
         uint4 *dst = reinterpret_cast<uint4 *>(tab);
         for (int i = t; i < a.n_layers * 4; i += kThreads) dst[i] = __ldg(src + i);
-        uint4 *xz = reinterpret_cast<uint4 *>(xbase);
-        for (int i = t; i < NB * (L.buf_bytes >> 4); i += kThreads) xz[i] = make_uint4(0u, 0u, 0u, 0u);
-        fence_proxy_async();  // the copy engine writes the same bytes later
+        for (int i = t; i < a.n_layers; i += kThreads) s_place[i] = __ldg(a.place + i);
     }
     if (t == 0) {
         for (int s = 0; s < S; ++s) {
@@ -230,7 +229,7 @@ __global__ void __launch_bounds__(kThreads, 1) k_decode_stream(const ChainArgs a
             mbar_init(&bar_empty[s], 1);   // the one unit warp that took the stage
             s_begun[s] = 0u;
         }
-        for (int b = 0; b < kMaxBufs; ++b) {
+        for (int b = 0; b < kDesc; ++b) {
             mbar_init(&bar_ready[b], 1);   // the fetch warp's arrival that announces the bytes; the copies report them
             mbar_init(&bar_free[b], kUW);  // every unit warp, once per layer
             s_unitdone[b] = 0u;
@@ -255,7 +254,7 @@ __global__ void __launch_bounds__(kThreads, 1) k_decode_stream(const ChainArgs a
         const int cnt = first < units ? (units - first + grid - 1) / grid : 0;
         s_cnt[l] = (uint16_t)cnt;
         s_lseq[l] = (uint32_t)(cnt * (ly.K / (int)ly.seg));
-        s_scr[l] = (uint32_t)scratch_layer_bytes(M, ly.K);
+        s_scr[l] = (uint32_t)scratch_layer_bytes(kRows, ly.K);
     }
     __syncthreads();
     if (warp == 0) {
@@ -339,23 +338,32 @@ __global__ void __launch_bounds__(kThreads, 1) k_decode_stream(const ChainArgs a
                 }
             }
     } else if (warp == kFetch) {
-        // ------------------------------------------------------------ fetch warp: prepared X of layer l into buffer l mod NB
+        // ------------------------------------------------------------ fetch warp: prepared X of layer l into its place
         size_t scr = 0;  // offset of the layer's scratch area
         int ready_upto = 0;  // layers below this one are known to be ready
+        int freed = 0;       // layers below this one have been released by the unit warps, in order
         int last_buf = -1;
         uint32_t last_phase = 0;
         for (int l = 0; l < a.n_layers; ++l) {
             const ChainLayer ly = tab[l];
-            const int K = ly.K, b = l % NB, ph = l / NB;
-            uint8_t *buf = xbase + b * L.buf_bytes;
+            const int K = ly.K, b = l % kDesc, ph = l / kDesc;
+            const XLayout L = x_layout(kRows, K);
+            const uint32_t place = s_place[l];
+            uint8_t *buf = xbase + (size_t)(place & 0xFFFFu) * 128;
             const uint8_t *g_head = a.scratch + scr;
             const uint8_t *g_codes = g_head + kHeadBlock;
-            scr += scratch_layer_bytes(M, K);
-            // the buffer was last read for layer l - NB; that layer's copies have landed (if no unit warp had a unit
-            // in it, nobody has waited for them yet)
-            if (l >= NB && !(wait_sleep(&bar_free[b], (uint32_t)(ph - 1) & 1u, abort_flag, a.spin) &&
-                             wait_sleep(&bar_ready[b], (uint32_t)(ph - 1) & 1u, abort_flag, a.spin)))
-                break;
+            scr += scratch_layer_bytes(kRows, K);
+            // The layers whose space (or whose barriers) this one takes over must have been released, and their copies
+            // must have landed (if no unit warp had a unit in such a layer, nobody has waited for them yet).  Layers
+            // are waited for in list order, so no barrier is ever more than one phase behind what is asked of it.
+            {
+                const int upto = max((int)(place >> 16), l - kDesc + 1);  // layers below `upto`
+                bool ok = true;
+                for (; freed < upto && ok; ++freed)
+                    ok = wait_sleep(&bar_free[freed % kDesc], (uint32_t)(freed / kDesc) & 1u, abort_flag, a.spin) &&
+                         wait_sleep(&bar_ready[freed % kDesc], (uint32_t)(freed / kDesc) & 1u, abort_flag, a.spin);
+                if (!ok) break;
+            }
             if (l >= ready_upto) {
                 // lane i looks at layer l + i: in a list of independent layers most are ready long before their turn
                 bool ok = false, stopped = false;
@@ -385,10 +393,10 @@ __global__ void __launch_bounds__(kThreads, 1) k_decode_stream(const ChainArgs a
             }
             if (lane == 0) {
                 s_fetched[b] = (uint32_t)ph + 1u;  // the barrier is in this layer's phase: it may be waited on
-                mbar_expect_tx(&bar_ready[b], (uint32_t)(kHeadBlock + M * K));
+                mbar_expect_tx(&bar_ready[b], (uint32_t)(kHeadBlock + kRows * K));
             }
             __syncwarp();
-            if (lane < M) bulk_load(buf + L.off_xq + (size_t)lane * L.pitch, g_codes + (size_t)lane * K, (uint32_t)K, &bar_ready[b]);
+            if (lane < kRows) bulk_load(buf + L.off_xq + (size_t)lane * L.pitch, g_codes + (size_t)lane * K, (uint32_t)K, &bar_ready[b]);
             if (lane == 30) bulk_load(buf, g_head, (uint32_t)kHeadBlock, &bar_ready[b]);
             // the unit warps without a unit in this layer pass it by: their arrivals on the buffer's barrier are made here
             // (the barrier is in this layer's phase: the one before was waited for above)
@@ -415,9 +423,9 @@ __global__ void __launch_bounds__(kThreads, 1) k_decode_stream(const ChainArgs a
             const int K = ly.K, ns = K >> 6;
             uint8_t *g_head = a.scratch + scr;
             uint8_t *g_codes = g_head + kHeadBlock;
-            uint8_t *g_mask = g_codes + scratch_codes_bytes(M, K);
+            uint8_t *g_mask = g_codes + scratch_codes_bytes(kRows, K);
             uint8_t *g_segflag = g_mask + K;
-            scr += scratch_layer_bytes(M, K);
+            scr += scratch_layer_bytes(kRows, K);
             int s = myw - (int)ly.slice_off;
             if (s < 0) s += NW;
             if (s >= ns) continue;
@@ -625,12 +633,13 @@ __global__ void __launch_bounds__(kThreads, 1) k_decode_stream(const ChainArgs a
             if (i0 >= cnt) continue;                             // nothing for this warp in this layer
             const int lseq = (int)s_lseq[l];                     // number of this CTA's stages before the layer
             const ChainLayer ly = tab[l];
-            const int K = ly.K, b = l % NB, ph = l / NB;
-            const uint8_t *buf = xbase + b * L.buf_bytes;
+            const int K = ly.K, b = l % kDesc, ph = l / kDesc;
+            const XLayout L = x_layout(kRows, K);
+            const uint8_t *buf = xbase + (size_t)(s_place[l] & 0xFFFFu) * 128;
             const XHeader *hdr = reinterpret_cast<const XHeader *>(buf);
             const int8_t *xq = reinterpret_cast<const int8_t *>(buf + L.off_xq);
             // (written in this launch by other SMs: read through L2; visible by way of the ready word and the buffer's barrier)
-            const uint8_t *g_mask = a.scratch + s_scr[l] + kHeadBlock + scratch_codes_bytes(M, ly.K);
+            const uint8_t *g_mask = a.scratch + s_scr[l] + kHeadBlock + scratch_codes_bytes(kRows, ly.K);
             const uint16_t *flaglist = reinterpret_cast<const uint16_t *>(buf + L.off_flaglist);
             const uint16_t *chlist = reinterpret_cast<const uint16_t *>(buf + L.off_chlist);
             const int seg = (int)ly.seg, nst = K / seg, segs = seg >> 6;
@@ -902,10 +911,66 @@ int chain_slot_bytes(int) { return 10 * 1024; }
 
 size_t chain_sync_bytes(int n_layers) { return (size_t)(n_layers + 1) * sizeof(LayerSync); }
 
+int chain_rows(int M) { return M == 1 ? 1 : M == 2 ? 2 : M <= 4 ? 4 : M <= 8 ? 8 : 16; }
+
 size_t chain_scratch_bytes(const ChainLayer *layers, int n_layers, int M) {
     size_t b = 0;
-    for (int l = 0; l < n_layers; ++l) b += scratch_layer_bytes(M, layers[l].K);
+    for (int l = 0; l < n_layers; ++l) b += scratch_layer_bytes(chain_rows(M), layers[l].K);
     return b;
+}
+
+// Shared memory of a CTA: ring stages, the layer table, and a region from which every layer's buffer of prepared X is
+// cut in list order, each as large as its own K needs, wrapping around at the end; a buffer may be filled when the
+// layers whose buffers it overlaps (all older ones with them: they are released in order) have been released.
+// The region gets what holds about six average layers or two of the largest, the ring the rest (two stages per unit
+// warp are enough: with one, the stage a warp has just released is refilled with that very warp's next unit and the
+// warp sees the whole memory latency on every unit); if that leaves the ring under four stages, the region shrinks
+// to two of the largest layers, then to one.
+bool chain_geometry(const ChainLayer *layers, int n_layers, int M, int slot_bytes, ChainGeometry *geo, uint32_t *place) {
+    const int rows = chain_rows(M);
+    const int avail = kMaxSmem - n_layers * (int)sizeof(ChainLayer);
+    long long sum = 0;
+    int maxbuf = 0;
+    for (int l = 0; l < n_layers; ++l) {
+        const int b = x_layout(rows, layers[l].K).buf_bytes;
+        sum += b;
+        if (b > maxbuf) maxbuf = b;
+    }
+    const int avg = (int)(sum / n_layers);
+    int region = 6 * avg > 2 * maxbuf ? 6 * avg : 2 * maxbuf;
+    int slots = (avail - region) / slot_bytes;
+    if (slots < 4) { region = 2 * maxbuf; slots = (avail - region) / slot_bytes; }
+    if (slots < 4) { region = maxbuf; slots = (avail - region) / slot_bytes; }
+    if (slots < 2) return false;
+    if (slots > 2 * kUW) slots = 2 * kUW;
+    geo->lgroups = slots >= kLW ? kLW : 2;
+    slots -= slots % geo->lgroups;  // a slot keeps its loader warp
+    geo->slots = slots;
+    region = (avail - slots * slot_bytes) & ~127;
+    if (region > 0xFFFF * 128) region = 0xFFFF * 128;
+    geo->xregion = region;
+    // the layers' places
+    struct Live { int layer, start, end; };
+    Live live[kDesc];
+    int nlive = 0, head = 0;
+    for (int l = 0; l < n_layers; ++l) {
+        const int size = x_layout(rows, layers[l].K).buf_bytes;
+        if (head + size > region) head = 0;
+        const int start = head, end = head + size;
+        int upto = 0;  // layers below this one must have been released
+        for (;;) {
+            bool clash = nlive == kDesc;
+            for (int i = 0; i < nlive && !clash; ++i) clash = live[i].start < end && start < live[i].end;
+            if (!clash) break;
+            upto = live[0].layer + 1;  // the oldest goes, whichever clashed
+            for (int i = 1; i < nlive; ++i) live[i - 1] = live[i];
+            --nlive;
+        }
+        live[nlive++] = Live{l, start, end};
+        place[l] = (uint32_t)(start / 128) | ((uint32_t)upto << 16);
+        head = end;
+    }
+    return true;
 }
 
 int chain_plan(ChainLayer *layers, int n_layers, int grid, int slot_bytes) {
@@ -931,7 +996,6 @@ namespace {
 
 template <int MT, int kDotM>
 cudaError_t launch_inst(ChainArgs a, cudaStream_t s) {
-    constexpr int kRows = kDotM > 0 ? kDotM : MT;
     auto kern = k_decode_stream<MT, kDotM>;
     static PerDevice<int> attr_set;
     const int dev = current_device();
@@ -944,23 +1008,8 @@ cudaError_t launch_inst(ChainArgs a, cudaStream_t s) {
             attr_set.have[dev] = true;
         }
     }
-    // As many buffers of prepared X (up to kMaxBufs) as leave the ring two stages per unit warp (with one, the stage
-    // a warp has just released is refilled with that very warp's next unit, and the warp sees the whole memory
-    // latency on every unit); two buffers if that leaves four stages (while one layer's products run, the next
-    // layer's X arrives); else one, and then at least two stages.
-    const XLayout L = x_layout(kRows, a.kmax);
-    const int table = a.n_layers * (int)sizeof(ChainLayer);
-    int nbuf = kMaxBufs;
-    while (nbuf > 2 && (kMaxSmem - table - nbuf * L.buf_bytes) / a.slot_bytes < 2 * kUW) --nbuf;
-    if (nbuf == 2 && (kMaxSmem - table - 2 * L.buf_bytes) / a.slot_bytes < 4) nbuf = 1;
-    int slots = (kMaxSmem - table - nbuf * L.buf_bytes) / a.slot_bytes;
-    if (slots > kMaxSlots) slots = kMaxSlots;
-    if (slots < 2) return cudaErrorInvalidValue;
-    a.nbuf = nbuf;
-    a.lgroups = slots >= kLW ? kLW : 2;
-    slots -= slots % a.lgroups;  // a slot keeps its loader warp
-    a.slots = slots;
-    const size_t smem = (size_t)slots * a.slot_bytes + table + (size_t)nbuf * L.buf_bytes;
+    const size_t smem = (size_t)a.slots * a.slot_bytes + (size_t)a.n_layers * sizeof(ChainLayer) + (size_t)a.xregion;
+    if (smem > (size_t)kMaxSmem) return cudaErrorInvalidValue;
     void *params[] = {&a};
     return cudaLaunchCooperativeKernel(reinterpret_cast<const void *>(kern), dim3(a.grid), dim3(kThreads), params, smem, s);
 }

@@ -220,8 +220,12 @@ struct ChainArgs {
     int32_t *dev_status;
     uint32_t spin;
     int slots, slot_bytes;         // ring geometry
-    int nbuf;                      // buffers of prepared X per CTA (set by the launcher)
-    int lgroups;                   // loader warps in use; divides slots (set by the launcher)
+    int lgroups;                   // loader warps in use; divides slots
+    int xregion;                   // bytes of the region the layers' buffers of prepared X are cut from
+    const uint32_t *place;         // [n_layers] device: where in the region, and after which layers' release (chain_geometry)
+};
+struct ChainGeometry {
+    int slots, lgroups, xregion;
 };
 // Fills unit_off / seg / slice_off of every entry (host copy of the table); returns the widest K, -1 if a layer
 // does not fit (or the grid is too small for the slice scheme).
@@ -229,6 +233,9 @@ int chain_plan(ChainLayer *layers, int n_layers, int grid, int slot_bytes);
 int chain_slot_bytes(int M);  // bytes of a ring stage for lists of M-row layers
 size_t chain_sync_bytes(int n_layers);
 size_t chain_scratch_bytes(const ChainLayer *layers, int n_layers, int M);
+int chain_rows(int M);  // rows of codes kept per layer: M rounded up to 1, 2, 4, 8, 16
+// Shared-memory geometry of a list and every layer's place in the region of prepared X; false: does not fit.
+bool chain_geometry(const ChainLayer *layers, int n_layers, int M, int slot_bytes, ChainGeometry *geo, uint32_t *place);
 bool chain_layer_supported(int M, int K, int N);
 cudaError_t launch_decode_chain(const ChainArgs &a, cudaStream_t s);  // cooperative launch, a.grid CTAs
 
