@@ -44,7 +44,9 @@ int muxq_int8_mma_peak(int mma_n, int iters, int ctas, unsigned long long *cycle
  * path without faulting, trapping or hanging anything:
  *   spin_limit           poll limit of the waits (0 = the kernels' own, which amount to about a second)
  *   prep_extra_arrivals  the grid barrier of the preparation kernel expects this many arrivals more than
- *                        there are CTAs, so every CTA's wait runs out
+ *                        there are CTAs, so every CTA's wait runs out; in a list of layers (muxq_chain_run) a
+ *                        layer flagged MUXQ_LAYER_WAIT_PREV likewise waits for that many CTAs more than
+ *                        store the layer before it
  *   gemm_skip_k_block    1 + the index of a K block whose operand loads the GEMM's producer warps leave
  *                        out (0 = none): the MMA warp's wait for that stage runs out
  * The switches are process-wide and apply to launches made after the call; NULL restores normal

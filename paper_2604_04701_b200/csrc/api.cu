@@ -595,6 +595,7 @@ int muxq_chain_run(const void *plan_host, void *plan_dev, muxq_chain_result *res
     a.results = reinterpret_cast<ChainResult *>(results);
     a.dev_status = dev_status;
     a.spin = test_hooks().spin_limit ? test_hooks().spin_limit : (1u << 22);
+    a.extra_arrivals = test_hooks().prep_extra_arrivals;
     a.slot_bytes = chain_slot_bytes(h->M);
     a.sync = pd + h->sync_off;
     a.scratch = pd + h->scratch_off;

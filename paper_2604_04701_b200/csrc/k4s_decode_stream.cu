@@ -431,7 +431,7 @@ __global__ void __launch_bounds__(kThreads, 1) k_decode_stream(const ChainArgs a
             if (s >= ns) continue;
             // X of this layer is Y of the layer before it: every CTA that has units of it must have stored its part
             if ((ly.flags & kChainWaitPrev) &&
-                !wait_count(&sync[l - 1].stored, (uint32_t)min(tab[l - 1].N >> 3, grid), abort_flag, g_abort, a.spin))
+                !wait_count(&sync[l - 1].stored, (uint32_t)min(tab[l - 1].N >> 3, grid) + a.extra_arrivals, abort_flag, g_abort, a.spin))
                 break;
             const int ch = s * 64 + cg * 8;
             uint4 v[4];

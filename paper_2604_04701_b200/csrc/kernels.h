@@ -219,6 +219,7 @@ struct ChainArgs {
     uint8_t *scratch;              // chain_scratch_bytes(...) of device memory: per-layer codes, masks, segment flags
     int32_t *dev_status;
     uint32_t spin;
+    uint32_t extra_arrivals;       // test hook: a layer that waits for the one before it expects this many CTAs more
     int slots, slot_bytes;         // ring geometry
     int lgroups;                   // loader warps in use; divides slots
     int xregion;                   // bytes of the region the layers' buffers of prepared X are cut from

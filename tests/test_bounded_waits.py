@@ -104,6 +104,47 @@ def test_gemm_stage_that_is_never_filled_times_out_and_recovers(mx, skip_block):
     assert _canaries_intact(raw, pad)
 
 
+def test_layer_list_wait_for_the_previous_layer_times_out_and_recovers(mx):
+    """Two layers, the second reads the first one's Y.  With the hook its slice warps wait for one CTA more
+    than stores that Y: their bounded wait runs out, they tell the other CTAs through the plan's abort word,
+    every role of every CTA leaves, and the launch ends with MUXQ_ERR_TIMEOUT.  The first layer has been
+    computed by then.  The next run of the same plan (which clears the plan's counters) is bit-exact."""
+    M, d = 4, 1280
+    p = mx.MuxqParams(max_outliers=1024)
+    x0, _ = synth.make_x(11, 1, M, d, 6, 30.0, 30.0)
+    ws = [synth.make_w(11, 20 + i, d, d) for i in range(2)]
+    wq = [mx.muxq_quantize(_dev(w), p, True, mx.Workspace(mx.muxq_small_workspace_bytes(d))) for w in ws]
+    y1 = torch.zeros(M, d, dtype=torch.float16, device="cuda")
+    raw, y2, pad = _guarded(M, d, torch.float16)
+    y2.zero_()
+    chain = mx.Chain([(_dev(x0), wq[0][0], wq[0][1], y1, 0), (y1, wq[1][0], wq[1][1], y2, mx.MUXQ_LAYER_WAIT_PREV)],
+                     p, mx.MUXQ_OUT_F16)
+
+    def f16_key(v):
+        u = v.view(np.uint16).astype(np.int32)
+        return np.where(u & 0x8000, -(u & 0x7FFF), u)
+
+    def check(y, x_in, w):
+        wq_o, sw_o = oracle.quantize_weight(w)
+        res = oracle.linear(x_in, wq_o, sw_o, cap=1024)
+        assert np.abs(f16_key(y.cpu().numpy()) - f16_key(res.y16)).max() <= 1
+
+    try:
+        mx.muxq_test_hooks(spin_limit=2048, prep_extra_arrivals=1)
+        chain.run()
+        assert chain.read_status() == mx.MUXQ_ERR_TIMEOUT
+        assert _canaries_intact(raw, pad)
+        check(y1, x0, ws[0])
+    finally:
+        mx.muxq_test_hooks()
+    chain.status.zero_()
+    chain.run()
+    assert chain.read_status() == 0
+    assert _canaries_intact(raw, pad)
+    check(y1, x0, ws[0])
+    check(y2, y1.cpu().numpy(), ws[1])
+
+
 def test_hooks_reject_a_negative_block_index(mx):
     with pytest.raises(mx.MuxqError):
         mx.muxq_test_hooks(gemm_skip_k_block=-1)

@@ -126,6 +126,31 @@ def test_dependent_layers_wait_for_their_input(mx, M):
             _check_layer(mx, bufs[i + 1], x_in, ws[i], p, mx.MUXQ_OUT_F16)
 
 
+@pytest.mark.parametrize("M", [1, 2, 4, 8, 16])
+def test_layers_with_more_outlier_channels_than_the_channel_list_holds(mx, M):
+    """Up to 64 outlier channels the Aux term comes from a list of channels; beyond that from the masked
+    64-byte segments.  100 and 300 outlier channels (and 5 for the list path next to them), both K shapes."""
+    shapes = [(1280, 1280), (5120, 1280), (1280, 3840), (5120, 264)]
+    n_out = [100, 300, 5, 64]
+    p = mx.MuxqParams(max_outliers=512)
+    L = []
+    for i, ((K, N), no) in enumerate(zip(shapes, n_out)):
+        x, _ = synth.make_x(40 + M, 10 + i, M, K, no, 40.0, 80.0)
+        w = synth.make_w(40 + M, 10 + i, K, N)
+        w_q, s_w = mx.muxq_quantize(_dev(w), p, True, mx.Workspace(mx.muxq_small_workspace_bytes(N)))
+        L.append((x, w, _dev(x), w_q, s_w))
+    for out_kind in (mx.MUXQ_OUT_ACC_I32, mx.MUXQ_OUT_F32):
+        ys = [torch.full((M, N), -7, dtype=_OUT[out_kind], device="cuda") for (_, N) in shapes]
+        chain = mx.Chain([(xd, w_q, s_w, y, 0) for (_, _, xd, w_q, s_w), y in zip(L, ys)], p, out_kind)
+        chain.run()
+        assert chain.read_status() == 0
+        results = chain.results.cpu().numpy()
+        for l, ((x, w, _, _, _), y) in enumerate(zip(L, ys)):
+            res = _check_layer(mx, y, x, w, p, out_kind)
+            assert results[l, 0] == res.r
+        assert results[0, 0] > 64 and results[1, 0] > 64 and results[2, 0] <= 64
+
+
 def test_a_layer_over_capacity_is_reported_and_the_list_goes_on(mx):
     M = 4
     shapes = [(1280, 1280), (1280, 1280), (1280, 1280)]
