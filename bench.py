@@ -54,6 +54,8 @@ TRAFFIC = {
                        "profiles/k_gemm_i8_pair_configs3.md"),
     "k_prep": (["k12_prep.cu", "quant.cuh"], "376646cd649c08db",
                {"cfg3": {"16384x1280": 46.9e6, "16384x5120": 328.9e6}}, "profiles/k_prep_configs3.md"),
+    "k_decode_stream": (["k4s_decode_stream.cu", "quant.cuh", "ptx.cuh"], "cfdb25baa3e94295",
+                        {"chain": 713.4e6}, "profiles/k_decode_stream_chain144.md"),
 }
 
 
@@ -533,7 +535,8 @@ def measure_decode(mx, torch, dev, peaks, p):
     wbytes = sum(K * N for K, N, _ in dlayers)
     sw1 = torch.full((1,), 0.02 / 127.0, device=dev)
     decode = {"workload": "configs[3]/[4] decode: 36 x (1280->3840, 1280->1280, 1280->5120, 5120->1280), "
-                          "8 outlier channels x60, per-tensor INT8, one fused launch per layer",
+                          "8 outlier channels x60, per-tensor INT8; us_per_layer etc.: one fused launch per layer (graph replay), "
+                          "one_launch: the whole list in one muxq_chain_run",
               "w_bytes": wbytes, "layers": len(dlayers), "hbm_peak_gbs": peaks["hbm_gbs"]}
     for Md in (1, 4, 16):
         dx = {K: torch.from_numpy(synth.make_x(3, 100 + K, Md, K, 8, 60.0, 60.0)[0]).to(dev) for K in (d, 4 * d)}
