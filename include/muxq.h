@@ -74,7 +74,7 @@ typedef struct muxq_params {
     int w_bits;       /* 2..8 (Eq. 2 uses 8) */
     int gran;         /* muxq_gran */
     int aux_scale;    /* muxq_aux_scale; MUXQ_AUX_OWN is taken by muxq_linear / _events / _host only */
-    int max_outliers; /* capacity of O, 1..1024; the Aux block and its cost grow with it (aux_cols below) */
+    int max_outliers; /* capacity of O, 1..8192 (every channel of the widest X); the Aux block and its cost grow with it (aux_cols below) */
 } muxq_params;
 
 /* threshold 6, exp factor 2, 8/8 bits, per tensor, shared Aux scale, capacity 64. */

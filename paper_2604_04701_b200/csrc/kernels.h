@@ -88,7 +88,7 @@ struct QuantActArgs {
 cudaError_t launch_quant_act(const QuantActArgs &a, cudaStream_t s);
 
 // Fused detect + redistribute + quantize (one cooperative launch, X read from HBM once).
-constexpr int kMaxOutlierCap = 1024;  // largest max_outliers the entry points accept
+constexpr int kMaxOutlierCap = 8192;  // largest max_outliers the entry points accept (every channel of the widest X)
 constexpr int kPrepColmaxReplicas = 8;
 constexpr int kPrepMaxK = 8192;
 // Bytes of replicated accumulators behind Ctrl for the widest supported K.  The region has the same place

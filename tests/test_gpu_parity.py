@@ -607,6 +607,32 @@ def test_aux_own_scale_layer_matches_oracle(mx, M, K, N, gran, e, n_out):
             assert f16_ulp_diff(y.cpu().numpy(), res.y16).max() <= 1
 
 
+# ------------------------------------------------------------------ an outlier set as large as K
+@pytest.mark.parametrize("M,K,N,gran", [(300, 1280, 256, 0), (300, 1280, 256, 1), (260, 5120, 136, 0), (4, 1280, 264, 0),
+                                        (16, 5120, 128, 1)])
+def test_every_channel_an_outlier_channel(mx, M, K, N, gran):
+    """A bulk wide enough that every channel holds an element above the threshold: O is all of K (beyond 1024
+    channels), Aux mirrors the whole of Body, and the layer still matches the oracle code for code."""
+    p = mx.MuxqParams(gran=gran, max_outliers=K)
+    x, w, _ = make_case(1700 + M + gran, M, K, N, n_out=8, mult=60.0, bulk="t4", bulk_scale=6.0 if M > 16 else 40.0)
+    wq, sw = oracle.quantize_weight(w, bits=p.w_bits, per_channel=gran == 1)
+    res = oracle.linear(x, wq, sw, tau=p.threshold, e=p.exp_factor, act_bits=p.act_bits, per_vector=gran == 1, cap=K)
+    assert res.r > 1024 and res.r >= 0.97 * K
+    y, ws, st, _, _ = run_linear(mx, x, w, p, mx.MUXQ_OUT_F32)
+    assert st == 0
+    v = ws_views(mx, ws, M, K, N, p)
+    assert v["n_outliers"] == res.r and np.array_equal(v["outlier_idx"][:res.r], res.O)
+    assert np.array_equal(v["s_x"], res.s_x)
+    if M > 16:
+        assert np.array_equal(v["body_q"], res.body_q)
+        c = (1 << p.exp_factor) - 1
+        assert np.array_equal(v["aux_q"][:, 0:c * res.r:c], res.aux_q)
+    assert rel_err32(y.cpu().numpy(), res.y32) <= 1e-5
+    acc = mx.muxq_linear(dev(x), *mx.muxq_quantize(dev(w), p, True, mx.Workspace(mx.muxq_small_workspace_bytes(N))),
+                         p, mx.Workspace(mx.muxq_workspace_bytes(M, K, N, p)), mx.MUXQ_OUT_ACC_I32)
+    assert np.array_equal(acc.cpu().numpy(), res.acc)
+
+
 # ------------------------------------------------------------------ many outlier channels (capacity up to 1024)
 @pytest.mark.parametrize("M,K,N,gran,own", [(300, 1024, 256, 0, 0), (300, 1024, 256, 1, 0), (8, 1024, 128, 0, 0),
                                              (200, 512, 136, 0, 1)])
