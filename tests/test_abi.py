@@ -40,7 +40,7 @@ def test_host_only_helpers(L):
     n = L.muxq_workspace_bytes(8192, 768, 2304, p)
     assert n >= 8192 * 768 + 8192 * 256 + 2304 * 256 and n % 1024 == 0
     assert L.muxq_workspace_bytes(0, 768, 768, p) == 0
-    assert L.muxq_workspace_bytes(128, 768, 768, L.MuxqParams(max_outliers=1025)) == 0
+    assert L.muxq_workspace_bytes(128, 768, 768, L.MuxqParams(max_outliers=8193)) == 0
     assert L.muxq_host_workspace_bytes(128, 768, 768, p, 0) >= L.muxq_workspace_bytes(128, 768, 768, p) + 128 * 768 * 4
     v = L.muxq_workspace_view(128, 768, 768, p)
     assert v.ld_body_q == 768 and v.aux_cols == 256 and v.body_q % 1024 == 0 and v.aux_q > v.body_q
