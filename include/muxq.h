@@ -193,6 +193,19 @@ int muxq_linear(const void *X_f16, int M, int K, int ldx, const int8_t *W_q, int
                 const float *s_w, int N, const muxq_params *p, void *Y, int ldy, int out_kind,
                 void *workspace, size_t workspace_bytes, int32_t *dev_status, void *stream);
 
+/*
+ * muxq_linear with the layer's additive term: Y[m, n] = dequantized value of Eq. 3 + bias[n].  The GPT-2
+ * projections the paper measures on (Section IV-C) carry such a term; the paper's equations end at Eq. 3, so the
+ * reading here is the plain one: one fp32 addition (round to nearest) after the two multiplications of Eq. 3, then
+ * the cast to the output type, fused into the epilogue of the product.  bias: device, fp32 [N], 16-byte aligned,
+ * constant while the call may be in flight; NULL gives muxq_linear.  MUXQ_OUT_ACC_I32 with a bias is
+ * MUXQ_ERR_INVALID_ARG (the accumulator has no scale yet), MUXQ_AUX_OWN with a bias MUXQ_ERR_UNSUPPORTED.
+ * Everything else as for muxq_linear.
+ */
+int muxq_linear_bias(const void *X_f16, int M, int K, int ldx, const int8_t *W_q, int ldw,
+                     const float *s_w, const float *bias_f32, int N, const muxq_params *p, void *Y, int ldy,
+                     int out_kind, void *workspace, size_t workspace_bytes, int32_t *dev_status, void *stream);
+
 /* Where muxq_linear leaves its intermediates inside the workspace (byte offsets). */
 typedef struct muxq_ws_view {
     size_t col_absmax;  /* float [K] */

@@ -153,8 +153,12 @@ class LinearResult:
 
 def linear(x: np.ndarray, w_q: np.ndarray, s_w: np.ndarray, *, tau: float = 6.0, e: int = 2,
            act_bits: int = 8, per_vector: bool = False, aux_own: bool = False, cap: int = 64,
-           rows: Optional[np.ndarray] = None, want_codes: bool = True) -> LinearResult:
+           rows: Optional[np.ndarray] = None, want_codes: bool = True,
+           bias: Optional[np.ndarray] = None) -> LinearResult:
     """Steps 1-6 and 8-10 for one call; w_q [K,N] and s_w come from quantize_weight.
+
+    bias: optional fp32 [N], the layer's additive term (the GPT-2 projections of Section IV-C carry one): added to
+    the dequantized fp32 value of Eq. 3 with one fp32 addition, before the cast to fp16.
 
     rows: optional int32 row subset for the products and the output (outputs are [len(rows), N]).
     """
@@ -189,6 +193,12 @@ def linear(x: np.ndarray, w_q: np.ndarray, s_w: np.ndarray, *, tau: float = 6.0,
                              _p(acc_b), _p(acc_a), _p(acc), _p(y32), _p(y16))
     if rc not in (OK, ERR_CAPACITY):
         raise ValueError(f"oracle_linear rc={rc}")
+    if bias is not None:
+        b32 = np.ascontiguousarray(bias, np.float32).reshape(1, N)
+        y32 = y32 + b32                       # float32 + float32: one IEEE addition per element, round to nearest even
+        assert y32.dtype == np.float32
+        with np.errstate(over="ignore"):
+            y16 = y32.astype(np.float16).view(np.uint16)   # round to nearest even, overflow to infinity
     rr = r.value
     return LinearResult(rc, cm, O[: min(rr, cap)].copy(), rr, s_x, s_a, bq,
                         None if aq is None else aq[:, : min(rr, cap)].copy(), acc_b, acc_a, acc,

@@ -21,7 +21,7 @@ MUXQ_OUT_F16, MUXQ_OUT_F32, MUXQ_OUT_ACC_I32 = 0, 1, 2
 EXPORTS = (
     "muxq_default_params", "muxq_aux_cols", "muxq_workspace_bytes", "muxq_small_workspace_bytes",
     "muxq_host_workspace_bytes", "muxq_workspace_init", "muxq_workspace_view", "muxq_detect_outliers", "muxq_build_aux",
-    "muxq_quantize", "muxq_gemm", "muxq_linear", "muxq_linear_events", "muxq_linear_host",
+    "muxq_quantize", "muxq_gemm", "muxq_linear", "muxq_linear_bias", "muxq_linear_events", "muxq_linear_host",
     "muxq_linear_decode_noalloc", "muxq_int8_mma_peak", "muxq_test_hooks", "muxq_read_status",
     "muxq_chain_plan_bytes", "muxq_chain_device_bytes", "muxq_chain_build", "muxq_chain_run",
     "muxq_status_string",
@@ -92,6 +92,7 @@ def lib() -> ctypes.CDLL:
         L.muxq_quantize.argtypes = [vp, i, i, i, pp, i, vp, vp, vp, vp, i, vp, i, vp, vp, sz, vp]; L.muxq_quantize.restype = i
         L.muxq_gemm.argtypes = [vp, i, vp, i, vp, i, vp, i, vp, i, i, i, pp, vp, vp, vp, i, i, vp, vp]; L.muxq_gemm.restype = i
         L.muxq_linear.argtypes = [vp, i, i, i, vp, i, vp, i, pp, vp, i, i, vp, sz, vp, vp]; L.muxq_linear.restype = i
+        L.muxq_linear_bias.argtypes = [vp, i, i, i, vp, i, vp, vp, i, pp, vp, i, i, vp, sz, vp, vp]; L.muxq_linear_bias.restype = i
         L.muxq_linear_events.argtypes = [vp, i, i, i, vp, i, vp, i, pp, vp, i, i, vp, sz, vp, vp, vp]; L.muxq_linear_events.restype = i
         L.muxq_linear_host.argtypes = [vp, i, i, vp, i, vp, i, pp, vp, i, vp, sz, vp, vp]; L.muxq_linear_host.restype = i
         L.muxq_linear_decode_noalloc.argtypes = [vp, i, i, i, vp, i, vp, i, pp, vp, i, i, vp, vp]; L.muxq_linear_decode_noalloc.restype = i
@@ -243,12 +244,20 @@ def muxq_gemm(body_q: torch.Tensor, aux_q: Optional[torch.Tensor], w_q: torch.Te
 
 
 def muxq_linear(X: torch.Tensor, w_q: torch.Tensor, s_w: torch.Tensor, p: MuxqParams, ws: Workspace,
-                out_kind: int = MUXQ_OUT_F16, out: Optional[torch.Tensor] = None) -> torch.Tensor:
-    """Y = MUXQ-quantized X.W; w_q [N,K] int8 and s_w from muxq_quantize(is_weight=True)."""
+                out_kind: int = MUXQ_OUT_F16, out: Optional[torch.Tensor] = None,
+                bias: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """Y = MUXQ-quantized X.W [+ bias]; w_q [N,K] int8 and s_w from muxq_quantize(is_weight=True); bias fp32 [N]."""
     assert X.is_cuda and X.dtype == torch.float16 and X.dim() == 2 and X.stride(1) == 1
     M, K = X.shape
     N = w_q.shape[0]
     Y = out if out is not None else _alloc_out(M, N, out_kind, X.device)
+    if bias is not None:
+        assert bias.is_cuda and bias.dtype == torch.float32 and bias.is_contiguous() and bias.numel() == N
+        _check("muxq_linear_bias",
+               lib().muxq_linear_bias(_ptr(X), M, K, X.stride(0), _ptr(w_q), w_q.stride(0), _ptr(s_w), _ptr(bias), N,
+                                      ctypes.byref(p.c()), _ptr(Y), Y.stride(0), out_kind, _ptr(ws.buf), ws.nbytes,
+                                      _ptr(ws.status), _stream()))
+        return Y
     _check("muxq_linear",
            lib().muxq_linear(_ptr(X), M, K, X.stride(0), _ptr(w_q), w_q.stride(0), _ptr(s_w), N,
                              ctypes.byref(p.c()), _ptr(Y), Y.stride(0), out_kind, _ptr(ws.buf), ws.nbytes,

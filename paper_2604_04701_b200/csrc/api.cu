@@ -276,8 +276,8 @@ int muxq_gemm(const int8_t *Body_q, int ld_a, const int8_t *Aux_q, int ld_aux, c
     return cuda_rc(launch_gemm(g, static_cast<cudaStream_t>(stream)));
 }
 
-static int linear_impl(const void *X, int M, int K, int ldx, const int8_t *W_q, int ldw, const float *s_w, int N,
-                       const muxq_params *p, void *Y, int ldy, int out_kind, void *workspace, size_t workspace_bytes,
+static int linear_impl(const void *X, int M, int K, int ldx, const int8_t *W_q, int ldw, const float *s_w,
+                       const float *bias, int N, const muxq_params *p, void *Y, int ldy, int out_kind, void *workspace, size_t workspace_bytes,
                        int32_t *dev_status, void *stream, void *const *events) {
     if (!X || !W_q || !s_w || !Y || !workspace || !dev_status || M <= 0 || K <= 0 || N <= 0 || ldx < K ||
         ldw < K || ldy < N || !params_ok(p) || out_kind < 0 || out_kind > 2)
@@ -288,6 +288,8 @@ static int linear_impl(const void *X, int M, int K, int ldx, const int8_t *W_q, 
         return MUXQ_ERR_UNSUPPORTED;
     const bool aux_own = p->aux_scale == MUXQ_AUX_OWN;
     if (aux_own && out_kind == MUXQ_OUT_ACC_I32) return MUXQ_ERR_UNSUPPORTED;  // there is no common accumulator
+    if (bias && out_kind == MUXQ_OUT_ACC_I32) return MUXQ_ERR_INVALID_ARG;     // the bias belongs to the dequantized output
+    if (bias && (aux_own || !aligned16(bias))) return MUXQ_ERR_UNSUPPORTED;
     const LinearWs w = linear_ws(M, K, N, p);
     if (workspace_bytes < w.total) return MUXQ_ERR_WORKSPACE;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
@@ -315,6 +317,7 @@ static int linear_impl(const void *X, int M, int K, int ldx, const int8_t *W_q, 
         k.M = M; k.K = K; k.ldx = ldx;
         k.w_q = W_q; k.ldw = ldw; k.N = N;
         k.s_w = s_w; k.per_vec = per_vec;
+        k.bias = bias;
         k.tau = p->threshold; k.exp_factor = p->exp_factor; k.qmax = qmax_of(p->act_bits);
         k.cap = p->max_outliers; k.c = (1 << p->exp_factor) - 1;
         k.Y = Y; k.ldy = ldy; k.out_kind = out_kind;
@@ -406,6 +409,7 @@ static int linear_impl(const void *X, int M, int K, int ldx, const int8_t *W_q, 
         k.M = M; k.K = K; k.N = N; k.c = c; k.cap = p->max_outliers;
         k.s_x = s_x; k.s_x_per_row = per_vec;
         k.s_w = s_w; k.s_w_per_col = per_vec;
+        k.bias = bias;
         k.Y = Y; k.ldy = ldy; k.out_kind = out_kind;
         e = launch_decode(k, s);
         mark(3);
@@ -445,6 +449,7 @@ static int linear_impl(const void *X, int M, int K, int ldx, const int8_t *W_q, 
     g.M = M; g.K = K; g.N = N; g.c = c; g.cap = p->max_outliers; g.aux_cols = w.aux_cols;
     g.s_x = s_x; g.s_x_per_row = per_vec;
     g.s_w = s_w; g.s_w_per_col = per_vec;
+    g.bias = bias;
     g.Y = Y; g.ldy = ldy; g.out_kind = out_kind;
     g.dev_status = dev_status;
     g.w_stable = 1;  // the kernel before this one in the stream is the preparation of X, which does not write W_q
@@ -456,16 +461,23 @@ static int linear_impl(const void *X, int M, int K, int ldx, const int8_t *W_q, 
 int muxq_linear(const void *X, int M, int K, int ldx, const int8_t *W_q, int ldw, const float *s_w, int N,
                 const muxq_params *p, void *Y, int ldy, int out_kind, void *workspace, size_t workspace_bytes,
                 int32_t *dev_status, void *stream) {
-    return linear_impl(X, M, K, ldx, W_q, ldw, s_w, N, p, Y, ldy, out_kind, workspace, workspace_bytes, dev_status,
-                       stream, nullptr);
+    return linear_impl(X, M, K, ldx, W_q, ldw, s_w, nullptr, N, p, Y, ldy, out_kind, workspace, workspace_bytes,
+                       dev_status, stream, nullptr);
+}
+
+int muxq_linear_bias(const void *X, int M, int K, int ldx, const int8_t *W_q, int ldw, const float *s_w,
+                     const float *bias, int N, const muxq_params *p, void *Y, int ldy, int out_kind, void *workspace,
+                     size_t workspace_bytes, int32_t *dev_status, void *stream) {
+    return linear_impl(X, M, K, ldx, W_q, ldw, s_w, bias, N, p, Y, ldy, out_kind, workspace, workspace_bytes,
+                       dev_status, stream, nullptr);
 }
 
 int muxq_linear_events(const void *X, int M, int K, int ldx, const int8_t *W_q, int ldw, const float *s_w, int N,
                        const muxq_params *p, void *Y, int ldy, int out_kind, void *workspace,
                        size_t workspace_bytes, int32_t *dev_status, void *stream, void *const *events) {
     if (!events) return MUXQ_ERR_INVALID_ARG;
-    return linear_impl(X, M, K, ldx, W_q, ldw, s_w, N, p, Y, ldy, out_kind, workspace, workspace_bytes, dev_status,
-                       stream, events);
+    return linear_impl(X, M, K, ldx, W_q, ldw, s_w, nullptr, N, p, Y, ldy, out_kind, workspace, workspace_bytes,
+                       dev_status, stream, events);
 }
 
 int muxq_linear_host(const void *X_host, int M, int K, const int8_t *W_q, int ldw, const float *s_w, int N,

@@ -25,6 +25,7 @@ struct GemmParams {
     const int32_t *n_outliers;
     const float *s_x;
     const float *s_w;
+    const float *bias;  // [N] fp32 or NULL: added to the dequantized value (one fp32 addition), then the cast
     int32_t *dev_status;
     int w_stable;  // the B operand may be read before the programmatic predecessor has finished
     uint32_t spin; // poll limit of the bounded waits
@@ -32,11 +33,12 @@ struct GemmParams {
 };
 
 // One 32-column chunk of one accumulator row: int32 -> fp32 (round to nearest even, exact below
-// 2^24) -> times the scale -> output type, written as 16-byte pieces into the warp's staging row
+// 2^24) -> times the scale [-> plus the layer's bias] -> output type, written as 16-byte pieces into the warp's staging row
 // with the 128-byte swizzle the TMA store expects (16-byte piece g of row `lane` sits at g ^ (lane & 7)).
 template <int kOut, bool kPerVec>
 __device__ __forceinline__ void convert_chunk(const uint32_t (&v)[32], uint4 *srow, int piece0, uint32_t sw_xor,
-                                              float sx, float sxw, const float *s_w_col, int cols_left) {
+                                              float sx, float sxw, const float *s_w_col, int cols_left,
+                                              const float *bias_col) {
     if constexpr (kOut == kOutI32) {
 #pragma unroll
         for (int g = 0; g < 8; ++g)
@@ -56,6 +58,14 @@ __device__ __forceinline__ void convert_chunk(const uint32_t (&v)[32], uint4 *sr
         f[4 * g + 1] = __fmul_rn(sc.y, __int2float_rn((int)v[4 * g + 1]));
         f[4 * g + 2] = __fmul_rn(sc.z, __int2float_rn((int)v[4 * g + 2]));
         f[4 * g + 3] = __fmul_rn(sc.w, __int2float_rn((int)v[4 * g + 3]));
+        if (bias_col) {  // warp-uniform; same address in every lane
+            const float4 bb = 4 * g < cols_left ? __ldg(reinterpret_cast<const float4 *>(bias_col) + g)
+                                                : make_float4(0.f, 0.f, 0.f, 0.f);
+            f[4 * g + 0] = __fadd_rn(f[4 * g + 0], bb.x);
+            f[4 * g + 1] = __fadd_rn(f[4 * g + 1], bb.y);
+            f[4 * g + 2] = __fadd_rn(f[4 * g + 2], bb.z);
+            f[4 * g + 3] = __fadd_rn(f[4 * g + 3], bb.w);
+        }
     }
     if (kOut == kOutF32) {
 #pragma unroll

@@ -204,7 +204,7 @@ k_gemm_i8(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
                 const int gcol = n0 + col0 + 32 * ch;
                 convert_chunk<kOut, kPerVec>(v[ch], reinterpret_cast<uint4 *>(stage + lane * 128),
                                              kOut == kOutF16 ? 4 * piece : 0, sw_xor, sx, sxw, p.s_w + gcol,
-                                             p.N - gcol);
+                                             p.N - gcol, p.bias ? p.bias + gcol : nullptr);
                 if (piece == kChunksPerBox - 1) {
                     fence_proxy_async();  // make the generic-proxy writes visible to the TMA engine
                     __syncwarp();
@@ -271,6 +271,7 @@ cudaError_t launch_gemm_inst(const GemmArgs &a, cudaStream_t s) {
     p.n_outliers = a.n_outliers;
     p.s_x = a.s_x;
     p.s_w = a.s_w;
+    p.bias = a.out_kind == kOutI32 ? nullptr : a.bias;
     p.dev_status = a.dev_status;
     p.w_stable = 0; p.spin = kSpinLimit; p.skip_kb = -1;
     int grid = p.tiles_m * p.tiles_n;

@@ -257,7 +257,7 @@ k_gemm_i8_pair(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                 const int gcol = n0 + col0 + 32 * ch;
                 convert_chunk<kOut, kPerVec>(v[ch], reinterpret_cast<uint4 *>(stage + lane * 128),
                                              kOut == kOutF16 ? 4 * piece : 0, sw_xor, sx, sxw, p.s_w + gcol,
-                                             p.N - gcol);
+                                             p.N - gcol, p.bias ? p.bias + gcol : nullptr);
                 if (piece == kChunksPerBox - 1) {
                     fence_proxy_async();
                     __syncwarp();
@@ -339,6 +339,7 @@ cudaError_t launch_pair_inst(const GemmArgs &a, cudaStream_t s) {
     p.n_outliers = a.n_outliers;
     p.s_x = a.s_x;
     p.s_w = a.s_w;
+    p.bias = a.out_kind == kOutI32 ? nullptr : a.bias;
     p.dev_status = a.dev_status;
     p.w_stable = a.w_stable;
     p.spin = test_hooks().spin_limit ? test_hooks().spin_limit : kSpinLimit;

@@ -60,7 +60,8 @@ __global__ void __launch_bounds__(kThreads) k_decode(const DecodeArgs a) {
                 if (a.out_kind == 2) {
                     reinterpret_cast<int32_t *>(a.Y)[o] = acc[m];
                 } else {
-                    const float y = __fmul_rn(__fmul_rn(sx, sw), __int2float_rn(acc[m]));
+                    float y = __fmul_rn(__fmul_rn(sx, sw), __int2float_rn(acc[m]));
+                    if (a.bias) y = __fadd_rn(y, __ldg(a.bias + n));
                     if (a.out_kind == 1) reinterpret_cast<float *>(a.Y)[o] = y;
                     else reinterpret_cast<__half *>(a.Y)[o] = __float2half_rn(y);
                 }

@@ -425,7 +425,8 @@ __global__ void __launch_bounds__(kT, 1) k_decode_fused(const DecodeFusedArgs a,
                 } else {
                     const float sx = s_rowscale[a.per_vec ? m : 0];
                     const float sw = a.per_vec ? __ldg(a.s_w + nn) : sw0;
-                    const float y = __fmul_rn(__fmul_rn(sx, sw), __int2float_rn(acc));  // Eq. 3
+                    float y = __fmul_rn(__fmul_rn(sx, sw), __int2float_rn(acc));  // Eq. 3
+                    if (a.bias) y = __fadd_rn(y, __ldg(a.bias + nn));
                     if (a.out_kind == 1) reinterpret_cast<float *>(a.Y)[o] = y;
                     else reinterpret_cast<__half *>(a.Y)[o] = __float2half_rn(y);
                 }

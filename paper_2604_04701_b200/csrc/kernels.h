@@ -152,6 +152,7 @@ struct GemmArgs {
     int c, cap, aux_cols;
     const float *s_x; int s_x_per_row;
     const float *s_w; int s_w_per_col;
+    const float *bias;  // [N] fp32 added after the dequantization, or NULL
     void *Y; int ldy; int out_kind;
     int32_t *dev_status;
     int w_stable;  // W_q is not written by the kernel before this one in the stream: its tiles may be fetched early
@@ -166,6 +167,7 @@ struct DecodeArgs {
     int M, K, N, c, cap;
     const float *s_x; int s_x_per_row;
     const float *s_w; int s_w_per_col;
+    const float *bias;  // [N] fp32 or NULL
     void *Y; int ldy; int out_kind;
 };
 cudaError_t launch_decode(const DecodeArgs &a, cudaStream_t s);
@@ -175,6 +177,7 @@ struct DecodeFusedArgs {
     const __half *X; int M, K, ldx;
     const int8_t *w_q; int ldw; int N;
     const float *s_w; int per_vec;      // per-token X scales and per-channel W scales, or one of each
+    const float *bias;                  // [N] fp32 added after the dequantization, or NULL
     float tau; int exp_factor, qmax, cap, c;
     void *Y; int ldy; int out_kind;
     float *colmax;                      // [K] out or NULL

@@ -607,6 +607,48 @@ def test_aux_own_scale_layer_matches_oracle(mx, M, K, N, gran, e, n_out):
             assert f16_ulp_diff(y.cpu().numpy(), res.y16).max() <= 1
 
 
+# ------------------------------------------------------------------ the layer's additive term (muxq_linear_bias)
+@pytest.mark.parametrize("M,K,N,gran", [(300, 768, 256, 0), (1000, 1024, 264, 1), (2600, 256, 776, 0), (1, 1280, 264, 0),
+                                        (7, 768, 136, 1), (16, 8320, 128, 0)])
+@pytest.mark.parametrize("out_kind", [0, 1])
+def test_linear_with_bias(mx, M, K, N, gran, out_kind):
+    """Prefill shapes (both GEMM kernels' epilogues, ragged tiles) and decode shapes (fused and two-kernel form):
+    fp32 outputs bit-equal to the oracle's one-addition reading, fp16 within 1 ulp."""
+    p = mx.MuxqParams(gran=gran)
+    x, w, _ = make_case(1800 + M + gran, M, K, N, n_out=5, mult=50.0)
+    bias = (synth.normal(1800 + M, 9, N) * 0.5).astype(np.float32)
+    wq, sw = oracle.quantize_weight(w, bits=p.w_bits, per_channel=gran == 1)
+    res = oracle.linear(x, wq, sw, per_vector=gran == 1, bias=bias, want_codes=False)
+    w_q, s_w = mx.muxq_quantize(dev(w), p, True, mx.Workspace(mx.muxq_small_workspace_bytes(N)))
+    ws = mx.Workspace(mx.muxq_workspace_bytes(M, K, N, p))
+    y = mx.muxq_linear(dev(x), w_q, s_w, p, ws, out_kind, bias=dev(bias))
+    assert mx.muxq_read_status(ws) == 0
+    g = y.cpu().numpy()
+    if out_kind == 1:
+        assert np.array_equal(g, res.y32)
+    else:
+        assert f16_ulp_diff(g, res.y16).max() <= 1
+    # without the term the same call gives the plain layer (the epilogue's branch is off, not stale)
+    y0 = mx.muxq_linear(dev(x), w_q, s_w, p, ws, mx.MUXQ_OUT_F32)
+    assert np.array_equal(y0.cpu().numpy(), oracle.linear(x, wq, sw, per_vector=gran == 1, want_codes=False).y32)
+
+
+def test_linear_bias_argument_errors(mx):
+    p = mx.MuxqParams()
+    x = torch.zeros(32, 256, dtype=torch.float16, device="cuda")
+    w_q = torch.zeros(128, 256, dtype=torch.int8, device="cuda")
+    s_w = torch.ones(1, device="cuda")
+    bias = torch.zeros(128, device="cuda")
+    ws = mx.Workspace(mx.muxq_workspace_bytes(32, 256, 128, p))
+    with pytest.raises(mx.MuxqError) as ei:
+        mx.muxq_linear(x, w_q, s_w, p, ws, mx.MUXQ_OUT_ACC_I32, bias=bias)
+    assert ei.value.status == mx.MUXQ_ERR_INVALID_ARG
+    pown = mx.MuxqParams(aux_scale=mx.MUXQ_AUX_OWN)
+    with pytest.raises(mx.MuxqError) as ei:
+        mx.muxq_linear(x, w_q, s_w, pown, mx.Workspace(mx.muxq_workspace_bytes(32, 256, 128, pown)), mx.MUXQ_OUT_F32, bias=bias)
+    assert ei.value.status == mx.MUXQ_ERR_UNSUPPORTED
+
+
 # ------------------------------------------------------------------ an outlier set as large as K
 @pytest.mark.parametrize("M,K,N,gran", [(300, 1280, 256, 0), (300, 1280, 256, 1), (260, 5120, 136, 0), (4, 1280, 264, 0),
                                         (16, 5120, 128, 1)])

@@ -305,6 +305,27 @@ def test_brute_force_tiny(seed, per_vector):
     assert np.array_equal(res.y32, np.array(y, np.float32).reshape(M, N))
 
 
+def test_bias_is_one_fp32_addition_after_eq3():
+    """The additive term of a projection: pinned through a different arithmetic route (Python floats are fp64; the
+    sum of two fp32 values is exact in fp64, so rounding it once to fp32 IS the correctly rounded fp32 sum), through
+    the fp16 cast of numpy, and through the special cases: a zero bias changes nothing, a bias of -y gives zero."""
+    x, w, _ = _rand_case(21, 9, 64, 24)
+    wq, sw = oracle.quantize_weight(w)
+    base = oracle.linear(x, wq, sw)
+    rng = np.random.default_rng(5)
+    bias = (rng.standard_normal(24) * 0.3).astype(np.float32)
+    res = oracle.linear(x, wq, sw, bias=bias)
+    want = [[np.float32(float(base.y32[m, n]) + float(bias[n])) for n in range(24)] for m in range(9)]
+    assert np.array_equal(res.y32, np.array(want, np.float32))
+    assert np.array_equal(res.y16.view(np.uint16), np.array(want, np.float32).astype(np.float16).view(np.uint16))
+    assert np.array_equal(res.acc, base.acc) and np.array_equal(res.body_q, base.body_q)
+    zero = oracle.linear(x, wq, sw, bias=np.zeros(24, np.float32))
+    assert np.array_equal(zero.y32, base.y32) and np.array_equal(zero.y16.view(np.uint16), base.y16.view(np.uint16))
+    # row 0 cancelled exactly
+    cancel = oracle.linear(x[:1], wq, sw, bias=-oracle.linear(x[:1], wq, sw).y32[0])
+    assert not cancel.y32.any()
+
+
 # ------------------------------------------------------------------ metamorphic relations
 def test_power_of_two_scaling():
     x, w, _ = _rand_case(31, 29, 64, 16, n_out=3)
