@@ -35,7 +35,7 @@ struct GemmParams {
 // One 32-column chunk of one accumulator row: int32 -> fp32 (round to nearest even, exact below
 // 2^24) -> times the scale [-> plus the layer's bias] -> output type, written as 16-byte pieces into the warp's staging row
 // with the 128-byte swizzle the TMA store expects (16-byte piece g of row `lane` sits at g ^ (lane & 7)).
-template <int kOut, bool kPerVec>
+template <int kOut, bool kPerVec, bool kBias>
 __device__ __forceinline__ void convert_chunk(const uint32_t (&v)[32], uint4 *srow, int piece0, uint32_t sw_xor,
                                               float sx, float sxw, const float *s_w_col, int cols_left,
                                               const float *bias_col) {
@@ -58,7 +58,7 @@ __device__ __forceinline__ void convert_chunk(const uint32_t (&v)[32], uint4 *sr
         f[4 * g + 1] = __fmul_rn(sc.y, __int2float_rn((int)v[4 * g + 1]));
         f[4 * g + 2] = __fmul_rn(sc.z, __int2float_rn((int)v[4 * g + 2]));
         f[4 * g + 3] = __fmul_rn(sc.w, __int2float_rn((int)v[4 * g + 3]));
-        if (bias_col) {  // warp-uniform; same address in every lane
+        if constexpr (kBias) {  // same address in every lane: one broadcast transaction
             const float4 bb = 4 * g < cols_left ? __ldg(reinterpret_cast<const float4 *>(bias_col) + g)
                                                 : make_float4(0.f, 0.f, 0.f, 0.f);
             f[4 * g + 0] = __fadd_rn(f[4 * g + 0], bb.x);

@@ -40,7 +40,7 @@ struct Cfg {
     static_assert(kStages >= 3, "operand ring too shallow");
 };
 
-template <int BN, int kOut, bool kPerVec>
+template <int BN, int kOut, bool kPerVec, bool kBias>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 k_gemm_i8(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_aux,
           const __grid_constant__ CUtensorMap tm_b, const __grid_constant__ CUtensorMap tm_baux,
@@ -202,9 +202,9 @@ k_gemm_i8(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
                     __syncwarp();
                 }
                 const int gcol = n0 + col0 + 32 * ch;
-                convert_chunk<kOut, kPerVec>(v[ch], reinterpret_cast<uint4 *>(stage + lane * 128),
+                convert_chunk<kOut, kPerVec, kBias>(v[ch], reinterpret_cast<uint4 *>(stage + lane * 128),
                                              kOut == kOutF16 ? 4 * piece : 0, sw_xor, sx, sxw, p.s_w + gcol,
-                                             p.N - gcol, p.bias ? p.bias + gcol : nullptr);
+                                             p.N - gcol, kBias ? p.bias + gcol : nullptr);
                 if (piece == kChunksPerBox - 1) {
                     fence_proxy_async();  // make the generic-proxy writes visible to the TMA engine
                     __syncwarp();
@@ -234,7 +234,7 @@ k_gemm_i8(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
     if (threadIdx.x == 0 && s_abort && p.dev_status) atomicMax(p.dev_status, kStatusTimeout);
 }
 
-template <int BN, int kOut, bool kPerVec>
+template <int BN, int kOut, bool kPerVec, bool kBias>
 cudaError_t launch_gemm_inst(const GemmArgs &a, cudaStream_t s) {
     using C = Cfg<BN>;
     static PerDevice<int> attr_set;  // per instantiation and device
@@ -243,7 +243,7 @@ cudaError_t launch_gemm_inst(const GemmArgs &a, cudaStream_t s) {
     {
         std::lock_guard<std::mutex> lock(device_mutex());
         if (!attr_set.have[dev]) {
-            cudaError_t e = cudaFuncSetAttribute(k_gemm_i8<BN, kOut, kPerVec>,
+            cudaError_t e = cudaFuncSetAttribute(k_gemm_i8<BN, kOut, kPerVec, kBias>,
                                                  cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
             if (e != cudaSuccess) return e;
             attr_set.have[dev] = true;
@@ -276,7 +276,7 @@ cudaError_t launch_gemm_inst(const GemmArgs &a, cudaStream_t s) {
     p.w_stable = 0; p.spin = kSpinLimit; p.skip_kb = -1;
     int grid = p.tiles_m * p.tiles_n;
     if (grid > num_sms()) grid = num_sms();
-    k_gemm_i8<BN, kOut, kPerVec><<<grid, kGemmThreads, C::kSmemBytes, s>>>(tm_a, tm_aux, tm_b, tm_baux, tm_y, p);
+    k_gemm_i8<BN, kOut, kPerVec, kBias><<<grid, kGemmThreads, C::kSmemBytes, s>>>(tm_a, tm_aux, tm_b, tm_baux, tm_y, p);
     return cudaGetLastError();
 }
 
@@ -284,9 +284,13 @@ template <int BN>
 cudaError_t launch_gemm_bn(const GemmArgs &a, cudaStream_t s) {
     const bool per_vec = a.s_x_per_row || a.s_w_per_col;  // the two granularities come as a pair
     switch (a.out_kind) {
-        case kOutF16: return per_vec ? launch_gemm_inst<BN, kOutF16, true>(a, s) : launch_gemm_inst<BN, kOutF16, false>(a, s);
-        case kOutF32: return per_vec ? launch_gemm_inst<BN, kOutF32, true>(a, s) : launch_gemm_inst<BN, kOutF32, false>(a, s);
-        default: return launch_gemm_inst<BN, kOutI32, false>(a, s);
+        case kOutF16:
+            if (a.bias) return per_vec ? launch_gemm_inst<BN, kOutF16, true, true>(a, s) : launch_gemm_inst<BN, kOutF16, false, true>(a, s);
+            return per_vec ? launch_gemm_inst<BN, kOutF16, true, false>(a, s) : launch_gemm_inst<BN, kOutF16, false, false>(a, s);
+        case kOutF32:
+            if (a.bias) return per_vec ? launch_gemm_inst<BN, kOutF32, true, true>(a, s) : launch_gemm_inst<BN, kOutF32, false, true>(a, s);
+            return per_vec ? launch_gemm_inst<BN, kOutF32, true, false>(a, s) : launch_gemm_inst<BN, kOutF32, false, false>(a, s);
+        default: return launch_gemm_inst<BN, kOutI32, false, false>(a, s);
     }
 }
 

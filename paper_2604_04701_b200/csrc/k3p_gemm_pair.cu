@@ -41,7 +41,7 @@ struct PairCfg {
     static_assert(kStages >= 4, "operand ring too shallow");
 };
 
-template <int BN, int kOut, bool kPerVec>
+template <int BN, int kOut, bool kPerVec, bool kBias>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 k_gemm_i8_pair(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_aux,
                const __grid_constant__ CUtensorMap tm_b, const __grid_constant__ CUtensorMap tm_baux,
@@ -255,9 +255,9 @@ k_gemm_i8_pair(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                     __syncwarp();
                 }
                 const int gcol = n0 + col0 + 32 * ch;
-                convert_chunk<kOut, kPerVec>(v[ch], reinterpret_cast<uint4 *>(stage + lane * 128),
+                convert_chunk<kOut, kPerVec, kBias>(v[ch], reinterpret_cast<uint4 *>(stage + lane * 128),
                                              kOut == kOutF16 ? 4 * piece : 0, sw_xor, sx, sxw, p.s_w + gcol,
-                                             p.N - gcol, p.bias ? p.bias + gcol : nullptr);
+                                             p.N - gcol, kBias ? p.bias + gcol : nullptr);
                 if (piece == kChunksPerBox - 1) {
                     fence_proxy_async();
                     __syncwarp();
@@ -286,10 +286,10 @@ k_gemm_i8_pair(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     if (threadIdx.x == 0 && s_abort && p.dev_status) atomicMax(p.dev_status, kStatusTimeout);
 }
 
-template <int BN, int kOut, bool kPerVec>
+template <int BN, int kOut, bool kPerVec, bool kBias>
 cudaError_t launch_pair_inst(const GemmArgs &a, cudaStream_t s) {
     using C = PairCfg<BN>;
-    auto kern = k_gemm_i8_pair<BN, kOut, kPerVec>;
+    auto kern = k_gemm_i8_pair<BN, kOut, kPerVec, kBias>;
     static PerDevice<int> cache;  // per instantiation and device: clusters of 2 that fit on the device at once
     const int dev = current_device();
     if (dev < 0) return cudaErrorInvalidDevice;
@@ -364,9 +364,13 @@ template <int BN>
 cudaError_t launch_pair_bn(const GemmArgs &a, cudaStream_t s) {
     const bool per_vec = a.s_x_per_row || a.s_w_per_col;
     switch (a.out_kind) {
-        case kOutF16: return per_vec ? launch_pair_inst<BN, kOutF16, true>(a, s) : launch_pair_inst<BN, kOutF16, false>(a, s);
-        case kOutF32: return per_vec ? launch_pair_inst<BN, kOutF32, true>(a, s) : launch_pair_inst<BN, kOutF32, false>(a, s);
-        default: return launch_pair_inst<BN, kOutI32, false>(a, s);
+        case kOutF16:
+            if (a.bias) return per_vec ? launch_pair_inst<BN, kOutF16, true, true>(a, s) : launch_pair_inst<BN, kOutF16, false, true>(a, s);
+            return per_vec ? launch_pair_inst<BN, kOutF16, true, false>(a, s) : launch_pair_inst<BN, kOutF16, false, false>(a, s);
+        case kOutF32:
+            if (a.bias) return per_vec ? launch_pair_inst<BN, kOutF32, true, true>(a, s) : launch_pair_inst<BN, kOutF32, false, true>(a, s);
+            return per_vec ? launch_pair_inst<BN, kOutF32, true, false>(a, s) : launch_pair_inst<BN, kOutF32, false, false>(a, s);
+        default: return launch_pair_inst<BN, kOutI32, false, false>(a, s);
     }
 }
 
