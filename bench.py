@@ -49,8 +49,8 @@ WORKLOAD_TEXT = {
 CSRC = os.path.join(ROOT, "paper_2604_04701_b200", "csrc")
 TRAFFIC = {
     # kernel key: (source files, sha16 of their concatenation at capture time, {workload: bytes per launch}, note)
-    "k_gemm_i8_pair": (["k3p_gemm_pair.cu", "gemm_common.cuh", "ptx.cuh"], "0d9613bb1c935026",
-                       {"cfg3": {"16384x1280->1280": 25.9e6, "16384x1280->5120": 138.5e6}},
+    "k_gemm_i8_pair": (["k3p_gemm_pair.cu", "gemm_common.cuh", "ptx.cuh"], "cf2bd61da2081cdb",
+                       {"cfg3": {"16384x1280->1280": 26.6e6, "16384x1280->5120": 138.1e6}},
                        "profiles/k_gemm_i8_pair_configs3.md"),
     "k_prep": (["k12_prep.cu", "quant.cuh"], "376646cd649c08db",
                {"cfg3": {"16384x1280": 46.9e6, "16384x5120": 328.9e6}}, "profiles/k_prep_configs3.md"),
