@@ -17,11 +17,11 @@
 //                   derives the slice's channel maxima and outlier flags (Section III-C) and merges the maxima of
 //                   Body (Eq. 4) into the layer's words in global memory; when all slices of the layer have done so
 //                   (a counter), the scale(s) of Eq. 1 are known and the warp writes its slice's INT8 codes and
-//                   its outlier mask to the layer's scratch area in global memory and counts itself done; the
-//                   last one to do so also writes the layer's header (scales, r, the list of 64-byte segments
-//                   that hold an outlier channel) and raises the layer's ready word.
+//                   its outlier mask to the layer's scratch area in global memory and counts itself done.  The
+//                   warp whose merge completed the first count writes the layer's header meanwhile (scales, r, the
+//                   list of 64-byte segments that hold an outlier channel) and counts that as one more part.
 //                   Every CTA used to do all of this for itself, which cost more than the weight stream.
-//   fetch warp      per layer, in order: once the layer is ready (one poll looks 32 layers ahead) and one of the
+//   fetch warp      per layer, in order: once all parts of the layer are there (one poll looks 32 layers ahead) and one of the
 //                   CTA's buffers in shared memory is free, has the copy engine bring header and codes there.
 //   unit warps      per layer: each unit is taken by ONE warp, which accumulates the unit's 8 x M outputs over all
 //                   of K in registers (4-way byte dot products for M <= 4, mma.sync m16n8k32 above), adds the Aux
@@ -130,11 +130,11 @@ __device__ __forceinline__ bool wait_count(const uint32_t *ctr, uint32_t want, v
 // Per layer, in global memory (zero when the launch starts): the counters and maxima the slice warps share.
 struct LayerSync {
     uint32_t merged;      // slices whose maxima and outlier counts are in
-    uint32_t coded;       // slices whose codes and mask are written
+    uint32_t coded;       // slices whose codes and mask are written, plus one for the layer's header
     uint32_t r;           // outlier channels found so far
     uint32_t stored;      // CTAs whose units of this layer are stored (counted only when the next layer waits)
     uint32_t bmax[16];    // bit patterns of the row maxima of Body (per tensor: word 0 only)
-    uint32_t ready;       // the layer's header, codes and mask are complete
+    uint32_t unused;
     uint32_t pad[11];
 };
 static_assert(sizeof(LayerSync) == 128, "per-layer words");
@@ -368,7 +368,8 @@ __global__ void __launch_bounds__(kThreads, 1) k_decode_stream(const ChainArgs a
                 // lane i looks at layer l + i: in a list of independent layers most are ready long before their turn
                 bool ok = false, stopped = false;
                 for (uint32_t i = 0; i < a.spin && !ok && !stopped; ++i) {
-                    const bool rdy = l + lane < a.n_layers && ld_acquire_u32(&sync[l + lane].ready) != 0u;
+                    const bool rdy = l + lane < a.n_layers &&
+                                     ld_acquire_u32(&sync[l + lane].coded) > (uint32_t)(tab[l + lane].K >> 6);  // all slices and the header
                     const uint32_t bal = __ballot_sync(0xffffffffu, rdy);
                     const int n = __ffs((int)~bal) - 1;  // consecutive ready layers from l on (-1: all 32)
                     if (n != 0) {
@@ -523,10 +524,69 @@ __global__ void __launch_bounds__(kThreads, 1) k_decode_stream(const ChainArgs a
                         }
                 }
             }
+            {
+                const uint32_t any = __ballot_sync(0xffffffffu, mask != 0u);
+                if (lane == 0) g_segflag[s] = any ? 1 : 0;
+            }
             __syncwarp();
+            uint32_t before = 0;
             if (lane == 0) {
                 __threadfence();
-                atomicAdd(&sync[l].merged, 1u);
+                before = atomicAdd(&sync[l].merged, 1u);
+            }
+            before = __shfl_sync(0xffffffffu, before, 0);
+            if (before + 1u == (uint32_t)ns) {
+                // ---- the last slice of the layer to be merged: everything the header needs is final (maxima, r, the
+                // slices' segment flags and channels), so this warp writes it now -- scales, r, flagged 64-byte segments
+                // in ascending order, per-layer result -- while the others already quantize, and counts it as one more
+                // coded part of the layer
+                __threadfence();
+                const int rh = (int)__ldcg(&sync[l].r);
+                const bool over = rh > a.cap;  // MUXQ_ERR_CAPACITY: no codes were written, Y of this layer is unspecified
+                XHeader *hdr = reinterpret_cast<XHeader *>(g_head);
+                uint16_t *flaglist = reinterpret_cast<uint16_t *>(g_head + kHeaderBytes);
+                float sc0 = 1.0f;
+                if (lane < 16) {
+                    const float mx = __uint_as_float(__ldcg(&sync[l].bmax[a.per_vec ? lane : 0]));
+                    sc0 = mx > 0.0f ? __fdiv_rn(mx, qf) : 1.0f;
+                    hdr->rowscale[lane] = sc0;
+                }
+                uint32_t bits = 0;  // this lane: segments 4 lane .. 4 lane + 3
+                if (!over) {
+                    const uint32_t w = __ldcg(reinterpret_cast<const uint32_t *>(g_segflag) + lane);
+#pragma unroll
+                    for (int j = 0; j < 4; ++j)
+                        if (4 * lane + j < ns && ((w >> (8 * j)) & 0xFFu)) bits |= 1u << j;
+                }
+                int pre = __popc(bits);  // inclusive prefix count over the lanes
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const int n = __shfl_up_sync(0xffffffffu, pre, o);
+                    if (lane >= o) pre += n;
+                }
+                const int nf = __shfl_sync(0xffffffffu, pre, 31);
+                int at = pre - __popc(bits);
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+                    if ((bits >> j) & 1u) flaglist[at++] = (uint16_t)(4 * lane + j);
+                if (lane == 0) {
+                    hdr->r = rh;
+                    hdr->nflag = nf;
+                    if (over && a.dev_status) atomicMax(a.dev_status, kStatusCapacity);
+                    if (a.results) {
+                        ChainResult rr;
+                        rr.n_outliers = rh;
+                        rr.status = over ? kStatusCapacity : 0;
+                        rr.s_x = sc0;
+                        rr.reserved = 0;
+                        a.results[l] = rr;
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) {
+                    __threadfence();
+                    atomicAdd(&sync[l].coded, 1u);
+                }
             }
             // ---- all slices merged: the scale(s) of Eq. 1 are final; codes of this slice
             if (!wait_count(&sync[l].merged, (uint32_t)ns, abort_flag, g_abort, a.spin)) break;
@@ -558,65 +618,11 @@ __global__ void __launch_bounds__(kThreads, 1) k_decode_stream(const ChainArgs a
                            ((mask & 128) ? 0xFF000000u : 0u);
                     *reinterpret_cast<uint2 *>(g_mask + ch) = mb;
                 }
-                const uint32_t any = __ballot_sync(0xffffffffu, mask != 0u);
-                if (lane == 0) g_segflag[s] = any ? 1 : 0;
             }
             __syncwarp();
-            uint32_t before = 0;
             if (lane == 0) {
                 __threadfence();
-                before = atomicAdd(&sync[l].coded, 1u);
-            }
-            before = __shfl_sync(0xffffffffu, before, 0);
-            if (before + 1u == (uint32_t)ns) {
-                // ---- the last slice of the layer: header block (scales, r, flagged 64-byte segments in ascending
-                // order), per-layer result, then the ready word
-                __threadfence();
-                const bool over = r > a.cap;  // MUXQ_ERR_CAPACITY: no codes were written, Y of this layer is unspecified
-                XHeader *hdr = reinterpret_cast<XHeader *>(g_head);
-                uint16_t *flaglist = reinterpret_cast<uint16_t *>(g_head + kHeaderBytes);
-                float sc0 = 1.0f;
-                if (lane < 16) {
-                    const float mx = __uint_as_float(__ldcg(&sync[l].bmax[a.per_vec ? lane : 0]));
-                    sc0 = mx > 0.0f ? __fdiv_rn(mx, qf) : 1.0f;
-                    hdr->rowscale[lane] = sc0;
-                }
-                uint32_t bits = 0;  // this lane: segments 4 lane .. 4 lane + 3
-                if (!over) {
-                    const uint32_t w = __ldcg(reinterpret_cast<const uint32_t *>(g_segflag) + lane);
-#pragma unroll
-                    for (int j = 0; j < 4; ++j)
-                        if (4 * lane + j < ns && ((w >> (8 * j)) & 0xFFu)) bits |= 1u << j;
-                }
-                int pre = __popc(bits);  // inclusive prefix count over the lanes
-#pragma unroll
-                for (int o = 1; o < 32; o <<= 1) {
-                    const int n = __shfl_up_sync(0xffffffffu, pre, o);
-                    if (lane >= o) pre += n;
-                }
-                const int nf = __shfl_sync(0xffffffffu, pre, 31);
-                int at = pre - __popc(bits);
-#pragma unroll
-                for (int j = 0; j < 4; ++j)
-                    if ((bits >> j) & 1u) flaglist[at++] = (uint16_t)(4 * lane + j);
-                if (lane == 0) {
-                    hdr->r = r;
-                    hdr->nflag = nf;
-                    if (over && a.dev_status) atomicMax(a.dev_status, kStatusCapacity);
-                    if (a.results) {
-                        ChainResult rr;
-                        rr.n_outliers = r;
-                        rr.status = over ? kStatusCapacity : 0;
-                        rr.s_x = sc0;
-                        rr.reserved = 0;
-                        a.results[l] = rr;
-                    }
-                }
-                __syncwarp();
-                if (lane == 0) {
-                    __threadfence();
-                    atomicExch(&sync[l].ready, 1u);
-                }
+                atomicAdd(&sync[l].coded, 1u);
             }
         }
     } else {
