@@ -676,7 +676,7 @@ __global__ void __launch_bounds__(kThreads, 1) k_decode_stream(const ChainArgs a
                     pos.use = (uint32_t)(seq0 / S);
                     // Body accumulators (several: consecutive products on one accumulator wait for each other) and the
                     // Aux accumulator over the outlier channels (Aux_q == Body_q[:, O], Eq. 5)
-                    constexpr int kAcc = (kDotM == 1 || kDotM == 2) ? 4 : 2;
+                    constexpr int kAcc = kDotM == 4 ? 2 : 4;
                     int accb[kAcc][4], acca[4] = {0, 0, 0, 0};
 #pragma unroll
                     for (int j = 0; j < kAcc; ++j) accb[j][0] = accb[j][1] = accb[j][2] = accb[j][3] = 0;
@@ -743,21 +743,22 @@ __global__ void __launch_bounds__(kThreads, 1) k_decode_stream(const ChainArgs a
                             } else {
                                 // mma.sync tiles: lane (g, q) supplies 16 bytes of token rows g and g + 8 and of W_q row
                                 // 8u + g per segment (the K order inside a segment permuted alike for both operands)
+                                // Four segments at a time, each on an accumulator of its own: all loads, then eight
+                                // products in four chains of two.
                                 int sgi = 0;
-                                for (; sgi + 2 <= segs; sgi += 2) {
-                                    uint4 w[2], alo[2], ahi[2];
+                                for (; sgi + 4 <= segs; sgi += 4) {
+                                    uint4 w[4], alo[4], ahi[4];
 #pragma unroll
-                                    for (int j = 0; j < 2; ++j) {
+                                    for (int j = 0; j < 4; ++j) {
                                         const int o = (sgi + j) * 64 + q * 16;
                                         w[j] = *reinterpret_cast<const uint4 *>(wrow + o);
                                         alo[j] = *reinterpret_cast<const uint4 *>(xseg + g * L.pitch + o);
                                         ahi[j] = MT == 16 ? *reinterpret_cast<const uint4 *>(xseg + (g + 8) * L.pitch + o) : make_uint4(0u, 0u, 0u, 0u);
                                     }
 #pragma unroll
-                                    for (int j = 0; j < 2; ++j) {
-                                        mma_s8(accb[0], alo[j].x, ahi[j].x, alo[j].y, ahi[j].y, w[j].x, w[j].y);
-                                        mma_s8(accb[1], alo[j].z, ahi[j].z, alo[j].w, ahi[j].w, w[j].z, w[j].w);
-                                    }
+                                    for (int j = 0; j < 4; ++j) mma_s8(accb[j], alo[j].x, ahi[j].x, alo[j].y, ahi[j].y, w[j].x, w[j].y);
+#pragma unroll
+                                    for (int j = 0; j < 4; ++j) mma_s8(accb[j], alo[j].z, ahi[j].z, alo[j].w, ahi[j].w, w[j].z, w[j].w);
                                 }
                                 for (; sgi < segs; ++sgi) {
                                     const int o = sgi * 64 + q * 16;
@@ -875,10 +876,13 @@ __global__ void __launch_bounds__(kThreads, 1) k_decode_stream(const ChainArgs a
                         }
                     } else {
                         // this lane holds token rows g and g + 8, output channels 8u + 2q and 8u + 2q + 1
-                        emit(g, u * 8 + 2 * q, accb[0][0] + accb[1][0] + a.c * acca[0]);
-                        emit(g, u * 8 + 2 * q + 1, accb[0][1] + accb[1][1] + a.c * acca[1]);
-                        emit(g + 8, u * 8 + 2 * q, accb[0][2] + accb[1][2] + a.c * acca[2]);
-                        emit(g + 8, u * 8 + 2 * q + 1, accb[0][3] + accb[1][3] + a.c * acca[3]);
+                        int v[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) v[e] = accb[0][e] + accb[1][e] + accb[2][e] + accb[3][e] + a.c * acca[e];
+                        emit(g, u * 8 + 2 * q, v[0]);
+                        emit(g, u * 8 + 2 * q + 1, v[1]);
+                        emit(g + 8, u * 8 + 2 * q, v[2]);
+                        emit(g + 8, u * 8 + 2 * q + 1, v[3]);
                     }
                 }
             }
