@@ -1006,6 +1006,8 @@ namespace {
 
 template <int MT, int kDotM>
 cudaError_t launch_inst(ChainArgs a, cudaStream_t s) {
+    // the plan's scratch areas and shared-memory places were laid out for chain_rows(M) rows of codes per layer
+    if (chain_rows(a.M) != (kDotM > 0 ? kDotM : MT)) return cudaErrorInvalidValue;
     auto kern = k_decode_stream<MT, kDotM>;
     static PerDevice<int> attr_set;
     const int dev = current_device();
