@@ -864,15 +864,33 @@ __global__ void __launch_bounds__(kThreads, 1) k_decode_stream(const ChainArgs a
                         }
                     };
                     if constexpr (kDotM > 0) {
-                        // the four lanes of a W_q row add up; lane q == 0 of row g holds output channel 8u + g
+                        // The four lanes of a W_q row (output channel 8u + g) add up.  With several token rows the sums
+                        // are spread over the four lanes on the way (lane q ends up with row q): three exchanges instead
+                        // of eight, and the rows are dequantized and stored side by side.
+                        int v[kDotM];
 #pragma unroll
                         for (int m = 0; m < kDotM; ++m) {
-                            int v = a.c * acca[m];
+                            v[m] = a.c * acca[m];
 #pragma unroll
-                            for (int j = 0; j < kAcc; ++j) v += accb[j][m];
-                            v += __shfl_xor_sync(0xffffffffu, v, 1);
-                            v += __shfl_xor_sync(0xffffffffu, v, 2);
-                            if (q == 0) emit(m, u * 8 + g, v);
+                            for (int j = 0; j < kAcc; ++j) v[m] += accb[j][m];
+                        }
+                        if constexpr (kDotM == 4) {
+                            const bool odd = (q & 1) != 0, hi = (q & 2) != 0;
+                            const int r0 = __shfl_xor_sync(0xffffffffu, odd ? v[0] : v[1], 1);
+                            const int r1 = __shfl_xor_sync(0xffffffffu, odd ? v[2] : v[3], 1);
+                            const int k0 = (odd ? v[1] : v[0]) + r0;  // rows 0 (even lanes) / 1 (odd lanes), two lanes' worth
+                            const int k1 = (odd ? v[3] : v[2]) + r1;  // rows 2 / 3
+                            const int r2 = __shfl_xor_sync(0xffffffffu, hi ? k0 : k1, 2);
+                            emit(q, u * 8 + g, (hi ? k1 : k0) + r2);
+                        } else if constexpr (kDotM == 2) {
+                            const bool odd = (q & 1) != 0;
+                            int k0 = (odd ? v[1] : v[0]) + __shfl_xor_sync(0xffffffffu, odd ? v[0] : v[1], 1);
+                            k0 += __shfl_xor_sync(0xffffffffu, k0, 2);
+                            if (q < 2) emit(q, u * 8 + g, k0);
+                        } else {
+                            int t0 = v[0] + __shfl_xor_sync(0xffffffffu, v[0], 1);
+                            t0 += __shfl_xor_sync(0xffffffffu, t0, 2);
+                            if (q == 0) emit(0, u * 8 + g, t0);
                         }
                     } else {
                         // this lane holds token rows g and g + 8, output channels 8u + 2q and 8u + 2q + 1
