@@ -208,6 +208,9 @@ __global__ void __launch_bounds__(kThreads, 1) k_decode_stream(const ChainArgs a
     const int t = threadIdx.x, lane = t & 31;
     const int warp = __shfl_sync(0xffffffffu, t >> 5, 0);  // warp-uniform by construction
     const int S = a.slots, M = a.M;
+    // n / S as a multiplication: exact for n * S < 2^32, far beyond any CTA's number of stages (a 32-bit division
+    // is some forty instructions, and the warps that need it are single-warp pipelines)
+    const uint32_t s_magic = 0xFFFFFFFFu / (uint32_t)S + 1u;
     const int grid = (int)gridDim.x, cta = (int)blockIdx.x;
     uint8_t *ring = smem;
     ChainLayer *tab = reinterpret_cast<ChainLayer *>(smem + (size_t)S * a.slot_bytes);
@@ -305,8 +308,8 @@ __global__ void __launch_bounds__(kThreads, 1) k_decode_stream(const ChainArgs a
             int i = (int)j / nst, st = (int)j - i * nst;                                    // its unit and K slice
             for (; j < nstage; j += LG) {
                 const uint32_t seq = lseq + j;
-                const int slot = (int)(seq % (uint32_t)S);
-                const uint32_t use = seq / (uint32_t)S;
+                const uint32_t use = __umulhi(seq, s_magic);
+                const int slot = (int)(seq - use * (uint32_t)S);
                 if (use > 0 && !wait_sleep(&bar_empty[slot], (use - 1u) & 1u, abort_flag, a.spin)) {
                     ok = false;
                     break;
@@ -672,8 +675,8 @@ __global__ void __launch_bounds__(kThreads, 1) k_decode_stream(const ChainArgs a
                     const int u = first + i * grid;
                     const int seq0 = lseq + i * nst;
                     RingPos pos;
-                    pos.slot = seq0 % S;
-                    pos.use = (uint32_t)(seq0 / S);
+                    pos.use = __umulhi((uint32_t)seq0, s_magic);
+                    pos.slot = seq0 - (int)pos.use * S;
                     // Body accumulators (several: consecutive products on one accumulator wait for each other) and the
                     // Aux accumulator over the outlier channels (Aux_q == Body_q[:, O], Eq. 5)
                     constexpr int kAcc = kDotM == 4 ? 2 : 4;
