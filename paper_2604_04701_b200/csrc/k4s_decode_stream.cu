@@ -256,7 +256,7 @@ __global__ void __launch_bounds__(kThreads, 1) k_decode_stream(const ChainArgs a
         const int units = ly.N >> 3, first = first_unit(ly);
         const int cnt = first < units ? (units - first + grid - 1) / grid : 0;
         s_cnt[l] = (uint16_t)cnt;
-        s_lseq[l] = (uint32_t)(cnt * (ly.K / (int)ly.seg));
+        s_lseq[l] = (uint32_t)(cnt * (int)ly.nst);
         s_scr[l] = (uint32_t)scratch_layer_bytes(kRows, ly.K);
     }
     __syncthreads();
@@ -300,11 +300,11 @@ __global__ void __launch_bounds__(kThreads, 1) k_decode_stream(const ChainArgs a
             if (cnt == 0) continue;
             const uint32_t lseq = s_lseq[l];  // number of this CTA's stages before the layer
             const ChainLayer ly = tab[l];
-            const int seg = (int)ly.seg, nst = ly.K / seg;
+            const int seg = (int)ly.seg, nst = (int)ly.nst;
             const int first = first_unit(ly);
             const uint32_t nstage = (uint32_t)(cnt * nst);
             const bool flat = seg == ly.ldw;
-            uint32_t j = (uint32_t)(wl + LG - (int)(lseq % (uint32_t)LG)) % (uint32_t)LG;  // first stage of the layer that is this warp's
+            uint32_t j = (uint32_t)(wl - (int)lseq) & (uint32_t)(LG - 1);  // first stage of the layer that is this warp's (LG is 4 or 2)
             int i = (int)j / nst, st = (int)j - i * nst;                                    // its unit and K slice
             for (; j < nstage; j += LG) {
                 const uint32_t seq = lseq + j;
@@ -651,7 +651,7 @@ __global__ void __launch_bounds__(kThreads, 1) k_decode_stream(const ChainArgs a
             const uint8_t *g_mask = a.scratch + s_scr[l] + kHeadBlock + scratch_codes_bytes(kRows, ly.K);
             const uint16_t *flaglist = reinterpret_cast<const uint16_t *>(buf + L.off_flaglist);
             const uint16_t *chlist = reinterpret_cast<const uint16_t *>(buf + L.off_chlist);
-            const int seg = (int)ly.seg, nst = K / seg, segs = seg >> 6;
+            const int seg = (int)ly.seg, nst = (int)ly.nst, segs = seg >> 6;
             const int first = first_unit(ly);
             // (a warp that has passed layers by must not take an older phase of the barrier for this one)
             {
@@ -1015,7 +1015,7 @@ int chain_plan(ChainLayer *layers, int n_layers, int grid, int slot_bytes) {
         ly.seg = (uint16_t)(ly.K / nst);
         ly.unit_off = (uint16_t)off;
         ly.slice_off = (uint16_t)soff;
-        ly.reserved = 0;
+        ly.nst = (uint16_t)nst;
         off = (off + (ly.N >> 3)) % grid;
         soff = (soff + (ly.K >> 6)) % (kSW * grid);
         if (ly.K > kmax) kmax = ly.K;

@@ -203,7 +203,7 @@ struct ChainLayer {                  // one entry of the device-resident layer t
     uint16_t unit_off;   // unit u of this layer goes to CTA (unit_off + u) mod grid
     uint16_t seg;        // bytes of each W_q row per ring stage (K / seg stages per unit of 8 rows)
     uint16_t slice_off;  // slice s of this layer's X goes to slice warp (slice_off + s) mod (kChainSliceWarps * grid)
-    uint16_t reserved;
+    uint16_t nst;        // K / seg
 };
 static_assert(sizeof(ChainLayer) == 64, "layer table entry");
 struct ChainResult {               // per layer, written by CTA 0 (optional)
