@@ -647,8 +647,6 @@ __global__ void __launch_bounds__(kThreads, 1) k_decode_stream(const ChainArgs a
             const uint8_t *buf = xbase + (size_t)(s_place[l] & 0xFFFFu) * 128;
             const XHeader *hdr = reinterpret_cast<const XHeader *>(buf);
             const int8_t *xq = reinterpret_cast<const int8_t *>(buf + L.off_xq);
-            // (written in this launch by other SMs: read through L2; visible by way of the ready word and the buffer's barrier)
-            const uint8_t *g_mask = a.scratch + s_scr[l] + kHeadBlock + scratch_codes_bytes(kRows, ly.K);
             const uint16_t *flaglist = reinterpret_cast<const uint16_t *>(buf + L.off_flaglist);
             const uint16_t *chlist = reinterpret_cast<const uint16_t *>(buf + L.off_chlist);
             const int seg = (int)ly.seg, nst = (int)ly.nst, segs = seg >> 6;
@@ -689,7 +687,7 @@ __global__ void __launch_bounds__(kThreads, 1) k_decode_stream(const ChainArgs a
                         // wait for a stage before the loaders have begun to fill it (by then the slot's previous use has
                         // been consumed and its phase is complete).  With more units per layer than ring slots a warp
                         // can get that far ahead.
-                        {
+                        if (s_begun[pos.slot] <= pos.use) {  // (one load for the whole warp; rarely taken)
                             uint32_t spins = 0;
                             while (s_begun[pos.slot] <= pos.use && ++spins < a.spin) {
                                 __nanosleep(40);
@@ -822,6 +820,9 @@ __global__ void __launch_bounds__(kThreads, 1) k_decode_stream(const ChainArgs a
                             } else {
                                 // many outlier channels: per flagged 64-byte segment, the same products as for Body with X
                                 // masked to the outlier channels
+                                // (the mask was written in this launch by other SMs: read through L2; visible by way of the
+                                // layer's count of parts and the buffer's barrier)
+                                const uint8_t *g_mask = a.scratch + s_scr[l] + kHeadBlock + scratch_codes_bytes(kRows, ly.K);
                                 const int seg0 = st * segs;
                                 for (int j = 0; j < nflag; ++j) {
                                     const int fs = (int)flaglist[j] - seg0;
