@@ -239,7 +239,8 @@ int muxq_linear_host(const void *X_f16_host, int M, int K, const int8_t *W_q, in
  * W_q is fetched while the layers before it are still being computed; a one-layer call cannot do that.
  *
  * muxq_layer: X [M, ldx] fp16, W_q [N, ldw] int8 and s_w from muxq_quantize(is_weight = 1), Y [M, ldy] by the
- * list's out_kind.  flags = MUXQ_LAYER_WAIT_PREV says that this layer's X is written by the layer before it
+ * list's out_kind; bias: fp32 [N] added after the dequantization as in muxq_linear_bias, or NULL (must be NULL
+ * with MUXQ_OUT_ACC_I32).  flags = MUXQ_LAYER_WAIT_PREV says that this layer's X is written by the layer before it
  * in the list (its Y, or memory derived from nothing else): the layer's activation work then starts only when
  * every CTA has counted its part of that Y as stored (bounded waits on counters in the plan's device memory).
  * Without the flag the layers are independent.  The activation work of a layer (Section III-C, Eq. 4, Eq. 1) is
@@ -271,6 +272,7 @@ typedef struct muxq_layer {
     int ldx, ldw, ldy;
     int K, N;
     int flags;
+    const float *bias; /* fp32 [N] added after the dequantization (as in muxq_linear_bias), or NULL */
 } muxq_layer;
 typedef struct muxq_chain_result {
     int32_t n_outliers; /* r of this layer's X */

@@ -323,13 +323,13 @@ MUXQ_LAYER_WAIT_PREV = 1
 class _CLayer(ctypes.Structure):
     _fields_ = [("X_f16", ctypes.c_void_p), ("W_q", ctypes.c_void_p), ("s_w", ctypes.c_void_p), ("Y", ctypes.c_void_p),
                 ("ldx", ctypes.c_int), ("ldw", ctypes.c_int), ("ldy", ctypes.c_int), ("K", ctypes.c_int),
-                ("N", ctypes.c_int), ("flags", ctypes.c_int)]
+                ("N", ctypes.c_int), ("flags", ctypes.c_int), ("bias", ctypes.c_void_p)]
 
 
 class Chain:
     """A list of decode-shaped layers run by one persistent launch (muxq_chain_build / muxq_chain_run).
 
-    layers: sequence of (X [M,K] f16, w_q [N,K] i8, s_w, Y [M,N], flags).  The tensors are kept alive by this
+    layers: sequence of (X [M,K] f16, w_q [N,K] i8, s_w, Y [M,N], flags[, bias f32 [N]]).  The tensors are kept alive by this
     object; results (one row of [r, status, s_x bits, 0] per layer, int32) and the status word live on the device."""
 
     def __init__(self, layers, p: MuxqParams, out_kind: int = MUXQ_OUT_F16):
@@ -338,10 +338,14 @@ class Chain:
         self.M = int(layers[0][0].shape[0])
         dev = layers[0][0].device
         arr = (_CLayer * n)()
-        for k, (X, w_q, s_w, Y, flags) in enumerate(layers):
+        for k, entry in enumerate(layers):
+            X, w_q, s_w, Y, flags = entry[:5]
+            bias = entry[5] if len(entry) > 5 else None
             assert X.is_cuda and X.dtype == torch.float16 and X.stride(1) == 1 and X.shape[0] == self.M
+            assert bias is None or (bias.is_cuda and bias.dtype == torch.float32 and bias.numel() == w_q.shape[0])
             arr[k] = _CLayer(X.data_ptr(), w_q.data_ptr(), s_w.data_ptr(), Y.data_ptr(), X.stride(0), w_q.stride(0),
-                             Y.stride(0), X.shape[1], w_q.shape[0], int(flags))
+                             Y.stride(0), X.shape[1], w_q.shape[0], int(flags),
+                             bias.data_ptr() if bias is not None else None)
         nbytes = int(lib().muxq_chain_plan_bytes(n))
         if nbytes == 0:
             raise MuxqError("muxq_chain_plan_bytes", MUXQ_ERR_INVALID_ARG)

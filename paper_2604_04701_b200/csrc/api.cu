@@ -557,7 +557,8 @@ int muxq_chain_build(const muxq_layer *layers, int n_layers, int M, const muxq_p
     for (int l = 0; l < n_layers; ++l) {
         const muxq_layer &in = layers[l];
         if (!in.X_f16 || !in.W_q || !in.s_w || !in.Y || in.K <= 0 || in.N <= 0 || in.ldx < in.K || in.ldw < in.K ||
-            in.ldy < in.N || (in.flags & ~MUXQ_LAYER_WAIT_PREV) || (l == 0 && in.flags))
+            in.ldy < in.N || (in.flags & ~MUXQ_LAYER_WAIT_PREV) || (l == 0 && in.flags) ||
+            (in.bias && out_kind == MUXQ_OUT_ACC_I32))
             return MUXQ_ERR_INVALID_ARG;
         if (!chain_layer_supported(M, in.K, in.N) || in.ldx % 8 || in.ldw % 16 || in.ldy % yal || !aligned16(in.X_f16) ||
             !aligned16(in.W_q) || !aligned16(in.Y) || (p->gran == MUXQ_PER_VECTOR && !aligned16(in.s_w)))
@@ -567,6 +568,8 @@ int muxq_chain_build(const muxq_layer *layers, int n_layers, int M, const muxq_p
         o.w_q = in.W_q;
         o.s_w = in.s_w;
         o.Y = in.Y;
+        o.bias = out_kind == MUXQ_OUT_ACC_I32 ? nullptr : in.bias;
+        o.reserved = 0;
         o.ldx = in.ldx; o.ldw = in.ldw; o.ldy = in.ldy; o.K = in.K; o.N = in.N;
         o.flags = (in.flags & MUXQ_LAYER_WAIT_PREV) ? kChainWaitPrev : 0;
     }

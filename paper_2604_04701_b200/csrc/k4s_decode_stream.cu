@@ -223,7 +223,7 @@ __global__ void __launch_bounds__(kThreads, 1) k_decode_stream(const ChainArgs a
     {
         const uint4 *src = reinterpret_cast<const uint4 *>(a.layers);
         uint4 *dst = reinterpret_cast<uint4 *>(tab);
-        for (int i = t; i < a.n_layers * 4; i += kThreads) dst[i] = __ldg(src + i);
+        for (int i = t; i < a.n_layers * (int)(sizeof(ChainLayer) / 16); i += kThreads) dst[i] = __ldg(src + i);
         for (int i = t; i < a.n_layers; i += kThreads) s_place[i] = __ldg(a.place + i);
     }
     if (t == 0) {
@@ -862,7 +862,8 @@ __global__ void __launch_bounds__(kThreads, 1) k_decode_stream(const ChainArgs a
                             reinterpret_cast<int32_t *>(ly.Y)[o] = acc;
                         } else {
                             const float ss = a.per_vec ? __fmul_rn(hdr->rowscale[m], __ldg(ly.s_w + n)) : ssw0;
-                            const float y = __fmul_rn(ss, __int2float_rn(acc));
+                            float y = __fmul_rn(ss, __int2float_rn(acc));
+                            if (ly.bias) y = __fadd_rn(y, __ldg(ly.bias + n));  // the layer's additive term, one fp32 addition
                             if (a.out_kind == 1) reinterpret_cast<float *>(ly.Y)[o] = y;
                             else reinterpret_cast<__half *>(ly.Y)[o] = __float2half_rn(y);
                         }

@@ -193,11 +193,13 @@ cudaError_t launch_decode_fused(const DecodeFusedArgs &a, cudaStream_t s);
 constexpr int kChainMaxLayers = 256;
 constexpr int kChainSliceWarps = 7;  // warps per CTA that prepare slices of X for the whole grid
 constexpr int kChainWaitPrev = 1;    // ChainLayer::flags bit 0: X of this layer is written by the layer before it
-struct ChainLayer {                  // one entry of the device-resident layer table, 64 bytes
+struct ChainLayer {                  // one entry of the device-resident layer table, 80 bytes
     const __half *X;
     const int8_t *w_q;
     const float *s_w;
     void *Y;
+    const float *bias;   // [N] fp32 added after the dequantization, or NULL
+    uint64_t reserved;
     int ldx, ldw, ldy, K, N, flags;
     // filled by the host (chain_plan):
     uint16_t unit_off;   // unit u of this layer goes to CTA (unit_off + u) mod grid
@@ -205,7 +207,7 @@ struct ChainLayer {                  // one entry of the device-resident layer t
     uint16_t slice_off;  // slice s of this layer's X goes to slice warp (slice_off + s) mod (kChainSliceWarps * grid)
     uint16_t nst;        // K / seg
 };
-static_assert(sizeof(ChainLayer) == 64, "layer table entry");
+static_assert(sizeof(ChainLayer) == 80, "layer table entry");
 struct ChainResult {               // per layer, written by CTA 0 (optional)
     int32_t n_outliers;
     int32_t status;                // 0 or MUXQ_ERR_CAPACITY

@@ -151,6 +151,31 @@ def test_layers_with_more_outlier_channels_than_the_channel_list_holds(mx, M):
         assert results[0, 0] > 64 and results[1, 0] > 64 and results[2, 0] <= 64
 
 
+@pytest.mark.parametrize("M", [1, 2, 4, 16])
+def test_layers_with_an_additive_term(mx, M):
+    """Every other layer of the list carries a bias (fp32 [N]): fp32 outputs bit-equal to the oracle's one-addition
+    reading, fp16 within 1 ulp; the layers without one are untouched by their neighbours' terms."""
+    shapes = [(1280, 1280), (5120, 264), (1280, 3840), (256, 72)]
+    p = mx.MuxqParams(max_outliers=32)
+    L = _make_layers(mx, shapes, M, p, seed=700 + M)
+    biases = [(synth.normal(700 + M, 50 + i, N) * 0.5).astype(np.float32) if i % 2 == 0 else None
+              for i, (_, N) in enumerate(shapes)]
+    for out_kind in (mx.MUXQ_OUT_F32, mx.MUXQ_OUT_F16):
+        ys = [torch.full((M, N), -7, dtype=_OUT[out_kind], device="cuda") for (_, N) in shapes]
+        chain = mx.Chain([(xd, w_q, s_w, y, 0, None if b is None else _dev(b))
+                          for (_, _, xd, w_q, s_w), y, b in zip(L, ys, biases)], p, out_kind)
+        chain.run()
+        assert chain.read_status() == 0
+        for (x, w, _, _, _), y, b in zip(L, ys, biases):
+            wq_o, sw_o = oracle.quantize_weight(w)
+            res = oracle.linear(x, wq_o, sw_o, cap=32, bias=b)
+            g = y.cpu().numpy()
+            if out_kind == mx.MUXQ_OUT_F32:
+                assert np.array_equal(g, res.y32)
+            else:
+                assert np.abs(_f16_key(g) - _f16_key(res.y16)).max() <= 1
+
+
 def test_a_layer_over_capacity_is_reported_and_the_list_goes_on(mx):
     M = 4
     shapes = [(1280, 1280), (1280, 1280), (1280, 1280)]
