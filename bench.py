@@ -54,8 +54,8 @@ TRAFFIC = {
                        "profiles/k_gemm_i8_pair_configs3.md"),
     "k_prep": (["k12_prep.cu", "quant.cuh"], "376646cd649c08db",
                {"cfg3": {"16384x1280": 46.9e6, "16384x5120": 328.9e6}}, "profiles/k_prep_configs3.md"),
-    "k_decode_stream": (["k4s_decode_stream.cu", "quant.cuh", "ptx.cuh"], "6a8bf51ebfadb0c1",
-                        {"chain": 713.1e6}, "profiles/k_decode_stream_chain144.md"),
+    "k_decode_stream": (["k4s_decode_stream.cu", "quant.cuh", "ptx.cuh"], "ecf2c0babe5cc1a0",
+                        {"chain": 712.4e6}, "profiles/k_decode_stream_chain144.md"),
 }
 
 

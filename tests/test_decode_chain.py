@@ -176,6 +176,29 @@ def test_layers_with_an_additive_term(mx, M):
                 assert np.abs(_f16_key(g) - _f16_key(res.y16)).max() <= 1
 
 
+def test_strided_operands(mx):
+    """X, W_q and Y as views into wider buffers (row pitches larger than K / N): the bytes between the rows are
+    neither read as data nor written."""
+    M, p = 4, mx.MuxqParams(max_outliers=32)
+    shapes = [(1280, 1280), (5120, 264), (256, 72)]
+    L = _make_layers(mx, shapes, M, p, seed=900)
+    layers, ys, pads = [], [], []
+    for (x, w, xd, w_q, s_w), (K, N) in zip(L, shapes):
+        xw = torch.full((M, K + 64), 1000.0, dtype=torch.float16, device="cuda")   # would flag channels if it were read
+        xw[:, :K] = xd
+        ww = torch.full((N, K + 128), 77, dtype=torch.int8, device="cuda")
+        ww[:, :K] = w_q
+        yw = torch.full((M, N + 24), -7.0, dtype=torch.float32, device="cuda")
+        layers.append((xw[:, :K], ww[:, :K], s_w, yw[:, :N], 0))
+        ys.append(yw)
+    chain = mx.Chain(layers, p, mx.MUXQ_OUT_F32)
+    chain.run()
+    assert chain.read_status() == 0
+    for (x, w, _, _, _), yw, (K, N) in zip(L, ys, shapes):
+        _check_layer(mx, yw[:, :N].contiguous(), x, w, p, mx.MUXQ_OUT_F32)
+        assert bool((yw[:, N:] == -7.0).all())
+
+
 def test_a_layer_over_capacity_is_reported_and_the_list_goes_on(mx):
     M = 4
     shapes = [(1280, 1280), (1280, 1280), (1280, 1280)]
